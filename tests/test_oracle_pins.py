@@ -1,0 +1,455 @@
+"""Pins for the float64 oracle: each test ties one part of it to something other than itself.
+
+  - exhaustive subset search and planted ties          -> top-k / top-c selection (Eq. 17, 22)
+  - dense MLP / textbook multi-head attention          -> expert math at k=n, c=m (Eq. 1, 5, 8-11)
+  - mask identity of Fig. 4                            -> causal mask handling
+  - special cases, bounds, symmetries                  -> routing structure (Eq. 20, 23, 26)
+  - central finite differences                         -> backward
+  - scalar-loop twin                                   -> array indexing
+  - planted mistakes                                   -> the pins above do catch a wrong oracle
+"""
+import math
+
+import numpy as np
+import pytest
+
+import uoe_inputs as gen
+from oracle import loops
+from oracle import uoe_oracle as orc
+
+
+def _inputs(w, blocks=("mlp", "att")):
+    x = gen.make_x(w).f64
+    out = dict(x=x, Wr=gen.make_router(w, "mlp").f64, Wra=gen.make_router(w, "att").f64)
+    if "mlp" in blocks:
+        W1, W2 = gen.make_mlp_weights(w)
+        out.update(W1=W1.f64, W2=W2.f64)
+    if "att" in blocks:
+        Wq, Wk, Wv, Wo = gen.make_attn_weights(w)
+        out.update(Wq=Wq.f64, Wk=Wk.f64, Wv=Wv.f64, Wo=Wo.f64)
+    return out
+
+
+def _boost_router(Wr, scale=40.0):
+    # larger router weights so that the gates are far from uniform in the tiny cases
+    return Wr * scale
+
+
+# ----------------------------------------------------------------------------------------------
+# generator sanity (the pins below rely on these inputs)
+# ----------------------------------------------------------------------------------------------
+
+def test_generator_is_counter_based_and_normal():
+    a = gen.normal(5, 2, (1000, 64))
+    b = gen.normal(5, 2, (1000, 64), chunk=999)
+    assert np.array_equal(a, b)
+    assert abs(a.mean()) < 0.02 and abs(a.std() - 1.0) < 0.02
+    assert abs(np.mean(a ** 4) - 3.0) < 0.15
+    assert not np.array_equal(a, gen.normal(5, 3, (1000, 64)))
+
+
+def test_bf16_rounding_is_nearest_even():
+    v = np.array([1.0, 1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8, 1.0 + 2 ** -7, -2.5, 3.140625], dtype=np.float32)
+    got = gen.bf16_bits_to_f64(gen.f32_to_bf16_bits(v))
+    # ties: 1+2^-8 is halfway between 1 and 1+2^-7 -> even mantissa (1.0); 1+3*2^-8 -> 1+2^-6
+    assert got.tolist() == [1.0, 1.0, 1.0 + 2 ** -6, 1.0 + 2 ** -7, -2.5, 3.140625]
+
+
+# ----------------------------------------------------------------------------------------------
+# activations against closed forms
+# ----------------------------------------------------------------------------------------------
+
+def test_activation_closed_forms():
+    h = np.array([0.0, 1.0, -1.0, 3.0])
+    assert np.allclose(orc.act_fn(h, "silu"), [0.0, 1 / (1 + math.e ** -1), -1 / (1 + math.e), 3 / (1 + math.e ** -3)], atol=1e-15)
+    # GELU(x) = x * Phi(x); Phi(1) = 0.841344746068543 (standard normal cdf)
+    assert np.allclose(orc.act_fn(h, "gelu_erf"), [0.0, 0.841344746068543, -0.158655253931457, 3 * 0.998650101968370], atol=1e-14)
+    assert np.allclose(orc.act_fn(h, "gelu_tanh"), orc.act_fn(h, "gelu_erf"), atol=2e-3)
+    for act in ("silu", "gelu_erf", "gelu_tanh", "identity"):
+        hh = np.linspace(-4, 4, 41)
+        fd = (orc.act_fn(hh + 1e-6, act) - orc.act_fn(hh - 1e-6, act)) / 2e-6
+        assert np.allclose(orc.act_grad(hh, act), fd, atol=1e-8)
+
+
+# ----------------------------------------------------------------------------------------------
+# selection: exhaustive search, ties, bounds
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n,k,m,c", [(4, 2, 6, 3), (5, 1, 5, 5), (3, 3, 4, 1), (5, 4, 6, 2)])
+def test_selection_matches_exhaustive_search(n, k, m, c):
+    w = gen.tiny(n=n, k=k, m=m, c=c, L=m * 4, L_valid=m * 4, d=8, d_ff=n * 4, H=0, d_h=0, B=4)
+    x = gen.make_x(w).f64
+    Wr = _boost_router(gen.make_router(w).f64)
+    r = orc.route(x, Wr, k, m, c)
+    for b in range(w.B):
+        # the chosen set must maximise the score sum among all subsets of that size
+        import itertools
+        best = max(itertools.combinations(range(n), k), key=lambda s: sum(r.p_samp[b, i] for i in s))
+        assert sorted(best) == r.expert_idx[b].tolist()
+        for s, i in enumerate(r.expert_idx[b]):
+            bestp = max(itertools.combinations(range(m), c), key=lambda q: sum(r.p_patch[b, i, j] for j in q))
+            assert sorted(bestp) == r.patch_idx[b, s].tolist()
+
+
+def test_selection_tie_goes_to_lower_index():
+    p_samp = np.array([[0.2, 0.3, 0.3, 0.2]])
+    p_patch = np.zeros((1, 4, 5))
+    p_patch[0, 1] = [0.5, 0.1, 0.5, 0.5, 0.1]
+    p_patch[0, 0] = [0.1, 0.1, 0.1, 0.1, 0.1]
+    cnt = np.full(5, 4)
+    e, p, em, pm = orc.select(p_samp, p_patch, cnt, k=3, c=2)
+    assert e[0].tolist() == [0, 1, 2]           # 0.2 tie between experts 0 and 3 -> 0
+    assert p[0, 1].tolist() == [0, 2]           # three-way tie at 0.5 -> patches 0 and 2
+    assert p[0, 0].tolist() == [0, 1]
+    assert em[0] == 0.0 and pm[0, 1] == 0.0
+    # the exhaustive search in the scalar twin follows the same rule
+    assert loops.best_subset(p_samp[0].tolist(), range(4), 3) == [0, 1, 2]
+    assert loops.best_subset(p_patch[0, 1].tolist(), range(5), 2) == [0, 2]
+
+
+def test_margin_definition():
+    p = np.array([[0.4, 0.1, 0.3, 0.2]])
+    e, _, em, _ = orc.select(p, np.full((1, 4, 2), 0.25), np.full(2, 1), k=2, c=2)
+    assert e[0].tolist() == [0, 2]
+    assert em[0] == pytest.approx((0.3 - 0.2) / 0.3)
+
+
+@pytest.mark.parametrize("L_valid", [24, 21, 17])
+def test_routing_bounds(L_valid):
+    w = gen.tiny(B=7, L_valid=L_valid)
+    x = gen.make_x(w).f64
+    r = orc.route(x, _boost_router(gen.make_router(w).f64), w.k, w.m, w.c, L_valid=L_valid)
+    assert np.allclose(r.p_samp.sum(axis=1), 1.0) and np.allclose(r.p_patch.sum(axis=1), 1.0)
+    assert r.load.sum() == w.B * w.k and r.load.min() >= 0 and r.load.max() <= w.B
+    cnt = orc.patch_valid_counts(w.L, w.m, L_valid)
+    n_elig = int((cnt > 0).sum())
+    for b in range(w.B):
+        assert np.all(np.diff(r.expert_idx[b]) > 0)
+        use = np.zeros(w.m, dtype=int)
+        for s in range(w.k):
+            sel = r.patch_idx[b, s][r.patch_idx[b, s] >= 0]
+            assert len(sel) == min(w.c, n_elig)
+            assert np.all(np.diff(sel) > 0) and sel.min() >= 0 and sel.max() < w.m
+            assert np.all(cnt[sel] > 0)
+            use[sel] += 1
+        assert use.max() <= w.k
+    assert np.all(np.diff(r.offsets) >= 0) and np.all(r.offsets % 128 == 0)
+    r1 = orc.route(x, _boost_router(gen.make_router(w).f64), w.k, w.m, w.c, L_valid=L_valid, row_align=1)
+    assert r1.offsets[-1] == w.B * w.k * w.c * w.l_p
+    # buffer rows: every (sample, expert) pair gets its own disjoint run of c*l_p rows inside its expert
+    seen = set()
+    for b in range(w.B):
+        for s in range(w.k):
+            row = orc.buffer_row(r1, b, s)
+            i = r1.expert_idx[b, s]
+            assert r1.offsets[i] <= row and row + w.l_a <= r1.offsets[i + 1]
+            assert row not in seen
+            seen.add(row)
+
+
+def test_patch_softmax_is_over_experts_not_patches():
+    # Eq. 14 normalises each patch column over the n experts.
+    w = gen.tiny()
+    x = gen.make_x(w).f64
+    Wr = _boost_router(gen.make_router(w).f64)
+    p_samp, p_patch, pool, samp, cnt = orc.router_probs(x, Wr, w.m, w.L)
+    b, j = 1, 2
+    logits = x[b, j * w.l_p:(j + 1) * w.l_p].mean(0) @ Wr
+    ref = np.exp(logits) / np.exp(logits).sum()
+    assert np.allclose(p_patch[b, :, j], ref, atol=1e-14)
+    sl = x[b].mean(0) @ Wr
+    assert np.allclose(p_samp[b], np.exp(sl) / np.exp(sl).sum(), atol=1e-14)
+
+
+# ----------------------------------------------------------------------------------------------
+# lossless decomposition: k=n, c=m reproduces the dense layer (Eq. 1, 5; Eq. 8-11)
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("act", ["silu", "gelu_erf", "gelu_tanh", "identity"])
+def test_uome_full_selection_equals_dense_mlp(act):
+    w = gen.tiny(k=4, c=6, act=act)
+    t = _inputs(w, ("mlp",))
+    r = orc.route(t["x"], t["Wr"], w.k, w.m, w.c, use_gate=False)
+    y = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, act)
+    A_I = np.concatenate([t["W1"][i] for i in range(w.n)], axis=1)     # [d, d_ff]: column blocks
+    A_O = np.concatenate([t["W2"][i] for i in range(w.n)], axis=0)     # [d_ff, d]: row blocks
+    dense = orc.act_fn(t["x"].reshape(-1, w.d) @ A_I, act) @ A_O
+    assert np.allclose(y - t["x"], dense.reshape(t["x"].shape), rtol=1e-12, atol=1e-13)
+
+
+def test_uome_full_selection_with_gates_scales_hidden_blocks():
+    w = gen.tiny(k=4, c=6)
+    t = _inputs(w, ("mlp",))
+    Wr = _boost_router(t["Wr"])
+    r = orc.route(t["x"], Wr, w.k, w.m, w.c, use_gate=True)
+    y = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, "silu")
+    A_I = np.concatenate(list(t["W1"]), axis=1)
+    A_O = np.concatenate(list(t["W2"]), axis=0)
+    hidden = orc.act_fn(t["x"] @ A_I, "silu")                          # [B, L, d_ff]
+    for b in range(w.B):
+        for tkn in range(w.L):
+            j = tkn // w.l_p
+            for i in range(w.n):
+                hidden[b, tkn, i * w.d_e:(i + 1) * w.d_e] *= r.p_samp[b, i] * r.p_patch[b, i, j]
+    assert np.allclose(y - t["x"], hidden @ A_O, rtol=1e-12, atol=1e-13)
+
+
+def _textbook_mha(x, WI_q, WI_k, WI_v, WO, heads, d_h, causal, L_valid):
+    """Plain multi-head attention on one sample, written independently of the oracle."""
+    L = x.shape[0]
+    q, k, v = x @ WI_q, x @ WI_k, x @ WI_v
+    out = np.zeros_like(q)
+    for h in range(heads):
+        for a in range(L):
+            w = np.full(L, -np.inf)
+            for b in range(L):
+                if b < L_valid and (not causal or b <= a):
+                    w[b] = q[a, h * d_h:(h + 1) * d_h] @ k[b, h * d_h:(h + 1) * d_h] / math.sqrt(d_h)
+            w = np.exp(w - w.max())
+            w /= w.sum()
+            out[a, h * d_h:(h + 1) * d_h] = w @ v[:, h * d_h:(h + 1) * d_h]
+    return out @ WO
+
+
+@pytest.mark.parametrize("causal", [False, True])
+@pytest.mark.parametrize("H,L_valid", [(4, 24), (8, 24), (4, 22)])
+def test_smha_full_selection_equals_multihead_attention(causal, H, L_valid):
+    w = gen.tiny(k=4, c=6, H=H, L_valid=L_valid, causal=causal)
+    t = _inputs(w, ("att",))
+    r = orc.route(t["x"], t["Wra"], w.k, w.m, w.c, L_valid=L_valid, use_gate=False)
+    y = orc.smha_forward(t["x"], t["Wq"], t["Wk"], t["Wv"], t["Wo"], r, w.d_h, causal)
+    cat = lambda W: np.concatenate(list(W), axis=1)
+    WO = np.concatenate(list(t["Wo"]), axis=0)
+    for b in range(w.B):
+        ref = _textbook_mha(t["x"][b], cat(t["Wq"]), cat(t["Wk"]), cat(t["Wv"]), WO, H, w.d_h, causal, L_valid)
+        assert np.allclose((y - t["x"])[b, :L_valid], ref[:L_valid], rtol=1e-11, atol=1e-12)
+        assert np.array_equal(y[b, L_valid:], t["x"][b, L_valid:])
+
+
+def test_fig4_mask_identity_and_its_negative():
+    L, l_p = 24, 4
+    full = np.tril(np.ones((L, L), dtype=bool))
+    tok = np.concatenate([np.arange(j * l_p, (j + 1) * l_p) for j in (1, 3, 4)])
+    assert np.array_equal(full[np.ix_(tok, tok)], np.tril(np.ones((len(tok),) * 2, dtype=bool)))
+    bad = np.concatenate([np.arange(j * l_p, (j + 1) * l_p) for j in (3, 1, 4)])      # unsorted
+    assert not np.array_equal(full[np.ix_(bad, bad)], np.tril(np.ones((len(bad),) * 2, dtype=bool)))
+
+
+def test_smha_causal_partial_selection_uses_leading_triangle():
+    # the oracle double-indexes the L x L mask; an attention over the gathered tokens with a plain
+    # l_a x l_a lower triangle (Fig. 4) must give the same result
+    w = gen.tiny(causal=True, B=2)
+    t = _inputs(w, ("att",))
+    r = orc.route(t["x"], _boost_router(t["Wra"]), w.k, w.m, w.c)
+    y = orc.smha_forward(t["x"], t["Wq"], t["Wk"], t["Wv"], t["Wo"], r, w.d_h, True)
+    for b in range(w.B):
+        acc = t["x"][b].copy()
+        for s, i in enumerate(r.expert_idx[b]):
+            tok = orc.gathered_tokens(r, b, s)
+            ref = _textbook_mha(t["x"][b, tok], t["Wq"][i], t["Wk"][i], t["Wv"][i], t["Wo"][i],
+                                w.d_g // w.d_h, w.d_h, True, len(tok))
+            g = np.repeat(r.gate[b, s], w.l_p)
+            acc[tok] += g[:, None] * ref
+        assert np.allclose(y[b], acc, rtol=1e-11, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------------------------
+# special cases and symmetries
+# ----------------------------------------------------------------------------------------------
+
+def test_c_equals_m_is_pure_expert_selection():
+    # Eq. 21-26: whole samples go to their top-k experts
+    w = gen.tiny(c=6)
+    t = _inputs(w, ("mlp",))
+    Wr = _boost_router(t["Wr"])
+    r = orc.route(t["x"], Wr, w.k, w.m, w.c, use_gate=False)
+    y = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, "silu")
+    for b in range(w.B):
+        sl = t["x"][b].mean(0) @ Wr
+        top = np.sort(np.argsort(-sl, kind="stable")[:w.k])
+        assert top.tolist() == r.expert_idx[b].tolist()
+        ref = t["x"][b].copy()
+        for i in top:
+            ref += orc.act_fn(t["x"][b] @ t["W1"][i], "silu") @ t["W2"][i]      # Eq. 25-26
+        assert np.allclose(y[b], ref, rtol=1e-12, atol=1e-13)
+
+
+def test_k_equals_n_is_pure_data_selection():
+    # Eq. 12-20: every expert takes its own top-c patches
+    w = gen.tiny(k=4)
+    t = _inputs(w, ("mlp",))
+    Wr = _boost_router(t["Wr"])
+    r = orc.route(t["x"], Wr, w.k, w.m, w.c, use_gate=False)
+    y = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, "silu")
+    for b in range(w.B):
+        ref = t["x"][b].copy()
+        xp = t["x"][b].reshape(w.m, w.l_p, w.d)
+        g = np.stack([orc.softmax(xp[j].mean(0) @ Wr, 0) for j in range(w.m)], axis=1)     # [n, m]
+        for i in range(w.n):
+            ids = np.sort(np.argsort(-g[i], kind="stable")[:w.c])                           # Eq. 17 + sort
+            assert ids.tolist() == r.patch_idx[b, i].tolist()
+            for j in ids:
+                ref[j * w.l_p:(j + 1) * w.l_p] += orc.act_fn(xp[j] @ t["W1"][i], "silu") @ t["W2"][i]
+        assert np.allclose(y[b], ref, rtol=1e-12, atol=1e-13)
+
+
+def test_unselected_patches_and_pad_rows_pass_through():
+    w = gen.tiny(L_valid=21)
+    t = _inputs(w)
+    r = orc.route(t["x"], _boost_router(t["Wr"]), w.k, w.m, w.c, L_valid=21)
+    y = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, "silu")
+    y2 = orc.smha_forward(t["x"], t["Wq"], t["Wk"], t["Wv"], t["Wo"], r, w.d_h, False)
+    for b in range(w.B):
+        used = set(int(j) for j in r.patch_idx[b].ravel() if j >= 0)
+        for j in range(w.m):
+            sl = slice(j * w.l_p, (j + 1) * w.l_p)
+            if j not in used:
+                assert np.array_equal(y[b, sl], t["x"][b, sl]) and np.array_equal(y2[b, sl], t["x"][b, sl])
+        assert np.array_equal(y[b, 21:], t["x"][b, 21:]) and np.array_equal(y2[b, 21:], t["x"][b, 21:])
+
+
+def test_batch_permutation_and_expert_permutation():
+    w = gen.tiny(B=5)
+    t = _inputs(w)
+    Wr = _boost_router(t["Wr"])
+    r = orc.route(t["x"], Wr, w.k, w.m, w.c)
+    y = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, "silu")
+    ya = orc.smha_forward(t["x"], t["Wq"], t["Wk"], t["Wv"], t["Wo"], r, w.d_h, True)
+    perm = np.array([3, 0, 4, 2, 1])
+    rp = orc.route(t["x"][perm], Wr, w.k, w.m, w.c)
+    assert np.allclose(orc.mlp_forward(t["x"][perm], t["W1"], t["W2"], rp, "silu"), y[perm], atol=1e-14)
+    ep = np.array([2, 0, 3, 1])
+    re = orc.route(t["x"], Wr[:, ep], w.k, w.m, w.c)
+    assert np.allclose(orc.mlp_forward(t["x"], t["W1"][ep], t["W2"][ep], re, "silu"), y, atol=1e-13)
+    assert np.allclose(orc.smha_forward(t["x"], t["Wq"][ep], t["Wk"][ep], t["Wv"][ep], t["Wo"][ep], re, w.d_h, True),
+                       ya, atol=1e-13)
+
+
+def test_identity_activation_is_linear_for_fixed_routing():
+    w = gen.tiny()
+    t = _inputs(w, ("mlp",))
+    r = orc.route(t["x"], _boost_router(t["Wr"]), w.k, w.m, w.c)
+    f = lambda xx: orc.mlp_forward(xx, t["W1"], t["W2"], r, "identity", residual=False)
+    x2 = gen.normal(99, 0, t["x"].shape)
+    assert np.allclose(f(2.0 * t["x"] - 3.0 * x2), 2.0 * f(t["x"]) - 3.0 * f(x2), atol=1e-12)
+
+
+def test_activation_sits_between_the_two_layers_only():
+    # phi(Y1 + Y2) != phi(Y1) + phi(Y2): an oracle that applied phi after the second layer per expert
+    # would break the dense equivalence; check the inequality the paper warns about on real numbers
+    w = gen.tiny(k=4, c=6)
+    t = _inputs(w, ("mlp",))
+    Y = [t["x"][0] @ t["W1"][i] @ t["W2"][i] for i in range(w.n)]
+    assert not np.allclose(orc.act_fn(sum(Y), "silu"), sum(orc.act_fn(v, "silu") for v in Y), atol=1e-6)
+
+
+def test_theoretical_cost_ratio():
+    # k/n = 1/2 in expert-selection mode, or c/m = 1/2 in data-selection mode, is half the dense rows
+    B, L = 8, 64
+    dense_rows = B * 4 * L                       # n experts x all tokens
+    assert orc.routed_rows(B, k=2, c=8, l_p=8) * 2 == dense_rows
+    assert orc.routed_rows(B, k=4, c=4, l_p=8) * 2 == dense_rows
+
+
+# ----------------------------------------------------------------------------------------------
+# scalar-loop twin
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("L_valid,causal,act", [(24, False, "silu"), (22, True, "gelu_erf"), (17, False, "gelu_tanh")])
+def test_array_oracle_equals_scalar_loops(L_valid, causal, act):
+    w = gen.tiny(B=2, L_valid=L_valid, causal=causal, act=act)
+    t = _inputs(w)
+    Wr = _boost_router(t["Wr"])
+    r = orc.route(t["x"], Wr, w.k, w.m, w.c, L_valid=L_valid)
+    lr = loops.route(t["x"].tolist(), Wr.tolist(), w.B, w.L, w.d, w.n, w.k, w.m, w.c, L_valid)
+    for b in range(w.B):
+        assert np.allclose(lr[b]["p_samp"], r.p_samp[b], atol=1e-13)
+        assert np.allclose(np.array(lr[b]["p_patch"]), r.p_patch[b], atol=1e-13)
+        assert [i for i, _, _ in lr[b]["sel"]] == r.expert_idx[b].tolist()
+        for s, (i, patches, g) in enumerate(lr[b]["sel"]):
+            got = [int(j) for j in r.patch_idx[b, s] if j >= 0]
+            assert patches == got
+            assert np.allclose(g, r.gate[b, s][:len(g)], atol=1e-14)
+    y = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, act)
+    yl = loops.mlp_forward(t["x"].tolist(), t["W1"].tolist(), t["W2"].tolist(), lr, w.B, w.L, w.d, w.d_e, w.m,
+                           L_valid, act)
+    assert np.allclose(np.array(yl), y, rtol=1e-12, atol=1e-12)
+    ya = orc.smha_forward(t["x"], t["Wq"], t["Wk"], t["Wv"], t["Wo"], r, w.d_h, causal)
+    yal = loops.smha_forward(t["x"].tolist(), t["Wq"].tolist(), t["Wk"].tolist(), t["Wv"].tolist(), t["Wo"].tolist(),
+                             lr, w.B, w.L, w.d, w.d_g, w.d_h, w.m, L_valid, causal)
+    assert np.allclose(np.array(yal), ya, rtol=1e-12, atol=1e-12)
+
+
+# ----------------------------------------------------------------------------------------------
+# backward: central finite differences with the selection frozen
+# ----------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("act,L_valid,use_gate", [("silu", 24, True), ("gelu_erf", 21, True), ("gelu_tanh", 24, False)])
+def test_backward_matches_finite_differences(act, L_valid, use_gate):
+    w = gen.tiny(B=2, L_valid=L_valid, act=act, d=8, d_ff=16)
+    t = _inputs(w, ("mlp",))
+    x, W1, W2 = t["x"], t["W1"], t["W2"]
+    Wr = _boost_router(t["Wr"], 10.0)
+    r = orc.route(x, Wr, w.k, w.m, w.c, L_valid=L_valid, use_gate=use_gate)
+    dy = gen.normal(7, 1, x.shape)
+    dy[:, L_valid:] = 0.0
+    dx, dW1, dW2, dWr, _ = orc.mlp_backward(x, W1, W2, Wr, r, dy, act, True, use_gate)
+
+    def loss(x_, W1_, W2_, Wr_):
+        rr = orc.with_selection(x_, Wr_, r.expert_idx, r.patch_idx, w.m, L_valid, use_gate)
+        return float(np.sum(orc.mlp_forward(x_, W1_, W2_, rr, act) * dy))
+
+    eps = 1e-5
+    for which, grad, arr in (("x", dx, x), ("W1", dW1, W1), ("W2", dW2, W2), ("Wr", dWr, Wr)):
+        for trial in range(3):
+            v = gen.normal(100 + trial, {"x": 0, "W1": 1, "W2": 2, "Wr": 3}[which], arr.shape)
+            if which == "x":
+                v[:, L_valid:] = 0.0
+            args_p = dict(x_=x, W1_=W1, W2_=W2, Wr_=Wr)
+            args_m = dict(args_p)
+            key = {"x": "x_", "W1": "W1_", "W2": "W2_", "Wr": "Wr_"}[which]
+            args_p[key] = arr + eps * v
+            args_m[key] = arr - eps * v
+            fd = (loss(**args_p) - loss(**args_m)) / (2 * eps)
+            an = float(np.sum(grad * v))
+            assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (which, fd, an)
+    if not use_gate:
+        assert np.all(dWr == 0.0)
+
+
+# ----------------------------------------------------------------------------------------------
+# planted mistakes: the pins above must notice a wrong oracle
+# ----------------------------------------------------------------------------------------------
+
+def test_planted_mistakes_are_caught(monkeypatch):
+    w = gen.tiny(k=4, c=6)
+    t = _inputs(w)
+    A_I = np.concatenate(list(t["W1"]), axis=1)
+    A_O = np.concatenate(list(t["W2"]), axis=0)
+    dense = (orc.act_fn(t["x"] @ A_I, "silu") @ A_O)
+    r = orc.route(t["x"], t["Wr"], w.k, w.m, w.c, use_gate=False)
+
+    def dense_ok():
+        y = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, "silu")
+        return np.allclose(y - t["x"], dense, rtol=1e-12, atol=1e-13)
+
+    assert dense_ok()
+    # (1) activation also after the second layer (the misprint in Eq. 39)
+    real_act = orc.act_fn
+    monkeypatch.setattr(orc, "act_fn", lambda h, a: real_act(real_act(h, a), a))
+    assert not dense_ok()
+    monkeypatch.setattr(orc, "act_fn", real_act)
+    # (2) experts' weight slices swapped between layers
+    y = orc.mlp_forward(t["x"], t["W1"], t["W2"][::-1], r, "silu")
+    assert not np.allclose(y - t["x"], dense, rtol=1e-9, atol=1e-10)
+    # (3) softmax over patches instead of experts changes the selection of some sample
+    w2 = gen.tiny(B=6)
+    x2 = gen.make_x(w2).f64
+    Wr2 = _boost_router(gen.make_router(w2).f64)
+    good = orc.route(x2, Wr2, w2.k, w2.m, w2.c)
+    real_sm = orc.softmax
+    p_samp, p_patch, pool, samp, cnt = orc.router_probs(x2, Wr2, w2.m, w2.L)
+    logits = np.einsum("bjd,dn->bnj", pool, Wr2)
+    wrong = real_sm(logits, axis=2)              # normalised over patches: not Eq. 14
+    _, pidx, _, _ = orc.select(p_samp, wrong, cnt, w2.k, w2.c)
+    assert not np.array_equal(pidx, good.patch_idx)
