@@ -1,0 +1,177 @@
+/*
+ * uoe.h -- C ABI of the Union-of-Experts routed hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library evaluates one Union-of-Experts block the way the paper states the problem
+ * (Section III): a transformer MLP (or the attention projections) is split column-wise /
+ * row-wise into n equivalent experts (Eq. 1-7, Eq. 8-11); every sample goes to its top-k of n
+ * experts (Eq. 21-23), every chosen expert takes at most c of the sample's m patches (Eq. 12-17),
+ * and the expert outputs are added back at the selected positions (Eq. 20, 26, 36, 40).
+ *
+ * Conventions for every entry point
+ *   - Pointers marked "device" are CUDA device pointers on the current device; `prob` is a host
+ *     pointer.  All arrays are dense, row-major, and 16-byte aligned.
+ *   - The caller owns every buffer, including the workspace `ws` (size from
+ *     uoe_workspace_bytes).  The library never allocates or frees device memory and never
+ *     synchronises, except uoe_read_device_status.  All work is enqueued on `cuda_stream`
+ *     (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - Outputs are overwritten, not accumulated into.
+ *   - Errors are return codes.  Arguments are validated on the host before anything is launched.
+ *     A device-side anomaly (a bounded wait that ran out, an index out of range) is recorded in
+ *     the first word of the workspace and reported by uoe_read_device_status; kernels never trap.
+ *   - Element type: `dtype` selects float32 or bfloat16 storage for x, weights and y.  Products are
+ *     accumulated in float32.  Routing probabilities and gates are always float32.
+ *
+ * Routed buffers.  Rows routed to expert i form one contiguous region that starts at row
+ * expert_offsets[i]; inside it the samples that chose i appear in ascending order, each with
+ * exactly l_a = c*l_p rows (its selected patches in ascending order; an unused slot, patch index
+ * -1, is l_p zero rows).  Every region is padded to a multiple of UOE_ROW_ALIGN rows, so
+ * expert_offsets[n] <= uoe_max_routed_rows(prob).
+ */
+#ifndef UOE_H_
+#define UOE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define UOE_ROW_ALIGN 128
+
+typedef enum {
+    UOE_OK = 0,
+    UOE_ERR_INVALID_ARG = 1,   /* null pointer, bad shape, misaligned buffer */
+    UOE_ERR_UNSUPPORTED = 2,   /* valid problem outside what the kernels cover */
+    UOE_ERR_WORKSPACE = 3,     /* ws_bytes smaller than uoe_workspace_bytes */
+    UOE_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed */
+    UOE_ERR_TIMEOUT = 5,       /* device status: a bounded wait inside a kernel ran out */
+    UOE_ERR_DEVICE_INDEX = 6   /* device status: a routing index was out of range */
+} uoe_status;
+
+typedef enum { UOE_F32 = 0, UOE_BF16 = 1 } uoe_dtype;
+
+typedef enum {
+    UOE_ACT_GELU_ERF = 0,
+    UOE_ACT_GELU_TANH = 1,
+    UOE_ACT_SILU = 2,          /* the paper's choice for UoME (below Eq. 39) */
+    UOE_ACT_IDENTITY = 3
+} uoe_act;
+
+enum {
+    UOE_FLAG_RESIDUAL = 1,     /* y = x + sum(...) (the selective residual of Eq. 20); else y = sum(...) */
+    UOE_FLAG_GATE = 2,         /* combine weight = P_samp[b,i] * P_patch[b,i,j]; else 1 (Eq. 20 literal) */
+    UOE_FLAG_CAUSAL = 4        /* SMHA: shared lower-triangular mask over the gathered tokens (Fig. 4) */
+};
+
+typedef enum { UOE_OP_ROUTE = 0, UOE_OP_MLP_FWD = 1, UOE_OP_MLP_BWD = 2, UOE_OP_SMHA_FWD = 3 } uoe_op;
+
+/* One Union-of-Experts block.  L must equal m * l_p; rows t >= L_valid of every sample are padding
+ * (they take no part in routing means, are masked as attention keys (Eq. 41), and y = x there). */
+typedef struct {
+    int32_t B;        /* samples */
+    int32_t L;        /* tokens per sample, padded: L = m * l_p */
+    int32_t L_valid;  /* real tokens per sample, 1 <= L_valid <= L */
+    int32_t d;        /* model width */
+    int32_t n;        /* experts */
+    int32_t k;        /* experts per sample, 1 <= k <= n */
+    int32_t m;        /* patches per sample */
+    int32_t c;        /* patches per expert, 1 <= c <= m */
+    int32_t d_e;      /* UoME: hidden width of one expert (d_ff / n); 0 if unused */
+    int32_t H;        /* SMHA: attention heads, H % n == 0; 0 if unused */
+    int32_t d_h;      /* SMHA: width of one head */
+    int32_t dtype;    /* uoe_dtype */
+    int32_t act;      /* uoe_act */
+    uint32_t flags;   /* UOE_FLAG_* */
+} uoe_problem;
+
+/* Upper bound on expert_offsets[n]: B*k*c*l_p rows plus per-expert padding.  Buffers indexed by routed
+ * row (saved_h, lse) must hold this many rows.  Returns 0 on an invalid problem. */
+int64_t uoe_max_routed_rows(const uoe_problem* prob);
+
+/* Bytes of device workspace that `op` (a uoe_op) needs for this problem (0 on an invalid problem). */
+size_t uoe_workspace_bytes(const uoe_problem* prob, int op);
+
+/*
+ * Router scoring and fused selection (Eq. 12-17 and 21-23, combined as in Fig. 3).
+ *   patch score   g'[b,i,j] = mean over the real tokens t of patch j of  x[b,t,:] . W_r[:,i]   (Eq. 13)
+ *   p_patch[b,:,j] = softmax over the n experts of g'[b,:,j]                                     (Eq. 14)
+ *   p_samp[b,:]    = softmax over experts of (mean over real tokens of x[b]) . W_r               (Eq. 21)
+ *   expert_idx[b,:] = the k experts with the largest p_samp, ascending (ties: lower index)       (Eq. 22)
+ *   patch_idx[b,s,:] = for the s-th chosen expert i, the min(c, #patches with a real token) patches
+ *                      with the largest p_patch[b,i,:], ascending; unused slots are -1            (Eq. 17)
+ *   gate[b,s,u]     = p_samp[b,i] * p_patch[b,i,patch] with UOE_FLAG_GATE, else 1; 0 in unused slots
+ *   expert_offsets  = row offsets of the per-expert regions (see "Routed buffers")               (Eq. 23)
+ * All arguments except prob are device pointers.  x [B,L,d] and W_r [d,n] have prob->dtype;
+ * the outputs are int32 / float32 with the shapes given.  Scores accumulate in float32.
+ */
+uoe_status uoe_route(const uoe_problem* prob, const void* x, const void* W_r,
+                     int32_t* expert_idx /* [B,k] */, int32_t* patch_idx /* [B,k,c] */,
+                     float* gate /* [B,k,c] */, float* p_samp /* [B,n] */, float* p_patch /* [B,n,m] */,
+                     int32_t* expert_offsets /* [n+1] */, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * UoME forward (Eq. 37-40 with the index-select of Eq. 18 and the index-add of Eq. 20):
+ *   y[b,t,:] = x[b,t,:] + sum over (expert i, patch j) that selected token t of
+ *              gate[b,i,j] * ( phi( x[b,t,:] W1[i] + b1[i] ) W2[i] + b2[i] )
+ * W1 [n,d,d_e] holds the column slices of the first layer, W2 [n,d_e,d] the row slices of the
+ * second (Eq. 1-7); no activation follows the second layer.  b1 [n,d_e], b2 [n,d] may be NULL
+ * (biases are supported for float32 only).  The routing arrays are the outputs of uoe_route or any
+ * arrays of the same form supplied by the caller (sorted, in range, offsets consistent with
+ * expert_idx).  With UOE_FLAG_GATE the combine weight is gate[b,s,u], otherwise 1.  saved_h, if
+ * not NULL, receives the pre-activation x W1[i] of every routed row,
+ * [uoe_max_routed_rows, d_e] in prob->dtype, for uoe_mlp_backward.  All pointers except prob are
+ * device pointers.
+ */
+uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, const void* W1, const void* W2,
+                           const void* b1, const void* b2,
+                           const int32_t* expert_idx, const int32_t* patch_idx, const float* gate,
+                           const int32_t* expert_offsets, void* y /* [B,L,d] */, void* saved_h,
+                           void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * UoME backward: gradients of sum(y * dy) with the selection (expert_idx, patch_idx) held constant.
+ * The paper gives no backward text; this is the derivative of Eq. 38-40 and, with UOE_FLAG_GATE, of
+ * the gate through both softmaxes (Eq. 14, 21) into W_r and x.
+ *   dx [B,L,d] in prob->dtype; dW1 [n,d,d_e], dW2 [n,d_e,d], dW_r [d,n] in float32, overwritten.
+ * saved_h is the array written by uoe_mlp_forward for the same inputs.  Biases are not supported
+ * here.  All pointers except prob are device pointers.
+ */
+uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, const void* W1, const void* W2,
+                            const void* W_r, const int32_t* expert_idx, const int32_t* patch_idx,
+                            const float* gate, const int32_t* expert_offsets,
+                            const float* p_samp, const float* p_patch, const void* saved_h,
+                            const void* dy /* [B,L,d] */, void* dx /* [B,L,d] */,
+                            float* dW1, float* dW2, float* dW_r,
+                            void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * SMHA forward (Eq. 27-30, 33-36; masks Eq. 41 and Fig. 4; RoPE of Eq. 32 not applied).
+ * Attention expert i owns the column slices Wq/Wk/Wv[i] [d, d_g] and the row slice Wo[i] [d_g, d]
+ * with d_g = (H/n)*d_h (Eq. 8-11).  For each sample b and chosen expert i the l_a gathered tokens
+ * attend to each other per head: softmax(q k^T / sqrt(d_h) + mask) v, where pad tokens are masked as
+ * keys and, with UOE_FLAG_CAUSAL, key position > query position in gathered order is masked.  The
+ * projected result is added back as in uoe_mlp_forward:  y = x + sum gate * (o Wo[i]).
+ * lse, if not NULL, receives the log-sum-exp of every (routed row, head of the expert):
+ * [uoe_max_routed_rows, H/n] float32.  All pointers except prob are device pointers.
+ */
+uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, const void* Wq, const void* Wk,
+                            const void* Wv, const void* Wo,
+                            const int32_t* expert_idx, const int32_t* patch_idx, const float* gate,
+                            const int32_t* expert_offsets, void* y /* [B,L,d] */, float* lse,
+                            void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Text for a status code (static storage). */
+const char* uoe_status_string(int status);
+
+/* Synchronises `cuda_stream`, reads the status word that the kernels of the last call on `ws` left
+ * in the workspace, and returns it (UOE_OK if nothing was recorded). */
+uoe_status uoe_read_device_status(void* ws, void* cuda_stream);
+
+/* Number of this library's kernel launches enqueued by this process so far (for benchmarks). */
+int64_t uoe_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* UOE_H_ */

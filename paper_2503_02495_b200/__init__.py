@@ -1,0 +1,11 @@
+"""Union-of-Experts routed hot path for B200: Python binding of the C-ABI library libuoe.so.
+
+Importing the package loads the shared library and fails if it has not been built
+(`python -m paper_2503_02495_b200.build`).  There is no CPU or PyTorch fallback.
+"""
+from .binding import (  # noqa: F401
+    LIB_PATH, Problem, Routing, UoeError, alloc_routing, alloc_saved_h, alloc_workspace, status_string,
+    uoe_launch_count, uoe_max_routed_rows, uoe_mlp_backward, uoe_mlp_forward, uoe_read_device_status, uoe_route,
+    uoe_smha_forward, uoe_workspace_bytes, UOE_OP_ROUTE, UOE_OP_MLP_FWD, UOE_OP_MLP_BWD, UOE_OP_SMHA_FWD,
+    UOE_ROW_ALIGN,
+)

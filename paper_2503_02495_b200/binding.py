@@ -1,0 +1,242 @@
+"""ctypes binding of libuoe.so: argument marshalling only.
+
+Every function here has the name and argument order of its C entry point (include/uoe.h), takes
+torch CUDA tensors, allocates the outputs and the workspace with torch, passes raw pointers and the
+current CUDA stream, and raises UoeError on a non-zero status.  No arithmetic of the method lives
+in Python.  If the shared library is missing, importing this module fails: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libuoe.so")
+
+UOE_ROW_ALIGN = 128
+UOE_F32, UOE_BF16 = 0, 1
+ACTS = {"gelu_erf": 0, "gelu_tanh": 1, "silu": 2, "identity": 3}
+UOE_FLAG_RESIDUAL, UOE_FLAG_GATE, UOE_FLAG_CAUSAL = 1, 2, 4
+UOE_OP_ROUTE, UOE_OP_MLP_FWD, UOE_OP_MLP_BWD, UOE_OP_SMHA_FWD = 0, 1, 2, 3
+
+
+class UoeError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class _Problem(ctypes.Structure):
+    _fields_ = [(f, ctypes.c_int32) for f in
+                ("B", "L", "L_valid", "d", "n", "k", "m", "c", "d_e", "H", "d_h", "dtype", "act")] + \
+               [("flags", ctypes.c_uint32)]
+
+
+@dataclass
+class Problem:
+    """Mirror of the C struct uoe_problem."""
+    B: int
+    L: int
+    L_valid: int
+    d: int
+    n: int
+    k: int
+    m: int
+    c: int
+    d_e: int = 0
+    H: int = 0
+    d_h: int = 0
+    dtype: str = "bf16"
+    act: str = "silu"
+    residual: bool = True
+    gate: bool = True
+    causal: bool = False
+
+    def c_struct(self) -> _Problem:
+        flags = (UOE_FLAG_RESIDUAL if self.residual else 0) | (UOE_FLAG_GATE if self.gate else 0) | \
+                (UOE_FLAG_CAUSAL if self.causal else 0)
+        return _Problem(self.B, self.L, self.L_valid, self.d, self.n, self.k, self.m, self.c, self.d_e, self.H,
+                        self.d_h, UOE_BF16 if self.dtype == "bf16" else UOE_F32, ACTS[self.act], flags)
+
+    @property
+    def torch_dtype(self):
+        return torch.bfloat16 if self.dtype == "bf16" else torch.float32
+
+    @property
+    def l_p(self) -> int:
+        return self.L // self.m
+
+    @property
+    def l_a(self) -> int:
+        return self.c * self.l_p
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2503_02495_b200.build` "
+                          "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, sz, i32p, f32p = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p
+    pp = ctypes.POINTER(_Problem)
+    lib.uoe_max_routed_rows.restype = ctypes.c_int64
+    lib.uoe_max_routed_rows.argtypes = [pp]
+    lib.uoe_workspace_bytes.restype = sz
+    lib.uoe_workspace_bytes.argtypes = [pp, ctypes.c_int]
+    lib.uoe_route.restype = ctypes.c_int
+    lib.uoe_route.argtypes = [pp, vp, vp, i32p, i32p, f32p, f32p, f32p, i32p, vp, sz, vp]
+    lib.uoe_mlp_forward.restype = ctypes.c_int
+    lib.uoe_mlp_forward.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, f32p, i32p, vp, vp, vp, sz, vp]
+    lib.uoe_mlp_backward.restype = ctypes.c_int
+    lib.uoe_mlp_backward.argtypes = [pp, vp, vp, vp, vp, i32p, i32p, f32p, i32p, f32p, f32p, vp, vp, vp, f32p, f32p,
+                                     f32p, vp, sz, vp]
+    lib.uoe_smha_forward.restype = ctypes.c_int
+    lib.uoe_smha_forward.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, f32p, i32p, vp, f32p, vp, sz, vp]
+    lib.uoe_status_string.restype = ctypes.c_char_p
+    lib.uoe_status_string.argtypes = [ctypes.c_int]
+    lib.uoe_read_device_status.restype = ctypes.c_int
+    lib.uoe_read_device_status.argtypes = [vp, vp]
+    lib.uoe_launch_count.restype = ctypes.c_int64
+    lib.uoe_launch_count.argtypes = []
+    return lib
+
+
+_lib = _load()
+
+
+def status_string(status: int) -> str:
+    return _lib.uoe_status_string(int(status)).decode()
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(st: int, where: str):
+    if st != 0:
+        raise UoeError(st, where)
+
+
+def _contig(t, dtype=None):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "tensors must be contiguous CUDA tensors"
+    if dtype is not None:
+        assert t.dtype == dtype, f"expected {dtype}, got {t.dtype}"
+    return t
+
+
+def uoe_max_routed_rows(prob: Problem) -> int:
+    return int(_lib.uoe_max_routed_rows(ctypes.byref(prob.c_struct())))
+
+
+def uoe_workspace_bytes(prob: Problem, op: int) -> int:
+    return int(_lib.uoe_workspace_bytes(ctypes.byref(prob.c_struct()), op))
+
+
+def uoe_launch_count() -> int:
+    return int(_lib.uoe_launch_count())
+
+
+def alloc_workspace(prob: Problem, op: int, device="cuda") -> torch.Tensor:
+    nbytes = uoe_workspace_bytes(prob, op)
+    if nbytes == 0:
+        raise UoeError(1, "uoe_workspace_bytes")
+    return torch.empty(nbytes, dtype=torch.uint8, device=device)
+
+
+def uoe_read_device_status(ws: torch.Tensor) -> int:
+    return int(_lib.uoe_read_device_status(_ptr(ws), _stream()))
+
+
+@dataclass
+class Routing:
+    expert_idx: torch.Tensor      # [B,k] int32
+    patch_idx: torch.Tensor       # [B,k,c] int32
+    gate: torch.Tensor            # [B,k,c] float32
+    p_samp: torch.Tensor          # [B,n] float32
+    p_patch: torch.Tensor         # [B,n,m] float32
+    expert_offsets: torch.Tensor  # [n+1] int32
+
+
+def alloc_routing(prob: Problem, device="cuda") -> Routing:
+    i32, f32 = torch.int32, torch.float32
+    return Routing(torch.empty(prob.B, prob.k, dtype=i32, device=device),
+                   torch.empty(prob.B, prob.k, prob.c, dtype=i32, device=device),
+                   torch.empty(prob.B, prob.k, prob.c, dtype=f32, device=device),
+                   torch.empty(prob.B, prob.n, dtype=f32, device=device),
+                   torch.empty(prob.B, prob.n, prob.m, dtype=f32, device=device),
+                   torch.empty(prob.n + 1, dtype=i32, device=device))
+
+
+def uoe_route(prob: Problem, x, W_r, out: Routing | None = None, ws=None, check: bool = True) -> Routing:
+    _contig(x, prob.torch_dtype)
+    _contig(W_r, prob.torch_dtype)
+    r = out if out is not None else alloc_routing(prob, x.device)
+    ws = ws if ws is not None else alloc_workspace(prob, UOE_OP_ROUTE, x.device)
+    st = _lib.uoe_route(ctypes.byref(prob.c_struct()), _ptr(x), _ptr(W_r), _ptr(r.expert_idx), _ptr(r.patch_idx),
+                        _ptr(r.gate), _ptr(r.p_samp), _ptr(r.p_patch), _ptr(r.expert_offsets), _ptr(ws), ws.numel(),
+                        _stream())
+    _check(st, "uoe_route")
+    if check:
+        _check(uoe_read_device_status(ws), "uoe_route (device)")
+    return r
+
+
+def uoe_mlp_forward(prob: Problem, x, W1, W2, r: Routing, b1=None, b2=None, y=None, saved_h=None, ws=None,
+                    check: bool = True):
+    for t in (x, W1, W2, b1, b2):
+        _contig(t, prob.torch_dtype)
+    y = y if y is not None else torch.empty_like(x)
+    ws = ws if ws is not None else alloc_workspace(prob, UOE_OP_MLP_FWD, x.device)
+    st = _lib.uoe_mlp_forward(ctypes.byref(prob.c_struct()), _ptr(x), _ptr(W1), _ptr(W2), _ptr(b1), _ptr(b2),
+                              _ptr(r.expert_idx), _ptr(r.patch_idx), _ptr(r.gate), _ptr(r.expert_offsets),
+                              _ptr(y), _ptr(saved_h), _ptr(ws), ws.numel(), _stream())
+    _check(st, "uoe_mlp_forward")
+    if check:
+        _check(uoe_read_device_status(ws), "uoe_mlp_forward (device)")
+    return y
+
+
+def alloc_saved_h(prob: Problem, device="cuda") -> torch.Tensor:
+    return torch.empty(uoe_max_routed_rows(prob), prob.d_e, dtype=prob.torch_dtype, device=device)
+
+
+def uoe_mlp_backward(prob: Problem, x, W1, W2, W_r, r: Routing, saved_h, dy, dx=None, dW1=None, dW2=None,
+                     dW_r=None, ws=None, check: bool = True):
+    for t in (x, W1, W2, W_r, saved_h, dy):
+        _contig(t, prob.torch_dtype)
+    f32 = torch.float32
+    dx = dx if dx is not None else torch.empty_like(x)
+    dW1 = dW1 if dW1 is not None else torch.empty(W1.shape, dtype=f32, device=x.device)
+    dW2 = dW2 if dW2 is not None else torch.empty(W2.shape, dtype=f32, device=x.device)
+    dW_r = dW_r if dW_r is not None else torch.empty(W_r.shape, dtype=f32, device=x.device)
+    ws = ws if ws is not None else alloc_workspace(prob, UOE_OP_MLP_BWD, x.device)
+    st = _lib.uoe_mlp_backward(ctypes.byref(prob.c_struct()), _ptr(x), _ptr(W1), _ptr(W2), _ptr(W_r),
+                               _ptr(r.expert_idx), _ptr(r.patch_idx), _ptr(r.gate), _ptr(r.expert_offsets),
+                               _ptr(r.p_samp), _ptr(r.p_patch), _ptr(saved_h), _ptr(dy), _ptr(dx), _ptr(dW1),
+                               _ptr(dW2), _ptr(dW_r), _ptr(ws), ws.numel(), _stream())
+    _check(st, "uoe_mlp_backward")
+    if check:
+        _check(uoe_read_device_status(ws), "uoe_mlp_backward (device)")
+    return dx, dW1, dW2, dW_r
+
+
+def uoe_smha_forward(prob: Problem, x, Wq, Wk, Wv, Wo, r: Routing, y=None, lse=None, ws=None, check: bool = True):
+    for t in (x, Wq, Wk, Wv, Wo):
+        _contig(t, prob.torch_dtype)
+    y = y if y is not None else torch.empty_like(x)
+    ws = ws if ws is not None else alloc_workspace(prob, UOE_OP_SMHA_FWD, x.device)
+    st = _lib.uoe_smha_forward(ctypes.byref(prob.c_struct()), _ptr(x), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(Wo),
+                               _ptr(r.expert_idx), _ptr(r.patch_idx), _ptr(r.gate), _ptr(r.expert_offsets),
+                               _ptr(y), _ptr(lse), _ptr(ws), ws.numel(), _stream())
+    _check(st, "uoe_smha_forward")
+    if check:
+        _check(uoe_read_device_status(ws), "uoe_smha_forward (device)")
+    return y

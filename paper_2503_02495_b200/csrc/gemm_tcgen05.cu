@@ -1,0 +1,245 @@
+// bf16 grouped expert GEMM on the tcgen05 tensor cores (Eq. 19 / 38 / 39: every expert applies its own
+// weight slice to the rows routed to it).
+//
+//   C[r, :] = epilogue( A[r, :] @ W[e(r)] ),  r over the routed rows, e(r) = expert whose region holds r
+//
+// One persistent CTA per SM walks the (128-row tile, BN-column tile) list; expert regions are padded
+// to 128 rows, so a row tile never straddles two experts.  Warp roles:
+//   warp 0     TMA producer: A tile [128 x 64] and B tile [64 x BN] per K step into a 128B-swizzled ring
+//   warp 1     MMA issuer: tcgen05.mma 128 x BN x 16 into one of two TMEM accumulators
+//   warps 2-5  epilogue: tcgen05.ld the accumulator (one row per thread), activation, bf16, global store
+// so the epilogue of tile t overlaps the main loop of tile t+1.
+#include "kernels.cuh"
+#include "tc.cuh"
+#include "tmap.cuh"
+
+namespace uoe {
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BK = 64;
+constexpr int kGemmThreads = 192;
+constexpr int A_BYTES = BM * BK * 2;     // 16 KB
+
+template <int BN> struct Cfg {
+    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int STAGE = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int TMEM_COLS = 2 * BN;               // two accumulators; 128, 256 or 512 columns
+    static constexpr int SMEM = STAGES * STAGE + 1024 /*align slack*/ + 512 /*barriers, offsets*/;
+};
+
+struct Ctl {                       // lives behind the stage ring
+    uint64_t full[8], empty[8], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    int offs[34];
+};
+
+template <int BN, bool B_KMAJOR>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                 __nv_bfloat16* __restrict__ C, __nv_bfloat16* __restrict__ pre, const int* __restrict__ offsets,
+                 int n, int K, int N, int act, int* status) {
+    using Cf = Cfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    Ctl* ctl = (Ctl*)(smem + Cf::STAGES * Cf::STAGE);
+    volatile int* abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < Cf::STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 128); }
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmA);
+        prefetch_tmap(&tmB);
+    }
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + n + 1) ctl->offs[threadIdx.x - 64] = offsets[threadIdx.x - 64];
+    if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    const int n_tiles = N / BN;
+    const int num_kb = K / BK;
+    const int total_tiles = (ctl->offs[n] / BM) * n_tiles;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------- TMA producer ----------------
+            int stage = 0;
+            uint32_t phase = 0;
+            uint32_t issued = 0, issued_parity = 0;      // per stage: a load is in flight with this parity
+            bool stop = false;
+            for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+                const int row0 = (tile / n_tiles) * BM, col0 = (tile % n_tiles) * BN;
+                int e = 0;
+                while (e + 1 < n && row0 >= ctl->offs[e + 1]) ++e;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) || *abort_flag) { stop = true; break; }
+                    uint8_t* sa = smem + stage * Cf::STAGE;
+                    uint8_t* sb = sa + A_BYTES;
+                    mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
+                    tma_load_2d(sa, &tmA, kb * BK, row0, &ctl->full[stage]);
+                    if (B_KMAJOR) {
+                        tma_load_3d(sb, &tmB, kb * BK, col0, e, &ctl->full[stage]);
+                    } else {
+#pragma unroll
+                        for (int q = 0; q < BN / 64; ++q)
+                            tma_load_3d(sb + q * 8192, &tmB, col0 + q * 64, kb * BK, e, &ctl->full[stage]);
+                    }
+                    issued |= 1u << stage;
+                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                    if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+            if (*abort_flag) {      // let this CTA's own copies land before it exits
+                for (int s = 0; s < Cf::STAGES; ++s)
+                    if (issued & (1u << s)) mbar_wait(&ctl->full[s], (issued_parity >> s) & 1, abort_flag, status);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------- MMA issuer ----------------
+            constexpr uint32_t idesc = instr_desc_bf16(BM, BN, false, !B_KMAJOR);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool stop = false;
+            for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+                if (!mbar_wait(&ctl->tempty[acc], acc_phase ^ 1, abort_flag, status) || *abort_flag) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&ctl->full[stage], phase, abort_flag, status) || *abort_flag) { stop = true; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + stage * Cf::STAGE);
+                    const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < BK / 16; ++ks) {
+                        const uint64_t ad = smem_desc(sa + ks * 32, 16, 1024);
+                        const uint64_t bd = B_KMAJOR ? smem_desc(sb + ks * 32, 16, 1024)
+                                                     : smem_desc(sb + ks * 2048, 8192, 1024);
+                        mma_bf16(d_tmem, ad, bd, idesc, (kb | ks) != 0);
+                    }
+                    mma_commit(&ctl->empty[stage]);
+                    if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (stop) break;
+                mma_commit(&ctl->tfull[acc]);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
+        const int quarter = warp & 3;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int row0 = (tile / n_tiles) * BM, col0 = (tile % n_tiles) * BN;
+            const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
+            if (!__all_sync(0xffffffffu, ready)) break;      // warp-uniform: tcgen05.ld below is warp-collective
+            tc_fence_after();
+            const size_t row = (size_t)row0 + quarter * 32 + lane;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+#pragma unroll 1
+            for (int ch = 0; ch < BN / 32; ++ch) {
+                uint32_t v[32];
+                tmem_ld32(taddr + ch * 32, v);
+                tmem_ld_wait();
+                uint4* out = (uint4*)(C + row * N + col0 + ch * 32);
+                if (pre) {
+                    uint4* po = (uint4*)(pre + row * N + col0 + ch * 32);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        uint4 w;
+                        w.x = pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1]));
+                        w.y = pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3]));
+                        w.z = pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5]));
+                        w.w = pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7]));
+                        po[q] = w;
+                    }
+                }
+                if (act != UOE_ACT_IDENTITY) {
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) v[q] = __float_as_uint(act_apply(__uint_as_float(v[q]), act));
+                }
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    uint4 w;
+                    w.x = pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1]));
+                    w.y = pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3]));
+                    w.z = pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5]));
+                    w.w = pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7]));
+                    out[q] = w;
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&ctl->tempty[acc]);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, Cf::TMEM_COLS);
+    }
+}
+
+template <int BN, bool B_KMAJOR>
+uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
+    using Cf = Cfg<BN>;
+    static bool attr_set = false;
+    auto kern = gemm_bf16_kernel<BN, B_KMAJOR>;
+    if (!attr_set) {
+        UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
+        attr_set = true;
+    }
+    CUtensorMap tmA, tmB;
+    {
+        const uint64_t dims[2] = {(uint64_t)g.K, (uint64_t)g.rows_max};
+        const uint64_t str[1] = {(uint64_t)g.K * 2};
+        const uint32_t box[2] = {BK, BM};
+        if (!make_tmap(&tmA, g.A, 2, dims, str, box)) return UOE_ERR_CUDA;
+    }
+    if (B_KMAJOR) {       // W [n, N, K]
+        const uint64_t dims[3] = {(uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.n};
+        const uint64_t str[2] = {(uint64_t)g.K * 2, (uint64_t)g.K * g.N * 2};
+        const uint32_t box[3] = {BK, BN, 1};
+        if (!make_tmap(&tmB, g.W, 3, dims, str, box)) return UOE_ERR_CUDA;
+    } else {              // W [n, K, N]
+        const uint64_t dims[3] = {(uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.n};
+        const uint64_t str[2] = {(uint64_t)g.N * 2, (uint64_t)g.K * g.N * 2};
+        const uint32_t box[3] = {64, BK, 1};
+        if (!make_tmap(&tmB, g.W, 3, dims, str, box)) return UOE_ERR_CUDA;
+    }
+    long long max_tiles = (g.rows_max / BM) * (g.N / BN);
+    int grid = (int)(max_tiles < sm_count() ? max_tiles : sm_count());
+    if (grid < 1) grid = 1;
+    kern<<<grid, kGemmThreads, Cf::SMEM, s>>>(tmA, tmB, (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.pre, g.offsets, g.n,
+                                              g.K, g.N, g.act, status);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
+
+}  // namespace
+
+uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s) {
+    if (g.K % BK != 0 || g.N % 64 != 0 || g.bias) return UOE_ERR_UNSUPPORTED;
+    if (g.rows_max % BM != 0) return UOE_ERR_INVALID_ARG;
+    const int bn = (g.N % 256 == 0) ? 256 : (g.N % 128 == 0 ? 128 : 64);
+    if (g.b_kmajor) {
+        if (bn == 256) return launch_one<256, true>(g, status, s);
+        if (bn == 128) return launch_one<128, true>(g, status, s);
+        return launch_one<64, true>(g, status, s);
+    }
+    if (bn == 256) return launch_one<256, false>(g, status, s);
+    if (bn == 128) return launch_one<128, false>(g, status, s);
+    return launch_one<64, false>(g, status, s);
+}
+
+}  // namespace uoe

@@ -1,0 +1,72 @@
+// uoe_mlp_forward: UoME forward (Eq. 37-40) as plan -> gather (Eq. 18) -> grouped GEMM1 + phi (Eq. 38)
+// -> grouped GEMM2 (Eq. 39) -> weighted combine (Eq. 20 / 40).
+#include "kernels.cuh"
+
+namespace uoe {
+
+struct MlpFwdWs { size_t plan, xg, a, z, total; };
+
+static MlpFwdWs mlp_fwd_ws(const Dims& D) {
+    WsCarver w;
+    w.take(kStatusBytes);
+    MlpFwdWs r;
+    r.plan = w.take(plan_bytes(D));
+    r.xg = w.take((size_t)D.Rmax * D.d * D.esize);
+    r.a = w.take((size_t)D.Rmax * D.d_e * D.esize);
+    r.z = w.take((size_t)D.Rmax * D.d * D.esize);
+    r.total = w.off;
+    return r;
+}
+
+size_t mlp_fwd_workspace_bytes(const Dims& D) { return mlp_fwd_ws(D).total; }
+
+}  // namespace uoe
+
+using namespace uoe;
+
+extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, const void* W1, const void* W2,
+                                      const void* b1, const void* b2, const int32_t* expert_idx,
+                                      const int32_t* patch_idx, const float* gate, const int32_t* expert_offsets,
+                                      void* y, void* saved_h, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Dims D;
+    uoe_status st = make_dims(prob, D);
+    if (st != UOE_OK) return st;
+    if (!x || !W1 || !W2 || !expert_idx || !patch_idx || !gate || !expert_offsets || !y || !ws) return UOE_ERR_INVALID_ARG;
+    if (D.d_e < 1) return UOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(W1) || !aligned16(W2) || !aligned16(y) || !aligned16(ws) ||
+        (saved_h && !aligned16(saved_h)))
+        return UOE_ERR_INVALID_ARG;
+    if ((D.d_e * D.esize) % 16 != 0) return UOE_ERR_UNSUPPORTED;
+    if (D.bf16 && (b1 || b2)) return UOE_ERR_UNSUPPORTED;
+    const MlpFwdWs W = mlp_fwd_ws(D);
+    if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    char* base = (char*)ws;
+    int* status = (int*)base;
+    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
+    const PlanPtrs P = plan_ptrs(D, base + W.plan);
+    void* xg = base + W.xg;
+    void* a = base + W.a;
+    void* z = base + W.z;
+
+    st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream);
+    if (st != UOE_OK) return st;
+    st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
+    if (st != UOE_OK) return st;
+
+    GemmArgs g1{xg, W1, b1, a, saved_h, expert_offsets, D.n, D.d, D.d_e, prob->act, false, D.Rmax};
+    GemmArgs g2{a, W2, b2, z, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
+    if (D.bf16) {
+        st = launch_gemm_bf16(g1, status, stream);
+        if (st != UOE_OK) return st;
+        st = launch_gemm_bf16(g2, status, stream);
+        if (st != UOE_OK) return st;
+    } else {
+        st = launch_gemm_f32(g1, stream);
+        if (st != UOE_OK) return st;
+        st = launch_gemm_f32(g2, stream);
+        if (st != UOE_OK) return st;
+    }
+    return launch_combine(D, x, z, P, (prob->flags & UOE_FLAG_RESIDUAL) != 0, (prob->flags & UOE_FLAG_GATE) != 0, y,
+                          stream);
+}

@@ -1,0 +1,250 @@
+// uoe_route: router scoring (Eq. 13-14, 21) and fused top-k expert / top-c patch selection
+// (Eq. 17, 22-23).  Two kernels:
+//   route_score_kernel  streams x once (16-byte loads) and leaves, per (patch, column chunk), the
+//                       partial dot products  sum_{t in patch} x[t, chunk] . W_r[chunk, i]
+//   route_select_kernel one CTA per sample: fixed-order sum of the partials, both softmaxes,
+//                       rank-based selection with warp ballots, gates; the last CTA to finish turns
+//                       the per-expert loads into row offsets.
+#include "kernels.cuh"
+
+namespace uoe {
+
+long long g_launch_count = 0;
+
+namespace {
+
+constexpr int kScoreThreads = 256;
+constexpr int kSelectThreads = 128;
+
+// grid (B*m, nchunks).  CT threads span the columns of a chunk (16 bytes each), 256/CT span rows.
+template <typename T>
+__global__ void __launch_bounds__(kScoreThreads)
+route_score_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ partial,
+                   int L, int Lv, int d, int n, int m, int l_p, int CT, int nchunks) {
+    constexpr int V = Vec16<T>::N;
+    const int bj = blockIdx.x, chunk = blockIdx.y;
+    const int b = bj / m, j = bj % m;
+    const int ct = threadIdx.x % CT, rt = threadIdx.x / CT, RT = kScoreThreads / CT;
+    const int col = (chunk * CT + ct) * V;
+    const int rows = max(0, min(l_p, Lv - j * l_p));
+
+    float cs[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) cs[v] = 0.f;
+    if (col < d) {
+        const T* base = x + ((size_t)b * L + (size_t)j * l_p) * d + col;
+        int r = rt;
+        for (; r + 3 * RT < rows; r += 4 * RT) {
+            uint4 q[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) q[u] = ld_stream16(base + (size_t)(r + u * RT) * d);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                float f[V];
+                unpack16<T>(q[u], f);
+#pragma unroll
+                for (int v = 0; v < V; ++v) cs[v] += f[v];
+            }
+        }
+        for (; r < rows; r += RT) {
+            float f[V];
+            unpack16<T>(ld_stream16(base + (size_t)r * d), f);
+#pragma unroll
+            for (int v = 0; v < V; ++v) cs[v] += f[v];
+        }
+    }
+
+    __shared__ float red[kScoreThreads / 32][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = 0; i < n; ++i) {
+        float a = 0.f;
+        if (col < d) {
+#pragma unroll
+            for (int v = 0; v < V; ++v) a += cs[v] * to_f32(W_r[(size_t)(col + v) * n + i]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if (lane == 0) red[warp][i] = a;
+    }
+    __syncthreads();
+    if (threadIdx.x < n) {
+        float s = 0.f;
+#pragma unroll
+        for (int wv = 0; wv < kScoreThreads / 32; ++wv) s += red[wv][threadIdx.x];
+        partial[((size_t)bj * nchunks + chunk) * n + threadIdx.x] = s;
+    }
+}
+
+// grid B.  Dynamic shared memory: n*m floats.
+__global__ void __launch_bounds__(kSelectThreads)
+route_select_kernel(const float* __restrict__ partial, int nchunks, int B, int Lv, int n, int k, int m, int c,
+                    int l_p, int use_gate, int* __restrict__ expert_idx, int* __restrict__ patch_idx,
+                    float* __restrict__ gate, float* __restrict__ p_samp, float* __restrict__ p_patch,
+                    int* __restrict__ offsets, int* __restrict__ load, int* __restrict__ ticket) {
+    extern __shared__ float pp[];          // [n][m]: raw sums, then probabilities
+    __shared__ float ps[32];               // sample gate
+    __shared__ int sel[32];                // chosen experts, ascending
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int n_elig = (Lv + l_p - 1) / l_p;       // patches holding at least one real token (a prefix)
+
+    for (int idx = tid; idx < n * m; idx += kSelectThreads) {
+        const int i = idx / m, j = idx % m;
+        const float* p = partial + ((size_t)(b * m + j) * nchunks) * n + i;
+        float s = 0.f;
+        for (int ch = 0; ch < nchunks; ++ch) s += p[(size_t)ch * n];
+        pp[idx] = s;
+    }
+    __syncthreads();
+    if (tid < n) {                          // Eq. 21: mean over the real tokens, then W_r
+        float s = 0.f;
+        for (int j = 0; j < m; ++j) s += pp[tid * m + j];
+        ps[tid] = s / (float)Lv;
+    }
+    __syncthreads();
+    for (int j = tid; j < m; j += kSelectThreads) {     // Eq. 14: softmax over the experts of patch j
+        const int cnt = max(0, min(l_p, Lv - j * l_p));
+        float mx = -INFINITY;
+        for (int i = 0; i < n; ++i) {
+            const float v = cnt > 0 ? pp[i * m + j] / (float)cnt : 0.f;
+            pp[i * m + j] = v;
+            mx = fmaxf(mx, v);
+        }
+        float sum = 0.f;
+        for (int i = 0; i < n; ++i) { const float e = expf(pp[i * m + j] - mx); pp[i * m + j] = e; sum += e; }
+        for (int i = 0; i < n; ++i) {
+            const float pr = pp[i * m + j] / sum;
+            pp[i * m + j] = pr;
+            p_patch[((size_t)b * n + i) * m + j] = pr;
+        }
+    }
+    if (warp == 0) {
+        const float v = lane < n ? ps[lane] : -INFINITY;
+        float mx = v;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float e = lane < n ? expf(v - mx) : 0.f;
+        float sum = e;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        const float pr = e / sum;
+        if (lane < n) { ps[lane] = pr; p_samp[(size_t)b * n + lane] = pr; }
+        // Eq. 22: rank = number of experts that beat this one (larger value, or equal with lower index)
+        int rank = 0;
+        for (int i = 0; i < n; ++i) {
+            const float w = __shfl_sync(0xffffffffu, pr, i);
+            rank += (w > pr) || (w == pr && i < lane);
+        }
+        const bool pick = lane < n && rank < k;
+        const unsigned mask = __ballot_sync(0xffffffffu, pick);
+        if (pick) {
+            const int s = __popc(mask & ((1u << lane) - 1u));
+            sel[s] = lane;
+            expert_idx[(size_t)b * k + s] = lane;
+            atomicAdd(&load[lane], 1);
+        }
+    }
+    __syncthreads();
+    const int take = min(c, n_elig);
+    for (int s = warp; s < k; s += kSelectThreads / 32) {       // Eq. 17 for the s-th chosen expert
+        const int i = sel[s];
+        const float* v_i = pp + i * m;
+        int* out_idx = patch_idx + ((size_t)b * k + s) * c;
+        float* out_gate = gate + ((size_t)b * k + s) * c;
+        int before = 0;
+        for (int j0 = 0; j0 < n_elig; j0 += 32) {
+            const int j = j0 + lane;
+            const bool valid = j < n_elig;
+            const float v = valid ? v_i[j] : 0.f;
+            int rank = 0;
+            if (valid)
+                for (int jj = 0; jj < n_elig; ++jj) {
+                    const float w = v_i[jj];
+                    rank += (w > v) || (w == v && jj < j);
+                }
+            const bool pick = valid && rank < take;
+            const unsigned mask = __ballot_sync(0xffffffffu, pick);
+            if (pick) {
+                const int pos = before + __popc(mask & ((1u << lane) - 1u));
+                out_idx[pos] = j;
+                out_gate[pos] = use_gate ? ps[i] * v : 1.0f;
+            }
+            before += __popc(mask);
+        }
+        for (int pos = before + lane; pos < c; pos += 32) { out_idx[pos] = -1; out_gate[pos] = 0.f; }
+    }
+    // Eq. 23 as row offsets: the last sample to arrive sums the loads
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const int t = atomicAdd(ticket, 1);
+        if (t == B - 1) {
+            __threadfence();
+            int off = 0;
+            const int rows_per_pair = c * l_p;
+            for (int i = 0; i < n; ++i) {
+                offsets[i] = off;
+                const int rows = atomicAdd(&load[i], 0) * rows_per_pair;
+                off += (rows + UOE_ROW_ALIGN - 1) / UOE_ROW_ALIGN * UOE_ROW_ALIGN;
+            }
+            offsets[n] = off;
+        }
+    }
+}
+
+struct RouteWs { size_t partial, total; int nchunks, CT; };
+
+RouteWs route_ws(const Dims& D) {
+    const int V = 16 / D.esize;
+    int CT = 64;
+    while (CT > 1 && (CT / 2) * V >= D.d) CT /= 2;
+    const int nchunks = (D.d + CT * V - 1) / (CT * V);
+    WsCarver w;
+    w.take(kStatusBytes);
+    RouteWs r;
+    r.partial = w.take((size_t)D.B * D.m * nchunks * D.n * sizeof(float));
+    r.total = w.off;
+    r.nchunks = nchunks;
+    r.CT = CT;
+    return r;
+}
+
+}  // namespace
+
+size_t route_workspace_bytes(const Dims& D) { return route_ws(D).total; }
+
+}  // namespace uoe
+
+using namespace uoe;
+
+extern "C" uoe_status uoe_route(const uoe_problem* prob, const void* x, const void* W_r, int32_t* expert_idx,
+                                int32_t* patch_idx, float* gate, float* p_samp, float* p_patch,
+                                int32_t* expert_offsets, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Dims D;
+    uoe_status st = make_dims(prob, D);
+    if (st != UOE_OK) return st;
+    if (!x || !W_r || !expert_idx || !patch_idx || !gate || !p_samp || !p_patch || !expert_offsets || !ws)
+        return UOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(ws)) return UOE_ERR_INVALID_ARG;
+    if ((size_t)D.n * D.m * sizeof(float) > 40 * 1024) return UOE_ERR_UNSUPPORTED;
+    const RouteWs W = route_ws(D);
+    if (W.nchunks > 65535) return UOE_ERR_UNSUPPORTED;
+    if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    char* base = (char*)ws;
+    int* status = (int*)base;          // word 0 status, word 1 ticket, words 8.. expert loads
+    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
+    float* partial = (float*)(base + W.partial);
+    dim3 grid(D.B * D.m, W.nchunks);
+    if (D.bf16)
+        route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, 0, stream>>>(
+            (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
+    else
+        route_score_kernel<float><<<grid, kScoreThreads, 0, stream>>>(
+            (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
+    UOE_LAUNCHED();
+    route_select_kernel<<<D.B, kSelectThreads, (size_t)D.n * D.m * sizeof(float), stream>>>(
+        partial, W.nchunks, D.B, D.Lv, D.n, D.k, D.m, D.c, D.l_p, (prob->flags & UOE_FLAG_GATE) ? 1 : 0,
+        expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, status + 8, status + 1);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}

@@ -1,0 +1,261 @@
+// Data movement around the expert GEMMs: the routing plan, the token gather (Eq. 18 / 24), the
+// weighted combine (Eq. 20 / 26 / 40), and the float32 grouped GEMM used by the float32 path.
+#include "kernels.cuh"
+
+namespace uoe {
+namespace {
+
+constexpr int kThreads = 256;
+
+// ---------------------------------------------------------------------------------------------
+// plan: grid B
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_idx, const float* __restrict__ gate,
+            const int* __restrict__ offsets, int B, int n, int k, int m, int c, int l_p,
+            int* __restrict__ pair_row, int* __restrict__ inv_row, float* __restrict__ inv_gate,
+            int* __restrict__ expert_end, int* status) {
+    __shared__ int my_e[32], cnt[32], prow[32];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int l_a = c * l_p;
+    if (tid < k) {
+        int e = expert_idx[b * k + tid];
+        if (e < 0 || e >= n) { set_status(status, UOE_ERR_DEVICE_INDEX); e = 0; }
+        my_e[tid] = e;
+        cnt[tid] = 0;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < b * k; idx += 128) {          // samples before b that chose the same expert
+        const int e = expert_idx[idx];
+        for (int s = 0; s < k; ++s)
+            if (my_e[s] == e) atomicAdd(&cnt[s], 1);
+    }
+    __syncthreads();
+    if (tid < k) {
+        const int row = offsets[my_e[tid]] + cnt[tid] * l_a;
+        prow[tid] = row;
+        pair_row[b * k + tid] = row;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < m * k; idx += 128) {
+        const int j = idx / k, s = idx % k;
+        const int* pi = patch_idx + ((size_t)b * k + s) * c;
+        int row = -1;
+        float g = 0.f;
+        for (int u = 0; u < c; ++u) {
+            const int pj = pi[u];
+            if (pj < -1 || pj >= m) set_status(status, UOE_ERR_DEVICE_INDEX);
+            if (pj == j) { row = prow[s] + u * l_p; g = gate[((size_t)b * k + s) * c + u]; }
+        }
+        inv_row[((size_t)b * m + j) * k + s] = row;
+        inv_gate[((size_t)b * m + j) * k + s] = g;
+    }
+    if (b == 0 && tid < n) {
+        int load = 0;
+        for (int idx = 0; idx < B * k; ++idx) load += (expert_idx[idx] == tid);
+        expert_end[tid] = offsets[tid] + load * l_a;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// gather: grid (B*k*c + n, nsplit); a patch is one contiguous slab of l_p*d elements on both sides
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads)
+gather_kernel(const uint4* __restrict__ src, const int* __restrict__ patch_idx, const int* __restrict__ offsets,
+              const int* __restrict__ pair_row, const int* __restrict__ expert_end,
+              uint4* __restrict__ dst, int n_slabs, int k, int c, int m, long long slab_vecs /* l_p*d*esize/16 */,
+              long long row_vecs /* d*esize/16 */, int l_p) {
+    const int bx = blockIdx.x;
+    long long count;                 // 16-byte pieces to write
+    const uint4* s = nullptr;
+    uint4* o;
+    if (bx < n_slabs) {
+        const int pair = bx / c, u = bx % c, b = pair / k;
+        const int j = patch_idx[bx];
+        o = dst + ((long long)pair_row[pair] + (long long)u * l_p) * row_vecs;
+        count = slab_vecs;
+        if (j >= 0 && j < m) s = src + ((long long)b * m + j) * slab_vecs;
+    } else {
+        const int i = bx - n_slabs;
+        const long long r0 = expert_end[i], r1 = offsets[i + 1];
+        o = dst + r0 * row_vecs;
+        count = (r1 - r0) * row_vecs;
+    }
+    const long long per = (count + gridDim.y - 1) / gridDim.y;
+    const long long lo = per * blockIdx.y, hi = min(count, lo + per);
+    if (s) {
+        long long i = lo + threadIdx.x;
+        for (; i + 3 * kThreads < hi; i += 4 * kThreads) {
+            uint4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q] = ld_stream16(s + i + q * kThreads);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) st_stream16(o + i + q * kThreads, v[q]);
+        }
+        for (; i < hi; i += kThreads) st_stream16(o + i, ld_stream16(s + i));
+    } else {
+        const uint4 z = make_uint4(0, 0, 0, 0);
+        for (long long i = lo + threadIdx.x; i < hi; i += kThreads) st_stream16(o + i, z);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// combine: grid (B*m, row groups)
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __restrict__ inv_row,
+               const float* __restrict__ inv_gate, T* __restrict__ y, int L, int Lv, int d, int m, int k,
+               int l_p, int residual, int use_gate, int rows_per_cta) {
+    constexpr int V = Vec16<T>::N;
+    __shared__ int srow[32];
+    __shared__ float sg[32];
+    const int bj = blockIdx.x, b = bj / m, j = bj % m;
+    const int r0 = blockIdx.y * rows_per_cta, r1 = min(l_p, r0 + rows_per_cta);
+    if (threadIdx.x < k) {
+        srow[threadIdx.x] = inv_row[(size_t)bj * k + threadIdx.x];
+        sg[threadIdx.x] = use_gate ? inv_gate[(size_t)bj * k + threadIdx.x] : 1.0f;
+    }
+    __syncthreads();
+    const int vpr = d / V;
+    const int total = (r1 - r0) * vpr;
+    for (int idx = threadIdx.x; idx < total; idx += kThreads) {
+        const int r = r0 + idx / vpr, cv = idx % vpr;
+        const int t = j * l_p + r;
+        const size_t xo = ((size_t)b * L + t) * d + (size_t)cv * V;
+        float acc[V];
+        if (residual) {
+            unpack16<T>(ld_stream16(x + xo), acc);
+        } else {
+#pragma unroll
+            for (int v = 0; v < V; ++v) acc[v] = 0.f;
+        }
+        if (t < Lv) {
+            for (int s = 0; s < k; ++s) {
+                if (srow[s] < 0) continue;
+                float f[V];
+                unpack16<T>(ld_stream16(z + ((size_t)(srow[s] + r)) * d + (size_t)cv * V), f);
+                const float g = sg[s];
+#pragma unroll
+                for (int v = 0; v < V; ++v) acc[v] = fmaf(g, f[v], acc[v]);
+            }
+        }
+        st_stream16(y + xo, pack16<T>(acc));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// float32 grouped GEMM (FFMA): 64x64 tile, 16-deep K step, 4x4 outputs per thread
+// ---------------------------------------------------------------------------------------------
+constexpr int BM = 64, BN = 64, BK = 16;
+
+__global__ void __launch_bounds__(256)
+gemm_f32_kernel(const float* __restrict__ A, const float* __restrict__ W, const float* __restrict__ bias,
+                float* __restrict__ C, float* __restrict__ pre, const int* __restrict__ offsets, int n, int K, int N,
+                int act, int b_kmajor) {
+    __shared__ float As[BK][BM + 4];
+    __shared__ float Bs[BK][BN + 4];
+    const int total_rows = offsets[n];
+    const int row0 = blockIdx.x * BM;
+    if (row0 >= total_rows) return;
+    int e = 0;
+    while (e + 1 < n && row0 >= offsets[e + 1]) ++e;       // regions are multiples of 128 rows: no tile straddles
+    const int col0 = blockIdx.y * BN;
+    const float* We = W + (size_t)e * K * N;
+    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < K; k0 += BK) {
+        for (int idx = threadIdx.x; idx < BM * BK; idx += 256) {
+            const int r = idx / BK, kk = idx % BK;
+            As[kk][r] = (k0 + kk < K) ? A[(size_t)(row0 + r) * K + k0 + kk] : 0.f;
+        }
+        for (int idx = threadIdx.x; idx < BK * BN; idx += 256) {
+            int kk, cc;
+            if (b_kmajor) { cc = idx / BK; kk = idx % BK; } else { kk = idx / BN; cc = idx % BN; }
+            float v = 0.f;
+            if (k0 + kk < K && col0 + cc < N)
+                v = b_kmajor ? We[(size_t)(col0 + cc) * K + k0 + kk] : We[(size_t)(k0 + kk) * N + col0 + cc];
+            Bs[kk][cc] = v;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[4], bb[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) bb[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], bb[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const size_t r = (size_t)row0 + ty * 4 + i;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int cc = col0 + tx * 4 + j;
+            if (cc >= N) continue;
+            float v = acc[i][j];
+            if (bias) v += bias[(size_t)e * N + cc];
+            if (pre) pre[r * N + cc] = v;
+            C[r * N + cc] = act_apply(v, act);
+        }
+    }
+}
+
+}  // namespace
+
+uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_idx, const float* gate,
+                       const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s) {
+    plan_kernel<<<D.B, 128, 0, s>>>(expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
+                                    P.pair_row, P.inv_row, P.inv_gate, P.expert_end, status);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
+
+uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, const int* offsets,
+                         const PlanPtrs& P, void* dst, cudaStream_t s) {
+    const long long row_vecs = (long long)D.d * D.esize / 16;
+    const long long slab_vecs = row_vecs * D.l_p;
+    const int n_slabs = D.B * D.k * D.c;
+    int nsplit = (int)((slab_vecs * 16 + 32767) / 32768);
+    if (nsplit < 1) nsplit = 1;
+    if (nsplit > 64) nsplit = 64;
+    dim3 grid(n_slabs + D.n, nsplit);
+    gather_kernel<<<grid, kThreads, 0, s>>>((const uint4*)src, patch_idx, offsets, P.pair_row, P.expert_end,
+                                            (uint4*)dst, n_slabs, D.k, D.c, D.m, slab_vecs, row_vecs, D.l_p);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
+
+uoe_status launch_combine(const Dims& D, const void* x, const void* z, const PlanPtrs& P, bool residual,
+                          bool use_gate, void* y, cudaStream_t s) {
+    int rows_per_cta = (int)(32768 / ((long long)D.d * D.esize));
+    if (rows_per_cta < 1) rows_per_cta = 1;
+    if (rows_per_cta > D.l_p) rows_per_cta = D.l_p;
+    dim3 grid(D.B * D.m, (D.l_p + rows_per_cta - 1) / rows_per_cta);
+    if (D.bf16)
+        combine_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(
+            (const __nv_bfloat16*)x, (const __nv_bfloat16*)z, P.inv_row, P.inv_gate, (__nv_bfloat16*)y, D.L, D.Lv,
+            D.d, D.m, D.k, D.l_p, residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta);
+    else
+        combine_kernel<float><<<grid, kThreads, 0, s>>>((const float*)x, (const float*)z, P.inv_row, P.inv_gate,
+                                                       (float*)y, D.L, D.Lv, D.d, D.m, D.k, D.l_p,
+                                                       residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
+
+uoe_status launch_gemm_f32(const GemmArgs& g, cudaStream_t s) {
+    dim3 grid((unsigned)((g.rows_max + BM - 1) / BM), (g.N + BN - 1) / BN);
+    gemm_f32_kernel<<<grid, 256, 0, s>>>((const float*)g.A, (const float*)g.W, (const float*)g.bias, (float*)g.C,
+                                         (float*)g.pre, g.offsets, g.n, g.K, g.N, g.act, g.b_kmajor ? 1 : 0);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
+
+}  // namespace uoe

@@ -1,0 +1,56 @@
+"""Host-side checks that need no GPU: the shared library loads, exports every symbol the header
+declares, and its launch-free entry points validate their arguments."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def uoe():
+    import __graft_entry__ as ge
+    ge.build()
+    import paper_2503_02495_b200 as mod
+    return mod
+
+
+def test_library_exports_every_declared_symbol(uoe):
+    header = open(os.path.join(ROOT, "include", "uoe.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    names = set(re.findall(r"\b(uoe_[a-z_0-9]+)\s*\(", header))
+    assert {"uoe_route", "uoe_mlp_forward", "uoe_mlp_backward", "uoe_smha_forward", "uoe_workspace_bytes",
+            "uoe_max_routed_rows", "uoe_status_string", "uoe_read_device_status", "uoe_launch_count"} <= names
+    lib = ctypes.CDLL(uoe.LIB_PATH)
+    for nm in names:
+        assert hasattr(lib, nm), nm
+
+
+def test_sizes_and_validation(uoe):
+    p = uoe.Problem(B=2, L=256, L_valid=256, d=256, n=4, k=2, m=8, c=4, d_e=256, dtype="f32", act="gelu_erf")
+    assert uoe.uoe_max_routed_rows(p) % uoe.UOE_ROW_ALIGN == 0
+    assert uoe.uoe_max_routed_rows(p) >= 2 * 2 * 4 * 32
+    assert uoe.uoe_workspace_bytes(p, uoe.UOE_OP_ROUTE) > 0
+    assert uoe.uoe_workspace_bytes(p, uoe.UOE_OP_MLP_FWD) >= uoe.uoe_max_routed_rows(p) * (256 + 256 + 256) * 4
+    bad = uoe.Problem(B=2, L=250, L_valid=250, d=256, n=4, k=2, m=8, c=4, d_e=256)      # L % m != 0
+    assert uoe.uoe_workspace_bytes(bad, uoe.UOE_OP_ROUTE) == 0
+    bad = uoe.Problem(B=2, L=256, L_valid=256, d=256, n=4, k=5, m=8, c=4, d_e=256)      # k > n
+    assert uoe.uoe_max_routed_rows(bad) == 0
+    bad = uoe.Problem(B=2, L=256, L_valid=300, d=256, n=4, k=2, m=8, c=4, d_e=256)      # L_valid > L
+    assert uoe.uoe_max_routed_rows(bad) == 0
+    assert uoe.status_string(0) == "ok" and "workspace" in uoe.status_string(3)
+
+
+def test_null_arguments_are_rejected_before_any_launch(uoe):
+    lib = ctypes.CDLL(uoe.LIB_PATH)
+    p = uoe.Problem(B=2, L=256, L_valid=256, d=256, n=4, k=2, m=8, c=4, d_e=256, dtype="f32").c_struct()
+    lib.uoe_route.restype = ctypes.c_int
+    st = lib.uoe_route(ctypes.byref(p), *([None] * 9), ctypes.c_size_t(0), None)
+    assert st == 1
+    lib.uoe_mlp_forward.restype = ctypes.c_int
+    st = lib.uoe_mlp_forward(ctypes.byref(p), *([None] * 12), ctypes.c_size_t(0), None)
+    assert st == 1
+    st = lib.uoe_route(None, *([None] * 9), ctypes.c_size_t(0), None)
+    assert st == 1

@@ -1,0 +1,85 @@
+"""GPU parity: uoe_route against the float64 oracle (Eq. 12-17, 21-23) on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import uoe_inputs as gen
+from oracle import uoe_oracle as orc
+from tests.helpers import check_routing, problem_of, to_dev
+
+pytestmark = pytest.mark.gpu
+
+CASES = {
+    "tiny": gen.tiny(),
+    "tiny_pad": gen.tiny(L_valid=21, B=5),
+    "tiny_k1": gen.tiny(k=1, c=1),
+    "tiny_full": gen.tiny(k=4, c=6),
+    "tiny_bf16": gen.tiny(dtype="bf16", d=64, B=7),
+    "wide_m": gen.tiny(B=3, m=48, c=20, L=96, L_valid=91, d=40, n=5, k=3, d_ff=40),
+    "cfg1": gen.WORKLOADS["cfg1_small_f32"],
+    "cfg2": gen.WORKLOADS["cfg2_lm"],
+    "cfg3": gen.WORKLOADS["cfg3_long"],
+    "cfg4": gen.WORKLOADS["cfg4_vit"],
+}
+
+
+@pytest.mark.parametrize("name", list(CASES))
+@pytest.mark.parametrize("use_gate", [True, False])
+def test_route_matches_oracle(name, use_gate):
+    import paper_2503_02495_b200 as uoe
+    w = CASES[name]
+    if name.startswith("cfg") and not use_gate:
+        pytest.skip("gate-off variant covered by the small cases")
+    x, Wr = gen.make_x(w), gen.make_router(w)
+    scale = 40.0 if name.startswith("tiny") or name == "wide_m" else 1.0
+    Wr = gen.store(Wr.f64 * scale, w.dtype)
+    prob = problem_of(w, "mlp", gate=use_gate)
+    r = uoe.uoe_route(prob, to_dev(x), to_dev(Wr))
+    ro = orc.route(x.f64, Wr.f64, w.k, w.m, w.c, L_valid=w.L_valid, use_gate=use_gate)
+    assert np.abs(r.p_samp.cpu().numpy() - ro.p_samp).max() < 2e-6
+    assert np.abs(r.p_patch.cpu().numpy() - ro.p_patch).max() < 2e-6
+    near_e, near_p = check_routing(r, ro)
+    print(f"{name}: near-tie mismatches experts={near_e} patches={near_p}")
+    if near_e == 0 and near_p == 0:
+        assert np.array_equal(r.expert_offsets.cpu().numpy(), ro.offsets)
+        g = r.gate.cpu().numpy()
+        assert np.abs(g - ro.gate).max() <= 1e-5 * max(1.0, np.abs(ro.gate).max())
+        assert np.all(g[r.patch_idx.cpu().numpy() < 0] == 0)
+    # structural invariants hold for any tie-break
+    e = r.expert_idx.cpu().numpy()
+    p = r.patch_idx.cpu().numpy()
+    assert np.all(np.diff(e, axis=1) > 0) and e.min() >= 0 and e.max() < w.n
+    n_elig = -(-w.L_valid // w.l_p)
+    for b in range(w.B):
+        for s in range(w.k):
+            sel = p[b, s][p[b, s] >= 0]
+            assert len(sel) == min(w.c, n_elig) and np.all(np.diff(sel) > 0) and sel.max() < n_elig
+            assert np.all(p[b, s][len(sel):] == -1)
+    off = r.expert_offsets.cpu().numpy()
+    load = np.bincount(e.ravel(), minlength=w.n)
+    exp = np.concatenate([[0], np.cumsum((load * w.l_a + 127) // 128 * 128)])
+    assert np.array_equal(off, exp)
+
+
+def test_route_planted_ties_take_lower_index():
+    import paper_2503_02495_b200 as uoe
+    # identical patches and a zero router: every probability ties exactly -> lowest indices win
+    w = gen.tiny(B=2)
+    x = np.tile(gen.normal(3, 0, (1, w.l_p, w.d)), (w.B, w.m, 1))
+    prob = problem_of(w, "mlp")
+    r = uoe.uoe_route(prob, torch.from_numpy(x.astype(np.float32)).cuda(),
+                      torch.zeros(w.d, w.n, device="cuda"))
+    assert r.expert_idx.cpu().tolist() == [[0, 1]] * w.B
+    assert r.patch_idx.cpu().tolist() == [[[0, 1, 2]] * w.k] * w.B
+    assert torch.allclose(r.gate.cpu(), torch.full((w.B, w.k, w.c), 1.0 / (w.n * w.n)))
+
+
+def test_route_is_deterministic():
+    import paper_2503_02495_b200 as uoe
+    w = gen.WORKLOADS["cfg2_lm"]
+    x, Wr = to_dev(gen.make_x(w)), to_dev(gen.make_router(w))
+    prob = problem_of(w, "mlp")
+    a = uoe.uoe_route(prob, x, Wr)
+    b = uoe.uoe_route(prob, x, Wr)
+    for f in ("expert_idx", "patch_idx", "gate", "p_samp", "p_patch", "expert_offsets"):
+        assert torch.equal(getattr(a, f), getattr(b, f)), f
