@@ -1,0 +1,242 @@
+// Selective multi-head attention core (Eq. 33-34 with the masks of Eq. 41 and Fig. 4): for every
+// (sample, chosen expert) pair and every head of that expert, softmax(q k^T / sqrt(d_h) + mask) v over
+// the pair's l_a gathered tokens.
+//
+// One CTA per (128-query tile, head, pair).  q, k, v are rows of the routed buffers [rows, d_g] (bf16),
+// so the pair's tokens are contiguous.  Per 128-key tile:
+//   S = Q K^T      tcgen05.mma 128x128x64, both operands K-major from TMA, accumulator in TMEM
+//   softmax        one query row per thread (TMEM lane = row): running max / sum in registers,
+//                  P rounded to bf16 and written to shared memory in the 128B-swizzled K-major layout
+//   O_t = P V      tcgen05.mma 128x64x128, V as the MN-major operand, fresh TMEM accumulator,
+//                  then O = alpha * O + O_t in registers
+// Masks: the real keys of a pair are a prefix of its gathered order (patches ascending, pad tokens at
+// the end of the sample), so key c is kept iff c < n_valid, and with the causal flag iff also
+// c <= query row (the shared lower triangle of Fig. 4).
+#include "kernels.cuh"
+#include "tc.cuh"
+#include "tmap.cuh"
+
+namespace uoe {
+namespace {
+
+using namespace tc;
+
+constexpr int TQ = 128, TK = 128, DH = 64;
+constexpr int kAttnThreads = 128;
+constexpr int TILE_BYTES = 128 * DH * 2;          // 16 KB: a [128 x 64] bf16 tile
+constexpr int ATTN_SMEM = TILE_BYTES * (1 + 2 + 2 + 2) + 1024 + 256;
+
+struct AttnCtl {
+    uint64_t bar_q, bar_kv[2], bar_s, bar_o;
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+__global__ void __launch_bounds__(kAttnThreads)
+attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+            const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
+            const int* __restrict__ pair_row, const int* __restrict__ patch_idx, int c, int l_p, int Lv, int l_a,
+            int d_g, int heads, int causal, float scale_log2, int* status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* sQ = smem;
+    uint8_t* sK = sQ + TILE_BYTES;                 // 2 stages
+    uint8_t* sV = sK + 2 * TILE_BYTES;             // 2 stages
+    uint8_t* sP = sV + 2 * TILE_BYTES;             // [128 x 128] bf16 as two [128 x 64] swizzled halves
+    AttnCtl* ctl = (AttnCtl*)(sP + 2 * TILE_BYTES);
+    volatile int* abort_flag = &ctl->abort_flag;
+    __shared__ int s_nvalid;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int qt = blockIdx.x, head = blockIdx.y, pair = blockIdx.z;
+    const int row_base = pair_row[pair];
+    const int q0 = qt * TQ;
+
+    if (tid == 0) {
+        mbar_init(&ctl->bar_q, 1);
+        mbar_init(&ctl->bar_kv[0], 1);
+        mbar_init(&ctl->bar_kv[1], 1);
+        mbar_init(&ctl->bar_s, 1);
+        mbar_init(&ctl->bar_o, 1);
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        // real keys of this pair: sum over its slots of the real tokens in the slot's patch
+        int nv = 0;
+        for (int u = 0; u < c; ++u) {
+            const int j = patch_idx[(size_t)pair * c + u];
+            if (j >= 0) nv += max(0, min(l_p, Lv - j * l_p));
+        }
+        s_nvalid = nv;
+    }
+    if (warp == 0) tmem_alloc(&ctl->tmem_base, 256);       // S: columns [0,128), O_t: [128,192)
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    const int n_valid = s_nvalid;
+
+    int kv_end = min(n_valid, l_a);
+    if (causal) kv_end = min(kv_end, q0 + TQ);
+    const int n_kv = (kv_end + TK - 1) / TK;               // >= 1: every pair holds a real token
+    const int col_h = head * DH;
+
+    if (tid == 0) {
+        mbar_arrive_expect_tx(&ctl->bar_q, TILE_BYTES);
+        tma_load_2d(sQ, &tmQ, col_h, row_base + q0, &ctl->bar_q);
+        for (int t = 0; t < 2 && t < n_kv; ++t) {
+            mbar_arrive_expect_tx(&ctl->bar_kv[t], 2 * TILE_BYTES);
+            tma_load_2d(sK + t * TILE_BYTES, &tmK, col_h, row_base + t * TK, &ctl->bar_kv[t]);
+            tma_load_2d(sV + t * TILE_BYTES, &tmV, col_h, row_base + t * TK, &ctl->bar_kv[t]);
+        }
+    }
+
+    constexpr uint32_t idesc_s = instr_desc_bf16(TQ, TK, false, false);
+    constexpr uint32_t idesc_o = instr_desc_bf16(TQ, DH, false, true);
+    const int qrow = q0 + warp * 32 + lane;                // query index inside the pair (TMEM lane)
+    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+
+    float o_acc[DH];
+#pragma unroll
+    for (int i = 0; i < DH; ++i) o_acc[i] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;
+    bool ok = true;
+
+    for (int it = 0; it < n_kv; ++it) {
+        const int st = it & 1;
+        // ---- S = Q K^T ----
+        if (tid == 0) {
+            if (it == 0) ok = mbar_wait(&ctl->bar_q, 0, abort_flag, status);
+            ok = mbar_wait(&ctl->bar_kv[st], (it >> 1) & 1, abort_flag, status) && ok;
+            tc_fence_after();
+            const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + st * TILE_BYTES);
+#pragma unroll
+            for (int ks = 0; ks < DH / 16; ++ks)
+                mma_bf16(tmem_base, smem_desc(qa + ks * 32, 16, 1024), smem_desc(ka + ks * 32, 16, 1024), idesc_s, ks != 0);
+            mma_commit(&ctl->bar_s);
+        }
+        ok = mbar_wait(&ctl->bar_s, it & 1, abort_flag, status);
+        if (!__all_sync(0xffffffffu, ok && !*abort_flag)) break;
+        tc_fence_after();
+
+        // ---- online softmax for this row ----
+        const int kv0 = it * TK;
+        float s_row[TK];
+#pragma unroll
+        for (int ch = 0; ch < TK / 32; ++ch) tmem_ld32(t_lane + ch * 32, (uint32_t*)(s_row + ch * 32));
+        tmem_ld_wait();
+        float m_new = m_run;
+#pragma unroll
+        for (int j = 0; j < TK; ++j) {
+            const int col = kv0 + j;
+            const bool keep = col < n_valid && col < l_a && (!causal || col <= qrow);
+            s_row[j] = keep ? s_row[j] * scale_log2 : -INFINITY;
+            m_new = fmaxf(m_new, s_row[j]);
+        }
+        // a row with no kept key so far keeps m = -inf; exp2(-inf - (-inf)) is avoided by the guard
+        const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+        const float alpha = exp2f(m_run - m_use);
+        float l_add = 0.f;
+        uint8_t* prow = sP + (size_t)(warp * 32 + lane) * 128;
+        const int sw = (warp * 32 + lane) & 7;
+#pragma unroll
+        for (int ch = 0; ch < TK / 8; ++ch) {                 // 16-byte chunks of 8 bf16
+            float p[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) { p[q] = exp2f(s_row[ch * 8 + q] - m_use); l_add += p[q]; }
+            uint4 w;
+            w.x = pack_bf16x2(p[0], p[1]); w.y = pack_bf16x2(p[2], p[3]);
+            w.z = pack_bf16x2(p[4], p[5]); w.w = pack_bf16x2(p[6], p[7]);
+            const int half = ch >> 3, cc = ch & 7;
+            *(uint4*)(prow + half * TILE_BYTES + ((cc ^ sw) << 4)) = w;
+        }
+        l_run = l_run * alpha + l_add;
+        m_run = m_new;
+        fence_async_smem();                  // generic-proxy writes of P -> visible to the tensor core
+        tc_fence_before();
+        __syncthreads();
+
+        // ---- O_t = P V ----
+        if (tid == 0) {
+            tc_fence_after();
+            const uint32_t pa = smem_u32(sP), va = smem_u32(sV + st * TILE_BYTES);
+#pragma unroll
+            for (int ks = 0; ks < TK / 16; ++ks)
+                mma_bf16(tmem_base + 128, smem_desc(pa + (ks >> 2) * TILE_BYTES + (ks & 3) * 32, 16, 1024),
+                         smem_desc(va + ks * 2048, 8192, 1024), idesc_o, ks != 0);
+            mma_commit(&ctl->bar_o);
+        }
+        ok = mbar_wait(&ctl->bar_o, it & 1, abort_flag, status);
+        if (!__all_sync(0xffffffffu, ok && !*abort_flag)) break;
+        tc_fence_after();
+        if (tid == 0 && it + 2 < n_kv) {     // both MMAs that read this stage are done: refill it
+            mbar_arrive_expect_tx(&ctl->bar_kv[st], 2 * TILE_BYTES);
+            tma_load_2d(sK + st * TILE_BYTES, &tmK, col_h, row_base + (it + 2) * TK, &ctl->bar_kv[st]);
+            tma_load_2d(sV + st * TILE_BYTES, &tmV, col_h, row_base + (it + 2) * TK, &ctl->bar_kv[st]);
+        }
+        {
+            float o_t[DH];
+            tmem_ld32(t_lane + 128, (uint32_t*)o_t);
+            tmem_ld32(t_lane + 160, (uint32_t*)(o_t + 32));
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < DH; ++i) o_acc[i] = o_acc[i] * alpha + o_t[i];
+        }
+        tc_fence_before();                   // S and O_t are read; the next iteration may overwrite them
+    }
+
+    if (qrow < l_a && !*abort_flag) {
+        const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
+        __nv_bfloat16* out = O + (size_t)(row_base + qrow) * d_g + col_h;
+#pragma unroll
+        for (int ch = 0; ch < DH / 8; ++ch) {
+            uint4 w;
+            w.x = pack_bf16x2(o_acc[ch * 8 + 0] * inv, o_acc[ch * 8 + 1] * inv);
+            w.y = pack_bf16x2(o_acc[ch * 8 + 2] * inv, o_acc[ch * 8 + 3] * inv);
+            w.z = pack_bf16x2(o_acc[ch * 8 + 4] * inv, o_acc[ch * 8 + 5] * inv);
+            w.w = pack_bf16x2(o_acc[ch * 8 + 6] * inv, o_acc[ch * 8 + 7] * inv);
+            ((uint4*)out)[ch] = w;
+        }
+        if (lse) lse[(size_t)(row_base + qrow) * heads + head] = (m_run + log2f(l_run)) * 0.69314718055994531f;
+    }
+    if (tid == 0 && *abort_flag) {           // let copies that may still be in flight land (bounded)
+        mbar_wait(&ctl->bar_q, 0, abort_flag, status);
+        for (int t = 0; t < 2 && t < n_kv; ++t) mbar_try_wait(&ctl->bar_kv[t], 0);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, 256);
+    }
+}
+
+}  // namespace
+
+// q, k, v, o: [rows_max, d_g] bf16 routed buffers.
+uoe_status launch_attention(const Dims& D, const void* q, const void* k, const void* v, void* o, float* lse,
+                            const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s) {
+    if (D.d_h != DH) return UOE_ERR_UNSUPPORTED;
+    static bool attr_set = false;
+    if (!attr_set) {
+        UOE_CUDA_OK(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM));
+        attr_set = true;
+    }
+    CUtensorMap tm[3];
+    const void* ptrs[3] = {q, k, v};
+    for (int i = 0; i < 3; ++i) {
+        const uint64_t dims[2] = {(uint64_t)D.d_g, (uint64_t)D.Rmax};
+        const uint64_t str[1] = {(uint64_t)D.d_g * 2};
+        const uint32_t box[2] = {DH, 128};
+        if (!make_tmap(&tm[i], ptrs[i], 2, dims, str, box)) return UOE_ERR_CUDA;
+    }
+    const int heads = D.d_g / DH;
+    dim3 grid((D.l_a + TQ - 1) / TQ, heads, D.B * D.k);
+    const float scale_log2 = 1.4426950408889634f / sqrtf((float)D.d_h);
+    attn_kernel<<<grid, kAttnThreads, ATTN_SMEM, s>>>(tm[0], tm[1], tm[2], (__nv_bfloat16*)o, lse, pair_row, patch_idx,
+                                                      D.c, D.l_p, D.Lv, D.l_a, D.d_g, heads, causal ? 1 : 0,
+                                                      scale_log2, status);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
+
+}  // namespace uoe

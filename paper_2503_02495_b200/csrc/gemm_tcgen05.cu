@@ -39,9 +39,11 @@ struct Ctl {                       // lives behind the stage ring
 
 template <int BN, bool B_KMAJOR>
 __global__ void __launch_bounds__(kGemmThreads, 1)
-gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                 __nv_bfloat16* __restrict__ C, __nv_bfloat16* __restrict__ pre, const int* __restrict__ offsets,
-                 int n, int K, int N, int act, int* status) {
+gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
+                 const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
+                 __nv_bfloat16* __restrict__ C0, __nv_bfloat16* __restrict__ C1, __nv_bfloat16* __restrict__ C2,
+                 __nv_bfloat16* __restrict__ pre, const int* __restrict__ offsets,
+                 int n, int K, int N, int nmat, int act, int* status) {
     using Cf = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -55,7 +57,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         ctl->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmA);
-        prefetch_tmap(&tmB);
+        prefetch_tmap(&tmB0);
     }
     if (threadIdx.x >= 64 && threadIdx.x < 64 + n + 1) ctl->offs[threadIdx.x - 64] = offsets[threadIdx.x - 64];
     if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
@@ -64,7 +66,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    const int n_tiles = N / BN;
+    // tile index -> (row tile, matrix, column tile); the matrices share the A tile, so they are adjacent
+    const int n_tiles_mat = N / BN;
+    const int n_tiles = n_tiles_mat * nmat;
     const int num_kb = K / BK;
     const int total_tiles = (ctl->offs[n] / BM) * n_tiles;
 
@@ -76,7 +80,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t issued = 0, issued_parity = 0;      // per stage: a load is in flight with this parity
             bool stop = false;
             for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
-                const int row0 = (tile / n_tiles) * BM, col0 = (tile % n_tiles) * BN;
+                const int row0 = (tile / n_tiles) * BM;
+                const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
+                const CUtensorMap* tmB = mat == 0 ? &tmB0 : (mat == 1 ? &tmB1 : &tmB2);
                 int e = 0;
                 while (e + 1 < n && row0 >= ctl->offs[e + 1]) ++e;
                 for (int kb = 0; kb < num_kb; ++kb) {
@@ -86,11 +92,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
                     tma_load_2d(sa, &tmA, kb * BK, row0, &ctl->full[stage]);
                     if (B_KMAJOR) {
-                        tma_load_3d(sb, &tmB, kb * BK, col0, e, &ctl->full[stage]);
+                        tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
                     } else {
 #pragma unroll
                         for (int q = 0; q < BN / 64; ++q)
-                            tma_load_3d(sb + q * 8192, &tmB, col0 + q * 64, kb * BK, e, &ctl->full[stage]);
+                            tma_load_3d(sb + q * 8192, tmB, col0 + q * 64, kb * BK, e, &ctl->full[stage]);
                     }
                     issued |= 1u << stage;
                     issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
@@ -139,7 +145,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-            const int row0 = (tile / n_tiles) * BM, col0 = (tile % n_tiles) * BN;
+            const int row0 = (tile / n_tiles) * BM;
+            const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
+            __nv_bfloat16* C = mat == 0 ? C0 : (mat == 1 ? C1 : C2);
             const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
             if (!__all_sync(0xffffffffu, ready)) break;      // warp-uniform: tcgen05.ld below is warp-collective
             tc_fence_after();
@@ -199,29 +207,34 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
         UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
         attr_set = true;
     }
-    CUtensorMap tmA, tmB;
+    CUtensorMap tmA, tmB[3];
     {
         const uint64_t dims[2] = {(uint64_t)g.K, (uint64_t)g.rows_max};
         const uint64_t str[1] = {(uint64_t)g.K * 2};
         const uint32_t box[2] = {BK, BM};
         if (!make_tmap(&tmA, g.A, 2, dims, str, box)) return UOE_ERR_CUDA;
     }
-    if (B_KMAJOR) {       // W [n, N, K]
-        const uint64_t dims[3] = {(uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.n};
-        const uint64_t str[2] = {(uint64_t)g.K * 2, (uint64_t)g.K * g.N * 2};
-        const uint32_t box[3] = {BK, BN, 1};
-        if (!make_tmap(&tmB, g.W, 3, dims, str, box)) return UOE_ERR_CUDA;
-    } else {              // W [n, K, N]
-        const uint64_t dims[3] = {(uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.n};
-        const uint64_t str[2] = {(uint64_t)g.N * 2, (uint64_t)g.K * g.N * 2};
-        const uint32_t box[3] = {64, BK, 1};
-        if (!make_tmap(&tmB, g.W, 3, dims, str, box)) return UOE_ERR_CUDA;
+    const int nmat = g.nmat < 1 ? 1 : g.nmat;
+    const void* Ws[3] = {g.W, g.W1 ? g.W1 : g.W, g.W2 ? g.W2 : g.W};
+    for (int q = 0; q < 3; ++q) {
+        if (B_KMAJOR) {       // W [n, N, K]
+            const uint64_t dims[3] = {(uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.n};
+            const uint64_t str[2] = {(uint64_t)g.K * 2, (uint64_t)g.K * g.N * 2};
+            const uint32_t box[3] = {BK, BN, 1};
+            if (!make_tmap(&tmB[q], Ws[q], 3, dims, str, box)) return UOE_ERR_CUDA;
+        } else {              // W [n, K, N]
+            const uint64_t dims[3] = {(uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.n};
+            const uint64_t str[2] = {(uint64_t)g.N * 2, (uint64_t)g.K * g.N * 2};
+            const uint32_t box[3] = {64, BK, 1};
+            if (!make_tmap(&tmB[q], Ws[q], 3, dims, str, box)) return UOE_ERR_CUDA;
+        }
     }
-    long long max_tiles = (g.rows_max / BM) * (g.N / BN);
+    long long max_tiles = (g.rows_max / BM) * (g.N / BN) * nmat;
     int grid = (int)(max_tiles < sm_count() ? max_tiles : sm_count());
     if (grid < 1) grid = 1;
-    kern<<<grid, kGemmThreads, Cf::SMEM, s>>>(tmA, tmB, (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.pre, g.offsets, g.n,
-                                              g.K, g.N, g.act, status);
+    kern<<<grid, kGemmThreads, Cf::SMEM, s>>>(tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
+                                              (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
+                                              nmat, g.act, status);
     UOE_LAUNCHED();
     return UOE_OK;
 }
@@ -229,7 +242,8 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
 }  // namespace
 
 uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s) {
-    if (g.K % BK != 0 || g.N % 64 != 0 || g.bias) return UOE_ERR_UNSUPPORTED;
+    if (g.K % BK != 0 || g.N % 64 != 0 || g.bias || g.nmat > 3) return UOE_ERR_UNSUPPORTED;
+    if (g.nmat > 1 && g.pre) return UOE_ERR_UNSUPPORTED;
     if (g.rows_max % BM != 0) return UOE_ERR_INVALID_ARG;
     const int bn = (g.N % 256 == 0) ? 256 : (g.N % 128 == 0 ? 128 : 64);
     if (g.b_kmajor) {

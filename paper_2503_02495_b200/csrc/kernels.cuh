@@ -37,8 +37,10 @@ uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_id
 
 // Eq. 18 / 24: copy the selected patches of `src` [B,L,d] into the routed buffer `dst` [rows,d];
 // unused slots and the padding rows of each expert region are zero-filled.
+// If tail is not null, rows [offsets[n], rows_max) of tail (rows of tail_row_bytes) are zero-filled too.
 uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, const int* offsets,
-                         const PlanPtrs& P, void* dst, cudaStream_t s);
+                         const PlanPtrs& P, void* dst, cudaStream_t s, void* tail = nullptr,
+                         long long tail_row_bytes = 0);
 
 // Eq. 20 / 26 / 36 / 40: y[b,t,:] = (residual ? x[b,t,:] : 0) + sum_s w_s * z[row_s(t),:], every output row
 // written once, contributions added in ascending slot order.  w_s = gate if use_gate else 1.
@@ -58,6 +60,13 @@ struct GemmArgs {
     int act;                // uoe_act applied in the epilogue (UOE_ACT_IDENTITY = none)
     bool b_kmajor;
     long long rows_max;     // host bound on offsets[n] (rows the buffers hold)
+    // bf16 path only: up to three weight tensors of the same shape applied to the same A in one launch
+    // (the q, k, v projections of Eq. 28-30); matrix q writes C (q = 0), C1, C2.
+    int nmat = 1;
+    const void* W1 = nullptr;
+    const void* W2 = nullptr;
+    void* C1 = nullptr;
+    void* C2 = nullptr;
 };
 uoe_status launch_gemm_f32(const GemmArgs& g, cudaStream_t s);
 uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s);

@@ -64,12 +64,17 @@ __global__ void __launch_bounds__(kThreads)
 gather_kernel(const uint4* __restrict__ src, const int* __restrict__ patch_idx, const int* __restrict__ offsets,
               const int* __restrict__ pair_row, const int* __restrict__ expert_end,
               uint4* __restrict__ dst, int n_slabs, int k, int c, int m, long long slab_vecs /* l_p*d*esize/16 */,
-              long long row_vecs /* d*esize/16 */, int l_p) {
+              long long row_vecs /* d*esize/16 */, int l_p, int n, uint4* __restrict__ tail, long long tail_row_vecs,
+              long long rows_max) {
     const int bx = blockIdx.x;
     long long count;                 // 16-byte pieces to write
     const uint4* s = nullptr;
     uint4* o;
-    if (bx < n_slabs) {
+    if (bx == n_slabs + n) {         // rows of `tail` that no kernel writes
+        const long long r0 = offsets[n];
+        o = tail + r0 * tail_row_vecs;
+        count = (rows_max - r0) * tail_row_vecs;
+    } else if (bx < n_slabs) {
         const int pair = bx / c, u = bx % c, b = pair / k;
         const int j = patch_idx[bx];
         o = dst + ((long long)pair_row[pair] + (long long)u * l_p) * row_vecs;
@@ -218,16 +223,17 @@ uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_id
 }
 
 uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, const int* offsets,
-                         const PlanPtrs& P, void* dst, cudaStream_t s) {
+                         const PlanPtrs& P, void* dst, cudaStream_t s, void* tail, long long tail_row_bytes) {
     const long long row_vecs = (long long)D.d * D.esize / 16;
     const long long slab_vecs = row_vecs * D.l_p;
     const int n_slabs = D.B * D.k * D.c;
     int nsplit = (int)((slab_vecs * 16 + 32767) / 32768);
     if (nsplit < 1) nsplit = 1;
     if (nsplit > 64) nsplit = 64;
-    dim3 grid(n_slabs + D.n, nsplit);
+    dim3 grid(n_slabs + D.n + (tail ? 1 : 0), nsplit);
     gather_kernel<<<grid, kThreads, 0, s>>>((const uint4*)src, patch_idx, offsets, P.pair_row, P.expert_end,
-                                            (uint4*)dst, n_slabs, D.k, D.c, D.m, slab_vecs, row_vecs, D.l_p);
+                                            (uint4*)dst, n_slabs, D.k, D.c, D.m, slab_vecs, row_vecs, D.l_p, D.n,
+                                            (uint4*)tail, tail_row_bytes / 16, D.Rmax);
     UOE_LAUNCHED();
     return UOE_OK;
 }

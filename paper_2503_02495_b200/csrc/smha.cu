@@ -1,8 +1,32 @@
-// uoe_smha_forward (Eq. 27-30, 33-36).
+// uoe_smha_forward: SMHA forward (Eq. 27-30, 33-36) as plan -> gather (Eq. 27) -> grouped q/k/v
+// projections in one launch (Eq. 28-30) -> attention over each pair's gathered tokens (Eq. 33-34)
+// -> grouped output projection (Eq. 35) -> weighted combine (Eq. 36).
 #include "kernels.cuh"
 
 namespace uoe {
-size_t smha_fwd_workspace_bytes(const Dims& D) { (void)D; return 0; }
+
+uoe_status launch_attention(const Dims& D, const void* q, const void* k, const void* v, void* o, float* lse,
+                            const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s);
+
+struct SmhaWs { size_t plan, xg, q, k, v, o, z, total; };
+
+static SmhaWs smha_ws(const Dims& D) {
+    WsCarver w;
+    w.take(kStatusBytes);
+    SmhaWs r;
+    r.plan = w.take(plan_bytes(D));
+    r.xg = w.take((size_t)D.Rmax * D.d * D.esize);
+    r.q = w.take((size_t)D.Rmax * D.d_g * D.esize);
+    r.k = w.take((size_t)D.Rmax * D.d_g * D.esize);
+    r.v = w.take((size_t)D.Rmax * D.d_g * D.esize);
+    r.o = w.take((size_t)D.Rmax * D.d_g * D.esize);
+    r.z = w.take((size_t)D.Rmax * D.d * D.esize);
+    r.total = w.off;
+    return r;
+}
+
+size_t smha_fwd_workspace_bytes(const Dims& D) { return smha_ws(D).total; }
+
 }  // namespace uoe
 
 using namespace uoe;
@@ -11,7 +35,41 @@ extern "C" uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, c
                                        const void* Wv, const void* Wo, const int32_t* expert_idx,
                                        const int32_t* patch_idx, const float* gate, const int32_t* expert_offsets,
                                        void* y, float* lse, void* ws, size_t ws_bytes, void* cuda_stream) {
-    (void)prob; (void)x; (void)Wq; (void)Wk; (void)Wv; (void)Wo; (void)expert_idx; (void)patch_idx; (void)gate;
-    (void)expert_offsets; (void)y; (void)lse; (void)ws; (void)ws_bytes; (void)cuda_stream;
-    return UOE_ERR_UNSUPPORTED;
+    Dims D;
+    uoe_status st = make_dims(prob, D);
+    if (st != UOE_OK) return st;
+    if (!x || !Wq || !Wk || !Wv || !Wo || !expert_idx || !patch_idx || !gate || !expert_offsets || !y || !ws)
+        return UOE_ERR_INVALID_ARG;
+    if (D.H < 1 || D.d_g < 1) return UOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(Wo) || !aligned16(y) ||
+        !aligned16(ws))
+        return UOE_ERR_INVALID_ARG;
+    if (!D.bf16 || D.d_h != 64) return UOE_ERR_UNSUPPORTED;     // tensor-core path: bf16, 64-wide heads
+    const SmhaWs W = smha_ws(D);
+    if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    char* base = (char*)ws;
+    int* status = (int*)base;
+    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
+    const PlanPtrs P = plan_ptrs(D, base + W.plan);
+    void *xg = base + W.xg, *q = base + W.q, *k = base + W.k, *v = base + W.v, *o = base + W.o, *z = base + W.z;
+
+    st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream);
+    if (st != UOE_OK) return st;
+    // rows of v past the last expert region are never written by the projection but may sit inside the
+    // last key tile of a pair: make them finite
+    st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream, v, (long long)D.d_g * D.esize);
+    if (st != UOE_OK) return st;
+    GemmArgs gq{xg, Wq, nullptr, q, nullptr, expert_offsets, D.n, D.d, D.d_g, UOE_ACT_IDENTITY, false, D.Rmax};
+    gq.nmat = 3; gq.W1 = Wk; gq.W2 = Wv; gq.C1 = k; gq.C2 = v;
+    st = launch_gemm_bf16(gq, status, stream);
+    if (st != UOE_OK) return st;
+    st = launch_attention(D, q, k, v, o, lse, P.pair_row, patch_idx, (prob->flags & UOE_FLAG_CAUSAL) != 0, status,
+                          stream);
+    if (st != UOE_OK) return st;
+    GemmArgs go{o, Wo, nullptr, z, nullptr, expert_offsets, D.n, D.d_g, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
+    st = launch_gemm_bf16(go, status, stream);
+    if (st != UOE_OK) return st;
+    return launch_combine(D, x, z, P, (prob->flags & UOE_FLAG_RESIDUAL) != 0, (prob->flags & UOE_FLAG_GATE) != 0, y,
+                          stream);
 }

@@ -1,0 +1,133 @@
+"""GPU parity: uoe_smha_forward against the float64 oracle (Eq. 27-30, 33-36, masks Eq. 41 / Fig. 4).
+
+As for the MLP, the oracle runs on the GPU's own selection; bfloat16 tolerance
+max|err| <= 2e-2 * max|ref|, applied to the attention term alone (RESIDUAL off) and to y.
+"""
+import numpy as np
+import pytest
+import torch
+
+import uoe_inputs as gen
+from oracle import uoe_oracle as orc
+from tests.helpers import problem_of, rel_inf, to_dev, to_f64
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-2
+
+
+def _w(**kw):
+    base = dict(B=3, L=96, L_valid=96, m=6, c=3, d=64, n=2, k=1, d_ff=128, H=2, d_h=64, dtype="bf16",
+                w_std=0.08, causal=False)
+    base.update(kw)
+    return gen.tiny(**base)
+
+
+CASES = {
+    "one_tile": _w(),
+    "one_tile_causal": _w(causal=True, k=2),
+    "pad": _w(L_valid=83, B=4, k=2),
+    "pad_causal": _w(L_valid=70, causal=True),
+    "two_heads_per_expert": _w(H=4, k=2),
+    "three_tiles_ragged": _w(B=2, L=512, L_valid=512, m=8, c=5, d=128, n=4, k=2, H=4),
+    "three_tiles_causal_pad": _w(B=2, L=512, L_valid=470, m=8, c=5, d=128, n=4, k=3, H=8, causal=True),
+    "full_selection": _w(k=2, c=6, causal=True),
+    "cfg2": gen.WORKLOADS["cfg2_lm"],
+    "cfg3": gen.WORKLOADS["cfg3_long"],
+    "cfg4": gen.WORKLOADS["cfg4_vit"],
+}
+
+
+def _run(w, residual, want_lse=False):
+    import paper_2503_02495_b200 as uoe
+    x, Wr = gen.make_x(w), gen.make_router(w, "att")
+    if not w.name.startswith("cfg"):
+        Wr = gen.store(Wr.f64 * 20, w.dtype)
+    Wq, Wk, Wv, Wo = gen.make_attn_weights(w)
+    prob = problem_of(w, "att", residual=residual)
+    xd = to_dev(x)
+    r = uoe.uoe_route(prob, xd, to_dev(Wr))
+    lse = None
+    if want_lse:
+        lse = torch.zeros(uoe.uoe_max_routed_rows(prob), w.d_g // w.d_h, device="cuda")
+    y = uoe.uoe_smha_forward(prob, xd, to_dev(Wq), to_dev(Wk), to_dev(Wv), to_dev(Wo), r, lse=lse)
+    ro = orc.with_selection(x.f64, Wr.f64, r.expert_idx.cpu().numpy(), r.patch_idx.cpu().numpy(), w.m, w.L_valid)
+    out = orc.smha_forward(x.f64, Wq.f64, Wk.f64, Wv.f64, Wo.f64, ro, w.d_h, w.causal, residual=residual,
+                           return_lse=want_lse)
+    return to_f64(y), out, x.f64, r, ro, lse
+
+
+@pytest.mark.parametrize("name", list(CASES))
+def test_attention_term_matches_oracle(name):
+    w = CASES[name]
+    y, ref, x, r, ro, _ = _run(w, residual=False)
+    err = rel_inf(y, ref)
+    print(f"{name}: max|err|/max|ref| = {err:.3e}")
+    assert err <= TOL
+    assert np.all(y[:, w.L_valid:] == 0)
+
+
+@pytest.mark.parametrize("name", ["one_tile", "pad_causal", "cfg2", "cfg4"])
+def test_residual_output_matches_oracle(name):
+    w = CASES[name]
+    y, ref, x, r, ro, _ = _run(w, residual=True)
+    assert rel_inf(y, ref) <= TOL
+    assert np.array_equal(y[:, w.L_valid:], x[:, w.L_valid:])
+
+
+def test_full_selection_equals_multihead_attention():
+    # k = n, c = m: the union of attention experts is plain causal multi-head attention (Eq. 8-11)
+    w = CASES["full_selection"]
+    y, ref, x, r, ro, _ = _run(w, residual=False)
+    assert rel_inf(y, ref) <= TOL
+    Wq, Wk, Wv, Wo = gen.make_attn_weights(w)
+    Q = x @ np.concatenate(list(Wq.f64), 1)
+    K = x @ np.concatenate(list(Wk.f64), 1)
+    V = x @ np.concatenate(list(Wv.f64), 1)
+    WO = np.concatenate(list(Wo.f64), 0)
+    for b in range(w.B):
+        o = np.zeros_like(Q[b])
+        for h in range(w.H):
+            sl = slice(h * w.d_h, (h + 1) * w.d_h)
+            s = Q[b][:, sl] @ K[b][:, sl].T / np.sqrt(w.d_h)
+            s = np.where(np.tril(np.ones_like(s, dtype=bool)), s, -np.inf)
+            p = np.exp(s - s.max(1, keepdims=True))
+            o[:, sl] = (p / p.sum(1, keepdims=True)) @ V[b][:, sl]
+        g = ro.gate[b]                      # [k, c] per-patch weights
+        dense = o @ WO
+        # with k = n and one head per expert, expert i contributes its own head: weight per (expert, patch)
+        acc = np.zeros_like(dense)
+        for i in range(w.n):
+            oi = np.zeros_like(o)
+            sl = slice(i * w.d_g, (i + 1) * w.d_g)
+            oi[:, sl] = o[:, sl]
+            acc += np.repeat(g[i], w.l_p)[:, None] * (oi @ WO)
+        assert rel_inf(y[b], acc) <= TOL
+
+
+def test_lse_output():
+    import paper_2503_02495_b200 as uoe
+    w = CASES["three_tiles_causal_pad"]
+    y, (ref, lse_ref), x, r, ro, lse = _run(w, residual=False, want_lse=True)
+    assert rel_inf(y, ref) <= TOL
+    lse = lse.cpu().numpy()
+    for b in range(w.B):
+        for s in range(w.k):
+            row = orc.buffer_row(ro, b, s)
+            tok = orc.gathered_tokens(ro, b, s)
+            valid = tok < w.L_valid
+            for hd in range(w.d_g // w.d_h):
+                got = lse[row:row + len(tok), hd][valid]
+                assert np.abs(got - lse_ref[(b, s, hd)][valid]).max() < 2e-2
+
+
+def test_unsupported_shapes_return_codes():
+    import paper_2503_02495_b200 as uoe
+    w = gen.tiny(dtype="bf16", d=64)          # d_h = 4
+    prob = problem_of(w, "att")
+    x, Wr = to_dev(gen.make_x(w)), to_dev(gen.make_router(w, "att"))
+    r = uoe.uoe_route(prob, x, Wr)
+    Wq, Wk, Wv, Wo = (to_dev(t) for t in gen.make_attn_weights(w))
+    with pytest.raises(uoe.UoeError) as ei:
+        uoe.uoe_smha_forward(prob, x, Wq, Wk, Wv, Wo, r)
+    assert ei.value.status == 2
