@@ -171,6 +171,17 @@ uoe_status uoe_read_device_status(void* ws, void* cuda_stream);
 /* Number of this library's kernel launches enqueued by this process so far (for benchmarks). */
 int64_t uoe_launch_count(void);
 
+/*
+ * Per-kernel timing for benchmarks (instrumentation; the paper times whole passes with a profiler,
+ * Section IV).  uoe_profile_enable(1) clears the record list and starts recording: from then on every
+ * kernel the library launches is bracketed by two CUDA events on its stream.  uoe_profile_enable(0)
+ * stops recording.  uoe_profile_get waits for record i to finish and returns its label (static
+ * storage) and duration in milliseconds.  Not thread-safe; leave it off outside measurements.
+ */
+void uoe_profile_enable(int on);
+int uoe_profile_count(void);
+uoe_status uoe_profile_get(int i, const char** name, float* ms);
+
 #ifdef __cplusplus
 }
 #endif

@@ -100,6 +100,12 @@ def _load():
     lib.uoe_read_device_status.argtypes = [vp, vp]
     lib.uoe_launch_count.restype = ctypes.c_int64
     lib.uoe_launch_count.argtypes = []
+    lib.uoe_profile_enable.restype = None
+    lib.uoe_profile_enable.argtypes = [ctypes.c_int]
+    lib.uoe_profile_count.restype = ctypes.c_int
+    lib.uoe_profile_count.argtypes = []
+    lib.uoe_profile_get.restype = ctypes.c_int
+    lib.uoe_profile_get.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float)]
     return lib
 
 
@@ -142,6 +148,20 @@ def uoe_workspace_bytes(prob: Problem, op: int) -> int:
 
 def uoe_launch_count() -> int:
     return int(_lib.uoe_launch_count())
+
+
+def uoe_profile_enable(on: bool) -> None:
+    _lib.uoe_profile_enable(1 if on else 0)
+
+
+def uoe_profile_records():
+    """[(label, milliseconds)] of every launch recorded since uoe_profile_enable(True)."""
+    out = []
+    for i in range(_lib.uoe_profile_count()):
+        name, ms = ctypes.c_char_p(), ctypes.c_float()
+        _check(_lib.uoe_profile_get(i, ctypes.byref(name), ctypes.byref(ms)), "uoe_profile_get")
+        out.append((name.value.decode(), float(ms.value)))
+    return out
 
 
 def alloc_workspace(prob: Problem, op: int, device="cuda") -> torch.Tensor:

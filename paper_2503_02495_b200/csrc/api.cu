@@ -1,7 +1,47 @@
 // Entry points that launch nothing: sizes, status text, status read-back, launch counter.
 #include "kernels.cuh"
 
+#include <vector>
+
+namespace uoe {
+namespace {
+struct ProfRec { const char* name; cudaEvent_t e0, e1; };
+bool g_prof_on = false;
+std::vector<ProfRec> g_prof;
+}  // namespace
+
+ProfScope::ProfScope(const char* name, cudaStream_t s) : slot(-1), stream(s) {
+    if (!g_prof_on) return;
+    ProfRec r{name, nullptr, nullptr};
+    if (cudaEventCreate(&r.e0) != cudaSuccess || cudaEventCreate(&r.e1) != cudaSuccess) return;
+    cudaEventRecord(r.e0, s);
+    g_prof.push_back(r);
+    slot = (int)g_prof.size() - 1;
+}
+ProfScope::~ProfScope() {
+    if (slot >= 0) cudaEventRecord(g_prof[slot].e1, stream);
+}
+}  // namespace uoe
+
 using namespace uoe;
+
+extern "C" void uoe_profile_enable(int on) {
+    if (on) {
+        for (auto& r : g_prof) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+        g_prof.clear();
+    }
+    g_prof_on = on != 0;
+}
+
+extern "C" int uoe_profile_count(void) { return (int)g_prof.size(); }
+
+extern "C" uoe_status uoe_profile_get(int i, const char** name, float* ms) {
+    if (i < 0 || i >= (int)g_prof.size() || !name || !ms) return UOE_ERR_INVALID_ARG;
+    if (cudaEventSynchronize(g_prof[i].e1) != cudaSuccess) return UOE_ERR_CUDA;
+    if (cudaEventElapsedTime(ms, g_prof[i].e0, g_prof[i].e1) != cudaSuccess) return UOE_ERR_CUDA;
+    *name = g_prof[i].name;
+    return UOE_OK;
+}
 
 extern "C" int64_t uoe_max_routed_rows(const uoe_problem* prob) {
     Dims D;

@@ -232,6 +232,7 @@ uoe_status launch_attention(const Dims& D, const void* q, const void* k, const v
     const int heads = D.d_g / DH;
     dim3 grid((D.l_a + TQ - 1) / TQ, heads, D.B * D.k);
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)D.d_h);
+    ProfScope ps("attention", s);
     attn_kernel<<<grid, kAttnThreads, ATTN_SMEM, s>>>(tm[0], tm[1], tm[2], (__nv_bfloat16*)o, lse, pair_row, patch_idx,
                                                       D.c, D.l_p, D.Lv, D.l_a, D.d_g, heads, causal ? 1 : 0,
                                                       scale_log2, status);

@@ -31,6 +31,15 @@ extern long long g_launch_count;   // kernels enqueued by this process (reported
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// While profiling is enabled (uoe_profile_enable), a ProfScope around a launch records a CUDA event
+// before and after it on the launching stream; otherwise it does nothing.
+struct ProfScope {
+    ProfScope(const char* name, cudaStream_t s);
+    ~ProfScope();
+    int slot;
+    cudaStream_t stream;
+};
+
 // Sizes derived from a problem (paper notation: l_p tokens per patch, l_a = c*l_p tokens per expert).
 struct Dims {
     int B, L, Lv, d, n, k, m, c, l_p, l_a, d_e, H, d_h, d_g;

@@ -232,6 +232,7 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     long long max_tiles = (g.rows_max / BM) * (g.N / BN) * nmat;
     int grid = (int)(max_tiles < sm_count() ? max_tiles : sm_count());
     if (grid < 1) grid = 1;
+    ProfScope ps(g.label, s);
     kern<<<grid, kGemmThreads, Cf::SMEM, s>>>(tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
                                               (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
                                               nmat, g.act, status);

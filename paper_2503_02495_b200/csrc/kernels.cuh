@@ -67,6 +67,7 @@ struct GemmArgs {
     const void* W2 = nullptr;
     void* C1 = nullptr;
     void* C2 = nullptr;
+    const char* label = "gemm";   // name under which the launch is profiled
 };
 uoe_status launch_gemm_f32(const GemmArgs& g, cudaStream_t s);
 uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s);

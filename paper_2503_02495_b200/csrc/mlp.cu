@@ -56,6 +56,8 @@ extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, co
 
     GemmArgs g1{xg, W1, b1, a, saved_h, expert_offsets, D.n, D.d, D.d_e, prob->act, false, D.Rmax};
     GemmArgs g2{a, W2, b2, z, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
+    g1.label = "gemm1_act";
+    g2.label = "gemm2";
     if (D.bf16) {
         st = launch_gemm_bf16(g1, status, stream);
         if (st != UOE_OK) return st;

@@ -235,13 +235,17 @@ extern "C" uoe_status uoe_route(const uoe_problem* prob, const void* x, const vo
     UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
     float* partial = (float*)(base + W.partial);
     dim3 grid(D.B * D.m, W.nchunks);
+    {
+    ProfScope ps("route_score", stream);
     if (D.bf16)
         route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, 0, stream>>>(
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
     else
         route_score_kernel<float><<<grid, kScoreThreads, 0, stream>>>(
             (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
+    }
     UOE_LAUNCHED();
+    ProfScope ps("route_select", stream);
     route_select_kernel<<<D.B, kSelectThreads, (size_t)D.n * D.m * sizeof(float), stream>>>(
         partial, W.nchunks, D.B, D.Lv, D.n, D.k, D.m, D.c, D.l_p, (prob->flags & UOE_FLAG_GATE) ? 1 : 0,
         expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, status + 8, status + 1);

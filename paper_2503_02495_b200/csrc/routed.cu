@@ -216,6 +216,7 @@ gemm_f32_kernel(const float* __restrict__ A, const float* __restrict__ W, const 
 
 uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_idx, const float* gate,
                        const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s) {
+    ProfScope ps("plan", s);
     plan_kernel<<<D.B, 128, 0, s>>>(expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
                                     P.pair_row, P.inv_row, P.inv_gate, P.expert_end, status);
     UOE_LAUNCHED();
@@ -231,6 +232,7 @@ uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, c
     if (nsplit < 1) nsplit = 1;
     if (nsplit > 64) nsplit = 64;
     dim3 grid(n_slabs + D.n + (tail ? 1 : 0), nsplit);
+    ProfScope ps("gather", s);
     gather_kernel<<<grid, kThreads, 0, s>>>((const uint4*)src, patch_idx, offsets, P.pair_row, P.expert_end,
                                             (uint4*)dst, n_slabs, D.k, D.c, D.m, slab_vecs, row_vecs, D.l_p, D.n,
                                             (uint4*)tail, tail_row_bytes / 16, D.Rmax);
@@ -244,6 +246,7 @@ uoe_status launch_combine(const Dims& D, const void* x, const void* z, const Pla
     if (rows_per_cta < 1) rows_per_cta = 1;
     if (rows_per_cta > D.l_p) rows_per_cta = D.l_p;
     dim3 grid(D.B * D.m, (D.l_p + rows_per_cta - 1) / rows_per_cta);
+    ProfScope ps("combine", s);
     if (D.bf16)
         combine_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)z, P.inv_row, P.inv_gate, (__nv_bfloat16*)y, D.L, D.Lv,
@@ -258,6 +261,7 @@ uoe_status launch_combine(const Dims& D, const void* x, const void* z, const Pla
 
 uoe_status launch_gemm_f32(const GemmArgs& g, cudaStream_t s) {
     dim3 grid((unsigned)((g.rows_max + BM - 1) / BM), (g.N + BN - 1) / BN);
+    ProfScope ps(g.label, s);
     gemm_f32_kernel<<<grid, 256, 0, s>>>((const float*)g.A, (const float*)g.W, (const float*)g.bias, (float*)g.C,
                                          (float*)g.pre, g.offsets, g.n, g.K, g.N, g.act, g.b_kmajor ? 1 : 0);
     UOE_LAUNCHED();

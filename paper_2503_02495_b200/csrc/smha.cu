@@ -61,6 +61,7 @@ extern "C" uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, c
     st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream, v, (long long)D.d_g * D.esize);
     if (st != UOE_OK) return st;
     GemmArgs gq{xg, Wq, nullptr, q, nullptr, expert_offsets, D.n, D.d, D.d_g, UOE_ACT_IDENTITY, false, D.Rmax};
+    gq.label = "qkv_proj";
     gq.nmat = 3; gq.W1 = Wk; gq.W2 = Wv; gq.C1 = k; gq.C2 = v;
     st = launch_gemm_bf16(gq, status, stream);
     if (st != UOE_OK) return st;
@@ -68,6 +69,7 @@ extern "C" uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, c
                           stream);
     if (st != UOE_OK) return st;
     GemmArgs go{o, Wo, nullptr, z, nullptr, expert_offsets, D.n, D.d_g, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
+    go.label = "out_proj";
     st = launch_gemm_bf16(go, status, stream);
     if (st != UOE_OK) return st;
     return launch_combine(D, x, z, P, (prob->flags & UOE_FLAG_RESIDUAL) != 0, (prob->flags & UOE_FLAG_GATE) != 0, y,
