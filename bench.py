@@ -1,0 +1,385 @@
+"""Benchmark of the UoE routed hot path: one step = one forward pass of a whole UoE block
+(router -> SMHA -> router -> UoME; a block without attention or without MLP skips that half; the scale
+workload adds the UoME backward) over one batch of seeded synthetic input.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2_lm] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is tokens/s with inputs resident in HBM; `e2e` is the same metric
+through the public API with host buffers (pinned host -> device copy of x and device -> host copy of the
+result inside the timed region).  L2 is flushed between timed steps (a 512 MB write), and every step is
+timed with its own pair of CUDA events on the launching stream.  `--impl reference` times the float64
+CPU oracle on the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import uoe_inputs as gen
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------------------------
+# algorithmic work per launch, by profile label
+# ------------------------------------------------------------------------------------------------
+
+def work_table(w: gen.Workload):
+    s = 2 if w.dtype == "bf16" else 4
+    R, d, n = w.R, w.d, w.n
+    x_bytes = w.B * w.L * d * s
+    t = {
+        "route_score": dict(flops=2 * w.B * w.L_valid * d * n, bytes=w.B * w.L_valid * d * s),
+        "gather": dict(flops=0, bytes=2 * R * d * s),
+        "combine": dict(flops=2 * R * d, bytes=R * d * s + 2 * x_bytes),
+        "route_select": dict(flops=0, bytes=0),
+        "plan": dict(flops=0, bytes=0),
+    }
+    if w.d_ff:
+        de = w.d_e
+        t["gemm1_act"] = dict(flops=2 * R * d * de, bytes=(R * d + R * de + n * d * de) * s)
+        t["gemm2"] = dict(flops=2 * R * de * d, bytes=(R * de + R * d + n * d * de) * s)
+    if w.H:
+        dg = w.d_g
+        att = 4 * w.l_a * w.l_a * dg * w.B * w.k
+        t["qkv_proj"] = dict(flops=6 * R * d * dg, bytes=(R * d + 3 * R * dg + 3 * n * d * dg) * s)
+        t["attention"] = dict(flops=att // 2 if w.causal else att, bytes=4 * R * dg * s)
+        t["out_proj"] = dict(flops=2 * R * dg * d, bytes=(R * dg + R * d + n * dg * d) * s)
+    return t
+
+
+def step_flops(w: gen.Workload) -> int:
+    t = work_table(w)
+    f = 0
+    if w.d_ff:
+        f += t["gemm1_act"]["flops"] + t["gemm2"]["flops"]
+    if w.H:
+        f += t["qkv_proj"]["flops"] + t["attention"]["flops"] + t["out_proj"]["flops"]
+    return f
+
+
+# ------------------------------------------------------------------------------------------------
+# inputs
+# ------------------------------------------------------------------------------------------------
+
+def host_inputs(w: gen.Workload):
+    d = dict(x=gen.make_x(w))
+    if w.H:
+        d["Wr_att"] = gen.make_router(w, "att")
+        d["Wq"], d["Wk"], d["Wv"], d["Wo"] = gen.make_attn_weights(w)
+    if w.d_ff:
+        d["Wr_mlp"] = gen.make_router(w, "mlp")
+        d["W1"], d["W2"] = gen.make_mlp_weights(w)
+    return d
+
+
+def oracle_step(w: gen.Workload, h, B=None):
+    """One block forward with the float64 oracle on the first B samples; returns seconds."""
+    from oracle import uoe_oracle as orc
+    B = w.B if B is None else B
+    x = h["x"].f64[:B]
+    t0 = time.perf_counter()
+    cur = x
+    if w.H:
+        r = orc.route(cur, h["Wr_att"].f64, w.k, w.m, w.c, L_valid=w.L_valid)
+        cur = orc.smha_forward(cur, h["Wq"].f64, h["Wk"].f64, h["Wv"].f64, h["Wo"].f64, r, w.d_h, w.causal)
+    if w.d_ff:
+        r = orc.route(cur, h["Wr_mlp"].f64, w.k, w.m, w.c, L_valid=w.L_valid)
+        cur = orc.mlp_forward(cur, h["W1"].f64, h["W2"].f64, r, w.act)
+    return time.perf_counter() - t0
+
+
+def blas_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        ns = [p.get("num_threads", 1) for p in threadpool_info()]
+        return max(ns) if ns else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_sample_B(w: gen.Workload) -> int:
+    """Samples of the workload the oracle is timed on: sized for seconds, not minutes."""
+    per_sample_gflop = step_flops(w) / w.B / 1e9
+    budget_gflop = 40.0            # roughly 1-3 s of float64 work per step on a few host cores
+    return max(1, min(w.B, int(budget_gflop / max(per_sample_gflop, 1e-9))))
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.proc = None
+        self.idx = gpu_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.idx}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [t.strip() for t in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1]))
+                    mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                   "samples": len(sm)}
+        return out
+
+
+# ------------------------------------------------------------------------------------------------
+# arms
+# ------------------------------------------------------------------------------------------------
+
+def base_line(w: gen.Workload, args, n_gpus: int):
+    return {
+        "metric": "UoME+SMHA layer tokens/s", "unit": "tokens/s", "n_gpus": n_gpus, "steps": args.steps,
+        "warmup": args.warmup, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "stands_in_for": w.stands_in_for, "B": w.B, "L": w.L, "L_valid": w.L_valid,
+                   "d": w.d, "n": w.n, "k": w.k, "m": w.m, "c": w.c, "d_ff": w.d_ff, "heads": w.H, "d_h": w.d_h,
+                   "causal": w.causal, "act": w.act, "blocks": ("smha+" if w.H else "") + ("uome" if w.d_ff else ""),
+                   "parallelism": f"replicas x{n_gpus}" if n_gpus > 1 else "single gpu",
+                   "l2": "flushed between timed steps (512 MB write)"},
+    }
+
+
+def run_reference(args, w: gen.Workload, rank: int, world: int):
+    if rank != 0:
+        return
+    h = host_inputs(w)
+    Bs = cpu_sample_B(w)
+    for _ in range(args.warmup):
+        oracle_step(w, h, Bs)
+    ts = [oracle_step(w, h, Bs) for _ in range(args.steps)]
+    sec = sum(ts) / len(ts)
+    tok_s = Bs * w.L_valid / sec
+    line = base_line(w, args, 1)
+    line.update({"impl": "reference", "value": tok_s, "ms_per_step": sec * 1e3, "dtype": "f64", "n_gpus": world,
+                 "tflops": step_flops(w) * Bs / w.B / sec / 1e12,
+                 "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+                                  "sample": f"first {Bs} of {w.B} samples, whole block, {args.steps} steps"},
+                 "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+                 "gpu_launches": 0})
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2503_02495_b200 as uoe
+    from paper_2503_02495_b200.block import UoEBlock
+    from tests.helpers import problem_of, to_dev
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    h = host_inputs(w)
+    wd = {k: to_dev(v, dev) for k, v in h.items() if k != "x"}
+    x_dev = to_dev(h["x"], dev)
+    blk = UoEBlock(problem_of(w, "att") if w.H else None, problem_of(w, "mlp") if w.d_ff else None, wd, dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        blk.forward(x_dev)
+    torch.cuda.synchronize()
+    st = blk.device_status()
+    if st != 0:
+        raise RuntimeError("device status after warm-up: " + uoe.status_string(st))
+
+    # ---- timed region: K steps, each with its own event pair, L2 flushed in between ----
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    launches0 = uoe.uoe_launch_count()
+    for e0, e1 in ev:
+        flush.zero_()
+        e0.record(stream)
+        blk.forward(x_dev)
+        e1.record(stream)
+    barrier()
+    launches = uoe.uoe_launch_count() - launches0
+    clocks = sampler.stop()
+    ms = [e0.elapsed_time(e1) for e0, e1 in ev]
+    ms_step = sum(ms) / len(ms)
+
+    # ---- end to end through the public API with host buffers ----
+    x_host = h["x"].raw
+    x_pin = torch.from_numpy(np.ascontiguousarray(x_host).view(np.int16 if w.dtype == "bf16" else np.float32)).pin_memory()
+    x_in = torch.empty_like(x_dev)
+    y_pin = torch.empty(x_pin.shape, dtype=x_pin.dtype).pin_memory()
+    e2e_t = []
+    for i in range(args.steps + 2):
+        flush.zero_()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        x_in.view(x_pin.dtype).copy_(x_pin, non_blocking=True)
+        out = blk.forward(x_in)
+        y_pin.copy_(out.view(x_pin.dtype), non_blocking=True)
+        torch.cuda.synchronize()
+        if i >= 2:
+            e2e_t.append(time.perf_counter() - t0)
+    e2e_ms = sum(e2e_t) / len(e2e_t) * 1e3
+
+    # ---- per-kernel durations (separate pass: the event pairs would perturb the timed region) ----
+    uoe.uoe_profile_enable(True)
+    for _ in range(min(args.steps, 20)):
+        flush.zero_()
+        blk.forward(x_dev)
+    torch.cuda.synchronize()
+    uoe.uoe_profile_enable(False)
+    recs = uoe.uoe_profile_records()
+    per = {}
+    for name, t in recs:
+        per.setdefault(name, []).append(t)
+
+    if world > 1:
+        tt = torch.tensor([ms_step, e2e_ms], device=dev)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms_step, e2e_ms = float(tt[0]), float(tt[1])
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_src = load_peaks()
+    tokens = w.B * w.L_valid * world
+    flops = step_flops(w) * world
+    work = work_table(w)
+    kern = []
+    tot = sum(sum(v) for v in per.values())
+    steps_prof = min(args.steps, 20)
+    for name, v in per.items():
+        avg = sum(v) / len(v)
+        wk = work.get(name, dict(flops=0, bytes=0))
+        kern.append({"kernel": name, "launches_per_step": len(v) / steps_prof, "avg_ms": avg,
+                     "share": sum(v) / tot if tot else 0.0,
+                     "tflops": wk["flops"] / avg / 1e9 if avg > 0 else 0.0,
+                     "gbs": wk["bytes"] / avg / 1e6 if avg > 0 else 0.0})
+    kern.sort(key=lambda r: -r["share"])
+    top = kern[0]
+    wk = work.get(top["kernel"], dict(flops=0, bytes=0))
+    t_tensor = wk["flops"] / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = wk["bytes"] / (peaks["hbm_gbs"] * 1e9)
+    if t_tensor >= t_hbm and wk["flops"] > 0:
+        roof = {"bound": "tensor", "achieved": top["tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+    else:
+        roof = {"bound": "hbm", "achieved": top["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": None, "kernel": top["kernel"],
+                 "avg_ms": top["avg_ms"], "share_of_kernel_time": top["share"], "peak_source": peak_src,
+                 "algorithmic_flops": wk["flops"], "algorithmic_bytes": wk["bytes"]})
+
+    # ---- CPU baseline: the oracle as it stands, on a bounded sample ----
+    Bs = cpu_sample_B(w)
+    oracle_step(w, h, Bs)
+    ts, t_begin = [], time.perf_counter()
+    while len(ts) < 3 or (time.perf_counter() - t_begin < 8.0 and len(ts) < 20):
+        ts.append(oracle_step(w, h, Bs))
+    cpu_sec = sum(ts) / len(ts)
+
+    line = base_line(w, args, world)
+    line.update({
+        "value": tokens / (ms_step * 1e-3), "ms_per_step": ms_step, "ms_per_step_min": min(ms),
+        "tflops": flops / (ms_step * 1e-3) / 1e12,
+        "frac_of_bf16_peak": flops / (ms_step * 1e-3) / 1e12 / (peaks["bf16_tflops"] * world),
+        "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(x_pin.numel() * x_pin.element_size()),
+                "d2h_bytes_per_step": int(y_pin.numel() * y_pin.element_size())},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roof,
+        "kernels": kern,
+        "cpu_baseline": {"value": Bs * w.L_valid / cpu_sec, "unit": "tokens/s", "cores": blas_threads(),
+                         "kind": "oracle", "sec_per_step": cpu_sec,
+                         "sample": f"first {Bs} of {w.B} samples, whole block, {len(ts)} steps"},
+    })
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="cfg2_lm", choices=sorted(gen.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    w = gen.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w, rank, world)
+    else:
+        run_ours(args, w, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,51 @@
+"""One UoE transformer block as a sequence of C-ABI calls with preallocated buffers.
+
+u = SMHA(h) (router, Eq. 27-36), out = UoME(u) (router, Eq. 37-40): each sub-block has its own router,
+as in Section III-C.  Nothing is computed here; the class only owns device buffers and issues the calls.
+"""
+from __future__ import annotations
+
+import torch
+
+from . import binding as B
+
+
+class UoEBlock:
+    def __init__(self, prob_att: B.Problem | None, prob_mlp: B.Problem | None, weights: dict, device="cuda",
+                 save_h: bool = False):
+        self.pa, self.pm, self.w = prob_att, prob_mlp, weights
+        p0 = prob_att or prob_mlp
+        self.u = torch.empty(p0.B, p0.L, p0.d, dtype=p0.torch_dtype, device=device)
+        self.out = torch.empty_like(self.u)
+        if prob_att is not None:
+            self.ra = B.alloc_routing(prob_att, device)
+            self.ws_ra = B.alloc_workspace(prob_att, B.UOE_OP_ROUTE, device)
+            self.ws_a = B.alloc_workspace(prob_att, B.UOE_OP_SMHA_FWD, device)
+        if prob_mlp is not None:
+            self.rm = B.alloc_routing(prob_mlp, device)
+            self.ws_rm = B.alloc_workspace(prob_mlp, B.UOE_OP_ROUTE, device)
+            self.ws_m = B.alloc_workspace(prob_mlp, B.UOE_OP_MLP_FWD, device)
+            self.saved_h = B.alloc_saved_h(prob_mlp, device) if save_h else None
+
+    def forward(self, h: torch.Tensor, check: bool = False) -> torch.Tensor:
+        w = self.w
+        cur = h
+        if self.pa is not None:
+            B.uoe_route(self.pa, cur, w["Wr_att"], out=self.ra, ws=self.ws_ra, check=check)
+            B.uoe_smha_forward(self.pa, cur, w["Wq"], w["Wk"], w["Wv"], w["Wo"], self.ra, y=self.u, ws=self.ws_a,
+                               check=check)
+            cur = self.u
+        if self.pm is not None:
+            B.uoe_route(self.pm, cur, w["Wr_mlp"], out=self.rm, ws=self.ws_rm, check=check)
+            B.uoe_mlp_forward(self.pm, cur, w["W1"], w["W2"], self.rm, y=self.out, saved_h=self.saved_h,
+                              ws=self.ws_m, check=check)
+            cur = self.out
+        return cur
+
+    def device_status(self) -> int:
+        worst = 0
+        for name in ("ws_ra", "ws_a", "ws_rm", "ws_m"):
+            ws = getattr(self, name, None)
+            if ws is not None:
+                worst = max(worst, B.uoe_read_device_status(ws))
+        return worst
