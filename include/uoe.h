@@ -46,7 +46,8 @@ typedef enum {
     UOE_ERR_WORKSPACE = 3,     /* ws_bytes smaller than uoe_workspace_bytes */
     UOE_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed */
     UOE_ERR_TIMEOUT = 5,       /* device status: a bounded wait inside a kernel ran out */
-    UOE_ERR_DEVICE_INDEX = 6   /* device status: a routing index was out of range */
+    UOE_ERR_DEVICE_INDEX = 6,  /* device status: a routing index was out of range */
+    UOE_ERR_STATIC_SCRATCH = 7 /* uoe_route_static: the problem needs more scratch than the built-in array holds */
 } uoe_status;
 
 typedef enum { UOE_F32 = 0, UOE_BF16 = 1 } uoe_dtype;
@@ -160,6 +161,37 @@ uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, const void* 
                             const int32_t* expert_idx, const int32_t* patch_idx, const float* gate,
                             const int32_t* expert_offsets, void* y /* [B,L,d] */, float* lse,
                             void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * uoe_route without a workspace argument and without any allocation.  (The paper has no counterpart;
+ * this exists for callers that cannot hand the library device memory of their own.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a region that must not
+ * synchronise the device or touch the allocator (a latency-critical serving loop, a plugin hosted by
+ * a framework that owns all device memory and offers no way to request scratch, start-up code that
+ * runs before the host application's memory pool exists).  Such a caller can pass its inputs and
+ * outputs but has nowhere to get the extra buffer that uoe_route needs for its partial scores.
+ *
+ * Here that buffer is a fixed array of UOE_ROUTE_STATIC_SCRATCH_BYTES compiled into the library's
+ * device image, so every GPU on which the library is loaded holds that many bytes until the process
+ * exits.  Results are identical to uoe_route.  Arguments are as for uoe_route, minus ws / ws_bytes.
+ *
+ *   - Limit: the problem must satisfy uoe_workspace_bytes(prob, UOE_OP_ROUTE) <=
+ *     UOE_ROUTE_STATIC_SCRATCH_BYTES; otherwise nothing is launched and UOE_ERR_STATIC_SCRATCH is returned.
+ *   - The first call on each device looks up the array's device address (a one-time set-up step, done
+ *     with that device current).  Make that first call before starting any stream capture.
+ *   - The function calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - All calls on a device share the one array, which still holds what the previous call left; the
+ *     counters that must start at zero are cleared on the stream at the start of every call.  Two calls
+ *     whose kernels may overlap on the GPU (different streams, no ordering between them) race on the
+ *     array and give wrong routing: order them, or use uoe_route with separate workspaces.
+ *   - No device status word is kept for this variant (uoe_read_device_status does not apply).
+ */
+#define UOE_ROUTE_STATIC_SCRATCH_BYTES (1 << 20)
+uoe_status uoe_route_static(const uoe_problem* prob, const void* x, const void* W_r,
+                            int32_t* expert_idx /* [B,k] */, int32_t* patch_idx /* [B,k,c] */,
+                            float* gate /* [B,k,c] */, float* p_samp /* [B,n] */, float* p_patch /* [B,n,m] */,
+                            int32_t* expert_offsets /* [n+1] */, void* cuda_stream);
 
 /* Text for a status code (static storage). */
 const char* uoe_status_string(int status);

@@ -87,6 +87,8 @@ def _load():
     lib.uoe_workspace_bytes.argtypes = [pp, ctypes.c_int]
     lib.uoe_route.restype = ctypes.c_int
     lib.uoe_route.argtypes = [pp, vp, vp, i32p, i32p, f32p, f32p, f32p, i32p, vp, sz, vp]
+    lib.uoe_route_static.restype = ctypes.c_int
+    lib.uoe_route_static.argtypes = [pp, vp, vp, i32p, i32p, f32p, f32p, f32p, i32p, vp]
     lib.uoe_mlp_forward.restype = ctypes.c_int
     lib.uoe_mlp_forward.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, f32p, i32p, vp, vp, vp, sz, vp]
     lib.uoe_mlp_backward.restype = ctypes.c_int
@@ -206,6 +208,23 @@ def uoe_route(prob: Problem, x, W_r, out: Routing | None = None, ws=None, check:
     _check(st, "uoe_route")
     if check:
         _check(uoe_read_device_status(ws), "uoe_route (device)")
+    return r
+
+
+UOE_ROUTE_STATIC_SCRATCH_BYTES = 1 << 20
+
+
+def uoe_route_static(prob: Problem, x, W_r, out: Routing | None = None) -> Routing:
+    """uoe_route for callers that cannot supply a workspace: the scratch is a fixed array inside the
+    library (limit UOE_ROUTE_STATIC_SCRATCH_BYTES).  Only the output tensors are created here, and only
+    when `out` is not given; the C call itself allocates nothing.  Calls on one device must not overlap."""
+    _contig(x, prob.torch_dtype)
+    _contig(W_r, prob.torch_dtype)
+    r = out if out is not None else alloc_routing(prob, x.device)
+    st = _lib.uoe_route_static(ctypes.byref(prob.c_struct()), _ptr(x), _ptr(W_r), _ptr(r.expert_idx),
+                               _ptr(r.patch_idx), _ptr(r.gate), _ptr(r.p_samp), _ptr(r.p_patch),
+                               _ptr(r.expert_offsets), _stream())
+    _check(st, "uoe_route_static")
     return r
 
 

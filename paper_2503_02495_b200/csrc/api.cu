@@ -70,6 +70,7 @@ extern "C" const char* uoe_status_string(int status) {
         case UOE_ERR_CUDA: return "CUDA call failed";
         case UOE_ERR_TIMEOUT: return "device wait timed out";
         case UOE_ERR_DEVICE_INDEX: return "routing index out of range";
+        case UOE_ERR_STATIC_SCRATCH: return "problem too large for the built-in static scratch of uoe_route_static";
         default: return "unknown status";
     }
 }

@@ -252,3 +252,66 @@ extern "C" uoe_status uoe_route(const uoe_problem* prob, const void* x, const vo
     UOE_LAUNCHED();
     return UOE_OK;
 }
+
+// ------------------------------------------------------------------------------------------------
+// uoe_route_static: the same two kernels with their scratch in a built-in device array
+// ------------------------------------------------------------------------------------------------
+
+// Scratch of uoe_route_static: the status block (ticket, expert loads) followed by the partial dot
+// products.  One copy per GPU that loads the library, held until the process exits.
+static __device__ __align__(256) unsigned char g_route_static_scratch[UOE_ROUTE_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+unsigned char* g_route_static_ptr[kMaxDevices] = {};    // device address of the array, per device
+
+// In host code `g_route_static_scratch` is only a handle; the address a kernel can use comes from
+// cudaGetSymbolAddress, asked once per device with that device current.
+uoe_status route_static_base(unsigned char** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return UOE_ERR_CUDA;
+    if (!g_route_static_ptr[dev]) {
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_route_static_scratch) != cudaSuccess || !p) return UOE_ERR_CUDA;
+        g_route_static_ptr[dev] = (unsigned char*)p;
+    }
+    *out = g_route_static_ptr[dev];
+    return UOE_OK;
+}
+}  // namespace
+
+extern "C" uoe_status uoe_route_static(const uoe_problem* prob, const void* x, const void* W_r,
+                                       int32_t* expert_idx, int32_t* patch_idx, float* gate, float* p_samp,
+                                       float* p_patch, int32_t* expert_offsets, void* cuda_stream) {
+    Dims D;
+    uoe_status st = make_dims(prob, D);
+    if (st != UOE_OK) return st;
+    if (!x || !W_r || !expert_idx || !patch_idx || !gate || !p_samp || !p_patch || !expert_offsets)
+        return UOE_ERR_INVALID_ARG;
+    if (!aligned16(x)) return UOE_ERR_INVALID_ARG;
+    if ((size_t)D.n * D.m * sizeof(float) > 40 * 1024) return UOE_ERR_UNSUPPORTED;
+    const RouteWs W = route_ws(D);
+    if (W.nchunks > 65535) return UOE_ERR_UNSUPPORTED;
+    if (W.total > (size_t)UOE_ROUTE_STATIC_SCRATCH_BYTES) return UOE_ERR_STATIC_SCRATCH;
+    unsigned char* base = nullptr;
+    st = route_static_base(&base);
+    if (st != UOE_OK) return st;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    int* status = (int*)base;
+    // the array keeps the previous call's ticket and expert loads: they must start at zero
+    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
+    float* partial = (float*)(base + W.partial);
+    dim3 grid(D.B * D.m, W.nchunks);
+    if (D.bf16)
+        route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, 0, stream>>>(
+            (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
+    else
+        route_score_kernel<float><<<grid, kScoreThreads, 0, stream>>>(
+            (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
+    UOE_LAUNCHED();
+    route_select_kernel<<<D.B, kSelectThreads, (size_t)D.n * D.m * sizeof(float), stream>>>(
+        partial, W.nchunks, D.B, D.Lv, D.n, D.k, D.m, D.c, D.l_p, (prob->flags & UOE_FLAG_GATE) ? 1 : 0,
+        expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, status + 8, status + 1);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
