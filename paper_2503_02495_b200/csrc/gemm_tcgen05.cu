@@ -37,13 +37,14 @@ struct Ctl {                       // lives behind the stage ring
     int offs[34];
 };
 
-template <int BN, bool B_KMAJOR>
+template <int BN, bool B_KMAJOR, bool BWD>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
                  __nv_bfloat16* __restrict__ C0, __nv_bfloat16* __restrict__ C1, __nv_bfloat16* __restrict__ C2,
                  __nv_bfloat16* __restrict__ pre, const int* __restrict__ offsets,
-                 int n, int K, int N, int nmat, int act, int* status) {
+                 int n, int K, int N, int nmat, int act, int* status, const __nv_bfloat16* __restrict__ bwd_h,
+                 const float* __restrict__ row_gate, const float* __restrict__ row_valid, float* __restrict__ dg_part) {
     using Cf = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -153,36 +154,64 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             tc_fence_after();
             const size_t row = (size_t)row0 + quarter * 32 + lane;
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+            auto pack8 = [](const float* f) {
+                uint4 w;
+                w.x = pack_bf16x2(f[0], f[1]); w.y = pack_bf16x2(f[2], f[3]);
+                w.z = pack_bf16x2(f[4], f[5]); w.w = pack_bf16x2(f[6], f[7]);
+                return w;
+            };
+            if constexpr (BWD) {
+                const float rg = row_gate[row], rv = row_valid[row];
+                float dsum = 0.f;
 #pragma unroll 1
-            for (int ch = 0; ch < BN / 32; ++ch) {
-                uint32_t v[32];
-                tmem_ld32(taddr + ch * 32, v);
-                tmem_ld_wait();
-                uint4* out = (uint4*)(C + row * N + col0 + ch * 32);
-                if (pre) {
-                    uint4* po = (uint4*)(pre + row * N + col0 + ch * 32);
+                for (int ch = 0; ch < BN / 32; ++ch) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + ch * 32, v);
+                    const uint4* hp = (const uint4*)(bwd_h + row * N + col0 + ch * 32);
+                    uint4 hv[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) hv[q] = hp[q];
+                    tmem_ld_wait();
+                    uint4* o_dh = (uint4*)(C + row * N + col0 + ch * 32);
+                    uint4* o_ag = (uint4*)(C1 + row * N + col0 + ch * 32);
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
-                        uint4 w;
-                        w.x = pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1]));
-                        w.y = pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3]));
-                        w.z = pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5]));
-                        w.w = pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7]));
-                        po[q] = w;
+                        float hh[8], dh[8], ag[8];
+                        unpack16<__nv_bfloat16>(hv[q], hh);
+#pragma unroll
+                        for (int t = 0; t < 8; ++t) {
+                            const float u = __uint_as_float(v[8 * q + t]);
+                            const float a = act_apply(hh[t], act);
+                            dsum = fmaf(u, a, dsum);
+                            dh[t] = rg * u * act_deriv(hh[t], act);
+                            ag[t] = rg * a;
+                        }
+                        o_dh[q] = pack8(dh);
+                        o_ag[q] = pack8(ag);
                     }
                 }
-                if (act != UOE_ACT_IDENTITY) {
+                dg_part[row * n_tiles_mat + (col0 / BN)] = rv * dsum;
+            } else {
+#pragma unroll 1
+                for (int ch = 0; ch < BN / 32; ++ch) {
+                    uint32_t v[32];
+                    tmem_ld32(taddr + ch * 32, v);
+                    tmem_ld_wait();
+                    float f[32];
 #pragma unroll
-                    for (int q = 0; q < 32; ++q) v[q] = __float_as_uint(act_apply(__uint_as_float(v[q]), act));
-                }
+                    for (int q = 0; q < 32; ++q) f[q] = __uint_as_float(v[q]);
+                    if (pre) {
+                        uint4* po = (uint4*)(pre + row * N + col0 + ch * 32);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    uint4 w;
-                    w.x = pack_bf16x2(__uint_as_float(v[8 * q + 0]), __uint_as_float(v[8 * q + 1]));
-                    w.y = pack_bf16x2(__uint_as_float(v[8 * q + 2]), __uint_as_float(v[8 * q + 3]));
-                    w.z = pack_bf16x2(__uint_as_float(v[8 * q + 4]), __uint_as_float(v[8 * q + 5]));
-                    w.w = pack_bf16x2(__uint_as_float(v[8 * q + 6]), __uint_as_float(v[8 * q + 7]));
-                    out[q] = w;
+                        for (int q = 0; q < 4; ++q) po[q] = pack8(f + 8 * q);
+                    }
+                    if (act != UOE_ACT_IDENTITY) {
+#pragma unroll
+                        for (int q = 0; q < 32; ++q) f[q] = act_apply(f[q], act);
+                    }
+                    uint4* out = (uint4*)(C + row * N + col0 + ch * 32);
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) out[q] = pack8(f + 8 * q);
                 }
             }
             tc_fence_before();
@@ -198,11 +227,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
-template <int BN, bool B_KMAJOR>
+template <int BN, bool B_KMAJOR, bool BWD>
 uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     using Cf = Cfg<BN>;
     static bool attr_set = false;
-    auto kern = gemm_bf16_kernel<BN, B_KMAJOR>;
+    auto kern = gemm_bf16_kernel<BN, B_KMAJOR, BWD>;
     if (!attr_set) {
         UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
         attr_set = true;
@@ -235,7 +264,8 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     ProfScope ps(g.label, s);
     kern<<<grid, kGemmThreads, Cf::SMEM, s>>>(tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
                                               (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
-                                              nmat, g.act, status);
+                                              nmat, g.act, status, (const __nv_bfloat16*)g.bwd_h, g.row_gate, g.row_valid,
+                                              g.dg_part);
     UOE_LAUNCHED();
     return UOE_OK;
 }
@@ -246,15 +276,22 @@ uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s) {
     if (g.K % BK != 0 || g.N % 64 != 0 || g.bias || g.nmat > 3) return UOE_ERR_UNSUPPORTED;
     if (g.nmat > 1 && g.pre) return UOE_ERR_UNSUPPORTED;
     if (g.rows_max % BM != 0) return UOE_ERR_INVALID_ARG;
-    const int bn = (g.N % 256 == 0) ? 256 : (g.N % 128 == 0 ? 128 : 64);
-    if (g.b_kmajor) {
-        if (bn == 256) return launch_one<256, true>(g, status, s);
-        if (bn == 128) return launch_one<128, true>(g, status, s);
-        return launch_one<64, true>(g, status, s);
+    const int bn = gemm_bf16_bn(g.N);
+    if (g.bwd) {          // backward epilogue: weights are read K-major ([n, N, K])
+        if (!g.b_kmajor || !g.bwd_h || !g.row_gate || !g.row_valid || !g.dg_part || !g.C1 || g.nmat > 1)
+            return UOE_ERR_INVALID_ARG;
+        if (bn == 256) return launch_one<256, true, true>(g, status, s);
+        if (bn == 128) return launch_one<128, true, true>(g, status, s);
+        return launch_one<64, true, true>(g, status, s);
     }
-    if (bn == 256) return launch_one<256, false>(g, status, s);
-    if (bn == 128) return launch_one<128, false>(g, status, s);
-    return launch_one<64, false>(g, status, s);
+    if (g.b_kmajor) {
+        if (bn == 256) return launch_one<256, true, false>(g, status, s);
+        if (bn == 128) return launch_one<128, true, false>(g, status, s);
+        return launch_one<64, true, false>(g, status, s);
+    }
+    if (bn == 256) return launch_one<256, false, false>(g, status, s);
+    if (bn == 128) return launch_one<128, false, false>(g, status, s);
+    return launch_one<64, false, false>(g, status, s);
 }
 
 }  // namespace uoe

@@ -16,11 +16,14 @@ struct PlanPtrs {
     int* inv_row;      // [B,m,k]  first routed row of patch j in slot s, or -1
     float* inv_gate;   // [B,m,k]
     int* expert_end;   // [n]      first padding row of expert i's region
+    float* row_gate;   // [Rmax]   backward only: combine weight of each routed row (0 on pad-token rows and unused slots)
+    float* row_valid;  // [Rmax]   backward only: 1 on rows that hold a real token, else 0
 };
-inline size_t plan_bytes(const Dims& D) {
-    return align_up((size_t)D.B * D.k * 4, 1024) + 2 * align_up((size_t)D.B * D.m * D.k * 4, 1024) + 1024;
+inline size_t plan_bytes(const Dims& D, bool with_rows = false) {
+    return align_up((size_t)D.B * D.k * 4, 1024) + 2 * align_up((size_t)D.B * D.m * D.k * 4, 1024) + 1024 +
+           (with_rows ? 2 * align_up((size_t)D.Rmax * 4, 1024) : 0);
 }
-inline PlanPtrs plan_ptrs(const Dims& D, char* base) {
+inline PlanPtrs plan_ptrs(const Dims& D, char* base, bool with_rows = false) {
     PlanPtrs p;
     p.pair_row = (int*)base;
     base += align_up((size_t)D.B * D.k * 4, 1024);
@@ -29,11 +32,16 @@ inline PlanPtrs plan_ptrs(const Dims& D, char* base) {
     p.inv_gate = (float*)base;
     base += align_up((size_t)D.B * D.m * D.k * 4, 1024);
     p.expert_end = (int*)base;
+    base += 1024;
+    p.row_gate = with_rows ? (float*)base : nullptr;
+    base += with_rows ? align_up((size_t)D.Rmax * 4, 1024) : 0;
+    p.row_valid = with_rows ? (float*)base : nullptr;
     return p;
 }
 
+// use_gate only matters for the per-row arrays of the backward (row_gate = gate or 1).
 uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_idx, const float* gate,
-                       const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s);
+                       const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s, bool use_gate = true);
 
 // Eq. 18 / 24: copy the selected patches of `src` [B,L,d] into the routed buffer `dst` [rows,d];
 // unused slots and the padding rows of each expert region are zero-filled.
@@ -44,8 +52,11 @@ uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, c
 
 // Eq. 20 / 26 / 36 / 40: y[b,t,:] = (residual ? x[b,t,:] : 0) + sum_s w_s * z[row_s(t),:], every output row
 // written once, contributions added in ascending slot order.  w_s = gate if use_gate else 1.
+// If G is not null (backward through the router), every real token of patch (b,j) also receives
+// sum_i W_r[:, i] * G[b, j, i]   (G [B, m, n] float32, W_r [d, n] in the element type).
 uoe_status launch_combine(const Dims& D, const void* x, const void* z, const PlanPtrs& P, bool residual,
-                          bool use_gate, void* y, cudaStream_t s);
+                          bool use_gate, void* y, cudaStream_t s, const float* G = nullptr,
+                          const void* W_r = nullptr);
 
 // Grouped GEMM over the routed rows: C[r,:] = epilogue(A[r,:] @ W[e(r)]) where e(r) is the expert whose
 // region holds row r.  W is [n, K, N] (b_kmajor = false: rows of K, N contiguous) or [n, N, K] (true).
@@ -68,7 +79,26 @@ struct GemmArgs {
     void* C1 = nullptr;
     void* C2 = nullptr;
     const char* label = "gemm";   // name under which the launch is profiled
+    // bf16 path, backward epilogue (bwd = true): with u = A @ W (the gradient w.r.t. the activation output,
+    // before the gate), h = bwd_h[r,:] the saved pre-activation:
+    //   C  [r,:] = row_gate[r] * u * phi'(h)         (gradient w.r.t. the pre-activation)
+    //   C1 [r,:] = row_gate[r] * phi(h)              (gated activation, operand of the weight gradient)
+    //   dg_part[r, column tile] = row_valid[r] * sum over the tile's columns of u * phi(h)
+    bool bwd = false;
+    const void* bwd_h = nullptr;
+    const float* row_gate = nullptr;
+    const float* row_valid = nullptr;
+    float* dg_part = nullptr;
 };
+
+// Column-tile width the bf16 grouped GEMM uses for N output columns (dg_part has N / that many columns).
+inline int gemm_bf16_bn(int N) { return (N % 256 == 0) ? 256 : (N % 128 == 0 ? 128 : 64); }
+
+// Per-expert weight gradient over ragged row counts:  dW[e] [M, N] (float32, overwritten) =
+// sum over the rows r of expert e's region of  P[r, 0:M]^T  Q[r, 0:N]   (P [rows, M], Q [rows, N], bf16).
+// Rows of a region beyond its real rows must be zero in P or Q.
+uoe_status launch_wgrad_bf16(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
+                             long long rows_max, const char* label, int* status, cudaStream_t s);
 uoe_status launch_gemm_f32(const GemmArgs& g, cudaStream_t s);
 uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s);
 

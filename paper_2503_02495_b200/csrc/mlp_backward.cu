@@ -1,8 +1,162 @@
-// uoe_mlp_backward (derivative of Eq. 38-40 with the selection held constant).
+// uoe_mlp_backward: gradients of sum(y * dy) for y = uoe_mlp_forward(x, ...) with the selection held
+// constant (derivative of Eq. 38-40; with gating also of Eq. 14 and 21 through the gate weights).
+//
+// In routed-row space, for a row r of expert i with combine weight w_r, saved pre-activation h_r:
+//   u_r  = dy_r A^O_i^T                      grouped GEMM (K-major weights), epilogue produces
+//   dh_r = w_r u_r * phi'(h_r)               -> buffer dh
+//   ag_r = w_r phi(h_r)                      -> buffer ag
+//   dgate(slab) = sum_r <u_r, phi(h_r)>      -> per-row partials, reduced per (sample, expert, patch)
+//   dA^O_i = ag^T dy_g,  dA^I_i = x_g^T dh   ragged-K weight-gradient GEMMs
+//   dx_g = dh A^I_i^T                        grouped GEMM, then combined back with unit weights
+// Router: dgate -> dP_samp, dP_patch -> softmax Jacobians -> per-(sample, patch) logit gradient G, which
+// feeds dW_r (through the pooled token sums) and one more term of dx.
 #include "kernels.cuh"
 
 namespace uoe {
-size_t mlp_bwd_workspace_bytes(const Dims& D) { (void)D; return 0; }
+namespace {
+
+constexpr int kThreads = 256;
+
+// grid B, 128 threads, dynamic smem 2*n*m floats.  G[b,j,i] = dlogit_patch[b,i,j]/cnt_j + dlogit_samp[b,i]/L_valid.
+__global__ void __launch_bounds__(128)
+router_bwd_kernel(const float* __restrict__ dg_part, int nt, const int* __restrict__ pair_row,
+                  const int* __restrict__ expert_idx, const int* __restrict__ patch_idx,
+                  const float* __restrict__ p_samp, const float* __restrict__ p_patch, int n, int k, int m, int c,
+                  int l_p, int Lv, float* __restrict__ G) {
+    extern __shared__ float sm[];
+    float* pp = sm;                 // [n][m] patch gate
+    float* dpp = sm + n * m;        // [n][m] its gradient
+    __shared__ float ps[32], dps[32], dls[32];
+    __shared__ float red[4];
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    for (int idx = tid; idx < n * m; idx += 128) { pp[idx] = p_patch[(size_t)b * n * m + idx]; dpp[idx] = 0.f; }
+    if (tid < n) { ps[tid] = p_samp[(size_t)b * n + tid]; dps[tid] = 0.f; }
+    __syncthreads();
+    // dgate of every selected (expert, patch) of this sample, summed in a fixed order
+    for (int su = 0; su < k * c; ++su) {
+        const int s = su / c, u = su % c;
+        const int j = patch_idx[((size_t)b * k + s) * c + u];
+        if (j < 0 || j >= m) continue;                    // uniform across the block
+        const int i = expert_idx[(size_t)b * k + s];
+        const float* src = dg_part + ((size_t)pair_row[b * k + s] + (size_t)u * l_p) * nt;
+        float a = 0.f;
+        for (int q = tid; q < l_p * nt; q += 128) a += src[q];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        if (lane == 0) red[warp] = a;
+        __syncthreads();
+        if (tid == 0) {
+            const float dg = (red[0] + red[1]) + (red[2] + red[3]);
+            dps[i] += dg * pp[i * m + j];                 // gate = P_samp * P_patch
+            dpp[i * m + j] += dg * ps[i];
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {                                       // softmax Jacobian of the sample gate (Eq. 21)
+        float dot = 0.f;
+        for (int i = 0; i < n; ++i) dot += ps[i] * dps[i];
+        for (int i = 0; i < n; ++i) dls[i] = ps[i] * (dps[i] - dot);
+    }
+    __syncthreads();
+    for (int j = tid; j < m; j += 128) {                  // softmax Jacobian of each patch gate (Eq. 14)
+        const int cnt = max(0, min(l_p, Lv - j * l_p));
+        float dot = 0.f;
+        for (int i = 0; i < n; ++i) dot += pp[i * m + j] * dpp[i * m + j];
+        for (int i = 0; i < n; ++i) {
+            const float dlp = pp[i * m + j] * (dpp[i * m + j] - dot);
+            G[((size_t)b * m + j) * n + i] = cnt > 0 ? dlp / (float)cnt + dls[i] / (float)Lv : 0.f;
+        }
+    }
+}
+
+// grid (B*m, column chunks): sum of the real rows of each patch, float32 [B*m, d]
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+pool_kernel(const T* __restrict__ x, float* __restrict__ pool, int L, int Lv, int d, int m, int l_p, int CT) {
+    constexpr int V = Vec16<T>::N;
+    __shared__ float red[kThreads * V];
+    const int bj = blockIdx.x, chunk = blockIdx.y, b = bj / m, j = bj % m;
+    const int ct = threadIdx.x % CT, rt = threadIdx.x / CT, RT = kThreads / CT;
+    const int col = (chunk * CT + ct) * V;
+    const int rows = max(0, min(l_p, Lv - j * l_p));
+    float cs[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) cs[v] = 0.f;
+    if (col < d) {
+        const T* base = x + ((size_t)b * L + (size_t)j * l_p) * d + col;
+        for (int r = rt; r < rows; r += RT) {
+            float f[V];
+            unpack16<T>(ld_stream16(base + (size_t)r * d), f);
+#pragma unroll
+            for (int v = 0; v < V; ++v) cs[v] += f[v];
+        }
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) red[(rt * CT + ct) * V + v] = cs[v];
+    __syncthreads();
+    if (rt == 0 && col < d) {
+        for (int q = 1; q < RT; ++q)
+#pragma unroll
+            for (int v = 0; v < V; ++v) cs[v] += red[(q * CT + ct) * V + v];
+#pragma unroll
+        for (int v = 0; v < V; ++v) pool[(size_t)bj * d + col + v] = cs[v];
+    }
+}
+
+// dW_r[dd, i] = sum over (b, j) of pool[bj, dd] * G[bj, i]; one thread per dd, fixed order over bj
+__global__ void __launch_bounds__(kThreads)
+dwr_kernel(const float* __restrict__ pool, const float* __restrict__ G, float* __restrict__ dW_r, int BM, int d, int n) {
+    __shared__ float sG[64 * 32];
+    const int dd = blockIdx.x * kThreads + threadIdx.x;
+    float acc[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) acc[i] = 0.f;
+    for (int b0 = 0; b0 < BM; b0 += 64) {
+        const int nb = min(64, BM - b0);
+        __syncthreads();
+        for (int q = threadIdx.x; q < nb * n; q += kThreads) sG[q] = G[(size_t)b0 * n + q];
+        __syncthreads();
+        if (dd < d) {
+            for (int q = 0; q < nb; ++q) {
+                const float p = pool[(size_t)(b0 + q) * d + dd];
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (i < n) acc[i] = fmaf(p, sG[q * n + i], acc[i]);
+            }
+        }
+    }
+    if (dd < d) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i < n) dW_r[(size_t)dd * n + i] = acc[i];
+    }
+}
+
+struct BwdWs { size_t plan, dyg, xg, dh, ag, dxg, dgp, G, pool, total; int nt; };
+
+BwdWs bwd_ws(const Dims& D) {
+    WsCarver w;
+    w.take(kStatusBytes);
+    BwdWs r;
+    r.nt = D.d_e / gemm_bf16_bn(D.d_e > 0 ? D.d_e : 64);
+    if (r.nt < 1) r.nt = 1;
+    r.plan = w.take(plan_bytes(D, true));
+    r.dyg = w.take((size_t)D.Rmax * D.d * D.esize);
+    r.xg = w.take((size_t)D.Rmax * D.d * D.esize);
+    r.dh = w.take((size_t)D.Rmax * D.d_e * D.esize);
+    r.ag = w.take((size_t)D.Rmax * D.d_e * D.esize);
+    r.dxg = w.take((size_t)D.Rmax * D.d * D.esize);
+    r.dgp = w.take((size_t)D.Rmax * r.nt * sizeof(float));
+    r.G = w.take((size_t)D.B * D.m * D.n * sizeof(float));
+    r.pool = w.take((size_t)D.B * D.m * D.d * sizeof(float));
+    r.total = w.off;
+    return r;
+}
+
+}  // namespace
+
+size_t mlp_bwd_workspace_bytes(const Dims& D) { return bwd_ws(D).total; }
+
 }  // namespace uoe
 
 using namespace uoe;
@@ -13,8 +167,80 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
                                        const float* p_patch, const void* saved_h, const void* dy, void* dx,
                                        float* dW1, float* dW2, float* dW_r, void* ws, size_t ws_bytes,
                                        void* cuda_stream) {
-    (void)prob; (void)x; (void)W1; (void)W2; (void)W_r; (void)expert_idx; (void)patch_idx; (void)gate;
-    (void)expert_offsets; (void)p_samp; (void)p_patch; (void)saved_h; (void)dy; (void)dx; (void)dW1; (void)dW2;
-    (void)dW_r; (void)ws; (void)ws_bytes; (void)cuda_stream;
-    return UOE_ERR_UNSUPPORTED;
+    Dims D;
+    uoe_status st = make_dims(prob, D);
+    if (st != UOE_OK) return st;
+    if (!x || !W1 || !W2 || !W_r || !expert_idx || !patch_idx || !gate || !expert_offsets || !p_samp || !p_patch ||
+        !saved_h || !dy || !dx || !dW1 || !dW2 || !dW_r || !ws)
+        return UOE_ERR_INVALID_ARG;
+    if (D.d_e < 1) return UOE_ERR_INVALID_ARG;
+    const void* al[] = {x, W1, W2, saved_h, dy, dx, dW1, dW2, ws};
+    for (const void* p : al)
+        if (!aligned16(p)) return UOE_ERR_INVALID_ARG;
+    // tensor-core path only: bf16, widths that tile the 128-row weight-gradient MMA
+    if (!D.bf16 || D.d % 128 != 0 || D.d_e % 128 != 0) return UOE_ERR_UNSUPPORTED;
+    if ((size_t)2 * D.n * D.m * sizeof(float) > 40 * 1024) return UOE_ERR_UNSUPPORTED;
+    const BwdWs W = bwd_ws(D);
+    if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const bool use_gate = (prob->flags & UOE_FLAG_GATE) != 0;
+    const bool residual = (prob->flags & UOE_FLAG_RESIDUAL) != 0;
+    char* base = (char*)ws;
+    int* status = (int*)base;
+    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
+    const PlanPtrs P = plan_ptrs(D, base + W.plan, true);
+    // rows of the per-row weights that belong to no pair (region padding) must read as zero
+    UOE_CUDA_OK(cudaMemsetAsync(P.row_gate, 0, 2 * align_up((size_t)D.Rmax * 4, 1024), stream));
+    void *dyg = base + W.dyg, *xg = base + W.xg, *dh = base + W.dh, *ag = base + W.ag, *dxg = base + W.dxg;
+    float* dgp = (float*)(base + W.dgp);
+    float* G = (float*)(base + W.G);
+    float* pool = (float*)(base + W.pool);
+
+    st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream, use_gate);
+    if (st != UOE_OK) return st;
+    st = launch_gather(D, dy, patch_idx, expert_offsets, P, dyg, stream);
+    if (st != UOE_OK) return st;
+    st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
+    if (st != UOE_OK) return st;
+
+    GemmArgs ga{dyg, W2, nullptr, dh, nullptr, expert_offsets, D.n, D.d, D.d_e, prob->act, true, D.Rmax};
+    ga.label = "bwd_da_dh";
+    ga.bwd = true; ga.bwd_h = saved_h; ga.row_gate = P.row_gate; ga.row_valid = P.row_valid; ga.dg_part = dgp; ga.C1 = ag;
+    st = launch_gemm_bf16(ga, status, stream);
+    if (st != UOE_OK) return st;
+    st = launch_wgrad_bf16(ag, dyg, dW2, expert_offsets, D.n, D.d_e, D.d, D.Rmax, "wgrad_W2", status, stream);
+    if (st != UOE_OK) return st;
+    GemmArgs gx{dh, W1, nullptr, dxg, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, true, D.Rmax};
+    gx.label = "bwd_dx";
+    st = launch_gemm_bf16(gx, status, stream);
+    if (st != UOE_OK) return st;
+    st = launch_wgrad_bf16(xg, dh, dW1, expert_offsets, D.n, D.d, D.d_e, D.Rmax, "wgrad_W1", status, stream);
+    if (st != UOE_OK) return st;
+
+    if (use_gate) {
+        {
+            ProfScope ps("router_bwd", stream);
+            router_bwd_kernel<<<D.B, 128, (size_t)2 * D.n * D.m * sizeof(float), stream>>>(
+                dgp, W.nt, P.pair_row, expert_idx, patch_idx, p_samp, p_patch, D.n, D.k, D.m, D.c, D.l_p, D.Lv, G);
+        }
+        UOE_LAUNCHED();
+        int CT = 64;
+        while (CT > 1 && (CT / 2) * 8 >= D.d) CT /= 2;
+        dim3 grid(D.B * D.m, (D.d + CT * 8 - 1) / (CT * 8));
+        {
+            ProfScope ps("pool", stream);
+            pool_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>((const __nv_bfloat16*)x, pool, D.L, D.Lv, D.d,
+                                                                      D.m, D.l_p, CT);
+        }
+        UOE_LAUNCHED();
+        {
+            ProfScope ps("dW_r", stream);
+            dwr_kernel<<<(D.d + kThreads - 1) / kThreads, kThreads, 0, stream>>>(pool, G, dW_r, D.B * D.m, D.d, D.n);
+        }
+        UOE_LAUNCHED();
+    } else {
+        UOE_CUDA_OK(cudaMemsetAsync(dW_r, 0, (size_t)D.d * D.n * sizeof(float), stream));
+    }
+    // dx = dy (selective residual) + the routed input gradients (the gate is already inside dh) + router term
+    return launch_combine(D, dy, dxg, P, residual, false, dx, stream, use_gate ? G : nullptr, W_r);
 }

@@ -14,7 +14,8 @@ __global__ void __launch_bounds__(128)
 plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_idx, const float* __restrict__ gate,
             const int* __restrict__ offsets, int B, int n, int k, int m, int c, int l_p,
             int* __restrict__ pair_row, int* __restrict__ inv_row, float* __restrict__ inv_gate,
-            int* __restrict__ expert_end, int* status) {
+            int* __restrict__ expert_end, int* status, float* __restrict__ row_gate, float* __restrict__ row_valid,
+            int Lv, int use_gate) {
     __shared__ int my_e[32], cnt[32], prow[32];
     const int b = blockIdx.x, tid = threadIdx.x;
     const int l_a = c * l_p;
@@ -54,6 +55,16 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
         int load = 0;
         for (int idx = 0; idx < B * k; ++idx) load += (expert_idx[idx] == tid);
         expert_end[tid] = offsets[tid] + load * l_a;
+    }
+    if (row_gate) {                          // per-row weights for the backward
+        for (int idx = tid; idx < k * l_a; idx += 128) {
+            const int s = idx / l_a, r = idx % l_a, u = r / l_p;
+            const int pj = patch_idx[((size_t)b * k + s) * c + u];
+            const bool real = pj >= 0 && pj < m && pj * l_p + (r % l_p) < Lv;
+            const float g = use_gate ? gate[((size_t)b * k + s) * c + u] : 1.0f;
+            row_gate[prow[s] + r] = real ? g : 0.f;
+            row_valid[prow[s] + r] = real ? 1.f : 0.f;
+        }
     }
 }
 
@@ -111,16 +122,19 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __restrict__ inv_row,
                const float* __restrict__ inv_gate, T* __restrict__ y, int L, int Lv, int d, int m, int k,
-               int l_p, int residual, int use_gate, int rows_per_cta) {
+               int l_p, int residual, int use_gate, int rows_per_cta, const float* __restrict__ G,
+               const T* __restrict__ W_r, int n) {
     constexpr int V = Vec16<T>::N;
     __shared__ int srow[32];
     __shared__ float sg[32];
+    __shared__ float sG[32];
     const int bj = blockIdx.x, b = bj / m, j = bj % m;
     const int r0 = blockIdx.y * rows_per_cta, r1 = min(l_p, r0 + rows_per_cta);
     if (threadIdx.x < k) {
         srow[threadIdx.x] = inv_row[(size_t)bj * k + threadIdx.x];
         sg[threadIdx.x] = use_gate ? inv_gate[(size_t)bj * k + threadIdx.x] : 1.0f;
     }
+    if (G && threadIdx.x < n) sG[threadIdx.x] = G[(size_t)bj * n + threadIdx.x];
     __syncthreads();
     const int vpr = d / V;
     const int total = (r1 - r0) * vpr;
@@ -143,6 +157,13 @@ combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __re
                 const float g = sg[s];
 #pragma unroll
                 for (int v = 0; v < V; ++v) acc[v] = fmaf(g, f[v], acc[v]);
+            }
+            if (G) {
+                for (int i = 0; i < n; ++i) {
+                    const float gi = sG[i];
+#pragma unroll
+                    for (int v = 0; v < V; ++v) acc[v] = fmaf(gi, to_f32(W_r[(size_t)(cv * V + v) * n + i]), acc[v]);
+                }
             }
         }
         st_stream16(y + xo, pack16<T>(acc));
@@ -215,10 +236,11 @@ gemm_f32_kernel(const float* __restrict__ A, const float* __restrict__ W, const 
 }  // namespace
 
 uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_idx, const float* gate,
-                       const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s) {
+                       const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s, bool use_gate) {
     ProfScope ps("plan", s);
     plan_kernel<<<D.B, 128, 0, s>>>(expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
-                                    P.pair_row, P.inv_row, P.inv_gate, P.expert_end, status);
+                                    P.pair_row, P.inv_row, P.inv_gate, P.expert_end, status, P.row_gate, P.row_valid,
+                                    D.Lv, use_gate ? 1 : 0);
     UOE_LAUNCHED();
     return UOE_OK;
 }
@@ -241,7 +263,7 @@ uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, c
 }
 
 uoe_status launch_combine(const Dims& D, const void* x, const void* z, const PlanPtrs& P, bool residual,
-                          bool use_gate, void* y, cudaStream_t s) {
+                          bool use_gate, void* y, cudaStream_t s, const float* G, const void* W_r) {
     int rows_per_cta = (int)(32768 / ((long long)D.d * D.esize));
     if (rows_per_cta < 1) rows_per_cta = 1;
     if (rows_per_cta > D.l_p) rows_per_cta = D.l_p;
@@ -250,11 +272,11 @@ uoe_status launch_combine(const Dims& D, const void* x, const void* z, const Pla
     if (D.bf16)
         combine_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)z, P.inv_row, P.inv_gate, (__nv_bfloat16*)y, D.L, D.Lv,
-            D.d, D.m, D.k, D.l_p, residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta);
+            D.d, D.m, D.k, D.l_p, residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, G, (const __nv_bfloat16*)W_r, D.n);
     else
         combine_kernel<float><<<grid, kThreads, 0, s>>>((const float*)x, (const float*)z, P.inv_row, P.inv_gate,
                                                        (float*)y, D.L, D.Lv, D.d, D.m, D.k, D.l_p,
-                                                       residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta);
+                                                       residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, G, (const float*)W_r, D.n);
     UOE_LAUNCHED();
     return UOE_OK;
 }

@@ -1,0 +1,208 @@
+// Per-expert weight gradients on the tcgen05 tensor cores (derivative of Eq. 38-39 with respect to
+// A^I_i and A^O_i):   dW[e] [M, N] = P_e^T Q_e,   P_e [rows_e, M], Q_e [rows_e, N] the rows of expert e's
+// region in two routed buffers.  The contraction runs over the ragged row count of each expert, so both
+// operands are "MN-major" for the MMA: a K step is 64 consecutive rows, each row contributing 128 bytes
+// (64 elements) per swizzled box.
+//
+// Persistent CTAs walk (expert, 128-row tile of M, BN-column tile of N); warp roles and the two-buffer
+// TMEM accumulator are the same as in the forward grouped GEMM.  The output is float32 and overwritten;
+// an expert with no rows gets zeros.
+#include "kernels.cuh"
+#include "tc.cuh"
+#include "tmap.cuh"
+
+namespace uoe {
+namespace {
+
+using namespace tc;
+
+constexpr int BM = 128, BK = 64;
+constexpr int kThreads = 192;
+constexpr int A_BYTES = BM * BK * 2;
+
+template <int BN> struct WCfg {
+    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int STAGE = A_BYTES + B_BYTES;
+    static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int TMEM_COLS = 2 * BN;
+    static constexpr int SMEM = STAGES * STAGE + 1024 + 512;
+};
+
+struct WCtl {
+    uint64_t full[8], empty[8], tfull[2], tempty[2];
+    uint32_t tmem_base;
+    int abort_flag;
+    int offs[34];
+};
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CUtensorMap tmQ,
+             float* __restrict__ dW, const int* __restrict__ offsets, int n, int M, int N, int* status) {
+    using Cf = WCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    WCtl* ctl = (WCtl*)(smem + Cf::STAGES * Cf::STAGE);
+    volatile int* abort_flag = &ctl->abort_flag;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < Cf::STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 128); }
+        ctl->abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tmap(&tmP);
+        prefetch_tmap(&tmQ);
+    }
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + n + 1) ctl->offs[threadIdx.x - 64] = offsets[threadIdx.x - 64];
+    if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    const int m_tiles = M / BM, n_tiles = N / BN;
+    const int per_expert = m_tiles * n_tiles;
+    const int total_tiles = n * per_expert;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0, issued = 0, issued_parity = 0;
+            bool stop = false;
+            for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+                const int e = tile / per_expert, rem = tile % per_expert;
+                const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
+                const int r0 = ctl->offs[e], num_kb = (ctl->offs[e + 1] - r0) / BK;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) || *abort_flag) { stop = true; break; }
+                    uint8_t* sa = smem + stage * Cf::STAGE;
+                    uint8_t* sb = sa + A_BYTES;
+                    mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
+#pragma unroll
+                    for (int q = 0; q < BM / 64; ++q)
+                        tma_load_2d(sa + q * 8192, &tmP, m0 + q * 64, r0 + kb * BK, &ctl->full[stage]);
+#pragma unroll
+                    for (int q = 0; q < BN / 64; ++q)
+                        tma_load_2d(sb + q * 8192, &tmQ, n0 + q * 64, r0 + kb * BK, &ctl->full[stage]);
+                    issued |= 1u << stage;
+                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                    if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
+                }
+            }
+            if (*abort_flag) {
+                for (int s = 0; s < Cf::STAGES; ++s)
+                    if (issued & (1u << s)) mbar_wait(&ctl->full[s], (issued_parity >> s) & 1, abort_flag, status);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_bf16(BM, BN, true, true);
+            int stage = 0, acc = 0;
+            uint32_t phase = 0, acc_phase = 0;
+            bool stop = false;
+            for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+                const int e = tile / per_expert;
+                const int num_kb = (ctl->offs[e + 1] - ctl->offs[e]) / BK;
+                if (!mbar_wait(&ctl->tempty[acc], acc_phase ^ 1, abort_flag, status) || *abort_flag) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < num_kb; ++kb) {
+                    if (!mbar_wait(&ctl->full[stage], phase, abort_flag, status) || *abort_flag) { stop = true; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + stage * Cf::STAGE);
+                    const uint32_t sb = sa + A_BYTES;
+#pragma unroll
+                    for (int ks = 0; ks < BK / 16; ++ks)
+                        mma_bf16(d_tmem, smem_desc(sa + ks * 2048, 8192, 1024), smem_desc(sb + ks * 2048, 8192, 1024),
+                                 idesc, (kb | ks) != 0);
+                    mma_commit(&ctl->empty[stage]);
+                    if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
+                }
+                if (stop) break;
+                mma_commit(&ctl->tfull[acc]);
+                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            }
+        }
+    } else {
+        const int quarter = warp & 3;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+            const int e = tile / per_expert, rem = tile % per_expert;
+            const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
+            const int num_kb = (ctl->offs[e + 1] - ctl->offs[e]) / BK;
+            const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
+            if (!__all_sync(0xffffffffu, ready)) break;
+            tc_fence_after();
+            float* out = dW + ((size_t)e * M + m0 + quarter * 32 + lane) * N + n0;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+#pragma unroll 1
+            for (int ch = 0; ch < BN / 32; ++ch) {
+                uint32_t v[32];
+                if (num_kb > 0) {
+                    tmem_ld32(taddr + ch * 32, v);
+                    tmem_ld_wait();
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 32; ++q) v[q] = 0u;
+                }
+                uint4* o4 = (uint4*)(out + ch * 32);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) o4[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+            }
+            tc_fence_before();
+            mbar_arrive(&ctl->tempty[acc]);
+            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tmem_dealloc(tmem_base, Cf::TMEM_COLS);
+    }
+}
+
+template <int BN>
+uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
+                    long long rows_max, const char* label, int* status, cudaStream_t s) {
+    using Cf = WCfg<BN>;
+    static bool attr_set = false;
+    auto kern = wgrad_kernel<BN>;
+    if (!attr_set) {
+        UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
+        attr_set = true;
+    }
+    CUtensorMap tmP, tmQ;
+    const uint32_t box[2] = {64, BK};
+    {
+        const uint64_t dims[2] = {(uint64_t)M, (uint64_t)rows_max};
+        const uint64_t str[1] = {(uint64_t)M * 2};
+        if (!make_tmap(&tmP, P, 2, dims, str, box)) return UOE_ERR_CUDA;
+    }
+    {
+        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)rows_max};
+        const uint64_t str[1] = {(uint64_t)N * 2};
+        if (!make_tmap(&tmQ, Q, 2, dims, str, box)) return UOE_ERR_CUDA;
+    }
+    const long long tiles = (long long)n * (M / BM) * (N / BN);
+    int grid = (int)(tiles < sm_count() ? tiles : sm_count());
+    ProfScope ps(label, s);
+    kern<<<grid, kThreads, Cf::SMEM, s>>>(tmP, tmQ, dW, offsets, n, M, N, status);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
+
+}  // namespace
+
+uoe_status launch_wgrad_bf16(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
+                             long long rows_max, const char* label, int* status, cudaStream_t s) {
+    if (M % BM != 0 || N % 64 != 0) return UOE_ERR_UNSUPPORTED;
+    const int bn = gemm_bf16_bn(N);
+    if (bn == 256) return launch_w<256>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
+    if (bn == 128) return launch_w<128>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
+    return launch_w<64>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
+}
+
+}  // namespace uoe
