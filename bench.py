@@ -62,6 +62,12 @@ def work_table(w: gen.Workload):
         de = w.d_e
         t["gemm1_act"] = dict(flops=2 * R * d * de, bytes=(R * d + R * de + n * d * de) * s)
         t["gemm2"] = dict(flops=2 * R * de * d, bytes=(R * de + R * d + n * d * de) * s)
+    if w.d_ff and w.backward:
+        de = w.d_e
+        for name in ("bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2"):
+            t[name] = dict(flops=2 * R * d * de, bytes=(R * d + 2 * R * de + n * d * de) * s)
+        t["wgrad_W1"]["bytes"] = t["wgrad_W2"]["bytes"] = (R * d + R * de) * s + n * d * de * 4
+        t["pool"] = dict(flops=0, bytes=x_bytes)
     if w.H:
         dg = w.d_g
         att = 4 * w.l_a * w.l_a * dg * w.B * w.k
@@ -76,6 +82,8 @@ def step_flops(w: gen.Workload) -> int:
     f = 0
     if w.d_ff:
         f += t["gemm1_act"]["flops"] + t["gemm2"]["flops"]
+    if w.d_ff and w.backward:
+        f += sum(t[k]["flops"] for k in ("bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2"))
     if w.H:
         f += t["qkv_proj"]["flops"] + t["attention"]["flops"] + t["out_proj"]["flops"]
     return f
@@ -93,6 +101,8 @@ def host_inputs(w: gen.Workload):
     if w.d_ff:
         d["Wr_mlp"] = gen.make_router(w, "mlp")
         d["W1"], d["W2"] = gen.make_mlp_weights(w)
+    if w.backward:
+        d["dy"] = gen.make_dy(w)
     return d
 
 
@@ -108,7 +118,10 @@ def oracle_step(w: gen.Workload, h, B=None):
         cur = orc.smha_forward(cur, h["Wq"].f64, h["Wk"].f64, h["Wv"].f64, h["Wo"].f64, r, w.d_h, w.causal)
     if w.d_ff:
         r = orc.route(cur, h["Wr_mlp"].f64, w.k, w.m, w.c, L_valid=w.L_valid)
-        cur = orc.mlp_forward(cur, h["W1"].f64, h["W2"].f64, r, w.act)
+        u = cur
+        cur = orc.mlp_forward(u, h["W1"].f64, h["W2"].f64, r, w.act)
+        if w.backward:
+            orc.mlp_backward(u, h["W1"].f64, h["W2"].f64, h["Wr_mlp"].f64, r, h["dy"].f64[:B], w.act)
     return time.perf_counter() - t0
 
 
@@ -193,7 +206,7 @@ def base_line(w: gen.Workload, args, n_gpus: int):
         "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "stands_in_for": w.stands_in_for, "B": w.B, "L": w.L, "L_valid": w.L_valid,
                    "d": w.d, "n": w.n, "k": w.k, "m": w.m, "c": w.c, "d_ff": w.d_ff, "heads": w.H, "d_h": w.d_h,
-                   "causal": w.causal, "act": w.act, "blocks": ("smha+" if w.H else "") + ("uome" if w.d_ff else ""),
+                   "causal": w.causal, "act": w.act, "blocks": ("smha+" if w.H else "") + ("uome" if w.d_ff else "") + ("+uome_backward" if w.backward else ""),
                    "parallelism": f"replicas x{n_gpus}" if n_gpus > 1 else "single gpu",
                    "l2": "flushed between timed steps (512 MB write)"},
     }
@@ -233,9 +246,18 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
         dist.init_process_group("nccl", device_id=dev)
 
     h = host_inputs(w)
-    wd = {k: to_dev(v, dev) for k, v in h.items() if k != "x"}
+    wd = {k: to_dev(v, dev) for k, v in h.items() if k not in ("x", "dy")}
     x_dev = to_dev(h["x"], dev)
-    blk = UoEBlock(problem_of(w, "att") if w.H else None, problem_of(w, "mlp") if w.d_ff else None, wd, dev)
+    dy_dev = to_dev(h["dy"], dev) if w.backward else None
+    blk = UoEBlock(problem_of(w, "att") if w.H else None, problem_of(w, "mlp") if w.d_ff else None, wd, dev,
+                   backward=w.backward)
+
+    def step(xin):
+        out = blk.forward(xin)
+        if w.backward:
+            blk.mlp_backward(xin, dy_dev)
+            return blk.dx
+        return out
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
@@ -245,7 +267,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
         torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
-        blk.forward(x_dev)
+        step(x_dev)
     torch.cuda.synchronize()
     st = blk.device_status()
     if st != 0:
@@ -260,7 +282,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
     for e0, e1 in ev:
         flush.zero_()
         e0.record(stream)
-        blk.forward(x_dev)
+        step(x_dev)
         e1.record(stream)
     barrier()
     launches = uoe.uoe_launch_count() - launches0
@@ -279,7 +301,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         x_in.view(x_pin.dtype).copy_(x_pin, non_blocking=True)
-        out = blk.forward(x_in)
+        out = step(x_in)
         y_pin.copy_(out.view(x_pin.dtype), non_blocking=True)
         torch.cuda.synchronize()
         if i >= 2:
@@ -290,7 +312,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
     uoe.uoe_profile_enable(True)
     for _ in range(min(args.steps, 20)):
         flush.zero_()
-        blk.forward(x_dev)
+        step(x_dev)
     torch.cuda.synchronize()
     uoe.uoe_profile_enable(False)
     recs = uoe.uoe_profile_records()

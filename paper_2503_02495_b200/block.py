@@ -12,7 +12,7 @@ from . import binding as B
 
 class UoEBlock:
     def __init__(self, prob_att: B.Problem | None, prob_mlp: B.Problem | None, weights: dict, device="cuda",
-                 save_h: bool = False):
+                 save_h: bool = False, backward: bool = False):
         self.pa, self.pm, self.w = prob_att, prob_mlp, weights
         p0 = prob_att or prob_mlp
         self.u = torch.empty(p0.B, p0.L, p0.d, dtype=p0.torch_dtype, device=device)
@@ -25,7 +25,15 @@ class UoEBlock:
             self.rm = B.alloc_routing(prob_mlp, device)
             self.ws_rm = B.alloc_workspace(prob_mlp, B.UOE_OP_ROUTE, device)
             self.ws_m = B.alloc_workspace(prob_mlp, B.UOE_OP_MLP_FWD, device)
-            self.saved_h = B.alloc_saved_h(prob_mlp, device) if save_h else None
+            self.saved_h = B.alloc_saved_h(prob_mlp, device) if (save_h or backward) else None
+            self.backward = backward
+            if backward:          # UoME backward buffers (Eq. 38-40 differentiated)
+                f32 = torch.float32
+                self.ws_b = B.alloc_workspace(prob_mlp, B.UOE_OP_MLP_BWD, device)
+                self.dx = torch.empty_like(self.u)
+                self.dW1 = torch.empty(weights["W1"].shape, dtype=f32, device=device)
+                self.dW2 = torch.empty(weights["W2"].shape, dtype=f32, device=device)
+                self.dWr = torch.empty(weights["Wr_mlp"].shape, dtype=f32, device=device)
 
     def forward(self, h: torch.Tensor, check: bool = False) -> torch.Tensor:
         w = self.w
@@ -42,9 +50,15 @@ class UoEBlock:
             cur = self.out
         return cur
 
+    def mlp_backward(self, h: torch.Tensor, dy: torch.Tensor, check: bool = False):
+        """Backward of the UoME half for the routing and saved pre-activations of the last forward(h)."""
+        w = self.w
+        return B.uoe_mlp_backward(self.pm, h, w["W1"], w["W2"], w["Wr_mlp"], self.rm, self.saved_h, dy, dx=self.dx,
+                                  dW1=self.dW1, dW2=self.dW2, dW_r=self.dWr, ws=self.ws_b, check=check)
+
     def device_status(self) -> int:
         worst = 0
-        for name in ("ws_ra", "ws_a", "ws_rm", "ws_m"):
+        for name in ("ws_ra", "ws_a", "ws_rm", "ws_m", "ws_b"):
             ws = getattr(self, name, None)
             if ws is not None:
                 worst = max(worst, B.uoe_read_device_status(ws))
