@@ -48,12 +48,11 @@ def test_scale_workload_forward_and_backward():
     ro1 = orc.with_selection(x.f64[b:b + 1], Wr.f64, e_gpu[b:b + 1], p_gpu[b:b + 1], w.m, w.L_valid)
     y_ref = orc.mlp_forward(x.f64[b:b + 1], W1.f64, W2.f64, ro1, w.act)
     assert rel_inf(to_f64(y[b]), y_ref[0]) <= TOL
-    assert rel_inf(to_f64(y[b]) - x.f64[b], y_ref[0] - x.f64[b]) <= 0.5      # y is rounded to bf16 around x
     dx_ref, _, _, dWr_ref1, _ = orc.mlp_backward(x.f64[b:b + 1], W1.f64, W2.f64, Wr.f64, ro1, dy.f64[b:b + 1], w.act)
     assert rel_inf(to_f64(dx[b]), dx_ref[0]) <= TOL
-    assert rel_inf(to_f64(dx[b]) - dy.f64[b], dx_ref[0] - dy.f64[b]) <= TOL       # the part that is not dy itself
 
-    # expert term alone (residual off) for the same sample, single-sample GPU calls
+    # y and dx are bf16 roundings of x + (small) and dy + (small): the small parts are compared with the
+    # residual off, in single-sample GPU calls
     prob1 = problem_of(w.replace(B=1), "mlp", residual=False)
     acc_dWr = torch.zeros_like(dWr)
     for bb in range(w.B):
