@@ -151,6 +151,29 @@ __device__ __forceinline__ float act_apply(float h, int act) {
     }
 }
 
+// phi applied in place to N values with the selection made once (keeps unrolled epilogues small)
+template <int N>
+__device__ __forceinline__ void act_apply_n(float* f, int act) {
+    switch (act) {
+        case UOE_ACT_GELU_ERF:
+#pragma unroll
+            for (int q = 0; q < N; ++q) f[q] = 0.5f * f[q] * (1.0f + erff(f[q] * 0.70710678118654752f));
+            break;
+        case UOE_ACT_GELU_TANH:
+#pragma unroll
+            for (int q = 0; q < N; ++q) {
+                const float u = 0.79788456080286536f * (f[q] + 0.044715f * f[q] * f[q] * f[q]);
+                f[q] = 0.5f * f[q] * (1.0f + tanhf(u));
+            }
+            break;
+        case UOE_ACT_SILU:
+#pragma unroll
+            for (int q = 0; q < N; ++q) f[q] = __fdividef(f[q], 1.0f + __expf(-f[q]));
+            break;
+        default: break;
+    }
+}
+
 __device__ __forceinline__ float act_deriv(float h, int act) {
     switch (act) {
         case UOE_ACT_GELU_ERF: {

@@ -205,10 +205,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
                         for (int q = 0; q < 4; ++q) po[q] = pack8(f + 8 * q);
                     }
-                    if (act != UOE_ACT_IDENTITY) {
-#pragma unroll
-                        for (int q = 0; q < 32; ++q) f[q] = act_apply(f[q], act);
-                    }
+                    act_apply_n<32>(f, act);
                     uint4* out = (uint4*)(C + row * N + col0 + ch * 32);
 #pragma unroll
                     for (int q = 0; q < 4; ++q) out[q] = pack8(f + 8 * q);

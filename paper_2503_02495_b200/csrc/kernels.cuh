@@ -52,11 +52,10 @@ uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, c
 
 // Eq. 20 / 26 / 36 / 40: y[b,t,:] = (residual ? x[b,t,:] : 0) + sum_s w_s * z[row_s(t),:], every output row
 // written once, contributions added in ascending slot order.  w_s = gate if use_gate else 1.
-// If G is not null (backward through the router), every real token of patch (b,j) also receives
-// sum_i W_r[:, i] * G[b, j, i]   (G [B, m, n] float32, W_r [d, n] in the element type).
+// If rvec is not null (backward through the router), every real token of patch (b,j) also receives the
+// vector rvec[b*m + j, :]  (float32 [B*m, d]).
 uoe_status launch_combine(const Dims& D, const void* x, const void* z, const PlanPtrs& P, bool residual,
-                          bool use_gate, void* y, cudaStream_t s, const float* G = nullptr,
-                          const void* W_r = nullptr);
+                          bool use_gate, void* y, cudaStream_t s, const float* rvec = nullptr);
 
 // Grouped GEMM over the routed rows: C[r,:] = epilogue(A[r,:] @ W[e(r)]) where e(r) is the expert whose
 // region holds row r.  W is [n, K, N] (b_kmajor = false: rows of K, N contiguous) or [n, N, K] (true).

@@ -103,6 +103,21 @@ pool_kernel(const T* __restrict__ x, float* __restrict__ pool, int L, int Lv, in
     }
 }
 
+// rvec[bj, dd] = sum_i W_r[dd, i] * G[bj, i]: what the router path adds to dx for every real token of patch bj
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+rvec_kernel(const T* __restrict__ W_r, const float* __restrict__ G, float* __restrict__ rvec, int d, int n) {
+    __shared__ float sG[32];
+    const int bj = blockIdx.x;
+    if (threadIdx.x < n) sG[threadIdx.x] = G[(size_t)bj * n + threadIdx.x];
+    __syncthreads();
+    for (int dd = threadIdx.x; dd < d; dd += kThreads) {
+        float a = 0.f;
+        for (int i = 0; i < n; ++i) a = fmaf(to_f32(W_r[(size_t)dd * n + i]), sG[i], a);
+        rvec[(size_t)bj * d + dd] = a;
+    }
+}
+
 // dW_r[dd, i] = sum over (b, j) of pool[bj, dd] * G[bj, i]; one thread per dd, fixed order over bj
 __global__ void __launch_bounds__(kThreads)
 dwr_kernel(const float* __restrict__ pool, const float* __restrict__ G, float* __restrict__ dW_r, int BM, int d, int n) {
@@ -132,7 +147,7 @@ dwr_kernel(const float* __restrict__ pool, const float* __restrict__ G, float* _
     }
 }
 
-struct BwdWs { size_t plan, dyg, xg, dh, ag, dxg, dgp, G, pool, total; int nt; };
+struct BwdWs { size_t plan, dyg, xg, dh, ag, dxg, dgp, G, pool, rvec, total; int nt; };
 
 BwdWs bwd_ws(const Dims& D) {
     WsCarver w;
@@ -149,6 +164,7 @@ BwdWs bwd_ws(const Dims& D) {
     r.dgp = w.take((size_t)D.Rmax * r.nt * sizeof(float));
     r.G = w.take((size_t)D.B * D.m * D.n * sizeof(float));
     r.pool = w.take((size_t)D.B * D.m * D.d * sizeof(float));
+    r.rvec = w.take((size_t)D.B * D.m * D.d * sizeof(float));
     r.total = w.off;
     return r;
 }
@@ -195,6 +211,7 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
     float* dgp = (float*)(base + W.dgp);
     float* G = (float*)(base + W.G);
     float* pool = (float*)(base + W.pool);
+    float* rvec = (float*)(base + W.rvec);
 
     st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream, use_gate);
     if (st != UOE_OK) return st;
@@ -238,9 +255,14 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
             dwr_kernel<<<(D.d + kThreads - 1) / kThreads, kThreads, 0, stream>>>(pool, G, dW_r, D.B * D.m, D.d, D.n);
         }
         UOE_LAUNCHED();
+        {
+            ProfScope ps("router_dx_vec", stream);
+            rvec_kernel<__nv_bfloat16><<<D.B * D.m, kThreads, 0, stream>>>((const __nv_bfloat16*)W_r, G, rvec, D.d, D.n);
+        }
+        UOE_LAUNCHED();
     } else {
         UOE_CUDA_OK(cudaMemsetAsync(dW_r, 0, (size_t)D.d * D.n * sizeof(float), stream));
     }
     // dx = dy (selective residual) + the routed input gradients (the gate is already inside dh) + router term
-    return launch_combine(D, dy, dxg, P, residual, false, dx, stream, use_gate ? G : nullptr, W_r);
+    return launch_combine(D, dy, dxg, P, residual, false, dx, stream, use_gate ? rvec : nullptr);
 }

@@ -17,16 +17,30 @@ constexpr int kScoreThreads = 256;
 constexpr int kSelectThreads = 128;
 
 // grid (B*m, nchunks).  CT threads span the columns of a chunk (16 bytes each), 256/CT span rows.
+// Dynamic shared memory: the W_r rows of this chunk, CT*V*n elements.
 template <typename T>
 __global__ void __launch_bounds__(kScoreThreads)
 route_score_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ partial,
                    int L, int Lv, int d, int n, int m, int l_p, int CT, int nchunks) {
     constexpr int V = Vec16<T>::N;
+    extern __shared__ uint4 s_w4[];                   // W_r[c0 : c0+cw, :] as stored
+    __shared__ float s_cs[kScoreThreads * V];         // per-thread column sums, later the partial dot products
+    __shared__ float s_col[64 * V];                   // column sums of the chunk
+    const T* s_w = (const T*)s_w4;
     const int bj = blockIdx.x, chunk = blockIdx.y;
     const int b = bj / m, j = bj % m;
-    const int ct = threadIdx.x % CT, rt = threadIdx.x / CT, RT = kScoreThreads / CT;
-    const int col = (chunk * CT + ct) * V;
+    const int tid = threadIdx.x;
+    const int ct = tid % CT, rt = tid / CT, RT = kScoreThreads / CT;
+    const int c0 = chunk * CT * V;
+    const int cw = min(CT * V, d - c0);               // columns of this chunk (a multiple of V)
+    const int col = c0 + ct * V;
     const int rows = max(0, min(l_p, Lv - j * l_p));
+
+    {   // stage the router rows of this chunk: cw*n elements, contiguous and 16-byte aligned
+        const uint4* src = (const uint4*)(W_r + (size_t)c0 * n);
+        const int nvec = cw * n / V;
+        for (int q = tid; q < nvec; q += kScoreThreads) s_w4[q] = src[q];
+    }
 
     float cs[V];
 #pragma unroll
@@ -34,12 +48,12 @@ route_score_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __
     if (col < d) {
         const T* base = x + ((size_t)b * L + (size_t)j * l_p) * d + col;
         int r = rt;
-        for (; r + 3 * RT < rows; r += 4 * RT) {
-            uint4 q[4];
+        for (; r + 7 * RT < rows; r += 8 * RT) {
+            uint4 q[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) q[u] = ld_stream16(base + (size_t)(r + u * RT) * d);
+            for (int u = 0; u < 8; ++u) q[u] = ld_stream16(base + (size_t)(r + u * RT) * d);
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
+            for (int u = 0; u < 8; ++u) {
                 float f[V];
                 unpack16<T>(q[u], f);
 #pragma unroll
@@ -53,25 +67,27 @@ route_score_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __
             for (int v = 0; v < V; ++v) cs[v] += f[v];
         }
     }
-
-    __shared__ float red[kScoreThreads / 32][32];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    for (int i = 0; i < n; ++i) {
+#pragma unroll
+    for (int v = 0; v < V; ++v) s_cs[tid * V + v] = cs[v];
+    __syncthreads();
+    for (int cc = tid; cc < cw; cc += kScoreThreads) {      // sum over the row threads, fixed order
         float a = 0.f;
-        if (col < d) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) a += cs[v] * to_f32(W_r[(size_t)(col + v) * n + i]);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-        if (lane == 0) red[warp][i] = a;
+        for (int q = 0; q < RT; ++q) a += s_cs[(q * CT + cc / V) * V + cc % V];
+        s_col[cc] = a;
     }
     __syncthreads();
-    if (threadIdx.x < n) {
-        float s = 0.f;
-#pragma unroll
-        for (int wv = 0; wv < kScoreThreads / 32; ++wv) s += red[wv][threadIdx.x];
-        partial[((size_t)bj * nchunks + chunk) * n + threadIdx.x] = s;
+    // dot products with the n router columns: thread (group g, expert i) strides over the chunk's columns
+    const int groups = kScoreThreads / n;
+    const int i = tid % n, g = tid / n;
+    float a = 0.f;
+    if (g < groups)
+        for (int cc = g; cc < cw; cc += groups) a = fmaf(s_col[cc], to_f32(s_w[cc * n + i]), a);
+    s_cs[tid] = a;
+    __syncthreads();
+    if (tid < n) {
+        float sum = 0.f;
+        for (int q = 0; q < groups; ++q) sum += s_cs[q * n + tid];
+        partial[((size_t)bj * nchunks + chunk) * n + tid] = sum;
     }
 }
 
@@ -224,7 +240,7 @@ extern "C" uoe_status uoe_route(const uoe_problem* prob, const void* x, const vo
     if (st != UOE_OK) return st;
     if (!x || !W_r || !expert_idx || !patch_idx || !gate || !p_samp || !p_patch || !expert_offsets || !ws)
         return UOE_ERR_INVALID_ARG;
-    if (!aligned16(x) || !aligned16(ws)) return UOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(W_r) || !aligned16(ws)) return UOE_ERR_INVALID_ARG;
     if ((size_t)D.n * D.m * sizeof(float) > 40 * 1024) return UOE_ERR_UNSUPPORTED;
     const RouteWs W = route_ws(D);
     if (W.nchunks > 65535) return UOE_ERR_UNSUPPORTED;
@@ -238,10 +254,10 @@ extern "C" uoe_status uoe_route(const uoe_problem* prob, const void* x, const vo
     {
     ProfScope ps("route_score", stream);
     if (D.bf16)
-        route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, 0, stream>>>(
+        route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
     else
-        route_score_kernel<float><<<grid, kScoreThreads, 0, stream>>>(
+        route_score_kernel<float><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
             (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
     }
     UOE_LAUNCHED();
@@ -288,7 +304,7 @@ extern "C" uoe_status uoe_route_static(const uoe_problem* prob, const void* x, c
     if (st != UOE_OK) return st;
     if (!x || !W_r || !expert_idx || !patch_idx || !gate || !p_samp || !p_patch || !expert_offsets)
         return UOE_ERR_INVALID_ARG;
-    if (!aligned16(x)) return UOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(W_r)) return UOE_ERR_INVALID_ARG;
     if ((size_t)D.n * D.m * sizeof(float) > 40 * 1024) return UOE_ERR_UNSUPPORTED;
     const RouteWs W = route_ws(D);
     if (W.nchunks > 65535) return UOE_ERR_UNSUPPORTED;
@@ -303,10 +319,10 @@ extern "C" uoe_status uoe_route_static(const uoe_problem* prob, const void* x, c
     float* partial = (float*)(base + W.partial);
     dim3 grid(D.B * D.m, W.nchunks);
     if (D.bf16)
-        route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, 0, stream>>>(
+        route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
     else
-        route_score_kernel<float><<<grid, kScoreThreads, 0, stream>>>(
+        route_score_kernel<float><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
             (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
     UOE_LAUNCHED();
     route_select_kernel<<<D.B, kSelectThreads, (size_t)D.n * D.m * sizeof(float), stream>>>(

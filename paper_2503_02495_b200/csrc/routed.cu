@@ -122,19 +122,16 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __restrict__ inv_row,
                const float* __restrict__ inv_gate, T* __restrict__ y, int L, int Lv, int d, int m, int k,
-               int l_p, int residual, int use_gate, int rows_per_cta, const float* __restrict__ G,
-               const T* __restrict__ W_r, int n) {
+               int l_p, int residual, int use_gate, int rows_per_cta, const float* __restrict__ rvec) {
     constexpr int V = Vec16<T>::N;
     __shared__ int srow[32];
     __shared__ float sg[32];
-    __shared__ float sG[32];
     const int bj = blockIdx.x, b = bj / m, j = bj % m;
     const int r0 = blockIdx.y * rows_per_cta, r1 = min(l_p, r0 + rows_per_cta);
     if (threadIdx.x < k) {
         srow[threadIdx.x] = inv_row[(size_t)bj * k + threadIdx.x];
         sg[threadIdx.x] = use_gate ? inv_gate[(size_t)bj * k + threadIdx.x] : 1.0f;
     }
-    if (G && threadIdx.x < n) sG[threadIdx.x] = G[(size_t)bj * n + threadIdx.x];
     __syncthreads();
     const int vpr = d / V;
     const int total = (r1 - r0) * vpr;
@@ -158,11 +155,12 @@ combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __re
 #pragma unroll
                 for (int v = 0; v < V; ++v) acc[v] = fmaf(g, f[v], acc[v]);
             }
-            if (G) {
-                for (int i = 0; i < n; ++i) {
-                    const float gi = sG[i];
+            if (rvec) {
+                const float* rp = rvec + (size_t)bj * d + (size_t)cv * V;
 #pragma unroll
-                    for (int v = 0; v < V; ++v) acc[v] = fmaf(gi, to_f32(W_r[(size_t)(cv * V + v) * n + i]), acc[v]);
+                for (int v = 0; v < V; v += 4) {
+                    const float4 q = *(const float4*)(rp + v);
+                    acc[v] += q.x; acc[v + 1] += q.y; acc[v + 2] += q.z; acc[v + 3] += q.w;
                 }
             }
         }
@@ -263,7 +261,7 @@ uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, c
 }
 
 uoe_status launch_combine(const Dims& D, const void* x, const void* z, const PlanPtrs& P, bool residual,
-                          bool use_gate, void* y, cudaStream_t s, const float* G, const void* W_r) {
+                          bool use_gate, void* y, cudaStream_t s, const float* rvec) {
     int rows_per_cta = (int)(32768 / ((long long)D.d * D.esize));
     if (rows_per_cta < 1) rows_per_cta = 1;
     if (rows_per_cta > D.l_p) rows_per_cta = D.l_p;
@@ -272,11 +270,11 @@ uoe_status launch_combine(const Dims& D, const void* x, const void* z, const Pla
     if (D.bf16)
         combine_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)z, P.inv_row, P.inv_gate, (__nv_bfloat16*)y, D.L, D.Lv,
-            D.d, D.m, D.k, D.l_p, residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, G, (const __nv_bfloat16*)W_r, D.n);
+            D.d, D.m, D.k, D.l_p, residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec);
     else
         combine_kernel<float><<<grid, kThreads, 0, s>>>((const float*)x, (const float*)z, P.inv_row, P.inv_gate,
                                                        (float*)y, D.L, D.Lv, D.d, D.m, D.k, D.l_p,
-                                                       residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, G, (const float*)W_r, D.n);
+                                                       residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec);
     UOE_LAUNCHED();
     return UOE_OK;
 }
