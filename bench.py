@@ -358,11 +358,13 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
 
     # ---- CPU baseline: the oracle as it stands, on a bounded sample ----
     Bs = cpu_sample_B(w)
-    oracle_step(w, h, Bs)
-    ts, t_begin = [], time.perf_counter()
-    while len(ts) < 3 or (time.perf_counter() - t_begin < 8.0 and len(ts) < 20):
-        ts.append(oracle_step(w, h, Bs))
-    cpu_sec = sum(ts) / len(ts)
+    ts = []
+    if not args.skip_cpu_baseline:
+        oracle_step(w, h, Bs)
+        t_begin = time.perf_counter()
+        while len(ts) < 3 or (time.perf_counter() - t_begin < 8.0 and len(ts) < 20):
+            ts.append(oracle_step(w, h, Bs))
+    cpu_sec = sum(ts) / len(ts) if ts else float("nan")
 
     line = base_line(w, args, world)
     line.update({
@@ -376,7 +378,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
         "clocks": clocks,
         "roofline": roof,
         "kernels": kern,
-        "cpu_baseline": {"value": Bs * w.L_valid / cpu_sec, "unit": "tokens/s", "cores": blas_threads(),
+        "cpu_baseline": {"value": (Bs * w.L_valid / cpu_sec) if ts else None, "unit": "tokens/s", "cores": blas_threads(),
                          "kind": "oracle", "sec_per_step": cpu_sec,
                          "sample": f"first {Bs} of {w.B} samples, whole block, {len(ts)} steps"},
     })
@@ -392,11 +394,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg2_lm", choices=sorted(gen.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (profiling on a smaller case)")
+    ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing (profiling runs)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     w = gen.WORKLOADS[args.workload]
+    if args.B > 0:
+        w = w.replace(B=args.B)
     if args.impl == "reference":
         run_reference(args, w, rank, world)
     else:
