@@ -212,6 +212,22 @@ def base_line(w: gen.Workload, args, n_gpus: int):
     }
 
 
+def max_over_ranks(values, world: int, device=None):
+    """Element-wise max of a list of floats over all ranks (the job is as slow as its slowest replica)."""
+    if world <= 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def job_throughput(w: gen.Workload, world: int, ms_per_step: float) -> float:
+    """Whole-job tokens/s of `world` replicas that each process the workload once per step."""
+    return w.B * w.L_valid * world / (ms_per_step * 1e-3)
+
+
 def run_reference(args, w: gen.Workload, rank: int, world: int):
     if rank != 0:
         return
@@ -320,10 +336,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
     for name, t in recs:
         per.setdefault(name, []).append(t)
 
-    if world > 1:
-        tt = torch.tensor([ms_step, e2e_ms], device=dev)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms_step, e2e_ms = float(tt[0]), float(tt[1])
+    ms_step, e2e_ms = max_over_ranks([ms_step, e2e_ms], world, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -368,7 +381,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
 
     line = base_line(w, args, world)
     line.update({
-        "value": tokens / (ms_step * 1e-3), "ms_per_step": ms_step, "ms_per_step_min": min(ms),
+        "value": job_throughput(w, world, ms_step), "ms_per_step": ms_step, "ms_per_step_min": min(ms),
         "tflops": flops / (ms_step * 1e-3) / 1e12,
         "frac_of_bf16_peak": flops / (ms_step * 1e-3) / 1e12 / (peaks["bf16_tflops"] * world),
         "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,

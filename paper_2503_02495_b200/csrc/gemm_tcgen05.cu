@@ -44,7 +44,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  __nv_bfloat16* __restrict__ C0, __nv_bfloat16* __restrict__ C1, __nv_bfloat16* __restrict__ C2,
                  __nv_bfloat16* __restrict__ pre, const int* __restrict__ offsets,
                  int n, int K, int N, int nmat, int act, int* status, const __nv_bfloat16* __restrict__ bwd_h,
-                 const float* __restrict__ row_gate, const float* __restrict__ row_valid, float* __restrict__ dg_part) {
+                 const float* __restrict__ row_gate, const float* __restrict__ row_valid, float* __restrict__ dg_part,
+                 const __grid_constant__ CUtensorMap tmX, const int* __restrict__ src_patch, int l_p, int Bm) {
     using Cf = Cfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -91,7 +92,16 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     uint8_t* sa = smem + stage * Cf::STAGE;
                     uint8_t* sb = sa + A_BYTES;
                     mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
-                    tma_load_2d(sa, &tmA, kb * BK, row0, &ctl->full[stage]);
+                    if (src_patch) {        // gather: one box per source patch, zero rows from an out-of-range patch
+                        const int nbox = BM / l_p;
+                        const int* sp = src_patch + (row0 / l_p);
+                        for (int q = 0; q < nbox; ++q) {
+                            const int src = sp[q];
+                            tma_load_3d(sa + q * l_p * 128, &tmX, kb * BK, 0, src >= 0 ? src : Bm, &ctl->full[stage]);
+                        }
+                    } else {
+                        tma_load_2d(sa, &tmA, kb * BK, row0, &ctl->full[stage]);
+                    }
                     if (B_KMAJOR) {
                         tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
                     } else {
@@ -233,12 +243,19 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
         UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
         attr_set = true;
     }
-    CUtensorMap tmA, tmB[3];
-    {
+    CUtensorMap tmA, tmB[3], tmX;
+    if (g.gather_x) {     // x as [Bm patches, l_p rows, K]; the 2-D map of A is unused
+        const uint64_t dims[3] = {(uint64_t)g.K, (uint64_t)g.l_p, (uint64_t)g.Bm};
+        const uint64_t str[2] = {(uint64_t)g.K * 2, (uint64_t)g.K * 2 * g.l_p};
+        const uint32_t box[3] = {BK, (uint32_t)g.l_p, 1};
+        if (!make_tmap(&tmX, g.gather_x, 3, dims, str, box)) return UOE_ERR_CUDA;
+        tmA = tmX;
+    } else {
         const uint64_t dims[2] = {(uint64_t)g.K, (uint64_t)g.rows_max};
         const uint64_t str[1] = {(uint64_t)g.K * 2};
         const uint32_t box[2] = {BK, BM};
         if (!make_tmap(&tmA, g.A, 2, dims, str, box)) return UOE_ERR_CUDA;
+        tmX = tmA;
     }
     const int nmat = g.nmat < 1 ? 1 : g.nmat;
     const void* Ws[3] = {g.W, g.W1 ? g.W1 : g.W, g.W2 ? g.W2 : g.W};
@@ -262,7 +279,7 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     kern<<<grid, kGemmThreads, Cf::SMEM, s>>>(tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
                                               (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
                                               nmat, g.act, status, (const __nv_bfloat16*)g.bwd_h, g.row_gate, g.row_valid,
-                                              g.dg_part);
+                                              g.dg_part, tmX, g.gather_x ? g.src_patch : nullptr, g.l_p, g.Bm);
     UOE_LAUNCHED();
     return UOE_OK;
 }
@@ -272,6 +289,7 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
 uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s) {
     if (g.K % BK != 0 || g.N % 64 != 0 || g.bias || g.nmat > 3) return UOE_ERR_UNSUPPORTED;
     if (g.nmat > 1 && g.pre) return UOE_ERR_UNSUPPORTED;
+    if (g.gather_x && (!g.src_patch || g.l_p < 8 || g.l_p % 8 != 0 || BM % g.l_p != 0)) return UOE_ERR_INVALID_ARG;
     if (g.rows_max % BM != 0) return UOE_ERR_INVALID_ARG;
     const int bn = gemm_bf16_bn(g.N);
     if (g.bwd) {          // backward epilogue: weights are read K-major ([n, N, K])

@@ -18,10 +18,16 @@ struct PlanPtrs {
     int* expert_end;   // [n]      first padding row of expert i's region
     float* row_gate;   // [Rmax]   backward only: combine weight of each routed row (0 on pad-token rows and unused slots)
     float* row_valid;  // [Rmax]   backward only: 1 on rows that hold a real token, else 0
+    int* src_patch;    // [Rmax/l_p] source patch (b*m + j) of every l_p-row block of the routed buffers, -1 = zero rows
 };
+// Gathering through the GEMM's own TMA loads needs whole patches inside a 128-row tile, 8-row swizzle groups
+// and 64-column K steps.
+inline bool can_fuse_gather(const Dims& D) {
+    return D.bf16 && D.l_p % 8 == 0 && 128 % D.l_p == 0 && D.d % 64 == 0;
+}
 inline size_t plan_bytes(const Dims& D, bool with_rows = false) {
     return align_up((size_t)D.B * D.k * 4, 1024) + 2 * align_up((size_t)D.B * D.m * D.k * 4, 1024) + 1024 +
-           (with_rows ? 2 * align_up((size_t)D.Rmax * 4, 1024) : 0);
+           (with_rows ? 2 * align_up((size_t)D.Rmax * 4, 1024) : 0) + align_up((size_t)(D.Rmax / D.l_p + 1) * 4, 1024);
 }
 inline PlanPtrs plan_ptrs(const Dims& D, char* base, bool with_rows = false) {
     PlanPtrs p;
@@ -36,12 +42,16 @@ inline PlanPtrs plan_ptrs(const Dims& D, char* base, bool with_rows = false) {
     p.row_gate = with_rows ? (float*)base : nullptr;
     base += with_rows ? align_up((size_t)D.Rmax * 4, 1024) : 0;
     p.row_valid = with_rows ? (float*)base : nullptr;
+    base += with_rows ? align_up((size_t)D.Rmax * 4, 1024) : 0;
+    p.src_patch = (int*)base;
     return p;
 }
 
 // use_gate only matters for the per-row arrays of the backward (row_gate = gate or 1).
+// If tail is not null, rows [offsets[n], Rmax) of tail (rows of tail_row_bytes) are zero-filled.
 uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_idx, const float* gate,
-                       const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s, bool use_gate = true);
+                       const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s, bool use_gate = true,
+                       void* tail = nullptr, long long tail_row_bytes = 0);
 
 // Eq. 18 / 24: copy the selected patches of `src` [B,L,d] into the routed buffer `dst` [rows,d];
 // unused slots and the padding rows of each expert region are zero-filled.
@@ -83,6 +93,11 @@ struct GemmArgs {
     //   C  [r,:] = row_gate[r] * u * phi'(h)         (gradient w.r.t. the pre-activation)
     //   C1 [r,:] = row_gate[r] * phi(h)              (gated activation, operand of the weight gradient)
     //   dg_part[r, column tile] = row_valid[r] * sum over the tile's columns of u * phi(h)
+    // bf16 path, gathered A (Eq. 18 inside the GEMM): if gather_x is not null, A is ignored and row block q of a
+    // tile is loaded from patch src_patch[tile*128/l_p + q] of gather_x [Bm patches, l_p, K]
+    const void* gather_x = nullptr;
+    const int* src_patch = nullptr;
+    int l_p = 0, Bm = 0;
     bool bwd = false;
     const void* bwd_h = nullptr;
     const float* row_gate = nullptr;

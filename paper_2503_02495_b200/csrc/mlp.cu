@@ -11,7 +11,7 @@ static MlpFwdWs mlp_fwd_ws(const Dims& D) {
     w.take(kStatusBytes);
     MlpFwdWs r;
     r.plan = w.take(plan_bytes(D));
-    r.xg = w.take((size_t)D.Rmax * D.d * D.esize);
+    r.xg = can_fuse_gather(D) ? 0 : w.take((size_t)D.Rmax * D.d * D.esize);     // the GEMM gathers x itself
     r.a = w.take((size_t)D.Rmax * D.d_e * D.esize);
     r.z = w.take((size_t)D.Rmax * D.d * D.esize);
     r.total = w.off;
@@ -51,10 +51,14 @@ extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, co
 
     st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream);
     if (st != UOE_OK) return st;
-    st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
-    if (st != UOE_OK) return st;
+    const bool fused = can_fuse_gather(D);
+    if (!fused) {
+        st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
+        if (st != UOE_OK) return st;
+    }
 
     GemmArgs g1{xg, W1, b1, a, saved_h, expert_offsets, D.n, D.d, D.d_e, prob->act, false, D.Rmax};
+    if (fused) { g1.gather_x = x; g1.src_patch = P.src_patch; g1.l_p = D.l_p; g1.Bm = D.B * D.m; }
     GemmArgs g2{a, W2, b2, z, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
     g1.label = "gemm1_act";
     g2.label = "gemm2";

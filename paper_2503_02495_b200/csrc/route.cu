@@ -21,7 +21,7 @@ constexpr int kSelectThreads = 128;
 template <typename T>
 __global__ void __launch_bounds__(kScoreThreads)
 route_score_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ partial,
-                   int L, int Lv, int d, int n, int m, int l_p, int CT, int nchunks) {
+                   int L, int Lv, int d, int n, int m, int l_p, int CT, int nchunks, int* __restrict__ counters) {
     constexpr int V = Vec16<T>::N;
     extern __shared__ uint4 s_w4[];                   // W_r[c0 : c0+cw, :] as stored
     __shared__ float s_cs[kScoreThreads * V];         // per-thread column sums, later the partial dot products
@@ -35,6 +35,8 @@ route_score_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __
     const int cw = min(CT * V, d - c0);               // columns of this chunk (a multiple of V)
     const int col = c0 + ct * V;
     const int rows = max(0, min(l_p, Lv - j * l_p));
+    // the selection kernel's ticket and expert loads (words 1 and 8..8+n of the status block) start at zero
+    if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 64) counters[tid] = 0;
 
     {   // stage the router rows of this chunk: cw*n elements, contiguous and 16-byte aligned
         const uint4* src = (const uint4*)(W_r + (size_t)c0 * n);
@@ -188,22 +190,27 @@ route_select_kernel(const float* __restrict__ partial, int nchunks, int B, int L
         }
         for (int pos = before + lane; pos < c; pos += 32) { out_idx[pos] = -1; out_gate[pos] = 0.f; }
     }
-    // Eq. 23 as row offsets: the last sample to arrive sums the loads
+    // Eq. 23 as row offsets: the last sample to arrive turns the loads into a prefix sum
+    __shared__ int s_last;
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        const int t = atomicAdd(ticket, 1);
-        if (t == B - 1) {
-            __threadfence();
-            int off = 0;
-            const int rows_per_pair = c * l_p;
-            for (int i = 0; i < n; ++i) {
-                offsets[i] = off;
-                const int rows = atomicAdd(&load[i], 0) * rows_per_pair;
-                off += (rows + UOE_ROW_ALIGN - 1) / UOE_ROW_ALIGN * UOE_ROW_ALIGN;
-            }
-            offsets[n] = off;
+        s_last = (atomicAdd(ticket, 1) == B - 1);
+    }
+    __syncthreads();
+    if (s_last && warp == 0) {
+        __threadfence();
+        const int rows_per_pair = c * l_p;
+        int rows = 0;
+        if (lane < n) rows = (__ldcg(load + lane) * rows_per_pair + UOE_ROW_ALIGN - 1) / UOE_ROW_ALIGN * UOE_ROW_ALIGN;
+        int incl = rows;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += v;
         }
+        if (lane < n) offsets[lane] = incl - rows;
+        if (lane == n - 1) offsets[n] = incl;
     }
 }
 
@@ -247,18 +254,17 @@ extern "C" uoe_status uoe_route(const uoe_problem* prob, const void* x, const vo
     if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     char* base = (char*)ws;
-    int* status = (int*)base;          // word 0 status, word 1 ticket, words 8.. expert loads
-    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
+    int* status = (int*)base;          // word 0 status, word 1 ticket, words 8.. expert loads (zeroed by the score kernel)
     float* partial = (float*)(base + W.partial);
     dim3 grid(D.B * D.m, W.nchunks);
     {
     ProfScope ps("route_score", stream);
     if (D.bf16)
         route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
-            (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
+            (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks, status);
     else
         route_score_kernel<float><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
-            (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
+            (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks, status);
     }
     UOE_LAUNCHED();
     ProfScope ps("route_select", stream);
@@ -314,16 +320,15 @@ extern "C" uoe_status uoe_route_static(const uoe_problem* prob, const void* x, c
     if (st != UOE_OK) return st;
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     int* status = (int*)base;
-    // the array keeps the previous call's ticket and expert loads: they must start at zero
-    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
+    // the array keeps the previous call's ticket and expert loads: the score kernel clears them first
     float* partial = (float*)(base + W.partial);
     dim3 grid(D.B * D.m, W.nchunks);
     if (D.bf16)
         route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
-            (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
+            (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks, status);
     else
         route_score_kernel<float><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
-            (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks);
+            (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks, status);
     UOE_LAUNCHED();
     route_select_kernel<<<D.B, kSelectThreads, (size_t)D.n * D.m * sizeof(float), stream>>>(
         partial, W.nchunks, D.B, D.Lv, D.n, D.k, D.m, D.c, D.l_p, (prob->flags & UOE_FLAG_GATE) ? 1 : 0,

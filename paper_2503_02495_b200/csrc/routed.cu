@@ -15,7 +15,8 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
             const int* __restrict__ offsets, int B, int n, int k, int m, int c, int l_p,
             int* __restrict__ pair_row, int* __restrict__ inv_row, float* __restrict__ inv_gate,
             int* __restrict__ expert_end, int* status, float* __restrict__ row_gate, float* __restrict__ row_valid,
-            int Lv, int use_gate) {
+            int Lv, int use_gate, int* __restrict__ src_patch, uint4* __restrict__ tail, long long tail_row_vecs,
+            long long rows_max) {
     __shared__ int my_e[32], cnt[32], prow[32];
     const int b = blockIdx.x, tid = threadIdx.x;
     const int l_a = c * l_p;
@@ -51,10 +52,28 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
         inv_row[((size_t)b * m + j) * k + s] = row;
         inv_gate[((size_t)b * m + j) * k + s] = g;
     }
+    __shared__ int s_end[32];
     if (b == 0 && tid < n) {
         int load = 0;
         for (int idx = 0; idx < B * k; ++idx) load += (expert_idx[idx] == tid);
-        expert_end[tid] = offsets[tid] + load * l_a;
+        s_end[tid] = expert_end[tid] = offsets[tid] + load * l_a;
+    }
+    // source patch of every l_p-row block (used when the GEMM gathers its own A operand)
+    for (int idx = tid; idx < k * c; idx += 128) {
+        const int s = idx / c, u = idx % c;
+        const int pj = patch_idx[((size_t)b * k + s) * c + u];
+        src_patch[prow[s] / l_p + u] = (pj >= 0 && pj < m) ? b * m + pj : -1;
+    }
+    if (b == 0) {
+        __syncthreads();
+        for (int i = 0; i < n; ++i)
+            for (int rb = s_end[i] / l_p + tid; rb < offsets[i + 1] / l_p; rb += 128) src_patch[rb] = -1;
+    }
+    if (tail) {
+        const long long r0 = offsets[n];
+        const long long total = (rows_max - r0) * tail_row_vecs;
+        for (long long q = (long long)b * 128 + tid; q < total; q += (long long)B * 128)
+            tail[r0 * tail_row_vecs + q] = make_uint4(0, 0, 0, 0);
     }
     if (row_gate) {                          // per-row weights for the backward
         for (int idx = tid; idx < k * l_a; idx += 128) {
@@ -234,11 +253,12 @@ gemm_f32_kernel(const float* __restrict__ A, const float* __restrict__ W, const 
 }  // namespace
 
 uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_idx, const float* gate,
-                       const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s, bool use_gate) {
+                       const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s, bool use_gate, void* tail,
+                       long long tail_row_bytes) {
     ProfScope ps("plan", s);
     plan_kernel<<<D.B, 128, 0, s>>>(expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
                                     P.pair_row, P.inv_row, P.inv_gate, P.expert_end, status, P.row_gate, P.row_valid,
-                                    D.Lv, use_gate ? 1 : 0);
+                                    D.Lv, use_gate ? 1 : 0, P.src_patch, (uint4*)tail, tail_row_bytes / 16, D.Rmax);
     UOE_LAUNCHED();
     return UOE_OK;
 }
@@ -248,9 +268,9 @@ uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, c
     const long long row_vecs = (long long)D.d * D.esize / 16;
     const long long slab_vecs = row_vecs * D.l_p;
     const int n_slabs = D.B * D.k * D.c;
-    int nsplit = (int)((slab_vecs * 16 + 32767) / 32768);
+    int nsplit = (int)((slab_vecs * 16 + 16383) / 16384);
     if (nsplit < 1) nsplit = 1;
-    if (nsplit > 64) nsplit = 64;
+    if (nsplit > 128) nsplit = 128;
     dim3 grid(n_slabs + D.n + (tail ? 1 : 0), nsplit);
     ProfScope ps("gather", s);
     gather_kernel<<<grid, kThreads, 0, s>>>((const uint4*)src, patch_idx, offsets, P.pair_row, P.expert_end,
@@ -262,7 +282,8 @@ uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, c
 
 uoe_status launch_combine(const Dims& D, const void* x, const void* z, const PlanPtrs& P, bool residual,
                           bool use_gate, void* y, cudaStream_t s, const float* rvec) {
-    int rows_per_cta = (int)(32768 / ((long long)D.d * D.esize));
+    // about two 16-byte vectors per thread: short dependent chains, many CTAs in flight
+    int rows_per_cta = (int)(2 * kThreads * 16 / ((long long)D.d * D.esize));
     if (rows_per_cta < 1) rows_per_cta = 1;
     if (rows_per_cta > D.l_p) rows_per_cta = D.l_p;
     dim3 grid(D.B * D.m, (D.l_p + rows_per_cta - 1) / rows_per_cta);

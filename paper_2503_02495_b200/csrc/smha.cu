@@ -15,7 +15,7 @@ static SmhaWs smha_ws(const Dims& D) {
     w.take(kStatusBytes);
     SmhaWs r;
     r.plan = w.take(plan_bytes(D));
-    r.xg = w.take((size_t)D.Rmax * D.d * D.esize);
+    r.xg = can_fuse_gather(D) ? 0 : w.take((size_t)D.Rmax * D.d * D.esize);     // the projection gathers x itself
     r.q = w.take((size_t)D.Rmax * D.d_g * D.esize);
     r.k = w.take((size_t)D.Rmax * D.d_g * D.esize);
     r.v = w.take((size_t)D.Rmax * D.d_g * D.esize);
@@ -54,13 +54,18 @@ extern "C" uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, c
     const PlanPtrs P = plan_ptrs(D, base + W.plan);
     void *xg = base + W.xg, *q = base + W.q, *k = base + W.k, *v = base + W.v, *o = base + W.o, *z = base + W.z;
 
-    st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream);
-    if (st != UOE_OK) return st;
     // rows of v past the last expert region are never written by the projection but may sit inside the
-    // last key tile of a pair: make them finite
-    st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream, v, (long long)D.d_g * D.esize);
+    // last key tile of a pair: the plan kernel makes them finite (zero)
+    const bool fused = can_fuse_gather(D);
+    st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream, true, v,
+                     (long long)D.d_g * D.esize);
     if (st != UOE_OK) return st;
+    if (!fused) {
+        st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
+        if (st != UOE_OK) return st;
+    }
     GemmArgs gq{xg, Wq, nullptr, q, nullptr, expert_offsets, D.n, D.d, D.d_g, UOE_ACT_IDENTITY, false, D.Rmax};
+    if (fused) { gq.gather_x = x; gq.src_patch = P.src_patch; gq.l_p = D.l_p; gq.Bm = D.B * D.m; }
     gq.label = "qkv_proj";
     gq.nmat = 3; gq.W1 = Wk; gq.W2 = Wv; gq.C1 = k; gq.C2 = v;
     st = launch_gemm_bf16(gq, status, stream);
