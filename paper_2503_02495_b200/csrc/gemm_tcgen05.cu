@@ -75,49 +75,49 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int total_tiles = (ctl->offs[n] / BM) * n_tiles;
 
     if (warp == 0) {
-        if (lane == 0) {
-            // ---------------- TMA producer ----------------
-            int stage = 0;
-            uint32_t phase = 0;
-            uint32_t issued = 0, issued_parity = 0;      // per stage: a load is in flight with this parity
-            bool stop = false;
-            for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
-                const int row0 = (tile / n_tiles) * BM;
-                const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
-                const CUtensorMap* tmB = mat == 0 ? &tmB0 : (mat == 1 ? &tmB1 : &tmB2);
-                int e = 0;
-                while (e + 1 < n && row0 >= ctl->offs[e + 1]) ++e;
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) || *abort_flag) { stop = true; break; }
-                    uint8_t* sa = smem + stage * Cf::STAGE;
-                    uint8_t* sb = sa + A_BYTES;
-                    mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
-                    if (src_patch) {        // gather: one box per source patch, zero rows from an out-of-range patch
-                        const int nbox = BM / l_p;
-                        const int* sp = src_patch + (row0 / l_p);
-                        for (int q = 0; q < nbox; ++q) {
-                            const int src = sp[q];
-                            tma_load_3d(sa + q * l_p * 128, &tmX, kb * BK, 0, src >= 0 ? src : Bm, &ctl->full[stage]);
-                        }
-                    } else {
-                        tma_load_2d(sa, &tmA, kb * BK, row0, &ctl->full[stage]);
-                    }
-                    if (B_KMAJOR) {
-                        tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
-                    } else {
-#pragma unroll
-                        for (int q = 0; q < BN / 64; ++q)
-                            tma_load_3d(sb + q * 8192, tmB, col0 + q * 64, kb * BK, e, &ctl->full[stage]);
-                    }
-                    issued |= 1u << stage;
-                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
-                    if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
+        // ---------------- TMA producer: lane 0 runs the pipeline, boxes are issued one per lane ----------------
+        int stage = 0;
+        uint32_t phase = 0;
+        uint32_t issued = 0, issued_parity = 0;      // per stage: a load is in flight with this parity
+        bool stop = false;
+        const int nbox_a = src_patch ? BM / l_p : 1;             // lanes 0..nbox_a-1 load A, lanes 16.. load B
+        constexpr int nbox_b = B_KMAJOR ? 1 : BN / 64;
+        for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+            const int row0 = (tile / n_tiles) * BM;
+            const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
+            const CUtensorMap* tmB = mat == 0 ? &tmB0 : (mat == 1 ? &tmB1 : &tmB2);
+            int e = 0;
+            while (e + 1 < n && row0 >= ctl->offs[e + 1]) ++e;
+            int my_src = 0;                                      // source patch of this lane's row block
+            if (src_patch && lane < nbox_a) {
+                my_src = src_patch[row0 / l_p + lane];
+                if (my_src < 0) my_src = Bm;                     // out of range: the box is zero-filled
+            }
+            for (int kb = 0; kb < num_kb; ++kb) {
+                int ok = 1;
+                if (lane == 0) ok = (mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) && !*abort_flag) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { stop = true; break; }
+                uint8_t* sa = smem + stage * Cf::STAGE;
+                uint8_t* sb = sa + A_BYTES;
+                if (lane == 0) mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
+                __syncwarp();
+                if (lane < nbox_a) {
+                    if (src_patch) tma_load_3d(sa + lane * l_p * 128, &tmX, kb * BK, 0, my_src, &ctl->full[stage]);
+                    else tma_load_2d(sa, &tmA, kb * BK, row0, &ctl->full[stage]);
+                } else if (lane >= 16 && lane < 16 + nbox_b) {
+                    const int q = lane - 16;
+                    if (B_KMAJOR) tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
+                    else tma_load_3d(sb + q * 8192, tmB, col0 + q * 64, kb * BK, e, &ctl->full[stage]);
                 }
+                issued |= 1u << stage;
+                issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
             }
-            if (*abort_flag) {      // let this CTA's own copies land before it exits
-                for (int s = 0; s < Cf::STAGES; ++s)
-                    if (issued & (1u << s)) mbar_wait(&ctl->full[s], (issued_parity >> s) & 1, abort_flag, status);
-            }
+        }
+        if (lane == 0 && *abort_flag) {      // let this CTA's own copies land before it exits
+            for (int s = 0; s < Cf::STAGES; ++s)
+                if (issued & (1u << s)) mbar_wait(&ctl->full[s], (issued_parity >> s) & 1, abort_flag, status);
         }
     } else if (warp == 1) {
         if (lane == 0) {

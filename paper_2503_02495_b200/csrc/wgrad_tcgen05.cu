@@ -66,34 +66,35 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
     const int total_tiles = n * per_expert;
 
     if (warp == 0) {
-        if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0, issued = 0, issued_parity = 0;
-            bool stop = false;
-            for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
-                const int e = tile / per_expert, rem = tile % per_expert;
-                const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
-                const int r0 = ctl->offs[e], num_kb = (ctl->offs[e + 1] - r0) / BK;
-                for (int kb = 0; kb < num_kb; ++kb) {
-                    if (!mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) || *abort_flag) { stop = true; break; }
-                    uint8_t* sa = smem + stage * Cf::STAGE;
-                    uint8_t* sb = sa + A_BYTES;
-                    mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
-#pragma unroll
-                    for (int q = 0; q < BM / 64; ++q)
-                        tma_load_2d(sa + q * 8192, &tmP, m0 + q * 64, r0 + kb * BK, &ctl->full[stage]);
-#pragma unroll
-                    for (int q = 0; q < BN / 64; ++q)
-                        tma_load_2d(sb + q * 8192, &tmQ, n0 + q * 64, r0 + kb * BK, &ctl->full[stage]);
-                    issued |= 1u << stage;
-                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
-                    if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
-                }
+        // TMA producer: lane 0 runs the pipeline, the 64-wide boxes are issued one per lane
+        int stage = 0;
+        uint32_t phase = 0, issued = 0, issued_parity = 0;
+        bool stop = false;
+        for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+            const int e = tile / per_expert, rem = tile % per_expert;
+            const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
+            const int r0 = ctl->offs[e], num_kb = (ctl->offs[e + 1] - r0) / BK;
+            for (int kb = 0; kb < num_kb; ++kb) {
+                int ok = 1;
+                if (lane == 0) ok = (mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) && !*abort_flag) ? 1 : 0;
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (!ok) { stop = true; break; }
+                uint8_t* sa = smem + stage * Cf::STAGE;
+                uint8_t* sb = sa + A_BYTES;
+                if (lane == 0) mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
+                __syncwarp();
+                if (lane < BM / 64)
+                    tma_load_2d(sa + lane * 8192, &tmP, m0 + lane * 64, r0 + kb * BK, &ctl->full[stage]);
+                else if (lane >= 16 && lane < 16 + BN / 64)
+                    tma_load_2d(sb + (lane - 16) * 8192, &tmQ, n0 + (lane - 16) * 64, r0 + kb * BK, &ctl->full[stage]);
+                issued |= 1u << stage;
+                issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
             }
-            if (*abort_flag) {
-                for (int s = 0; s < Cf::STAGES; ++s)
-                    if (issued & (1u << s)) mbar_wait(&ctl->full[s], (issued_parity >> s) & 1, abort_flag, status);
-            }
+        }
+        if (lane == 0 && *abort_flag) {
+            for (int s = 0; s < Cf::STAGES; ++s)
+                if (issued & (1u << s)) mbar_wait(&ctl->full[s], (issued_parity >> s) & 1, abort_flag, status);
         }
     } else if (warp == 1) {
         if (lane == 0) {
