@@ -248,18 +248,14 @@ def run_reference(args, w: gen.Workload, rank: int, world: int):
     print(json.dumps(line), flush=True)
 
 
-def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
+def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int, with_e2e: bool):
+    """Times `steps` steps of workload w on this rank's GPU.  Returns a dict with the per-step milliseconds
+    (device events, L2 flushed between steps), launches, clocks, per-kernel records and the e2e time."""
     import torch
-    import torch.distributed as dist
 
     import paper_2503_02495_b200 as uoe
     from paper_2503_02495_b200.block import UoEBlock
     from tests.helpers import problem_of, to_dev
-
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
 
     h = host_inputs(w)
     wd = {k: to_dev(v, dev) for k, v in h.items() if k not in ("x", "dy")}
@@ -267,6 +263,8 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
     dy_dev = to_dev(h["dy"], dev) if w.backward else None
     blk = UoEBlock(problem_of(w, "att") if w.H else None, problem_of(w, "mlp") if w.d_ff else None, wd, dev,
                    backward=w.backward)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
 
     def step(xin):
         out = blk.forward(xin)
@@ -274,15 +272,14 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
             blk.mlp_backward(xin, dy_dev)
             return blk.dx
         return out
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
-    stream = torch.cuda.current_stream()
 
     def barrier():
         if world > 1:
+            import torch.distributed as dist
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(max(warmup, 3)):
         step(x_dev)
     torch.cuda.synchronize()
     st = blk.device_status()
@@ -290,9 +287,9 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
         raise RuntimeError("device status after warm-up: " + uoe.status_string(st))
 
     # ---- timed region: K steps, each with its own event pair, L2 flushed in between ----
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(dev.index or 0)
     sampler.start()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     barrier()
     launches0 = uoe.uoe_launch_count()
     for e0, e1 in ev:
@@ -304,51 +301,43 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
     launches = uoe.uoe_launch_count() - launches0
     clocks = sampler.stop()
     ms = [e0.elapsed_time(e1) for e0, e1 in ev]
-    ms_step = sum(ms) / len(ms)
+    res = {"ms_step": sum(ms) / len(ms), "ms_min": min(ms), "launches": int(launches), "clocks": clocks, "host": h}
 
     # ---- end to end through the public API with host buffers ----
-    x_host = h["x"].raw
-    x_pin = torch.from_numpy(np.ascontiguousarray(x_host).view(np.int16 if w.dtype == "bf16" else np.float32)).pin_memory()
-    x_in = torch.empty_like(x_dev)
-    y_pin = torch.empty(x_pin.shape, dtype=x_pin.dtype).pin_memory()
-    e2e_t = []
-    for i in range(args.steps + 2):
-        flush.zero_()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        x_in.view(x_pin.dtype).copy_(x_pin, non_blocking=True)
-        out = step(x_in)
-        y_pin.copy_(out.view(x_pin.dtype), non_blocking=True)
-        torch.cuda.synchronize()
-        if i >= 2:
-            e2e_t.append(time.perf_counter() - t0)
-    e2e_ms = sum(e2e_t) / len(e2e_t) * 1e3
+    if with_e2e:
+        x_host = h["x"].raw
+        x_pin = torch.from_numpy(np.ascontiguousarray(x_host).view(np.int16 if w.dtype == "bf16" else np.float32)).pin_memory()
+        x_in = torch.empty_like(x_dev)
+        y_pin = torch.empty(x_pin.shape, dtype=x_pin.dtype).pin_memory()
+        e2e_t = []
+        for i in range(steps + 2):
+            flush.zero_()
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            x_in.view(x_pin.dtype).copy_(x_pin, non_blocking=True)
+            out = step(x_in)
+            y_pin.copy_(out.view(x_pin.dtype), non_blocking=True)
+            torch.cuda.synchronize()
+            if i >= 2:
+                e2e_t.append(time.perf_counter() - t0)
+        res["e2e_ms"] = sum(e2e_t) / len(e2e_t) * 1e3
+        res["h2d"] = int(x_pin.numel() * x_pin.element_size())
+        res["d2h"] = int(y_pin.numel() * y_pin.element_size())
 
     # ---- per-kernel durations (separate pass: the event pairs would perturb the timed region) ----
+    steps_prof = min(steps, 20)
     uoe.uoe_profile_enable(True)
-    for _ in range(min(args.steps, 20)):
+    for _ in range(steps_prof):
         flush.zero_()
         step(x_dev)
     torch.cuda.synchronize()
     uoe.uoe_profile_enable(False)
-    recs = uoe.uoe_profile_records()
     per = {}
-    for name, t in recs:
+    for name, t in uoe.uoe_profile_records():
         per.setdefault(name, []).append(t)
-
-    ms_step, e2e_ms = max_over_ranks([ms_step, e2e_ms], world, dev)
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
-
-    peaks, peak_src = load_peaks()
-    tokens = w.B * w.L_valid * world
-    flops = step_flops(w) * world
     work = work_table(w)
-    kern = []
     tot = sum(sum(v) for v in per.values())
-    steps_prof = min(args.steps, 20)
+    kern = []
     for name, v in per.items():
         avg = sum(v) / len(v)
         wk = work.get(name, dict(flops=0, bytes=0))
@@ -357,8 +346,18 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
                      "tflops": wk["flops"] / avg / 1e9 if avg > 0 else 0.0,
                      "gbs": wk["bytes"] / avg / 1e6 if avg > 0 else 0.0})
     kern.sort(key=lambda r: -r["share"])
-    top = kern[0]
-    wk = work.get(top["kernel"], dict(flops=0, bytes=0))
+    res["kernels"] = kern
+    del blk, flush
+    torch.cuda.empty_cache()
+    return res
+
+
+TENSOR_KERNELS = ("gemm1_act", "gemm2", "qkv_proj", "out_proj", "attention", "bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2")
+HBM_KERNELS = ("route_score", "gather", "combine", "pool")
+
+
+def roofline_of(top, w: gen.Workload, peaks, peak_src):
+    wk = work_table(w).get(top["kernel"], dict(flops=0, bytes=0))
     t_tensor = wk["flops"] / (peaks["bf16_tflops"] * 1e12)
     t_hbm = wk["bytes"] / (peaks["hbm_gbs"] * 1e9)
     if t_tensor >= t_hbm and wk["flops"] > 0:
@@ -368,8 +367,33 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
     roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": None, "kernel": top["kernel"],
                  "avg_ms": top["avg_ms"], "share_of_kernel_time": top["share"], "peak_source": peak_src,
                  "algorithmic_flops": wk["flops"], "algorithmic_bytes": wk["bytes"]})
+    return roof
+
+
+def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
+    import torch
+    import torch.distributed as dist
+
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    m = measure_gpu(args, w, dev, world, args.steps, args.warmup, True)
+    ms_step, e2e_ms = max_over_ranks([m["ms_step"], m["e2e_ms"]], world, dev)
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_src = load_peaks()
+    tokens = w.B * w.L_valid * world
+    flops = step_flops(w) * world
+    kern = m["kernels"]
+    roof = roofline_of(kern[0], w, peaks, peak_src)
 
     # ---- CPU baseline: the oracle as it stands, on a bounded sample ----
+    h = m["host"]
     Bs = cpu_sample_B(w)
     ts = []
     if not args.skip_cpu_baseline:
@@ -381,20 +405,44 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
 
     line = base_line(w, args, world)
     line.update({
-        "value": job_throughput(w, world, ms_step), "ms_per_step": ms_step, "ms_per_step_min": min(ms),
+        "value": job_throughput(w, world, ms_step), "ms_per_step": ms_step, "ms_per_step_min": m["ms_min"],
         "tflops": flops / (ms_step * 1e-3) / 1e12,
         "frac_of_bf16_peak": flops / (ms_step * 1e-3) / 1e12 / (peaks["bf16_tflops"] * world),
         "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": int(x_pin.numel() * x_pin.element_size()),
-                "d2h_bytes_per_step": int(y_pin.numel() * y_pin.element_size())},
-        "gpu_launches": int(launches),
-        "clocks": clocks,
+                "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"]},
+        "gpu_launches": m["launches"],
+        "clocks": m["clocks"],
         "roofline": roof,
         "kernels": kern,
         "cpu_baseline": {"value": (Bs * w.L_valid / cpu_sec) if ts else None, "unit": "tokens/s", "cores": blas_threads(),
-                         "kind": "oracle", "sec_per_step": cpu_sec,
+                         "kind": "oracle", "sec_per_step": cpu_sec if ts else None,
                          "sample": f"first {Bs} of {w.B} samples, whole block, {len(ts)} steps"},
     })
+    del m, h
+
+    # ---- the large MLP workload (forward + backward), where the tensor-core and HBM targets are quoted ----
+    if world == 1 and not args.no_scale and w.name != "cfg5_scale" and args.B == 0:
+        ws = gen.WORKLOADS["cfg5_scale"]
+        ms5 = measure_gpu(args, ws, dev, 1, 10, 3, False)
+        k5 = {r["kernel"]: r for r in ms5["kernels"]}
+        tens = [k5[n] for n in TENSOR_KERNELS if n in k5]
+        wt = work_table(ws)
+        tf_sum = sum(wt[r["kernel"]]["flops"] for r in tens)
+        tm_sum = sum(r["avg_ms"] * r["launches_per_step"] for r in tens)
+        line["scale_workload"] = {
+            "workload": ws.name, "blocks": "uome forward + backward", "B": ws.B, "L": ws.L, "d": ws.d, "d_ff": ws.d_ff,
+            "n": ws.n, "k": ws.k, "m": ws.m, "c": ws.c, "steps": 10,
+            "ms_per_step": ms5["ms_step"], "tokens_per_s": ws.B * ws.L_valid / (ms5["ms_step"] * 1e-3),
+            "tflops": step_flops(ws) / (ms5["ms_step"] * 1e-3) / 1e12,
+            "frac_of_bf16_peak": step_flops(ws) / (ms5["ms_step"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
+            "grouped_gemm_tflops": tf_sum / tm_sum / 1e9 if tm_sum > 0 else None,
+            "grouped_gemm_frac_of_bf16_peak": tf_sum / tm_sum / 1e9 / peaks["bf16_tflops"] if tm_sum > 0 else None,
+            "hbm_kernels": {n: {"gbs": k5[n]["gbs"], "frac_of_hbm_peak": k5[n]["gbs"] / peaks["hbm_gbs"]}
+                            for n in HBM_KERNELS if n in k5},
+            "gpu_launches": ms5["launches"], "clocks": ms5["clocks"],
+            "roofline": roofline_of(ms5["kernels"][0], ws, peaks, peak_src),
+            "kernels": [{kk: (round(vv, 5) if isinstance(vv, float) else vv) for kk, vv in r.items()} for r in ms5["kernels"]],
+        }
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -409,6 +457,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (profiling on a smaller case)")
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing (profiling runs)")
+    ap.add_argument("--no-scale", action="store_true", help="do not add the scale workload's summary to the line")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
