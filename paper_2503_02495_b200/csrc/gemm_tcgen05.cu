@@ -3,12 +3,20 @@
 //
 //   C[r, :] = epilogue( A[r, :] @ W[e(r)] ),  r over the routed rows, e(r) = expert whose region holds r
 //
-// One persistent CTA per SM walks the (128-row tile, BN-column tile) list; expert regions are padded
-// to 128 rows, so a row tile never straddles two experts.  Warp roles:
-//   warp 0     TMA producer: A tile [128 x 64] and B tile [64 x BN] per K step into a 128B-swizzled ring
-//   warp 1     MMA issuer: tcgen05.mma 128 x BN x 16 into one of two TMEM accumulators
-//   warps 2-5  epilogue: tcgen05.ld the accumulator (one row per thread), activation, bf16, global store
-// so the epilogue of tile t overlaps the main loop of tile t+1.
+// One persistent CTA per SM walks the (row tile, BN-column tile) list; expert regions are padded to 128
+// rows, so a 128-row block never straddles two experts.  Warp roles:
+//   warp 0      TMA producer (lane 0 runs the pipeline; the boxes of a stage are issued one per lane):
+//               A tile [MT*128 x 64] and B tile [64 x BN] per K step into a 128B-swizzled ring
+//   warp 1      MMA issuer: tcgen05.mma 128 x BN x 16 into TMEM accumulators
+//   warps 2..   epilogue: tcgen05.ld the accumulator (one row per thread), activation, bf16, global store
+// Two tile heights:
+//   MT = 1  128-row tiles, two TMEM accumulators: the epilogue of tile t overlaps the main loop of tile t+1
+//   MT = 2  256-row tiles (two 128-row accumulators fed by the same B stage): a third fewer operand bytes
+//           per flop, which is what bounds the ring at large K (the ring holds ~1 us of MMA work against an
+//           L2/HBM latency of the same order); one accumulator set, drained by eight epilogue warps.
+//           A 256-row unit at the end of an expert region may hold a single 128-row block ("half tile").
+// The A operand is either a routed buffer (2-D tensor map) or gathered on the fly from x, one TMA box per
+// source patch (Eq. 18 inside the GEMM).
 #include "kernels.cuh"
 #include "tc.cuh"
 #include "tmap.cuh"
@@ -19,15 +27,18 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BK = 64;
-constexpr int kGemmThreads = 192;
-constexpr int A_BYTES = BM * BK * 2;     // 16 KB
+constexpr int A_BLOCK_BYTES = BM * BK * 2;     // 16 KB per 128-row block
 
-template <int BN> struct Cfg {
+template <int BN, int MT> struct Cfg {
+    static constexpr int A_BYTES = MT * A_BLOCK_BYTES;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
-    static constexpr int TMEM_COLS = 2 * BN;               // two accumulators; 128, 256 or 512 columns
-    static constexpr int SMEM = STAGES * STAGE + 1024 /*align slack*/ + 512 /*barriers, offsets*/;
+    static constexpr int STAGES = (MT == 2) ? 3 : ((BN == 256) ? 4 : (BN == 128 ? 6 : 8));
+    static constexpr int NACC = (MT == 2) ? 1 : 2;                 // accumulator sets in TMEM
+    static constexpr int TMEM_COLS = 2 * BN;                       // MT=1: two sets; MT=2: one set of two blocks
+    static constexpr int EPI_WARPS = 4 * MT;
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;
+    static constexpr int SMEM = STAGES * STAGE + 1024 /*align slack*/ + 1024 /*barriers, offsets*/;
 };
 
 struct Ctl {                       // lives behind the stage ring
@@ -35,10 +46,11 @@ struct Ctl {                       // lives behind the stage ring
     uint32_t tmem_base;
     int abort_flag;
     int offs[34];
+    int tstart[34];                // first row tile of each expert (prefix sum), tstart[n] = number of row tiles
 };
 
-template <int BN, bool B_KMAJOR, bool BWD>
-__global__ void __launch_bounds__(kGemmThreads, 1)
+template <int BN, bool B_KMAJOR, bool BWD, int MT>
+__global__ void __launch_bounds__(Cfg<BN, MT>::THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
                  __nv_bfloat16* __restrict__ C0, __nv_bfloat16* __restrict__ C1, __nv_bfloat16* __restrict__ C2,
@@ -46,7 +58,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  int n, int K, int N, int nmat, int act, int* status, const __nv_bfloat16* __restrict__ bwd_h,
                  const float* __restrict__ row_gate, const float* __restrict__ row_valid, float* __restrict__ dg_part,
                  const __grid_constant__ CUtensorMap tmX, const int* __restrict__ src_patch, int l_p, int Bm) {
-    using Cf = Cfg<BN>;
+    using Cf = Cfg<BN, MT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     Ctl* ctl = (Ctl*)(smem + Cf::STAGES * Cf::STAGE);
@@ -55,13 +67,28 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < Cf::STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 128); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 32 * Cf::EPI_WARPS); }
         ctl->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB0);
     }
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + n + 1) ctl->offs[threadIdx.x - 64] = offsets[threadIdx.x - 64];
+    if (warp == 2) {                // offsets and the row-tile prefix over experts (n <= 31 here)
+        int o = 0;
+        if (lane <= n) o = offsets[lane];
+        const int o1 = __shfl_down_sync(0xffffffffu, o, 1);
+        const int blocks = lane < n ? (o1 - o) / BM : 0;
+        const int tiles = (blocks + MT - 1) / MT;
+        int incl = tiles;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const int v = __shfl_up_sync(0xffffffffu, incl, d);
+            if (lane >= d) incl += v;
+        }
+        if (lane <= n) ctl->offs[lane] = o;
+        if (lane < n) ctl->tstart[lane] = incl - tiles;
+        if (lane == n - 1) ctl->tstart[n] = incl;
+    }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
     tc_fence_before();
     __syncthreads();
@@ -72,43 +99,52 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int n_tiles_mat = N / BN;
     const int n_tiles = n_tiles_mat * nmat;
     const int num_kb = K / BK;
-    const int total_tiles = (ctl->offs[n] / BM) * n_tiles;
+    const int total_tiles = ctl->tstart[n] * n_tiles;
+
+    // row tile -> expert, first row, number of 128-row blocks it holds
+    auto locate = [&](int row_tile, int& e, int& row0, int& blocks) {
+        e = 0;
+        while (e + 1 < n && row_tile >= ctl->tstart[e + 1]) ++e;
+        const int i = row_tile - ctl->tstart[e];
+        row0 = ctl->offs[e] + i * (MT * BM);
+        blocks = min(MT, (ctl->offs[e + 1] - row0) / BM);
+    };
 
     if (warp == 0) {
-        // ---------------- TMA producer: lane 0 runs the pipeline, boxes are issued one per lane ----------------
+        // ---------------- TMA producer ----------------
         int stage = 0;
         uint32_t phase = 0;
         uint32_t issued = 0, issued_parity = 0;      // per stage: a load is in flight with this parity
         bool stop = false;
-        const int nbox_a = src_patch ? BM / l_p : 1;             // lanes 0..nbox_a-1 load A, lanes 16.. load B
         constexpr int nbox_b = B_KMAJOR ? 1 : BN / 64;
         for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
-            const int row0 = (tile / n_tiles) * BM;
+            int e, row0, blocks;
+            locate(tile / n_tiles, e, row0, blocks);
             const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
             const CUtensorMap* tmB = mat == 0 ? &tmB0 : (mat == 1 ? &tmB1 : &tmB2);
-            int e = 0;
-            while (e + 1 < n && row0 >= ctl->offs[e + 1]) ++e;
-            int my_src = 0;                                      // source patch of this lane's row block
+            const int nbox_a = src_patch ? blocks * (BM / l_p) : blocks;      // <= 32
+            int my_src = 0;                                                     // source patch of this lane's box
             if (src_patch && lane < nbox_a) {
                 my_src = src_patch[row0 / l_p + lane];
-                if (my_src < 0) my_src = Bm;                     // out of range: the box is zero-filled
+                if (my_src < 0) my_src = Bm;                                    // out of range: zero-filled box
             }
+            const uint32_t stage_bytes = blocks * A_BLOCK_BYTES + Cf::B_BYTES;
             for (int kb = 0; kb < num_kb; ++kb) {
                 int ok = 1;
                 if (lane == 0) ok = (mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) && !*abort_flag) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { stop = true; break; }
                 uint8_t* sa = smem + stage * Cf::STAGE;
-                uint8_t* sb = sa + A_BYTES;
-                if (lane == 0) mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
+                uint8_t* sb = sa + Cf::A_BYTES;
+                if (lane == 0) mbar_arrive_expect_tx(&ctl->full[stage], stage_bytes);
                 __syncwarp();
                 if (lane < nbox_a) {
                     if (src_patch) tma_load_3d(sa + lane * l_p * 128, &tmX, kb * BK, 0, my_src, &ctl->full[stage]);
-                    else tma_load_2d(sa, &tmA, kb * BK, row0, &ctl->full[stage]);
-                } else if (lane >= 16 && lane < 16 + nbox_b) {
-                    const int q = lane - 16;
+                    else tma_load_2d(sa + lane * A_BLOCK_BYTES, &tmA, kb * BK, row0 + lane * BM, &ctl->full[stage]);
+                }
+                if (lane < nbox_b) {
                     if (B_KMAJOR) tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
-                    else tma_load_3d(sb + q * 8192, tmB, col0 + q * 64, kb * BK, e, &ctl->full[stage]);
+                    else tma_load_3d(sb + lane * 8192, tmB, col0 + lane * 64, kb * BK, e, &ctl->full[stage]);
                 }
                 issued |= 1u << stage;
                 issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
@@ -127,103 +163,112 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             uint32_t phase = 0, acc_phase = 0;
             bool stop = false;
             for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+                int e, row0, blocks;
+                locate(tile / n_tiles, e, row0, blocks);
                 if (!mbar_wait(&ctl->tempty[acc], acc_phase ^ 1, abort_flag, status) || *abort_flag) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * BN;
+                const uint32_t d_tmem = tmem_base + acc * BN;        // MT=2: acc is always 0, block h at column h*BN
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&ctl->full[stage], phase, abort_flag, status) || *abort_flag) { stop = true; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(smem + stage * Cf::STAGE);
-                    const uint32_t sb = sa + A_BYTES;
+                    const uint32_t sb = sa + Cf::A_BYTES;
 #pragma unroll
                     for (int ks = 0; ks < BK / 16; ++ks) {
-                        const uint64_t ad = smem_desc(sa + ks * 32, 16, 1024);
                         const uint64_t bd = B_KMAJOR ? smem_desc(sb + ks * 32, 16, 1024)
                                                      : smem_desc(sb + ks * 2048, 8192, 1024);
-                        mma_bf16(d_tmem, ad, bd, idesc, (kb | ks) != 0);
+#pragma unroll
+                        for (int h = 0; h < MT; ++h)
+                            if (h < blocks)
+                                mma_bf16(d_tmem + h * BN, smem_desc(sa + h * A_BLOCK_BYTES + ks * 32, 16, 1024), bd, idesc,
+                                         (kb | ks) != 0);
                     }
                     mma_commit(&ctl->empty[stage]);
                     if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (stop) break;
                 mma_commit(&ctl->tfull[acc]);
-                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+                if (++acc == Cf::NACC) { acc = 0; acc_phase ^= 1; }
             }
         }
     } else {
-        // ---------------- epilogue: warps 2..5, TMEM lane quarter = warp % 4 ----------------
+        // ---------------- epilogue: warp w drains 128-row block (w-2)/4, TMEM lane quarter w % 4 ----------------
         const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
         int acc = 0;
         uint32_t acc_phase = 0;
+        auto pack8 = [](const float* f) {
+            uint4 w;
+            w.x = pack_bf16x2(f[0], f[1]); w.y = pack_bf16x2(f[2], f[3]);
+            w.z = pack_bf16x2(f[4], f[5]); w.w = pack_bf16x2(f[6], f[7]);
+            return w;
+        };
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-            const int row0 = (tile / n_tiles) * BM;
+            int e, row0, blocks;
+            locate(tile / n_tiles, e, row0, blocks);
             const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
             __nv_bfloat16* C = mat == 0 ? C0 : (mat == 1 ? C1 : C2);
             const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
             if (!__all_sync(0xffffffffu, ready)) break;      // warp-uniform: tcgen05.ld below is warp-collective
             tc_fence_after();
-            const size_t row = (size_t)row0 + quarter * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
-            auto pack8 = [](const float* f) {
-                uint4 w;
-                w.x = pack_bf16x2(f[0], f[1]); w.y = pack_bf16x2(f[2], f[3]);
-                w.z = pack_bf16x2(f[4], f[5]); w.w = pack_bf16x2(f[6], f[7]);
-                return w;
-            };
-            if constexpr (BWD) {
-                const float rg = row_gate[row], rv = row_valid[row];
-                float dsum = 0.f;
+            if (half < blocks) {
+                const size_t row = (size_t)row0 + half * BM + quarter * 32 + lane;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (MT == 2 ? half * BN : acc * BN);
+                if constexpr (BWD) {
+                    const float rg = row_gate[row], rv = row_valid[row];
+                    float dsum = 0.f;
 #pragma unroll 1
-                for (int ch = 0; ch < BN / 32; ++ch) {
-                    uint32_t v[32];
-                    tmem_ld32(taddr + ch * 32, v);
-                    const uint4* hp = (const uint4*)(bwd_h + row * N + col0 + ch * 32);
-                    uint4 hv[4];
+                    for (int ch = 0; ch < BN / 32; ++ch) {
+                        uint32_t v[32];
+                        tmem_ld32(taddr + ch * 32, v);
+                        const uint4* hp = (const uint4*)(bwd_h + row * N + col0 + ch * 32);
+                        uint4 hv[4];
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) hv[q] = hp[q];
-                    tmem_ld_wait();
-                    uint4* o_dh = (uint4*)(C + row * N + col0 + ch * 32);
-                    uint4* o_ag = (uint4*)(C1 + row * N + col0 + ch * 32);
+                        for (int q = 0; q < 4; ++q) hv[q] = hp[q];
+                        tmem_ld_wait();
+                        uint4* o_dh = (uint4*)(C + row * N + col0 + ch * 32);
+                        uint4* o_ag = (uint4*)(C1 + row * N + col0 + ch * 32);
 #pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        float hh[8], dh[8], ag[8];
-                        unpack16<__nv_bfloat16>(hv[q], hh);
+                        for (int q = 0; q < 4; ++q) {
+                            float hh[8], dh[8], ag[8];
+                            unpack16<__nv_bfloat16>(hv[q], hh);
 #pragma unroll
-                        for (int t = 0; t < 8; ++t) {
-                            const float u = __uint_as_float(v[8 * q + t]);
-                            const float a = act_apply(hh[t], act);
-                            dsum = fmaf(u, a, dsum);
-                            dh[t] = rg * u * act_deriv(hh[t], act);
-                            ag[t] = rg * a;
+                            for (int t = 0; t < 8; ++t) {
+                                const float u = __uint_as_float(v[8 * q + t]);
+                                const float a = act_apply(hh[t], act);
+                                dsum = fmaf(u, a, dsum);
+                                dh[t] = rg * u * act_deriv(hh[t], act);
+                                ag[t] = rg * a;
+                            }
+                            o_dh[q] = pack8(dh);
+                            o_ag[q] = pack8(ag);
                         }
-                        o_dh[q] = pack8(dh);
-                        o_ag[q] = pack8(ag);
                     }
-                }
-                dg_part[row * n_tiles_mat + (col0 / BN)] = rv * dsum;
-            } else {
+                    dg_part[row * n_tiles_mat + (col0 / BN)] = rv * dsum;
+                } else {
 #pragma unroll 1
-                for (int ch = 0; ch < BN / 32; ++ch) {
-                    uint32_t v[32];
-                    tmem_ld32(taddr + ch * 32, v);
-                    tmem_ld_wait();
-                    float f[32];
+                    for (int ch = 0; ch < BN / 32; ++ch) {
+                        uint32_t v[32];
+                        tmem_ld32(taddr + ch * 32, v);
+                        tmem_ld_wait();
+                        float f[32];
 #pragma unroll
-                    for (int q = 0; q < 32; ++q) f[q] = __uint_as_float(v[q]);
-                    if (pre) {
-                        uint4* po = (uint4*)(pre + row * N + col0 + ch * 32);
+                        for (int q = 0; q < 32; ++q) f[q] = __uint_as_float(v[q]);
+                        if (pre) {
+                            uint4* po = (uint4*)(pre + row * N + col0 + ch * 32);
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) po[q] = pack8(f + 8 * q);
+                            for (int q = 0; q < 4; ++q) po[q] = pack8(f + 8 * q);
+                        }
+                        act_apply_n<32>(f, act);
+                        uint4* out = (uint4*)(C + row * N + col0 + ch * 32);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) out[q] = pack8(f + 8 * q);
                     }
-                    act_apply_n<32>(f, act);
-                    uint4* out = (uint4*)(C + row * N + col0 + ch * 32);
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) out[q] = pack8(f + 8 * q);
                 }
             }
             tc_fence_before();
             mbar_arrive(&ctl->tempty[acc]);
-            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            if (++acc == Cf::NACC) { acc = 0; acc_phase ^= 1; }
         }
     }
     tc_fence_before();
@@ -234,11 +279,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
 }
 
-template <int BN, bool B_KMAJOR, bool BWD>
+template <int BN, bool B_KMAJOR, bool BWD, int MT>
 uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
-    using Cf = Cfg<BN>;
+    using Cf = Cfg<BN, MT>;
     static bool attr_set = false;
-    auto kern = gemm_bf16_kernel<BN, B_KMAJOR, BWD>;
+    auto kern = gemm_bf16_kernel<BN, B_KMAJOR, BWD, MT>;
     if (!attr_set) {
         UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
         attr_set = true;
@@ -272,16 +317,28 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
             if (!make_tmap(&tmB[q], Ws[q], 3, dims, str, box)) return UOE_ERR_CUDA;
         }
     }
-    long long max_tiles = (g.rows_max / BM) * (g.N / BN) * nmat;
+    long long max_tiles = ((g.rows_max / BM + MT - 1) / MT + g.n) * (g.N / BN) * nmat;
     int grid = (int)(max_tiles < sm_count() ? max_tiles : sm_count());
     if (grid < 1) grid = 1;
     ProfScope ps(g.label, s);
-    kern<<<grid, kGemmThreads, Cf::SMEM, s>>>(tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
-                                              (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
-                                              nmat, g.act, status, (const __nv_bfloat16*)g.bwd_h, g.row_gate, g.row_valid,
-                                              g.dg_part, tmX, g.gather_x ? g.src_patch : nullptr, g.l_p, g.Bm);
+    kern<<<grid, Cf::THREADS, Cf::SMEM, s>>>(tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
+                                             (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
+                                             nmat, g.act, status, (const __nv_bfloat16*)g.bwd_h, g.row_gate, g.row_valid,
+                                             g.dg_part, tmX, g.gather_x ? g.src_patch : nullptr, g.l_p, g.Bm);
     UOE_LAUNCHED();
     return UOE_OK;
+}
+
+template <bool B_KMAJOR, bool BWD>
+uoe_status dispatch(const GemmArgs& g, int* status, cudaStream_t s) {
+    const int bn = gemm_bf16_bn(g.N);
+    // 256-row tiles pay off when every SM still gets several of them and the K loop is long enough to be
+    // bound by operand delivery rather than by the prologue
+    const long long tiles256 = (g.rows_max / 256) * (g.N / 256);
+    if (bn == 256 && g.K >= 1024 && tiles256 >= 2 * sm_count()) return launch_one<256, B_KMAJOR, BWD, 2>(g, status, s);
+    if (bn == 256) return launch_one<256, B_KMAJOR, BWD, 1>(g, status, s);
+    if (bn == 128) return launch_one<128, B_KMAJOR, BWD, 1>(g, status, s);
+    return launch_one<64, B_KMAJOR, BWD, 1>(g, status, s);
 }
 
 }  // namespace
@@ -290,23 +347,14 @@ uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s) {
     if (g.K % BK != 0 || g.N % 64 != 0 || g.bias || g.nmat > 3) return UOE_ERR_UNSUPPORTED;
     if (g.nmat > 1 && g.pre) return UOE_ERR_UNSUPPORTED;
     if (g.gather_x && (!g.src_patch || g.l_p < 8 || g.l_p % 8 != 0 || BM % g.l_p != 0)) return UOE_ERR_INVALID_ARG;
-    if (g.rows_max % BM != 0) return UOE_ERR_INVALID_ARG;
-    const int bn = gemm_bf16_bn(g.N);
+    if (g.rows_max % BM != 0 || g.n > 31) return UOE_ERR_UNSUPPORTED;
     if (g.bwd) {          // backward epilogue: weights are read K-major ([n, N, K])
         if (!g.b_kmajor || !g.bwd_h || !g.row_gate || !g.row_valid || !g.dg_part || !g.C1 || g.nmat > 1)
             return UOE_ERR_INVALID_ARG;
-        if (bn == 256) return launch_one<256, true, true>(g, status, s);
-        if (bn == 128) return launch_one<128, true, true>(g, status, s);
-        return launch_one<64, true, true>(g, status, s);
+        return dispatch<true, true>(g, status, s);
     }
-    if (g.b_kmajor) {
-        if (bn == 256) return launch_one<256, true, false>(g, status, s);
-        if (bn == 128) return launch_one<128, true, false>(g, status, s);
-        return launch_one<64, true, false>(g, status, s);
-    }
-    if (bn == 256) return launch_one<256, false, false>(g, status, s);
-    if (bn == 128) return launch_one<128, false, false>(g, status, s);
-    return launch_one<64, false, false>(g, status, s);
+    if (g.b_kmajor) return dispatch<true, false>(g, status, s);
+    return dispatch<false, false>(g, status, s);
 }
 
 }  // namespace uoe

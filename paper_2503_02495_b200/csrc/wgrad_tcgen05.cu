@@ -17,14 +17,19 @@ namespace {
 using namespace tc;
 
 constexpr int BM = 128, BK = 64;
-constexpr int kThreads = 192;
-constexpr int A_BYTES = BM * BK * 2;
+constexpr int A_BLOCK_BYTES = BM * BK * 2;
 
-template <int BN> struct WCfg {
+// MT = 2: 256 x BN output tiles (two 128-row accumulators fed by the same Q stage), one accumulator set
+// drained by eight epilogue warps; MT = 1: 128 x BN tiles with two accumulator sets.
+template <int BN, int MT> struct WCfg {
+    static constexpr int A_BYTES = MT * A_BLOCK_BYTES;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (BN == 256) ? 4 : (BN == 128 ? 6 : 8);
+    static constexpr int STAGES = (MT == 2) ? 3 : ((BN == 256) ? 4 : (BN == 128 ? 6 : 8));
+    static constexpr int NACC = (MT == 2) ? 1 : 2;
     static constexpr int TMEM_COLS = 2 * BN;
+    static constexpr int EPI_WARPS = 4 * MT;
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;
     static constexpr int SMEM = STAGES * STAGE + 1024 + 512;
 };
 
@@ -35,11 +40,11 @@ struct WCtl {
     int offs[34];
 };
 
-template <int BN>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int BN, int MT>
+__global__ void __launch_bounds__(WCfg<BN, MT>::THREADS, 1)
 wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CUtensorMap tmQ,
              float* __restrict__ dW, const int* __restrict__ offsets, int n, int M, int N, int* status) {
-    using Cf = WCfg<BN>;
+    using Cf = WCfg<BN, MT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     WCtl* ctl = (WCtl*)(smem + Cf::STAGES * Cf::STAGE);
@@ -48,7 +53,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < Cf::STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 128); }
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 32 * Cf::EPI_WARPS); }
         ctl->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmP);
@@ -61,7 +66,8 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
-    const int m_tiles = M / BM, n_tiles = N / BN;
+    constexpr int TM = MT * BM;
+    const int m_tiles = M / TM, n_tiles = N / BN;
     const int per_expert = m_tiles * n_tiles;
     const int total_tiles = n * per_expert;
 
@@ -72,7 +78,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         bool stop = false;
         for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
             const int e = tile / per_expert, rem = tile % per_expert;
-            const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
+            const int m0 = (rem / n_tiles) * TM, n0 = (rem % n_tiles) * BN;
             const int r0 = ctl->offs[e], num_kb = (ctl->offs[e + 1] - r0) / BK;
             for (int kb = 0; kb < num_kb; ++kb) {
                 int ok = 1;
@@ -80,10 +86,10 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (!ok) { stop = true; break; }
                 uint8_t* sa = smem + stage * Cf::STAGE;
-                uint8_t* sb = sa + A_BYTES;
+                uint8_t* sb = sa + Cf::A_BYTES;
                 if (lane == 0) mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
                 __syncwarp();
-                if (lane < BM / 64)
+                if (lane < TM / 64)
                     tma_load_2d(sa + lane * 8192, &tmP, m0 + lane * 64, r0 + kb * BK, &ctl->full[stage]);
                 else if (lane >= 16 && lane < 16 + BN / 64)
                     tma_load_2d(sb + (lane - 16) * 8192, &tmQ, n0 + (lane - 16) * 64, r0 + kb * BK, &ctl->full[stage]);
@@ -112,32 +118,37 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
                     if (!mbar_wait(&ctl->full[stage], phase, abort_flag, status) || *abort_flag) { stop = true; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(smem + stage * Cf::STAGE);
-                    const uint32_t sb = sa + A_BYTES;
+                    const uint32_t sb = sa + Cf::A_BYTES;
 #pragma unroll
-                    for (int ks = 0; ks < BK / 16; ++ks)
-                        mma_bf16(d_tmem, smem_desc(sa + ks * 2048, 8192, 1024), smem_desc(sb + ks * 2048, 8192, 1024),
-                                 idesc, (kb | ks) != 0);
+                    for (int ks = 0; ks < BK / 16; ++ks) {
+                        const uint64_t bd = smem_desc(sb + ks * 2048, 8192, 1024);
+#pragma unroll
+                        for (int h = 0; h < MT; ++h)
+                            mma_bf16(d_tmem + h * BN, smem_desc(sa + h * A_BLOCK_BYTES + ks * 2048, 8192, 1024), bd, idesc,
+                                     (kb | ks) != 0);
+                    }
                     mma_commit(&ctl->empty[stage]);
                     if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (stop) break;
                 mma_commit(&ctl->tfull[acc]);
-                if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+                if (++acc == Cf::NACC) { acc = 0; acc_phase ^= 1; }
             }
         }
     } else {
         const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             const int e = tile / per_expert, rem = tile % per_expert;
-            const int m0 = (rem / n_tiles) * BM, n0 = (rem % n_tiles) * BN;
+            const int m0 = (rem / n_tiles) * TM, n0 = (rem % n_tiles) * BN;
             const int num_kb = (ctl->offs[e + 1] - ctl->offs[e]) / BK;
             const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
             if (!__all_sync(0xffffffffu, ready)) break;
             tc_fence_after();
-            float* out = dW + ((size_t)e * M + m0 + quarter * 32 + lane) * N + n0;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+            float* out = dW + ((size_t)e * M + m0 + half * BM + quarter * 32 + lane) * N + n0;
+            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (MT == 2 ? half * BN : acc * BN);
 #pragma unroll 1
             for (int ch = 0; ch < BN / 32; ++ch) {
                 uint32_t v[32];
@@ -154,7 +165,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
             }
             tc_fence_before();
             mbar_arrive(&ctl->tempty[acc]);
-            if (++acc == 2) { acc = 0; acc_phase ^= 1; }
+            if (++acc == Cf::NACC) { acc = 0; acc_phase ^= 1; }
         }
     }
     tc_fence_before();
@@ -165,12 +176,12 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
     }
 }
 
-template <int BN>
+template <int BN, int MT>
 uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
                     long long rows_max, const char* label, int* status, cudaStream_t s) {
-    using Cf = WCfg<BN>;
+    using Cf = WCfg<BN, MT>;
     static bool attr_set = false;
-    auto kern = wgrad_kernel<BN>;
+    auto kern = wgrad_kernel<BN, MT>;
     if (!attr_set) {
         UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
         attr_set = true;
@@ -187,10 +198,10 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
         const uint64_t str[1] = {(uint64_t)N * 2};
         if (!make_tmap(&tmQ, Q, 2, dims, str, box)) return UOE_ERR_CUDA;
     }
-    const long long tiles = (long long)n * (M / BM) * (N / BN);
+    const long long tiles = (long long)n * (M / (MT * BM)) * (N / BN);
     int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     ProfScope ps(label, s);
-    kern<<<grid, kThreads, Cf::SMEM, s>>>(tmP, tmQ, dW, offsets, n, M, N, status);
+    kern<<<grid, Cf::THREADS, Cf::SMEM, s>>>(tmP, tmQ, dW, offsets, n, M, N, status);
     UOE_LAUNCHED();
     return UOE_OK;
 }
@@ -199,11 +210,14 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
 
 uoe_status launch_wgrad_bf16(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
                              long long rows_max, const char* label, int* status, cudaStream_t s) {
-    if (M % BM != 0 || N % 64 != 0) return UOE_ERR_UNSUPPORTED;
+    if (M % BM != 0 || N % 64 != 0 || n > 32) return UOE_ERR_UNSUPPORTED;
     const int bn = gemm_bf16_bn(N);
-    if (bn == 256) return launch_w<256>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
-    if (bn == 128) return launch_w<128>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
-    return launch_w<64>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
+    // 256-row output tiles when the weight matrices are large enough to keep every SM busy with them
+    if (bn == 256 && M % 256 == 0 && (long long)n * (M / 256) * (N / 256) >= 2 * sm_count())
+        return launch_w<256, 2>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
+    if (bn == 256) return launch_w<256, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
+    if (bn == 128) return launch_w<128, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
+    return launch_w<64, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
 }
 
 }  // namespace uoe

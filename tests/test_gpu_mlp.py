@@ -27,6 +27,8 @@ CASES = {
     "small_bf16": gen.tiny(B=3, L=96, L_valid=96, m=6, c=3, d=64, n=4, k=2, d_ff=256, dtype="bf16", w_std=0.05),
     "pad_bf16": gen.tiny(B=5, L=112, L_valid=100, m=7, c=4, d=128, n=3, k=2, d_ff=192, dtype="bf16", w_std=0.05,
                          act="gelu_erf"),
+    # long K and many row tiles: the 256-row tile variant, with regions of 3*load 128-row blocks (half tiles)
+    "tall_tiles": gen.tiny(B=40, L=1152, L_valid=1152, m=9, c=3, d=1024, n=4, k=2, d_ff=4096, dtype="bf16", w_std=0.02),
     "cfg2": gen.WORKLOADS["cfg2_lm"],
     "cfg3": gen.WORKLOADS["cfg3_long"],
     "cfg4": gen.WORKLOADS["cfg4_vit"],
@@ -52,7 +54,7 @@ def _run(w, residual, use_gate, router_scale=1.0):
 @pytest.mark.parametrize("name", list(CASES))
 def test_expert_term_matches_oracle(name):
     w = CASES[name]
-    scale = 20.0 if not name.startswith("cfg") else 1.0
+    scale = 20.0 if not (name.startswith("cfg") or name == "tall_tiles") else 1.0
     y, ref, x, r = _run(w, residual=False, use_gate=True, router_scale=scale)
     err = rel_inf(y, ref)
     print(f"{name}: max|err|/max|ref| = {err:.3e}")

@@ -29,6 +29,8 @@ CASES = {
     "full": _w(k=4, c=6),
     "wide": _w(B=3, d=256, d_ff=1024, n=4, k=3, L=256, L_valid=250, m=8, c=5),
     "skewed": _w(B=9, n=5, k=2, d_ff=640),
+    # long K and many row tiles: 256-row GEMM tiles with half tiles at the region ends
+    "tall_tiles": _w(B=40, L=1152, L_valid=1152, m=9, c=3, d=1024, n=4, k=2, d_ff=4096, w_std=0.02),
 }
 
 
@@ -54,6 +56,8 @@ def _run(w, residual, use_gate, skew=0.0):
 @pytest.mark.parametrize("residual", [False, True])
 def test_backward_matches_oracle(name, residual):
     w = CASES[name]
+    if name == "tall_tiles" and residual:
+        pytest.skip("large case: run once")
     got, ref, ro = _run(w, residual, True, skew=3.0 if name == "skewed" else 0.0)
     for nm, g, r in zip(("dx", "dW1", "dW2", "dW_r"), got, ref[:4]):
         err = rel_inf(g, r)
