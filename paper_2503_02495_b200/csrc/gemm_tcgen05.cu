@@ -8,7 +8,9 @@
 //   warp 0      TMA producer (lane 0 runs the pipeline; the boxes of a stage are issued one per lane):
 //               A tile [MT*128 x 64] and B tile [64 x BN] per K step into a 128B-swizzled ring
 //   warp 1      MMA issuer: tcgen05.mma 128 x BN x 16 into TMEM accumulators
-//   warps 2..   epilogue: tcgen05.ld the accumulator (one row per thread), activation, bf16, global store
+//   warps 2..   epilogue: tcgen05.ld the accumulator (one row per thread), activation, bf16, then a
+//               [32 rows x 64 columns] piece per warp staged in swizzled shared memory and written with one
+//               TMA tensor store (full 128-byte lines instead of 16-byte scattered stores)
 // Two tile heights:
 //   MT = 1  128-row tiles, two TMEM accumulators: the epilogue of tile t overlaps the main loop of tile t+1
 //   MT = 2  256-row tiles (two 128-row accumulators fed by the same B stage): a third fewer operand bytes
@@ -38,7 +40,8 @@ template <int BN, int MT> struct Cfg {
     static constexpr int TMEM_COLS = 2 * BN;                       // MT=1: two sets; MT=2: one set of two blocks
     static constexpr int EPI_WARPS = 4 * MT;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
-    static constexpr int SMEM = STAGES * STAGE + 1024 /*align slack*/ + 1024 /*barriers, offsets*/;
+    static constexpr int STG_BYTES = 32 * 128;                     // one epilogue warp's staging piece
+    static constexpr int SMEM = STAGES * STAGE + 1024 /*align slack*/ + 1024 /*barriers, offsets*/ + EPI_WARPS * STG_BYTES;
 };
 
 struct Ctl {                       // lives behind the stage ring
@@ -57,7 +60,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  __nv_bfloat16* __restrict__ pre, const int* __restrict__ offsets,
                  int n, int K, int N, int nmat, int act, int* status, const __nv_bfloat16* __restrict__ bwd_h,
                  const float* __restrict__ row_gate, const float* __restrict__ row_valid, float* __restrict__ dg_part,
-                 const __grid_constant__ CUtensorMap tmX, const int* __restrict__ src_patch, int l_p, int Bm) {
+                 const __grid_constant__ CUtensorMap tmX, const int* __restrict__ src_patch, int l_p, int Bm,
+                 const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
+                 const __grid_constant__ CUtensorMap tmC2, const __grid_constant__ CUtensorMap tmPre) {
     using Cf = Cfg<BN, MT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -203,66 +208,73 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             w.z = pack_bf16x2(f[4], f[5]); w.w = pack_bf16x2(f[6], f[7]);
             return w;
         };
+        uint8_t* stg = smem + Cf::STAGES * Cf::STAGE + 1024 + (warp - 2) * Cf::STG_BYTES;
+        // 64 values of this thread's row -> bf16 -> this warp's staging piece (row = lane, 128B swizzle) -> TMA store
+        auto stage_store = [&](const float* f, const CUtensorMap* tm, int c0, int r0) {
+            if (lane == 0) bulk_wait_read();          // the previous store has finished reading the piece
+            __syncwarp();
+#pragma unroll
+            for (int c = 0; c < 8; ++c) *(uint4*)(stg + lane * 128 + ((c ^ (lane & 7)) << 4)) = pack8(f + 8 * c);
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) { tma_store_2d(tm, stg, c0, r0); bulk_commit(); }
+        };
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
             int e, row0, blocks;
             locate(tile / n_tiles, e, row0, blocks);
             const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
-            __nv_bfloat16* C = mat == 0 ? C0 : (mat == 1 ? C1 : C2);
+            const CUtensorMap* tmC = mat == 0 ? &tmC0 : (mat == 1 ? &tmC1 : &tmC2);
             const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
             if (!__all_sync(0xffffffffu, ready)) break;      // warp-uniform: tcgen05.ld below is warp-collective
             tc_fence_after();
             if (half < blocks) {
-                const size_t row = (size_t)row0 + half * BM + quarter * 32 + lane;
+                const int wrow0 = row0 + half * BM + quarter * 32;       // first row of this warp's piece
+                const size_t row = (size_t)wrow0 + lane;
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (MT == 2 ? half * BN : acc * BN);
                 if constexpr (BWD) {
                     const float rg = row_gate[row], rv = row_valid[row];
                     float dsum = 0.f;
 #pragma unroll 1
-                    for (int ch = 0; ch < BN / 32; ++ch) {
-                        uint32_t v[32];
-                        tmem_ld32(taddr + ch * 32, v);
-                        const uint4* hp = (const uint4*)(bwd_h + row * N + col0 + ch * 32);
-                        uint4 hv[4];
+                    for (int g = 0; g < BN / 64; ++g) {
+                        uint32_t v[64];
+                        tmem_ld32(taddr + g * 64, v);
+                        tmem_ld32(taddr + g * 64 + 32, v + 32);
+                        const uint4* hp = (const uint4*)(bwd_h + row * N + col0 + g * 64);
+                        uint4 hv[8];
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) hv[q] = hp[q];
+                        for (int q = 0; q < 8; ++q) hv[q] = hp[q];
                         tmem_ld_wait();
-                        uint4* o_dh = (uint4*)(C + row * N + col0 + ch * 32);
-                        uint4* o_ag = (uint4*)(C1 + row * N + col0 + ch * 32);
+                        float dh[64], ag[64];
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            float hh[8], dh[8], ag[8];
+                        for (int q = 0; q < 8; ++q) {
+                            float hh[8];
                             unpack16<__nv_bfloat16>(hv[q], hh);
 #pragma unroll
                             for (int t = 0; t < 8; ++t) {
                                 const float u = __uint_as_float(v[8 * q + t]);
                                 const float a = act_apply(hh[t], act);
                                 dsum = fmaf(u, a, dsum);
-                                dh[t] = rg * u * act_deriv(hh[t], act);
-                                ag[t] = rg * a;
+                                dh[8 * q + t] = rg * u * act_deriv(hh[t], act);
+                                ag[8 * q + t] = rg * a;
                             }
-                            o_dh[q] = pack8(dh);
-                            o_ag[q] = pack8(ag);
                         }
+                        stage_store(dh, &tmC0, col0 + g * 64, wrow0);
+                        stage_store(ag, &tmC1, col0 + g * 64, wrow0);
                     }
                     dg_part[row * n_tiles_mat + (col0 / BN)] = rv * dsum;
                 } else {
 #pragma unroll 1
-                    for (int ch = 0; ch < BN / 32; ++ch) {
-                        uint32_t v[32];
-                        tmem_ld32(taddr + ch * 32, v);
+                    for (int g = 0; g < BN / 64; ++g) {
+                        uint32_t v[64];
+                        tmem_ld32(taddr + g * 64, v);
+                        tmem_ld32(taddr + g * 64 + 32, v + 32);
                         tmem_ld_wait();
-                        float f[32];
+                        float f[64];
 #pragma unroll
-                        for (int q = 0; q < 32; ++q) f[q] = __uint_as_float(v[q]);
-                        if (pre) {
-                            uint4* po = (uint4*)(pre + row * N + col0 + ch * 32);
-#pragma unroll
-                            for (int q = 0; q < 4; ++q) po[q] = pack8(f + 8 * q);
-                        }
-                        act_apply_n<32>(f, act);
-                        uint4* out = (uint4*)(C + row * N + col0 + ch * 32);
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) out[q] = pack8(f + 8 * q);
+                        for (int q = 0; q < 64; ++q) f[q] = __uint_as_float(v[q]);
+                        if (pre) stage_store(f, &tmPre, col0 + g * 64, wrow0);
+                        act_apply_n<64>(f, act);
+                        stage_store(f, tmC, col0 + g * 64, wrow0);
                     }
                 }
             }
@@ -271,6 +283,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (++acc == Cf::NACC) { acc = 0; acc_phase ^= 1; }
         }
     }
+    if (warp >= 2 && lane == 0) bulk_wait_all();       // this warp's tensor stores are complete
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -317,6 +330,17 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
             if (!make_tmap(&tmB[q], Ws[q], 3, dims, str, box)) return UOE_ERR_CUDA;
         }
     }
+    // outputs as [rows_max, N], written in [32 rows x 64 columns] pieces
+    CUtensorMap tmC[3], tmPre;
+    {
+        const uint64_t dims[2] = {(uint64_t)g.N, (uint64_t)g.rows_max};
+        const uint64_t str[1] = {(uint64_t)g.N * 2};
+        const uint32_t box[2] = {64, 32};
+        const void* Cs[3] = {g.C, g.C1 ? g.C1 : g.C, g.C2 ? g.C2 : g.C};
+        for (int q = 0; q < 3; ++q)
+            if (!make_tmap(&tmC[q], Cs[q], 2, dims, str, box)) return UOE_ERR_CUDA;
+        if (!make_tmap(&tmPre, g.pre ? g.pre : g.C, 2, dims, str, box)) return UOE_ERR_CUDA;
+    }
     long long max_tiles = ((g.rows_max / BM + MT - 1) / MT + g.n) * (g.N / BN) * nmat;
     int grid = (int)(max_tiles < sm_count() ? max_tiles : sm_count());
     if (grid < 1) grid = 1;
@@ -324,7 +348,8 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     kern<<<grid, Cf::THREADS, Cf::SMEM, s>>>(tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
                                              (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
                                              nmat, g.act, status, (const __nv_bfloat16*)g.bwd_h, g.row_gate, g.row_valid,
-                                             g.dg_part, tmX, g.gather_x ? g.src_patch : nullptr, g.l_p, g.Bm);
+                                             g.dg_part, tmX, g.gather_x ? g.src_patch : nullptr, g.l_p, g.Bm, tmC[0],
+                                             tmC[1], tmC[2], tmPre);
     UOE_LAUNCHED();
     return UOE_OK;
 }
