@@ -1,7 +1,7 @@
 """Union-of-Experts routed hot path for B200: Python binding of the C-ABI library libuoe.so.
 
 Importing the package loads the shared library and fails if it has not been built
-(`python -m paper_2503_02495_b200.build`).  There is no CPU or PyTorch fallback.
+(`python paper_2503_02495_b200/build.py`).  There is no CPU or PyTorch fallback.
 """
 from .binding import (  # noqa: F401
     LIB_PATH, Problem, Routing, UoeError, alloc_routing, alloc_saved_h, alloc_workspace, status_string,

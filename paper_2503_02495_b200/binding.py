@@ -76,7 +76,7 @@ class Problem:
 
 def _load():
     if not os.path.exists(LIB_PATH):
-        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2503_02495_b200.build` "
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python paper_2503_02495_b200/build.py` "
                           "(there is no fallback path)")
     lib = ctypes.CDLL(LIB_PATH)
     vp, sz, i32p, f32p = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p

@@ -1,4 +1,4 @@
-"""Builds libuoe.so (all CUDA sources, sm_100a) next to this file.  Usage: python -m paper_2503_02495_b200.build"""
+"""Builds libuoe.so (all CUDA sources, sm_100a) next to this file.  Usage: python paper_2503_02495_b200/build.py"""
 from __future__ import annotations
 
 import os
