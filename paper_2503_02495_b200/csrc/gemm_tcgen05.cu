@@ -360,7 +360,9 @@ uoe_status dispatch(const GemmArgs& g, int* status, cudaStream_t s) {
     // 256-row tiles pay off when every SM still gets several of them and the K loop is long enough to be
     // bound by operand delivery rather than by the prologue
     const long long tiles256 = (g.rows_max / 256) * (g.N / 256);
-    if (bn == 256 && g.K >= 1024 && tiles256 >= 2 * sm_count()) return launch_one<256, B_KMAJOR, BWD, 2>(g, status, s);
+    // (the backward epilogue is long: it stays on 128-row tiles, where it overlaps the next tile's main loop)
+    if (!BWD && bn == 256 && g.K >= 1024 && tiles256 >= 2 * sm_count())
+        return launch_one<256, B_KMAJOR, BWD, 2>(g, status, s);
     if (bn == 256) return launch_one<256, B_KMAJOR, BWD, 1>(g, status, s);
     if (bn == 128) return launch_one<128, B_KMAJOR, BWD, 1>(g, status, s);
     return launch_one<64, B_KMAJOR, BWD, 1>(g, status, s);

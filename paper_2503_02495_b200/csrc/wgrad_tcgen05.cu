@@ -5,8 +5,9 @@
 // (64 elements) per swizzled box.
 //
 // Persistent CTAs walk (expert, 128-row tile of M, BN-column tile of N); warp roles and the two-buffer
-// TMEM accumulator are the same as in the forward grouped GEMM.  The output is float32 and overwritten;
-// an expert with no rows gets zeros.
+// TMEM accumulator are the same as in the forward grouped GEMM.  The output is float32 and overwritten
+// (each epilogue warp stages [32 rows x 32 columns] in swizzled shared memory and issues one TMA tensor
+// store); an expert with no rows gets zeros.
 #include "kernels.cuh"
 #include "tc.cuh"
 #include "tmap.cuh"
@@ -30,7 +31,8 @@ template <int BN, int MT> struct WCfg {
     static constexpr int TMEM_COLS = 2 * BN;
     static constexpr int EPI_WARPS = 4 * MT;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
-    static constexpr int SMEM = STAGES * STAGE + 1024 + 512;
+    static constexpr int STG_BYTES = 32 * 128;
+    static constexpr int SMEM = STAGES * STAGE + 1024 + 1024 + EPI_WARPS * STG_BYTES;
 };
 
 struct WCtl {
@@ -43,7 +45,8 @@ struct WCtl {
 template <int BN, int MT>
 __global__ void __launch_bounds__(WCfg<BN, MT>::THREADS, 1)
 wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CUtensorMap tmQ,
-             float* __restrict__ dW, const int* __restrict__ offsets, int n, int M, int N, int* status) {
+             const __grid_constant__ CUtensorMap tmW, const int* __restrict__ offsets, int n, int M, int N,
+             int* status) {
     using Cf = WCfg<BN, MT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -147,8 +150,9 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
             const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
             if (!__all_sync(0xffffffffu, ready)) break;
             tc_fence_after();
-            float* out = dW + ((size_t)e * M + m0 + half * BM + quarter * 32 + lane) * N + n0;
+            const int wrow0 = e * M + m0 + half * BM + quarter * 32;      // first row of this warp's piece in [n*M, N]
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (MT == 2 ? half * BN : acc * BN);
+            uint8_t* stg = smem + Cf::STAGES * Cf::STAGE + 1024 + (warp - 2) * Cf::STG_BYTES;
 #pragma unroll 1
             for (int ch = 0; ch < BN / 32; ++ch) {
                 uint32_t v[32];
@@ -159,15 +163,21 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
 #pragma unroll
                     for (int q = 0; q < 32; ++q) v[q] = 0u;
                 }
-                uint4* o4 = (uint4*)(out + ch * 32);
+                if (lane == 0) bulk_wait_read();      // the previous store has finished reading the piece
+                __syncwarp();
 #pragma unroll
-                for (int q = 0; q < 8; ++q) o4[q] = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                for (int q = 0; q < 8; ++q)
+                    *(uint4*)(stg + lane * 128 + ((q ^ (lane & 7)) << 4)) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) { tma_store_2d(&tmW, stg, n0 + ch * 32, wrow0); bulk_commit(); }
             }
             tc_fence_before();
             mbar_arrive(&ctl->tempty[acc]);
             if (++acc == Cf::NACC) { acc = 0; acc_phase ^= 1; }
         }
     }
+    if (warp >= 2 && lane == 0) bulk_wait_all();
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
@@ -198,10 +208,17 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
         const uint64_t str[1] = {(uint64_t)N * 2};
         if (!make_tmap(&tmQ, Q, 2, dims, str, box)) return UOE_ERR_CUDA;
     }
+    CUtensorMap tmW;      // dW as [n*M, N] float32, written in [32 x 32] pieces
+    {
+        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)n * M};
+        const uint64_t str[1] = {(uint64_t)N * 4};
+        const uint32_t wbox[2] = {32, 32};
+        if (!make_tmap(&tmW, dW, 2, dims, str, wbox, CU_TENSOR_MAP_DATA_TYPE_FLOAT32)) return UOE_ERR_CUDA;
+    }
     const long long tiles = (long long)n * (M / (MT * BM)) * (N / BN);
     int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     ProfScope ps(label, s);
-    kern<<<grid, Cf::THREADS, Cf::SMEM, s>>>(tmP, tmQ, dW, offsets, n, M, N, status);
+    kern<<<grid, Cf::THREADS, Cf::SMEM, s>>>(tmP, tmQ, tmW, offsets, n, M, N, status);
     UOE_LAUNCHED();
     return UOE_OK;
 }
