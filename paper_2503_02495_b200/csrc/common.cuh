@@ -174,6 +174,44 @@ __device__ __forceinline__ void act_apply_n(float* f, int act) {
     }
 }
 
+// phi(h) and phi'(h) for N values with the selection made once; sub-expressions are shared
+// (SiLU: s = sigmoid(h), phi = h s, phi' = s (1 + h (1 - s))).
+template <int N>
+__device__ __forceinline__ void act_and_deriv_n(const float* h, float* a, float* d, int act) {
+    switch (act) {
+        case UOE_ACT_SILU:
+#pragma unroll
+            for (int q = 0; q < N; ++q) {
+                const float s = __fdividef(1.0f, 1.0f + __expf(-h[q]));
+                a[q] = h[q] * s;
+                d[q] = s * (1.0f + h[q] * (1.0f - s));
+            }
+            break;
+        case UOE_ACT_GELU_ERF:
+#pragma unroll
+            for (int q = 0; q < N; ++q) {
+                const float cdf = 0.5f * (1.0f + erff(h[q] * 0.70710678118654752f));
+                a[q] = h[q] * cdf;
+                d[q] = cdf + h[q] * 0.39894228040143268f * __expf(-0.5f * h[q] * h[q]);
+            }
+            break;
+        case UOE_ACT_GELU_TANH:
+#pragma unroll
+            for (int q = 0; q < N; ++q) {
+                const float u = 0.79788456080286536f * (h[q] + 0.044715f * h[q] * h[q] * h[q]);
+                const float t = tanhf(u);
+                const float du = 0.79788456080286536f * (1.0f + 3.0f * 0.044715f * h[q] * h[q]);
+                a[q] = 0.5f * h[q] * (1.0f + t);
+                d[q] = 0.5f * (1.0f + t) + 0.5f * h[q] * (1.0f - t * t) * du;
+            }
+            break;
+        default:
+#pragma unroll
+            for (int q = 0; q < N; ++q) { a[q] = h[q]; d[q] = 1.0f; }
+            break;
+    }
+}
+
 __device__ __forceinline__ float act_deriv(float h, int act) {
     switch (act) {
         case UOE_ACT_GELU_ERF: {

@@ -246,17 +246,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         tmem_ld_wait();
                         float dh[64], ag[64];
 #pragma unroll
-                        for (int q = 0; q < 8; ++q) {
-                            float hh[8];
-                            unpack16<__nv_bfloat16>(hv[q], hh);
+                        for (int q = 0; q < 8; ++q) unpack16<__nv_bfloat16>(hv[q], dh + 8 * q);     // h
+                        act_and_deriv_n<64>(dh, ag, dh, act);                                         // ag = phi(h), dh = phi'(h)
 #pragma unroll
-                            for (int t = 0; t < 8; ++t) {
-                                const float u = __uint_as_float(v[8 * q + t]);
-                                const float a = act_apply(hh[t], act);
-                                dsum = fmaf(u, a, dsum);
-                                dh[8 * q + t] = rg * u * act_deriv(hh[t], act);
-                                ag[8 * q + t] = rg * a;
-                            }
+                        for (int q = 0; q < 64; ++q) {
+                            const float u = __uint_as_float(v[q]);
+                            dsum = fmaf(u, ag[q], dsum);
+                            dh[q] = rg * u * dh[q];
+                            ag[q] = rg * ag[q];
                         }
                         stage_store(dh, &tmC0, col0 + g * 64, wrow0);
                         stage_store(ag, &tmC1, col0 + g * 64, wrow0);
@@ -361,8 +358,9 @@ uoe_status dispatch(const GemmArgs& g, int* status, cudaStream_t s) {
     // bound by operand delivery rather than by the prologue
     const long long tiles256 = (g.rows_max / 256) * (g.N / 256);
     // (the backward epilogue is long: it stays on 128-row tiles, where it overlaps the next tile's main loop)
-    if (!BWD && bn == 256 && g.K >= 1024 && tiles256 >= 2 * sm_count())
-        return launch_one<256, B_KMAJOR, BWD, 2>(g, status, s);
+    if constexpr (!BWD) {
+        if (bn == 256 && g.K >= 1024 && tiles256 >= 2 * sm_count()) return launch_one<256, B_KMAJOR, BWD, 2>(g, status, s);
+    }
     if (bn == 256) return launch_one<256, B_KMAJOR, BWD, 1>(g, status, s);
     if (bn == 128) return launch_one<128, B_KMAJOR, BWD, 1>(g, status, s);
     return launch_one<64, B_KMAJOR, BWD, 1>(g, status, s);
