@@ -17,9 +17,27 @@ namespace {
 
 constexpr int kThreads = 256;
 
+// dgate[b,s,u] = sum over the slab's rows and column tiles of the per-row partials; one warp per slab,
+// fixed summation order.  grid ceil(B*k*c / 4), 128 threads.
+__global__ void __launch_bounds__(128)
+dgate_kernel(const float* __restrict__ dg_part, int nt, const int* __restrict__ pair_row,
+             const int* __restrict__ patch_idx, int n_slabs, int c, int m, int l_p, float* __restrict__ dgate) {
+    const int slab = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (slab >= n_slabs) return;
+    const int j = patch_idx[slab];
+    float a = 0.f;
+    if (j >= 0 && j < m) {
+        const float* src = dg_part + ((size_t)pair_row[slab / c] + (size_t)(slab % c) * l_p) * nt;
+        for (int q = lane; q < l_p * nt; q += 32) a += src[q];
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+    if (lane == 0) dgate[slab] = a;
+}
+
 // grid B, 128 threads, dynamic smem 2*n*m floats.  G[b,j,i] = dlogit_patch[b,i,j]/cnt_j + dlogit_samp[b,i]/L_valid.
 __global__ void __launch_bounds__(128)
-router_bwd_kernel(const float* __restrict__ dg_part, int nt, const int* __restrict__ pair_row,
+router_bwd_kernel(const float* __restrict__ dgate,
                   const int* __restrict__ expert_idx, const int* __restrict__ patch_idx,
                   const float* __restrict__ p_samp, const float* __restrict__ p_patch, int n, int k, int m, int c,
                   int l_p, int Lv, float* __restrict__ G) {
@@ -27,31 +45,24 @@ router_bwd_kernel(const float* __restrict__ dg_part, int nt, const int* __restri
     float* pp = sm;                 // [n][m] patch gate
     float* dpp = sm + n * m;        // [n][m] its gradient
     __shared__ float ps[32], dps[32], dls[32];
-    __shared__ float red[4];
-    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = blockIdx.x, tid = threadIdx.x;
     for (int idx = tid; idx < n * m; idx += 128) { pp[idx] = p_patch[(size_t)b * n * m + idx]; dpp[idx] = 0.f; }
     if (tid < n) { ps[tid] = p_samp[(size_t)b * n + tid]; dps[tid] = 0.f; }
     __syncthreads();
-    // dgate of every selected (expert, patch) of this sample, summed in a fixed order
-    for (int su = 0; su < k * c; ++su) {
-        const int s = su / c, u = su % c;
-        const int j = patch_idx[((size_t)b * k + s) * c + u];
-        if (j < 0 || j >= m) continue;                    // uniform across the block
-        const int i = expert_idx[(size_t)b * k + s];
-        const float* src = dg_part + ((size_t)pair_row[b * k + s] + (size_t)u * l_p) * nt;
-        float a = 0.f;
-        for (int q = tid; q < l_p * nt; q += 128) a += src[q];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
-        if (lane == 0) red[warp] = a;
-        __syncthreads();
-        if (tid == 0) {
-            const float dg = (red[0] + red[1]) + (red[2] + red[3]);
-            dps[i] += dg * pp[i * m + j];                 // gate = P_samp * P_patch
-            dpp[i * m + j] += dg * ps[i];
+    // gate = P_samp * P_patch: each chosen expert's slots are handled by one thread, in slot order
+    if (tid < k) {
+        const int i = expert_idx[(size_t)b * k + tid];
+        float acc = 0.f;
+        for (int u = 0; u < c; ++u) {
+            const int j = patch_idx[((size_t)b * k + tid) * c + u];
+            if (j < 0 || j >= m) continue;
+            const float dg = dgate[((size_t)b * k + tid) * c + u];
+            acc += dg * pp[i * m + j];
+            dpp[i * m + j] = dg * ps[i];          // one (expert, patch) pair per slot: no other writer
         }
-        __syncthreads();
+        dps[i] = acc;
     }
+    __syncthreads();
     if (tid == 0) {                                       // softmax Jacobian of the sample gate (Eq. 21)
         float dot = 0.f;
         for (int i = 0; i < n; ++i) dot += ps[i] * dps[i];
@@ -118,16 +129,21 @@ rvec_kernel(const T* __restrict__ W_r, const float* __restrict__ G, float* __res
     }
 }
 
-// dW_r[dd, i] = sum over (b, j) of pool[bj, dd] * G[bj, i]; one thread per dd, fixed order over bj
+// dW_r[dd, i] = sum over (b, j) of pool[bj, dd] * G[bj, i] in two fixed-order stages: grid (d/256, S) partial sums
+// over S chunks of bj, then a sum over the chunks.
+constexpr int kDwrSplit = 16;
 __global__ void __launch_bounds__(kThreads)
-dwr_kernel(const float* __restrict__ pool, const float* __restrict__ G, float* __restrict__ dW_r, int BM, int d, int n) {
+dwr_partial_kernel(const float* __restrict__ pool, const float* __restrict__ G, float* __restrict__ part, int BM, int d,
+                   int n) {
     __shared__ float sG[64 * 32];
     const int dd = blockIdx.x * kThreads + threadIdx.x;
+    const int per = (BM + kDwrSplit - 1) / kDwrSplit;
+    const int lo = blockIdx.y * per, hi = min(BM, lo + per);
     float acc[32];
 #pragma unroll
     for (int i = 0; i < 32; ++i) acc[i] = 0.f;
-    for (int b0 = 0; b0 < BM; b0 += 64) {
-        const int nb = min(64, BM - b0);
+    for (int b0 = lo; b0 < hi; b0 += 64) {
+        const int nb = min(64, hi - b0);
         __syncthreads();
         for (int q = threadIdx.x; q < nb * n; q += kThreads) sG[q] = G[(size_t)b0 * n + q];
         __syncthreads();
@@ -143,11 +159,19 @@ dwr_kernel(const float* __restrict__ pool, const float* __restrict__ G, float* _
     if (dd < d) {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
-            if (i < n) dW_r[(size_t)dd * n + i] = acc[i];
+            if (i < n) part[((size_t)blockIdx.y * d + dd) * n + i] = acc[i];
     }
 }
+__global__ void __launch_bounds__(kThreads)
+dwr_sum_kernel(const float* __restrict__ part, float* __restrict__ dW_r, int total) {
+    const int idx = blockIdx.x * kThreads + threadIdx.x;
+    if (idx >= total) return;
+    float a = 0.f;
+    for (int s = 0; s < kDwrSplit; ++s) a += part[(size_t)s * total + idx];
+    dW_r[idx] = a;
+}
 
-struct BwdWs { size_t plan, dyg, xg, dh, ag, dxg, dgp, G, pool, rvec, total; int nt; };
+struct BwdWs { size_t plan, dyg, xg, dh, ag, dxg, dgp, G, pool, rvec, dgate, wpart, total; int nt; };
 
 BwdWs bwd_ws(const Dims& D) {
     WsCarver w;
@@ -165,6 +189,8 @@ BwdWs bwd_ws(const Dims& D) {
     r.G = w.take((size_t)D.B * D.m * D.n * sizeof(float));
     r.pool = w.take((size_t)D.B * D.m * D.d * sizeof(float));
     r.rvec = w.take((size_t)D.B * D.m * D.d * sizeof(float));
+    r.dgate = w.take((size_t)D.B * D.k * D.c * sizeof(float));
+    r.wpart = w.take((size_t)kDwrSplit * D.d * D.n * sizeof(float));
     r.total = w.off;
     return r;
 }
@@ -212,6 +238,8 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
     float* G = (float*)(base + W.G);
     float* pool = (float*)(base + W.pool);
     float* rvec = (float*)(base + W.rvec);
+    float* dgate = (float*)(base + W.dgate);
+    float* wpart = (float*)(base + W.wpart);
 
     st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream, use_gate);
     if (st != UOE_OK) return st;
@@ -236,9 +264,16 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
 
     if (use_gate) {
         {
+            ProfScope ps("dgate", stream);
+            const int n_slabs = D.B * D.k * D.c;
+            dgate_kernel<<<(n_slabs + 3) / 4, 128, 0, stream>>>(dgp, W.nt, P.pair_row, patch_idx, n_slabs, D.c, D.m, D.l_p,
+                                                               dgate);
+        }
+        UOE_LAUNCHED();
+        {
             ProfScope ps("router_bwd", stream);
             router_bwd_kernel<<<D.B, 128, (size_t)2 * D.n * D.m * sizeof(float), stream>>>(
-                dgp, W.nt, P.pair_row, expert_idx, patch_idx, p_samp, p_patch, D.n, D.k, D.m, D.c, D.l_p, D.Lv, G);
+                dgate, expert_idx, patch_idx, p_samp, p_patch, D.n, D.k, D.m, D.c, D.l_p, D.Lv, G);
         }
         UOE_LAUNCHED();
         int CT = 64;
@@ -252,7 +287,14 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
         UOE_LAUNCHED();
         {
             ProfScope ps("dW_r", stream);
-            dwr_kernel<<<(D.d + kThreads - 1) / kThreads, kThreads, 0, stream>>>(pool, G, dW_r, D.B * D.m, D.d, D.n);
+            dim3 g2((D.d + kThreads - 1) / kThreads, kDwrSplit);
+            dwr_partial_kernel<<<g2, kThreads, 0, stream>>>(pool, G, wpart, D.B * D.m, D.d, D.n);
+        }
+        UOE_LAUNCHED();
+        {
+            ProfScope ps("dW_r_sum", stream);
+            const int total = D.d * D.n;
+            dwr_sum_kernel<<<(total + kThreads - 1) / kThreads, kThreads, 0, stream>>>(wpart, dW_r, total);
         }
         UOE_LAUNCHED();
         {
