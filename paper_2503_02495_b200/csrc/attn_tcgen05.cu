@@ -37,6 +37,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
             const int* __restrict__ pair_row, const int* __restrict__ patch_idx, int c, int l_p, int Lv, int l_a,
             int d_g, int heads, int causal, float scale_log2, int* status) {
+    pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;
@@ -49,9 +50,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int qt = blockIdx.x, head = blockIdx.y, pair = blockIdx.z;
-    const int row_base = pair_row[pair];
     const int q0 = qt * TQ;
 
+    if (warp == 0) tmem_alloc(&ctl->tmem_base, 256);       // S: columns [0,128), O_t: [128,192)
+    pdl_wait();                                             // from here on: data written by earlier kernels
+    const int row_base = pair_row[pair];
     if (tid == 0) {
         mbar_init(&ctl->bar_q, 1);
         mbar_init(&ctl->bar_kv[0], 1);
@@ -68,7 +71,6 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
         s_nvalid = nv;
     }
-    if (warp == 0) tmem_alloc(&ctl->tmem_base, 256);       // S: columns [0,128), O_t: [128,192)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -233,7 +235,7 @@ uoe_status launch_attention(const Dims& D, const void* q, const void* k, const v
     dim3 grid((D.l_a + TQ - 1) / TQ, heads, D.B * D.k);
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)D.d_h);
     ProfScope ps("attention", s);
-    attn_kernel<<<grid, kAttnThreads, ATTN_SMEM, s>>>(tm[0], tm[1], tm[2], (__nv_bfloat16*)o, lse, pair_row, patch_idx,
+    launch_k(attn_kernel, grid, dim3(kAttnThreads), ATTN_SMEM, s, tm[0], tm[1], tm[2], (__nv_bfloat16*)o, lse, pair_row, patch_idx,
                                                       D.c, D.l_p, D.Lv, D.l_a, D.d_g, heads, causal ? 1 : 0,
                                                       scale_log2, status);
     UOE_LAUNCHED();

@@ -31,6 +31,25 @@ extern long long g_launch_count;   // kernels enqueued by this process (reported
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// Every kernel is launched with programmatic stream serialization allowed: the next kernel in the stream may
+// be scheduled, and run up to its pdl_wait(), while this one is still executing, which hides launch and
+// prologue latency between the short kernels of a call.  Kernels call pdl_trigger() first (dependents may
+// be launched once all CTAs of this grid have started) and pdl_wait() before touching global memory.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // While profiling is enabled (uoe_profile_enable), a ProfScope around a launch records a CUDA event
 // before and after it on the launching stream; otherwise it does nothing.
 struct ProfScope {
@@ -81,6 +100,13 @@ struct WsCarver {
     size_t take(size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; }
 };
 constexpr size_t kStatusBytes = 1024;
+
+// ------------------------------------------------------------------------------------------------
+// device side: programmatic dependent launch
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+// returns when every kernel this one depends on has completed and its writes are visible
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
 // ------------------------------------------------------------------------------------------------
 // device side: elements

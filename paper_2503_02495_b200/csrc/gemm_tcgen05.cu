@@ -63,6 +63,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmX, const int* __restrict__ src_patch, int l_p, int Bm,
                  const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                  const __grid_constant__ CUtensorMap tmC2, const __grid_constant__ CUtensorMap tmPre) {
+    pdl_trigger();
     using Cf = Cfg<BN, MT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -78,6 +79,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB0);
     }
+    if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
+    pdl_wait();                     // everything above touches only this CTA's own resources
     if (warp == 2) {                // offsets and the row-tile prefix over experts (n <= 31 here)
         int o = 0;
         if (lane <= n) o = offsets[lane];
@@ -94,7 +97,6 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (lane < n) ctl->tstart[lane] = incl - tiles;
         if (lane == n - 1) ctl->tstart[n] = incl;
     }
-    if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -342,7 +344,7 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     int grid = (int)(max_tiles < sm_count() ? max_tiles : sm_count());
     if (grid < 1) grid = 1;
     ProfScope ps(g.label, s);
-    kern<<<grid, Cf::THREADS, Cf::SMEM, s>>>(tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
+    launch_k(kern, grid, dim3(Cf::THREADS), Cf::SMEM, s, tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
                                              (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
                                              nmat, g.act, status, (const __nv_bfloat16*)g.bwd_h, g.row_gate, g.row_valid,
                                              g.dg_part, tmX, g.gather_x ? g.src_patch : nullptr, g.l_p, g.Bm, tmC[0],

@@ -22,6 +22,8 @@ constexpr int kThreads = 256;
 __global__ void __launch_bounds__(128)
 dgate_kernel(const float* __restrict__ dg_part, int nt, const int* __restrict__ pair_row,
              const int* __restrict__ patch_idx, int n_slabs, int c, int m, int l_p, float* __restrict__ dgate) {
+    pdl_trigger();
+    pdl_wait();
     const int slab = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
     if (slab >= n_slabs) return;
     const int j = patch_idx[slab];
@@ -41,6 +43,8 @@ router_bwd_kernel(const float* __restrict__ dgate,
                   const int* __restrict__ expert_idx, const int* __restrict__ patch_idx,
                   const float* __restrict__ p_samp, const float* __restrict__ p_patch, int n, int k, int m, int c,
                   int l_p, int Lv, float* __restrict__ G) {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ float sm[];
     float* pp = sm;                 // [n][m] patch gate
     float* dpp = sm + n * m;        // [n][m] its gradient
@@ -84,6 +88,8 @@ router_bwd_kernel(const float* __restrict__ dgate,
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 pool_kernel(const T* __restrict__ x, float* __restrict__ pool, int L, int Lv, int d, int m, int l_p, int CT) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int V = Vec16<T>::N;
     __shared__ float red[kThreads * V];
     const int bj = blockIdx.x, chunk = blockIdx.y, b = bj / m, j = bj % m;
@@ -118,6 +124,8 @@ pool_kernel(const T* __restrict__ x, float* __restrict__ pool, int L, int Lv, in
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
 rvec_kernel(const T* __restrict__ W_r, const float* __restrict__ G, float* __restrict__ rvec, int d, int n) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float sG[32];
     const int bj = blockIdx.x;
     if (threadIdx.x < n) sG[threadIdx.x] = G[(size_t)bj * n + threadIdx.x];
@@ -135,6 +143,8 @@ constexpr int kDwrSplit = 16;
 __global__ void __launch_bounds__(kThreads)
 dwr_partial_kernel(const float* __restrict__ pool, const float* __restrict__ G, float* __restrict__ part, int BM, int d,
                    int n) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float sG[64 * 32];
     const int dd = blockIdx.x * kThreads + threadIdx.x;
     const int per = (BM + kDwrSplit - 1) / kDwrSplit;
@@ -164,6 +174,8 @@ dwr_partial_kernel(const float* __restrict__ pool, const float* __restrict__ G, 
 }
 __global__ void __launch_bounds__(kThreads)
 dwr_sum_kernel(const float* __restrict__ part, float* __restrict__ dW_r, int total) {
+    pdl_trigger();
+    pdl_wait();
     const int idx = blockIdx.x * kThreads + threadIdx.x;
     if (idx >= total) return;
     float a = 0.f;
@@ -266,13 +278,13 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
         {
             ProfScope ps("dgate", stream);
             const int n_slabs = D.B * D.k * D.c;
-            dgate_kernel<<<(n_slabs + 3) / 4, 128, 0, stream>>>(dgp, W.nt, P.pair_row, patch_idx, n_slabs, D.c, D.m, D.l_p,
+            launch_k(dgate_kernel, dim3((n_slabs + 3) / 4), dim3(128), 0, stream, dgp, W.nt, P.pair_row, patch_idx, n_slabs, D.c, D.m, D.l_p,
                                                                dgate);
         }
         UOE_LAUNCHED();
         {
             ProfScope ps("router_bwd", stream);
-            router_bwd_kernel<<<D.B, 128, (size_t)2 * D.n * D.m * sizeof(float), stream>>>(
+            launch_k(router_bwd_kernel, dim3(D.B), dim3(128), (size_t)2 * D.n * D.m * sizeof(float), stream, 
                 dgate, expert_idx, patch_idx, p_samp, p_patch, D.n, D.k, D.m, D.c, D.l_p, D.Lv, G);
         }
         UOE_LAUNCHED();
@@ -281,25 +293,25 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
         dim3 grid(D.B * D.m, (D.d + CT * 8 - 1) / (CT * 8));
         {
             ProfScope ps("pool", stream);
-            pool_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>((const __nv_bfloat16*)x, pool, D.L, D.Lv, D.d,
+            launch_k(pool_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, stream, (const __nv_bfloat16*)x, pool, D.L, D.Lv, D.d,
                                                                       D.m, D.l_p, CT);
         }
         UOE_LAUNCHED();
         {
             ProfScope ps("dW_r", stream);
             dim3 g2((D.d + kThreads - 1) / kThreads, kDwrSplit);
-            dwr_partial_kernel<<<g2, kThreads, 0, stream>>>(pool, G, wpart, D.B * D.m, D.d, D.n);
+            launch_k(dwr_partial_kernel, g2, dim3(kThreads), 0, stream, pool, G, wpart, D.B * D.m, D.d, D.n);
         }
         UOE_LAUNCHED();
         {
             ProfScope ps("dW_r_sum", stream);
             const int total = D.d * D.n;
-            dwr_sum_kernel<<<(total + kThreads - 1) / kThreads, kThreads, 0, stream>>>(wpart, dW_r, total);
+            launch_k(dwr_sum_kernel, dim3((total + kThreads - 1) / kThreads), dim3(kThreads), 0, stream, wpart, dW_r, total);
         }
         UOE_LAUNCHED();
         {
             ProfScope ps("router_dx_vec", stream);
-            rvec_kernel<__nv_bfloat16><<<D.B * D.m, kThreads, 0, stream>>>((const __nv_bfloat16*)W_r, G, rvec, D.d, D.n);
+            launch_k(rvec_kernel<__nv_bfloat16>, dim3(D.B * D.m), dim3(kThreads), 0, stream, (const __nv_bfloat16*)W_r, G, rvec, D.d, D.n);
         }
         UOE_LAUNCHED();
     } else {

@@ -22,6 +22,8 @@ template <typename T>
 __global__ void __launch_bounds__(kScoreThreads)
 route_score_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ partial,
                    int L, int Lv, int d, int n, int m, int l_p, int CT, int nchunks, int* __restrict__ counters) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int V = Vec16<T>::N;
     extern __shared__ uint4 s_w4[];                   // W_r[c0 : c0+cw, :] as stored
     __shared__ float s_cs[kScoreThreads * V];         // per-thread column sums, later the partial dot products
@@ -99,6 +101,8 @@ route_select_kernel(const float* __restrict__ partial, int nchunks, int B, int L
                     int l_p, int use_gate, int* __restrict__ expert_idx, int* __restrict__ patch_idx,
                     float* __restrict__ gate, float* __restrict__ p_samp, float* __restrict__ p_patch,
                     int* __restrict__ offsets, int* __restrict__ load, int* __restrict__ ticket) {
+    pdl_trigger();
+    pdl_wait();
     extern __shared__ float pp[];          // [n][m]: raw sums, then probabilities
     __shared__ float ps[32];               // sample gate
     __shared__ int sel[32];                // chosen experts, ascending
@@ -260,15 +264,15 @@ extern "C" uoe_status uoe_route(const uoe_problem* prob, const void* x, const vo
     {
     ProfScope ps("route_score", stream);
     if (D.bf16)
-        route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
+        launch_k(route_score_kernel<__nv_bfloat16>, grid, dim3(kScoreThreads), (size_t)W.CT * 16 * D.n, stream, 
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks, status);
     else
-        route_score_kernel<float><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
+        launch_k(route_score_kernel<float>, grid, dim3(kScoreThreads), (size_t)W.CT * 16 * D.n, stream, 
             (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks, status);
     }
     UOE_LAUNCHED();
     ProfScope ps("route_select", stream);
-    route_select_kernel<<<D.B, kSelectThreads, (size_t)D.n * D.m * sizeof(float), stream>>>(
+    launch_k(route_select_kernel, dim3(D.B), dim3(kSelectThreads), (size_t)D.n * D.m * sizeof(float), stream, 
         partial, W.nchunks, D.B, D.Lv, D.n, D.k, D.m, D.c, D.l_p, (prob->flags & UOE_FLAG_GATE) ? 1 : 0,
         expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, status + 8, status + 1);
     UOE_LAUNCHED();
@@ -324,13 +328,13 @@ extern "C" uoe_status uoe_route_static(const uoe_problem* prob, const void* x, c
     float* partial = (float*)(base + W.partial);
     dim3 grid(D.B * D.m, W.nchunks);
     if (D.bf16)
-        route_score_kernel<__nv_bfloat16><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
+        launch_k(route_score_kernel<__nv_bfloat16>, grid, dim3(kScoreThreads), (size_t)W.CT * 16 * D.n, stream, 
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks, status);
     else
-        route_score_kernel<float><<<grid, kScoreThreads, (size_t)W.CT * 16 * D.n, stream>>>(
+        launch_k(route_score_kernel<float>, grid, dim3(kScoreThreads), (size_t)W.CT * 16 * D.n, stream, 
             (const float*)x, (const float*)W_r, partial, D.L, D.Lv, D.d, D.n, D.m, D.l_p, W.CT, W.nchunks, status);
     UOE_LAUNCHED();
-    route_select_kernel<<<D.B, kSelectThreads, (size_t)D.n * D.m * sizeof(float), stream>>>(
+    launch_k(route_select_kernel, dim3(D.B), dim3(kSelectThreads), (size_t)D.n * D.m * sizeof(float), stream, 
         partial, W.nchunks, D.B, D.Lv, D.n, D.k, D.m, D.c, D.l_p, (prob->flags & UOE_FLAG_GATE) ? 1 : 0,
         expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, status + 8, status + 1);
     UOE_LAUNCHED();

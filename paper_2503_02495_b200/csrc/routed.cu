@@ -17,6 +17,8 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
             int* __restrict__ expert_end, int* status, float* __restrict__ row_gate, float* __restrict__ row_valid,
             int Lv, int use_gate, int* __restrict__ src_patch, uint4* __restrict__ tail, long long tail_row_vecs,
             long long rows_max) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ int my_e[32], cnt[32], prow[32];
     const int b = blockIdx.x, tid = threadIdx.x;
     const int l_a = c * l_p;
@@ -96,6 +98,8 @@ gather_kernel(const uint4* __restrict__ src, const int* __restrict__ patch_idx, 
               uint4* __restrict__ dst, int n_slabs, int k, int c, int m, long long slab_vecs /* l_p*d*esize/16 */,
               long long row_vecs /* d*esize/16 */, int l_p, int n, uint4* __restrict__ tail, long long tail_row_vecs,
               long long rows_max) {
+    pdl_trigger();
+    pdl_wait();
     const int bx = blockIdx.x;
     long long count;                 // 16-byte pieces to write
     const uint4* s = nullptr;
@@ -142,6 +146,8 @@ __global__ void __launch_bounds__(kThreads)
 combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __restrict__ inv_row,
                const float* __restrict__ inv_gate, T* __restrict__ y, int L, int Lv, int d, int m, int k,
                int l_p, int residual, int use_gate, int rows_per_cta, const float* __restrict__ rvec) {
+    pdl_trigger();
+    pdl_wait();
     constexpr int V = Vec16<T>::N;
     __shared__ int srow[32];
     __shared__ float sg[32];
@@ -196,6 +202,8 @@ __global__ void __launch_bounds__(256)
 gemm_f32_kernel(const float* __restrict__ A, const float* __restrict__ W, const float* __restrict__ bias,
                 float* __restrict__ C, float* __restrict__ pre, const int* __restrict__ offsets, int n, int K, int N,
                 int act, int b_kmajor) {
+    pdl_trigger();
+    pdl_wait();
     __shared__ float As[BK][BM + 4];
     __shared__ float Bs[BK][BN + 4];
     const int total_rows = offsets[n];
@@ -256,7 +264,7 @@ uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_id
                        const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s, bool use_gate, void* tail,
                        long long tail_row_bytes) {
     ProfScope ps("plan", s);
-    plan_kernel<<<D.B, 128, 0, s>>>(expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
+    launch_k(plan_kernel, dim3(D.B), dim3(128), 0, s, expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
                                     P.pair_row, P.inv_row, P.inv_gate, P.expert_end, status, P.row_gate, P.row_valid,
                                     D.Lv, use_gate ? 1 : 0, P.src_patch, (uint4*)tail, tail_row_bytes / 16, D.Rmax);
     UOE_LAUNCHED();
@@ -273,7 +281,7 @@ uoe_status launch_gather(const Dims& D, const void* src, const int* patch_idx, c
     if (nsplit > 128) nsplit = 128;
     dim3 grid(n_slabs + D.n + (tail ? 1 : 0), nsplit);
     ProfScope ps("gather", s);
-    gather_kernel<<<grid, kThreads, 0, s>>>((const uint4*)src, patch_idx, offsets, P.pair_row, P.expert_end,
+    launch_k(gather_kernel, grid, dim3(kThreads), 0, s, (const uint4*)src, patch_idx, offsets, P.pair_row, P.expert_end,
                                             (uint4*)dst, n_slabs, D.k, D.c, D.m, slab_vecs, row_vecs, D.l_p, D.n,
                                             (uint4*)tail, tail_row_bytes / 16, D.Rmax);
     UOE_LAUNCHED();
@@ -289,11 +297,11 @@ uoe_status launch_combine(const Dims& D, const void* x, const void* z, const Pla
     dim3 grid(D.B * D.m, (D.l_p + rows_per_cta - 1) / rows_per_cta);
     ProfScope ps("combine", s);
     if (D.bf16)
-        combine_kernel<__nv_bfloat16><<<grid, kThreads, 0, s>>>(
+        launch_k(combine_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, s, 
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)z, P.inv_row, P.inv_gate, (__nv_bfloat16*)y, D.L, D.Lv,
             D.d, D.m, D.k, D.l_p, residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec);
     else
-        combine_kernel<float><<<grid, kThreads, 0, s>>>((const float*)x, (const float*)z, P.inv_row, P.inv_gate,
+        launch_k(combine_kernel<float>, grid, dim3(kThreads), 0, s, (const float*)x, (const float*)z, P.inv_row, P.inv_gate,
                                                        (float*)y, D.L, D.Lv, D.d, D.m, D.k, D.l_p,
                                                        residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec);
     UOE_LAUNCHED();
@@ -303,7 +311,7 @@ uoe_status launch_combine(const Dims& D, const void* x, const void* z, const Pla
 uoe_status launch_gemm_f32(const GemmArgs& g, cudaStream_t s) {
     dim3 grid((unsigned)((g.rows_max + BM - 1) / BM), (g.N + BN - 1) / BN);
     ProfScope ps(g.label, s);
-    gemm_f32_kernel<<<grid, 256, 0, s>>>((const float*)g.A, (const float*)g.W, (const float*)g.bias, (float*)g.C,
+    launch_k(gemm_f32_kernel, grid, dim3(256), 0, s, (const float*)g.A, (const float*)g.W, (const float*)g.bias, (float*)g.C,
                                          (float*)g.pre, g.offsets, g.n, g.K, g.N, g.act, g.b_kmajor ? 1 : 0);
     UOE_LAUNCHED();
     return UOE_OK;

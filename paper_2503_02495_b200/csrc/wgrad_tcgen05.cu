@@ -47,6 +47,7 @@ __global__ void __launch_bounds__(WCfg<BN, MT>::THREADS, 1)
 wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CUtensorMap tmQ,
              const __grid_constant__ CUtensorMap tmW, const int* __restrict__ offsets, int n, int M, int N,
              int* status) {
+    pdl_trigger();
     using Cf = WCfg<BN, MT>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -62,8 +63,9 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         prefetch_tmap(&tmP);
         prefetch_tmap(&tmQ);
     }
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + n + 1) ctl->offs[threadIdx.x - 64] = offsets[threadIdx.x - 64];
     if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
+    pdl_wait();                     // everything above touches only this CTA's own resources
+    if (threadIdx.x >= 64 && threadIdx.x < 64 + n + 1) ctl->offs[threadIdx.x - 64] = offsets[threadIdx.x - 64];
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -218,7 +220,7 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
     const long long tiles = (long long)n * (M / (MT * BM)) * (N / BN);
     int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     ProfScope ps(label, s);
-    kern<<<grid, Cf::THREADS, Cf::SMEM, s>>>(tmP, tmQ, tmW, offsets, n, M, N, status);
+    launch_k(kern, grid, dim3(Cf::THREADS), Cf::SMEM, s, tmP, tmQ, tmW, offsets, n, M, N, status);
     UOE_LAUNCHED();
     return UOE_OK;
 }
