@@ -19,7 +19,8 @@ rank, world = dist.get_rank(), dist.get_world_size()
 w = gen.WORKLOADS["cfg2_lm"]
 ms, e2e = bench.max_over_ranks([1.0 + rank, 5.0 - rank], world)
 out = {"rank": rank, "ms": ms, "e2e": e2e, "value": bench.job_throughput(w, world, ms)}
-print("RESULT " + json.dumps(out), flush=True)
+with open(os.path.join(sys.argv[2], "rank%d.json" % rank), "w") as f:   # one file per rank: stdout of two ranks can interleave
+    json.dump(out, f)
 dist.barrier()
 dist.destroy_process_group()
 """
@@ -35,10 +36,9 @@ def _torchrun(args, timeout=300):
 def test_max_over_ranks_and_job_throughput(tmp_path):
     worker = tmp_path / "worker.py"
     worker.write_text(WORKER)
-    r = _torchrun([str(worker), ROOT])
+    r = _torchrun([str(worker), ROOT, str(tmp_path)])
     assert r.returncode == 0, r.stderr[-2000:]
-    res = [json.loads(l.split("RESULT ", 1)[1]) for l in r.stdout.splitlines() if "RESULT " in l]
-    assert len(res) == 2
+    res = [json.loads((tmp_path / ("rank%d.json" % i)).read_text()) for i in range(2)]
     for d in res:
         assert d["ms"] == 2.0 and d["e2e"] == 5.0                 # slowest rank decides
         assert d["value"] == pytest.approx(2 * 16 * 512 / 2e-3)    # both replicas' tokens over that time
