@@ -16,9 +16,7 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
-import tempfile
 import time
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
@@ -52,10 +50,9 @@ def work_table(w: gen.Workload):
     R, d, n = w.R, w.d, w.n
     x_bytes = w.B * w.L * d * s
     t = {
-        "route_score": dict(flops=2 * w.B * w.L_valid * d * n, bytes=w.B * w.L_valid * d * s),
+        "route": dict(flops=2 * w.B * w.L_valid * d * n, bytes=w.B * w.L_valid * d * s),
         "gather": dict(flops=0, bytes=2 * R * d * s),
         "combine": dict(flops=2 * R * d, bytes=R * d * s + 2 * x_bytes),
-        "route_select": dict(flops=0, bytes=0),
         "plan": dict(flops=0, bytes=0),
     }
     if w.d_ff:
@@ -146,52 +143,77 @@ def cpu_sample_B(w: gen.Workload) -> int:
 # ------------------------------------------------------------------------------------------------
 
 class ClockSampler:
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """SM clock and clock-event reasons of one GPU, read (never set) through NVML from a background thread
+    every few milliseconds while the timed region runs."""
 
-    def __init__(self, gpu_index: int):
-        self.path = tempfile.mktemp(suffix=".csv")
-        self.proc = None
-        self.idx = gpu_index
-
-    def start(self):
+    def __init__(self, torch_device_index: int, period_s: float = 0.005):
+        import threading
+        self.period = period_s
+        self.sm, self.reasons, self.power = [], set(), []
+        self.sm_max = None
+        self._stop = threading.Event()
+        self._thread = None
+        self._h = None
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.idx}", f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
-                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+            import pynvml
+            import torch
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            h = None
+            try:
+                uuid = str(torch.cuda.get_device_properties(torch_device_index).uuid)
+                h = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode() if not uuid.startswith("GPU-") else uuid.encode())
+            except Exception:
+                h = pynvml.nvmlDeviceGetHandleByIndex(torch_device_index)
+            self._h = h
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
         except Exception:
-            self.proc = None
+            self._h = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
-        if self.proc is None:
-            return out
-        self.proc.terminate()
+    def _sample(self):
+        nv, h = self._nv, self._h
+        self.sm.append(float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+        r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
+        for name, bit in (("hw_slowdown", nv.nvmlClocksEventReasonHwSlowdown),
+                          ("hw_thermal_slowdown", nv.nvmlClocksEventReasonHwThermalSlowdown),
+                          ("sw_thermal_slowdown", nv.nvmlClocksEventReasonSwThermalSlowdown),
+                          ("sw_power_cap", nv.nvmlClocksEventReasonSwPowerCap)):
+            if r & bit:
+                self.reasons.add(name)
         try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        try:
-            for line in open(self.path):
-                f = [t.strip() for t in line.split(",")]
-                if len(f) < 9:
-                    continue
-                try:
-                    sm.append(float(f[1]))
-                    mx.append(float(f[2]))
-                except ValueError:
-                    continue
-                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
-                    if v.lower().startswith("active"):
-                        reasons.add(name)
-            os.unlink(self.path)
+            self.power.append(nv.nvmlDeviceGetPowerUsage(h) / 1000.0)
         except Exception:
             pass
-        if sm:
-            out = {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "reasons": sorted(reasons),
-                   "samples": len(sm)}
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                self._sample()
+            except Exception:
+                break
+            self._stop.wait(self.period)
+
+    def start(self):
+        if self._h is None:
+            return
+        import threading
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": []}
+        if self._thread is None:
+            return out
+        try:
+            self._sample()          # at least one reading taken while the last timed kernels are in flight
+        except Exception:
+            pass
+        self._stop.set()
+        self._thread.join(timeout=2)
+        if self.sm:
+            out = {"sm_mhz": statistics.median(self.sm), "sm_min_mhz": min(self.sm), "sm_max_mhz": self.sm_max,
+                   "reasons": sorted(self.reasons), "samples": len(self.sm),
+                   "power_w_max": max(self.power) if self.power else None, "source": "nvml"}
         return out
 
 
@@ -353,7 +375,7 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
 
 
 TENSOR_KERNELS = ("gemm1_act", "gemm2", "qkv_proj", "out_proj", "attention", "bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2")
-HBM_KERNELS = ("route_score", "gather", "combine", "pool")
+HBM_KERNELS = ("route", "gather", "combine", "pool")
 
 
 def roofline_of(top, w: gen.Workload, peaks, peak_src):
@@ -451,7 +473,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default="cfg2_lm", choices=sorted(gen.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

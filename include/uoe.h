@@ -18,6 +18,10 @@
  *   - Errors are return codes.  Arguments are validated on the host before anything is launched.
  *     A device-side anomaly (a bounded wait that ran out, an index out of range) is recorded in
  *     the first word of the workspace and reported by uoe_read_device_status; kernels never trap.
+ *     That word is sticky: it keeps the first anomaly recorded since it was last cleared, and no
+ *     call clears it on its own (a clear on the stream would sit between the kernels of
+ *     consecutive calls and stop them from overlapping).  A new workspace is prepared once with
+ *     uoe_workspace_init; uoe_read_device_status clears the word after reporting an anomaly.
  *   - Element type: `dtype` selects float32 or bfloat16 storage for x, weights and y.  Products are
  *     accumulated in float32.  Routing probabilities and gates are always float32.
  *
@@ -196,8 +200,14 @@ uoe_status uoe_route_static(const uoe_problem* prob, const void* x, const void* 
 /* Text for a status code (static storage). */
 const char* uoe_status_string(int status);
 
-/* Synchronises `cuda_stream`, reads the status word that the kernels of the last call on `ws` left
- * in the workspace, and returns it (UOE_OK if nothing was recorded). */
+/* Prepares a new workspace (device pointer, at least 1024 bytes): enqueues on `cuda_stream` the zeroing of its
+ * control block (the first 64 KB, or all of a smaller workspace: the status word and the counters that the
+ * kernels leave at zero again after every call).  Call it once per workspace, before the first call that
+ * uses it. */
+uoe_status uoe_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* Synchronises `cuda_stream`, reads the status word of workspace `ws` and returns it: UOE_OK, or the first
+ * anomaly a kernel recorded there since the word was last cleared.  A reported anomaly is cleared. */
 uoe_status uoe_read_device_status(void* ws, void* cuda_stream);
 
 /* Number of this library's kernel launches enqueued by this process so far (for benchmarks). */

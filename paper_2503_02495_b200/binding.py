@@ -98,6 +98,8 @@ def _load():
     lib.uoe_smha_forward.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, f32p, i32p, vp, f32p, vp, sz, vp]
     lib.uoe_status_string.restype = ctypes.c_char_p
     lib.uoe_status_string.argtypes = [ctypes.c_int]
+    lib.uoe_workspace_init.restype = ctypes.c_int
+    lib.uoe_workspace_init.argtypes = [vp, sz, vp]
     lib.uoe_read_device_status.restype = ctypes.c_int
     lib.uoe_read_device_status.argtypes = [vp, vp]
     lib.uoe_launch_count.restype = ctypes.c_int64
@@ -170,7 +172,10 @@ def alloc_workspace(prob: Problem, op: int, device="cuda") -> torch.Tensor:
     nbytes = uoe_workspace_bytes(prob, op)
     if nbytes == 0:
         raise UoeError(1, "uoe_workspace_bytes")
-    return torch.empty(nbytes, dtype=torch.uint8, device=device)
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    with torch.cuda.device(ws.device):
+        _check(_lib.uoe_workspace_init(_ptr(ws), nbytes, _stream()), "uoe_workspace_init")
+    return ws
 
 
 def uoe_read_device_status(ws: torch.Tensor) -> int:

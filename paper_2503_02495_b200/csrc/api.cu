@@ -75,12 +75,23 @@ extern "C" const char* uoe_status_string(int status) {
     }
 }
 
+extern "C" uoe_status uoe_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream) {
+    if (!ws || ws_bytes < kStatusBytes) return UOE_ERR_INVALID_ARG;
+    const size_t bytes = ws_bytes < kControlBytes ? ws_bytes : kControlBytes;
+    if (cudaMemsetAsync(ws, 0, bytes, (cudaStream_t)cuda_stream) != cudaSuccess) return UOE_ERR_CUDA;
+    return UOE_OK;
+}
+
 extern "C" uoe_status uoe_read_device_status(void* ws, void* cuda_stream) {
     if (!ws) return UOE_ERR_INVALID_ARG;
     int v = 0;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     if (cudaMemcpyAsync(&v, ws, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess) return UOE_ERR_CUDA;
     if (cudaStreamSynchronize(s) != cudaSuccess) return UOE_ERR_CUDA;
+    if (v != 0) {      // read and clear: the next anomaly can be recorded again
+        if (cudaMemsetAsync(ws, 0, sizeof(int), s) != cudaSuccess) return UOE_ERR_CUDA;
+        if (cudaStreamSynchronize(s) != cudaSuccess) return UOE_ERR_CUDA;
+    }
     return (uoe_status)v;
 }
 

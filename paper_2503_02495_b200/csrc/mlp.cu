@@ -43,7 +43,6 @@ extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, co
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     char* base = (char*)ws;
     int* status = (int*)base;
-    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
     const PlanPtrs P = plan_ptrs(D, base + W.plan);
     void* xg = base + W.xg;
     void* a = base + W.a;

@@ -84,15 +84,16 @@ router_bwd_kernel(const float* __restrict__ dgate,
     }
 }
 
-// grid (B*m, column chunks): sum of the real rows of each patch, float32 [B*m, d]
+// grid B*m * column chunks (chunk fastest, so concurrent CTAs read x linearly): sum of the real rows of each
+// patch, float32 [B*m, d]
 template <typename T>
 __global__ void __launch_bounds__(kThreads)
-pool_kernel(const T* __restrict__ x, float* __restrict__ pool, int L, int Lv, int d, int m, int l_p, int CT) {
+pool_kernel(const T* __restrict__ x, float* __restrict__ pool, int L, int Lv, int d, int m, int l_p, int CT, int nchunks) {
     pdl_trigger();
     pdl_wait();
     constexpr int V = Vec16<T>::N;
     __shared__ float red[kThreads * V];
-    const int bj = blockIdx.x, chunk = blockIdx.y, b = bj / m, j = bj % m;
+    const int bj = blockIdx.x / nchunks, chunk = blockIdx.x % nchunks, b = bj / m, j = bj % m;
     const int ct = threadIdx.x % CT, rt = threadIdx.x / CT, RT = kThreads / CT;
     const int col = (chunk * CT + ct) * V;
     const int rows = max(0, min(l_p, Lv - j * l_p));
@@ -101,7 +102,20 @@ pool_kernel(const T* __restrict__ x, float* __restrict__ pool, int L, int Lv, in
     for (int v = 0; v < V; ++v) cs[v] = 0.f;
     if (col < d) {
         const T* base = x + ((size_t)b * L + (size_t)j * l_p) * d + col;
-        for (int r = rt; r < rows; r += RT) {
+        int r = rt;
+        for (; r + 7 * RT < rows; r += 8 * RT) {
+            uint4 q[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) q[u] = ld_stream16(base + (size_t)(r + u * RT) * d);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                float f[V];
+                unpack16<T>(q[u], f);
+#pragma unroll
+                for (int v = 0; v < V; ++v) cs[v] += f[v];
+            }
+        }
+        for (; r < rows; r += RT) {
             float f[V];
             unpack16<T>(ld_stream16(base + (size_t)r * d), f);
 #pragma unroll
@@ -241,7 +255,6 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
     const bool residual = (prob->flags & UOE_FLAG_RESIDUAL) != 0;
     char* base = (char*)ws;
     int* status = (int*)base;
-    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
     const PlanPtrs P = plan_ptrs(D, base + W.plan, true);
     // rows of the per-row weights that belong to no pair (region padding) must read as zero
     UOE_CUDA_OK(cudaMemsetAsync(P.row_gate, 0, 2 * align_up((size_t)D.Rmax * 4, 1024), stream));
@@ -290,11 +303,12 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
         UOE_LAUNCHED();
         int CT = 64;
         while (CT > 1 && (CT / 2) * 8 >= D.d) CT /= 2;
-        dim3 grid(D.B * D.m, (D.d + CT * 8 - 1) / (CT * 8));
+        const int nchunks = (D.d + CT * 8 - 1) / (CT * 8);
+        dim3 grid((unsigned)(D.B * D.m * nchunks));
         {
             ProfScope ps("pool", stream);
             launch_k(pool_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, stream, (const __nv_bfloat16*)x, pool, D.L, D.Lv, D.d,
-                                                                      D.m, D.l_p, CT);
+                                                                      D.m, D.l_p, CT, nchunks);
         }
         UOE_LAUNCHED();
         {

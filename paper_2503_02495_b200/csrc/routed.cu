@@ -8,7 +8,9 @@ namespace {
 constexpr int kThreads = 256;
 
 // ---------------------------------------------------------------------------------------------
-// plan: grid B
+// plan: grid B, 128 threads, dynamic shared memory 8*k*c bytes.  Everything a sample needs from global memory
+// (its routing arrays, the offsets, the expert choices of the samples before it) is fetched in one round of
+// independent loads; the rest runs out of shared memory.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(128)
 plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_idx, const float* __restrict__ gate,
@@ -19,60 +21,64 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
             long long rows_max) {
     pdl_trigger();
     pdl_wait();
-    __shared__ int my_e[32], cnt[32], prow[32];
+    extern __shared__ int s_dyn[];
+    int* s_pi = s_dyn;                         // [k*c] patch indices of this sample
+    float* s_g = (float*)(s_dyn + k * c);      // [k*c] gates
+    __shared__ int my_e[32], prow[32], hist[33], offs[34];
     const int b = blockIdx.x, tid = threadIdx.x;
     const int l_a = c * l_p;
+    if (tid < 33) hist[tid] = 0;
+    __syncthreads();
+    // ---- one round of loads ----
     if (tid < k) {
         int e = expert_idx[b * k + tid];
         if (e < 0 || e >= n) { set_status(status, UOE_ERR_DEVICE_INDEX); e = 0; }
         my_e[tid] = e;
-        cnt[tid] = 0;
     }
-    __syncthreads();
-    for (int idx = tid; idx < b * k; idx += 128) {          // samples before b that chose the same expert
+    if (tid <= n) offs[tid] = offsets[tid];
+    for (int idx = tid; idx < k * c; idx += 128) {
+        const int pj = patch_idx[(size_t)b * k * c + idx];
+        if (pj < -1 || pj >= m) set_status(status, UOE_ERR_DEVICE_INDEX);
+        s_pi[idx] = pj;
+        s_g[idx] = gate[(size_t)b * k * c + idx];
+    }
+    for (int idx = tid; idx < b * k; idx += 128) {          // choices of the samples before b, per expert
         const int e = expert_idx[idx];
-        for (int s = 0; s < k; ++s)
-            if (my_e[s] == e) atomicAdd(&cnt[s], 1);
+        if (e >= 0 && e < n) atomicAdd(&hist[e], 1);
     }
     __syncthreads();
     if (tid < k) {
-        const int row = offsets[my_e[tid]] + cnt[tid] * l_a;
+        const int row = offs[my_e[tid]] + hist[my_e[tid]] * l_a;
         prow[tid] = row;
         pair_row[b * k + tid] = row;
     }
     __syncthreads();
-    for (int idx = tid; idx < m * k; idx += 128) {
+    for (int idx = tid; idx < m * k; idx += 128) {          // inverse map: which routed rows feed patch j
         const int j = idx / k, s = idx % k;
-        const int* pi = patch_idx + ((size_t)b * k + s) * c;
         int row = -1;
         float g = 0.f;
-        for (int u = 0; u < c; ++u) {
-            const int pj = pi[u];
-            if (pj < -1 || pj >= m) set_status(status, UOE_ERR_DEVICE_INDEX);
-            if (pj == j) { row = prow[s] + u * l_p; g = gate[((size_t)b * k + s) * c + u]; }
-        }
+        for (int u = 0; u < c; ++u)
+            if (s_pi[s * c + u] == j) { row = prow[s] + u * l_p; g = s_g[s * c + u]; }
         inv_row[((size_t)b * m + j) * k + s] = row;
         inv_gate[((size_t)b * m + j) * k + s] = g;
-    }
-    __shared__ int s_end[32];
-    if (b == 0 && tid < n) {
-        int load = 0;
-        for (int idx = 0; idx < B * k; ++idx) load += (expert_idx[idx] == tid);
-        s_end[tid] = expert_end[tid] = offsets[tid] + load * l_a;
     }
     // source patch of every l_p-row block (used when the GEMM gathers its own A operand)
     for (int idx = tid; idx < k * c; idx += 128) {
         const int s = idx / c, u = idx % c;
-        const int pj = patch_idx[((size_t)b * k + s) * c + u];
+        const int pj = s_pi[idx];
         src_patch[prow[s] / l_p + u] = (pj >= 0 && pj < m) ? b * m + pj : -1;
     }
-    if (b == 0) {
+    if (b == B - 1) {          // the last sample has seen every choice: ends of the expert regions, padding blocks
+        __shared__ int s_end[32];
+        if (tid < k) atomicAdd(&hist[my_e[tid]], 1);
+        __syncthreads();
+        if (tid < n) s_end[tid] = expert_end[tid] = offs[tid] + hist[tid] * l_a;
         __syncthreads();
         for (int i = 0; i < n; ++i)
-            for (int rb = s_end[i] / l_p + tid; rb < offsets[i + 1] / l_p; rb += 128) src_patch[rb] = -1;
+            for (int rb = s_end[i] / l_p + tid; rb < offs[i + 1] / l_p; rb += 128) src_patch[rb] = -1;
     }
     if (tail) {
-        const long long r0 = offsets[n];
+        const long long r0 = offs[n];
         const long long total = (rows_max - r0) * tail_row_vecs;
         for (long long q = (long long)b * 128 + tid; q < total; q += (long long)B * 128)
             tail[r0 * tail_row_vecs + q] = make_uint4(0, 0, 0, 0);
@@ -80,9 +86,9 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
     if (row_gate) {                          // per-row weights for the backward
         for (int idx = tid; idx < k * l_a; idx += 128) {
             const int s = idx / l_a, r = idx % l_a, u = r / l_p;
-            const int pj = patch_idx[((size_t)b * k + s) * c + u];
+            const int pj = s_pi[s * c + u];
             const bool real = pj >= 0 && pj < m && pj * l_p + (r % l_p) < Lv;
-            const float g = use_gate ? gate[((size_t)b * k + s) * c + u] : 1.0f;
+            const float g = use_gate ? s_g[s * c + u] : 1.0f;
             row_gate[prow[s] + r] = real ? g : 0.f;
             row_valid[prow[s] + r] = real ? 1.f : 0.f;
         }
@@ -164,28 +170,40 @@ combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __re
         const int r = r0 + idx / vpr, cv = idx % vpr;
         const int t = j * l_p + r;
         const size_t xo = ((size_t)b * L + t) * d + (size_t)cv * V;
+        // the loads of a round (x and up to four slots) are issued together, then added in ascending slot order
+        const bool real = t < Lv;
+        uint4 xv = make_uint4(0, 0, 0, 0), q[4];
+        if (residual) xv = ld_stream16(x + xo);
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            if (real && u < k && srow[u] >= 0) q[u] = ld_stream16(z + ((size_t)(srow[u] + r)) * d + (size_t)cv * V);
         float acc[V];
-        if (residual) {
-            unpack16<T>(ld_stream16(x + xo), acc);
-        } else {
+        unpack16<T>(xv, acc);
+        if (real) {
+            for (int s0 = 0; s0 < k; s0 += 4) {
+                if (s0 > 0) {
 #pragma unroll
-            for (int v = 0; v < V; ++v) acc[v] = 0.f;
-        }
-        if (t < Lv) {
-            for (int s = 0; s < k; ++s) {
-                if (srow[s] < 0) continue;
-                float f[V];
-                unpack16<T>(ld_stream16(z + ((size_t)(srow[s] + r)) * d + (size_t)cv * V), f);
-                const float g = sg[s];
+                    for (int u = 0; u < 4; ++u)
+                        if (s0 + u < k && srow[s0 + u] >= 0)
+                            q[u] = ld_stream16(z + ((size_t)(srow[s0 + u] + r)) * d + (size_t)cv * V);
+                }
 #pragma unroll
-                for (int v = 0; v < V; ++v) acc[v] = fmaf(g, f[v], acc[v]);
+                for (int u = 0; u < 4; ++u) {
+                    if (s0 + u < k && srow[s0 + u] >= 0) {
+                        float f[V];
+                        unpack16<T>(q[u], f);
+                        const float g = sg[s0 + u];
+#pragma unroll
+                        for (int v = 0; v < V; ++v) acc[v] = fmaf(g, f[v], acc[v]);
+                    }
+                }
             }
             if (rvec) {
                 const float* rp = rvec + (size_t)bj * d + (size_t)cv * V;
 #pragma unroll
                 for (int v = 0; v < V; v += 4) {
-                    const float4 q = *(const float4*)(rp + v);
-                    acc[v] += q.x; acc[v + 1] += q.y; acc[v + 2] += q.z; acc[v + 3] += q.w;
+                    const float4 rq = *(const float4*)(rp + v);
+                    acc[v] += rq.x; acc[v + 1] += rq.y; acc[v + 2] += rq.z; acc[v + 3] += rq.w;
                 }
             }
         }
@@ -263,8 +281,10 @@ gemm_f32_kernel(const float* __restrict__ A, const float* __restrict__ W, const 
 uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_idx, const float* gate,
                        const int* offsets, const PlanPtrs& P, int* status, cudaStream_t s, bool use_gate, void* tail,
                        long long tail_row_bytes) {
+    const size_t smem = (size_t)D.k * D.c * 8;
+    if (smem > 32 * 1024) return UOE_ERR_UNSUPPORTED;      // a sample's routing arrays live in shared memory
     ProfScope ps("plan", s);
-    launch_k(plan_kernel, dim3(D.B), dim3(128), 0, s, expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
+    launch_k(plan_kernel, dim3(D.B), dim3(128), smem, s, expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
                                     P.pair_row, P.inv_row, P.inv_gate, P.expert_end, status, P.row_gate, P.row_valid,
                                     D.Lv, use_gate ? 1 : 0, P.src_patch, (uint4*)tail, tail_row_bytes / 16, D.Rmax);
     UOE_LAUNCHED();

@@ -50,7 +50,6 @@ extern "C" uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, c
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     char* base = (char*)ws;
     int* status = (int*)base;
-    UOE_CUDA_OK(cudaMemsetAsync(base, 0, kStatusBytes, stream));
     const PlanPtrs P = plan_ptrs(D, base + W.plan);
     void *xg = base + W.xg, *q = base + W.q, *k = base + W.k, *v = base + W.v, *o = base + W.o, *z = base + W.z;
 

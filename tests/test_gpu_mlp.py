@@ -131,6 +131,9 @@ def test_bad_arguments_return_codes():
     r = uoe.uoe_route(prob, x, Wr)
     bad = uoe.Routing(r.expert_idx.clone().fill_(99), r.patch_idx, r.gate, r.p_samp, r.p_patch, r.expert_offsets)
     W1, W2 = gen.make_mlp_weights(w)
+    ws = uoe.alloc_workspace(prob, uoe.UOE_OP_MLP_FWD)
     with pytest.raises(uoe.UoeError) as ei:
-        uoe.uoe_mlp_forward(prob, x, to_dev(W1), to_dev(W2), bad)
+        uoe.uoe_mlp_forward(prob, x, to_dev(W1), to_dev(W2), bad, ws=ws)
     assert ei.value.status == 6      # recorded on the device, nothing faulted
+    assert uoe.uoe_read_device_status(ws) == 0       # reporting an anomaly clears the sticky status word
+    uoe.uoe_mlp_forward(prob, x, to_dev(W1), to_dev(W2), r, ws=ws)      # and the workspace is usable again
