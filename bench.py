@@ -289,6 +289,12 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
     stream = torch.cuda.current_stream()
 
     def step(xin):
+        if args.part == "route":          # the router alone (profiling): one uoe_route call on the block's input
+            if blk.pm is not None:
+                uoe.uoe_route(blk.pm, xin, wd["Wr_mlp"], out=blk.rm, ws=blk.ws_rm, check=False)
+                return blk.rm.gate
+            uoe.uoe_route(blk.pa, xin, wd["Wr_att"], out=blk.ra, ws=blk.ws_ra, check=False)
+            return blk.ra.gate
         out = blk.forward(xin)
         if w.backward:
             blk.mlp_backward(xin, dy_dev)
@@ -338,7 +344,8 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
             t0 = time.perf_counter()
             x_in.view(x_pin.dtype).copy_(x_pin, non_blocking=True)
             out = step(x_in)
-            y_pin.copy_(out.view(x_pin.dtype), non_blocking=True)
+            if out.shape == x_in.shape:
+                y_pin.copy_(out.view(x_pin.dtype), non_blocking=True)
             torch.cuda.synchronize()
             if i >= 2:
                 e2e_t.append(time.perf_counter() - t0)
@@ -479,6 +486,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (profiling on a smaller case)")
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing (profiling runs)")
+    ap.add_argument("--part", default="all", choices=["all", "route"], help="time only a part of the step (profiling runs)")
     ap.add_argument("--no-scale", action="store_true", help="do not add the scale workload's summary to the line")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))

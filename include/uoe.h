@@ -191,7 +191,7 @@ uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, const void* 
  *     array and give wrong routing: order them, or use uoe_route with separate workspaces.
  *   - No device status word is kept for this variant (uoe_read_device_status does not apply).
  */
-#define UOE_ROUTE_STATIC_SCRATCH_BYTES (1 << 20)
+#define UOE_ROUTE_STATIC_SCRATCH_BYTES (8 << 20)
 uoe_status uoe_route_static(const uoe_problem* prob, const void* x, const void* W_r,
                             int32_t* expert_idx /* [B,k] */, int32_t* patch_idx /* [B,k,c] */,
                             float* gate /* [B,k,c] */, float* p_samp /* [B,n] */, float* p_patch /* [B,n,m] */,
@@ -201,7 +201,7 @@ uoe_status uoe_route_static(const uoe_problem* prob, const void* x, const void* 
 const char* uoe_status_string(int status);
 
 /* Prepares a new workspace (device pointer, at least 1024 bytes): enqueues on `cuda_stream` the zeroing of its
- * control block (the first 64 KB, or all of a smaller workspace: the status word and the counters that the
+ * control block (the first 1 MiB, or all of a smaller workspace: the status word and the counters that the
  * kernels leave at zero again after every call).  Call it once per workspace, before the first call that
  * uses it. */
 uoe_status uoe_workspace_init(void* ws, size_t ws_bytes, void* cuda_stream);

@@ -11,7 +11,7 @@ std::vector<ProfRec> g_prof;
 }  // namespace
 
 ProfScope::ProfScope(const char* name, cudaStream_t s) : slot(-1), stream(s) {
-    if (!g_prof_on) return;
+    if (!g_prof_on || !name) return;
     ProfRec r{name, nullptr, nullptr};
     if (cudaEventCreate(&r.e0) != cudaSuccess || cudaEventCreate(&r.e1) != cudaSuccess) return;
     cudaEventRecord(r.e0, s);

@@ -100,7 +100,7 @@ struct WsCarver {
     size_t take(size_t bytes) { size_t o = off; off = align_up(off + bytes, 1024); return o; }
 };
 constexpr size_t kStatusBytes = 1024;
-constexpr size_t kControlBytes = 64 * 1024;    // what uoe_workspace_init zeroes: the status block and the counters after it
+constexpr size_t kControlBytes = 1024 * 1024;    // what uoe_workspace_init zeroes: the status block and the counters after it
 
 // ------------------------------------------------------------------------------------------------
 // device side: programmatic dependent launch

@@ -141,164 +141,372 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
     }
 }
 
-// grid B*m * nchunks * rsplit, column chunk fastest: a CTA takes one column chunk of one row slice of a patch,
-// and CTAs that run at the same time cover neighbouring chunks of the same rows, so together they read x
-// linearly.  CT threads span the columns of the chunk (16 bytes each), 256/CT span rows.
-// Dynamic shared memory: the W_r rows of this chunk, CT*V*n elements (staged with cp.async behind the x loads);
-// the CTA that ends up running a sample's selection reuses it for the n*m gate values.
-template <typename T>
-__global__ void __launch_bounds__(kScoreThreads)
-route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ partial,
-             int B, int L, int Lv, int d, int n, int k, int m, int c, int l_p, int CT, int nchunks, int rsplit,
-             int rows_per_cta, int use_gate, int* __restrict__ expert_idx, int* __restrict__ patch_idx,
-             float* __restrict__ gate, float* __restrict__ p_samp, float* __restrict__ p_patch,
-             int* __restrict__ offsets, int* __restrict__ ctl /* word 1: ticket, words 8..: expert loads */,
-             int* __restrict__ sample_ticket /* [B] */) {
+// Three steps, in one kernel (MODE 0) or two (MODE 1, then route_patch_scores_kernel):
+//   1. grid B*m * nchunks * rsplit, column chunk fastest: a CTA takes one column chunk of one row slice of a
+//      patch, sums its rows per column and stores the sums, pool_part[patch, row slice, column].  CTAs that run
+//      at the same time cover neighbouring chunks of the same rows, so together they read x linearly.  CT
+//      threads span the columns of the chunk (16 bytes each), 256/CT span rows.
+//   2. one CTA per patch (MODE 0: the CTA that completes the patch; else the second kernel) adds the row slices in
+//      fixed order and multiplies by W_r:  scores[patch, i] = sum over the patch's real tokens of x[t,:] . W_r[:,i]
+//   3. the CTA that completes a sample runs its selection (select_sample).
+// MODE 0 serves small inputs, where a second launch costs more than the work; two kernels serve large ones,
+// where step 1 should be nothing but streaming.
+// Dynamic shared memory: max(n*m floats for step 3, the blocks of W_r rows for step 2).
+
+template <typename T, int MODE>
+__global__ void __launch_bounds__(kScoreThreads, MODE == 1 ? 6 : 5)
+route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ pool_part,
+             float* __restrict__ scores, int B, int L, int Lv, int d, int n, int k, int m, int c, int l_p, int CT,
+             int nchunks, int rsplit, int rows_per_cta, int wblk_bytes, int csplit, int use_gate,
+             int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
+             float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
+             int* __restrict__ ctl /* word 1: ticket, words 8..: expert loads */, int* __restrict__ sample_ticket /* [B] */,
+             int* __restrict__ patch_ticket /* [B*m] */) {
     pdl_trigger();
     pdl_wait();
     constexpr int V = Vec16<T>::N;
-    extern __shared__ uint4 s_w4[];                   // W_r[c0 : c0+cw, :] as stored
-    __shared__ float s_cs[kScoreThreads * V];         // per-thread column sums, later the partial dot products
-    __shared__ float s_col[64 * V];                   // column sums of the chunk
-    const T* s_w = (const T*)s_w4;
-    const int nparts = nchunks * rsplit;
-    const int bj = blockIdx.x / nparts, part = blockIdx.x % nparts;
-    const int chunk = part % nchunks, rs = part / nchunks;
-    const int b = bj / m, j = bj % m;
+    constexpr int NT = kScoreThreads;
+    extern __shared__ uint4 s_dyn4[];
+    __shared__ __align__(16) float s_cs[NT * V];                    // column sums across row threads; later pooled columns, dot partials
+    __shared__ int s_mine;
     const int tid = threadIdx.x;
-    const int ct = tid % CT, rt = tid / CT, RT = kScoreThreads / CT;
-    const int c0 = chunk * CT * V;
-    const int cw = min(CT * V, d - c0);               // columns of this chunk (a multiple of V)
-    const int col = c0 + ct * V;
-    const int row_lo = rs * rows_per_cta;
-    const int rows = min(max(0, min(l_p, Lv - j * l_p)), row_lo + rows_per_cta);      // this slice: [row_lo, rows)
+    const int nparts = nchunks * rsplit;
+    const int bj = blockIdx.x / nparts;
+    const int cpart = 0;
+    const int b = bj / m, j = bj % m;
 
-    {   // stage the router rows of this chunk: cw*n elements, contiguous and 16-byte aligned
+    // step 2 set-up (used by the CTA that completes a patch)
+    const int groups = NT / n;                    // thread (group g, expert i) strides over the columns
+    const int i = tid % n, g = tid / n;
+    int cb = (wblk_bytes / (n * (int)sizeof(T))) / V * V;
+    cb = min(cb, NT * V);
+    const int cols_per_part = ((d + csplit - 1) / csplit + V - 1) / V * V;
+    const int col_lo = cpart * cols_per_part, col_hi = min(d, col_lo + cols_per_part);
+    const int nblk = col_hi > col_lo ? (col_hi - col_lo + cb - 1) / cb : 0;
+    const float* pp_bj = pool_part + (size_t)bj * rsplit * d;
+    auto stage_w = [&](int blk) {
+        const int c0 = col_lo + blk * cb, cw = min(cb, col_hi - c0);
         const uint4* src = (const uint4*)(W_r + (size_t)c0 * n);
-        const int nvec = cw * n / V;
-        for (int q = tid; q < nvec; q += kScoreThreads)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(s_w4 + q)), "l"(src + q) : "memory");
+        uint4* dst = s_dyn4 + (blk & 1) * (wblk_bytes / 16);
+        const int nvec = cw * n * (int)sizeof(T) / 16;
+        for (int q = tid; q < nvec; q += NT)
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(dst + q)), "l"(src + q) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
-    }
+    };
+    // a patch that is one CTA's work (one part, all columns in one block) never leaves the CTA: its pooled sums
+    // stay in shared memory, no ticket is taken, and the W_r rows are fetched behind the x loads
+    const bool direct = MODE == 0 && nparts == 1 && d <= cb;
+    if (direct) stage_w(0);
 
-    float cs[V];
+    {
+        // ---- 1. column sums of this CTA's rows ----
+        const int part = blockIdx.x % nparts;
+        const int chunk = part % nchunks, rs = part / nchunks;
+        const int ct = tid % CT, rt = tid / CT, RT = NT / CT;
+        const int col = (chunk * CT + ct) * V;
+        const int row_lo = rs * rows_per_cta;
+        const int rows = min(max(0, min(l_p, Lv - j * l_p)), row_lo + rows_per_cta);      // this slice: [row_lo, rows)
+        float cs[V];
 #pragma unroll
-    for (int v = 0; v < V; ++v) cs[v] = 0.f;
-    if (col < d) {
-        const T* base = x + ((size_t)b * L + (size_t)j * l_p) * d + col;
-        int r = row_lo + rt;
-        for (; r + 7 * RT < rows; r += 8 * RT) {
-            uint4 q[8];
+        for (int v = 0; v < V; ++v) cs[v] = 0.f;
+        if (col < d) {
+            const T* base = x + ((size_t)b * L + (size_t)j * l_p) * d + col;
+            int r = row_lo + rt;
+            for (; r + 7 * RT < rows; r += 8 * RT) {
+                uint4 q[8];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) q[u] = ld_stream16(base + (size_t)(r + u * RT) * d);
+                for (int u = 0; u < 8; ++u) q[u] = ld_stream16(base + (size_t)(r + u * RT) * d);
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+                for (int u = 0; u < 8; ++u) {
+                    float f[V];
+                    unpack16<T>(q[u], f);
+#pragma unroll
+                    for (int v = 0; v < V; ++v) cs[v] += f[v];
+                }
+            }
+            for (; r < rows; r += RT) {
                 float f[V];
-                unpack16<T>(q[u], f);
+                unpack16<T>(ld_stream16(base + (size_t)r * d), f);
 #pragma unroll
                 for (int v = 0; v < V; ++v) cs[v] += f[v];
             }
         }
-        for (; r < rows; r += RT) {
-            float f[V];
-            unpack16<T>(ld_stream16(base + (size_t)r * d), f);
+        if (RT > 1) {                           // sum over the row threads, fixed order
 #pragma unroll
-            for (int v = 0; v < V; ++v) cs[v] += f[v];
+            for (int v = 0; v < V; ++v) s_cs[tid * V + v] = cs[v];
+            __syncthreads();
+            if (rt == 0)
+                for (int q = 1; q < RT; ++q)
+#pragma unroll
+                    for (int v = 0; v < V; ++v) cs[v] += s_cs[(q * CT + ct) * V + v];
+        }
+        if (direct) {
+            if (rt == 0 && col < d) {
+#pragma unroll
+                for (int v = 0; v < V; ++v) s_cs[col + v] = cs[v];      // slot 0 of this thread's own column group
+            }
+        } else {
+            if (rt == 0 && col < d) {
+                float4* dst = (float4*)(pool_part + ((size_t)bj * rsplit + rs) * d + col);
+#pragma unroll
+                for (int v = 0; v < V; v += 4) dst[v / 4] = make_float4(cs[v], cs[v + 1], cs[v + 2], cs[v + 3]);
+            }
+            if constexpr (MODE == 1) return;
+            __threadfence();
+            __syncthreads();
+            if (tid == 0) {
+                __threadfence();
+                s_mine = (atomicAdd(&patch_ticket[bj], 1) == nparts - 1);
+                if (s_mine) patch_ticket[bj] = 0;         // left at zero for the next call
+            }
+            __syncthreads();
+            if (!s_mine) return;
+            __threadfence();
+        }
+    }
+
+    if constexpr (MODE != 1) {
+        // ---- 2. scores[bj, cpart, :] = pooled columns . W_r over this CTA's column range, W_r rows staged block
+        //         by block in shared memory (double-buffered when the range takes more than one block) ----
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        if (!direct && nblk > 0) stage_w(0);
+        for (int blk = 0; blk < nblk; ++blk) {
+            const int c0 = col_lo + blk * cb, cw = min(cb, col_hi - c0);
+            if (blk + 1 < nblk) stage_w(blk + 1);
+            for (int q4 = direct ? cw : tid; q4 < cw / 4; q4 += NT) {        // add the row slices, fixed order, loads batched by four
+                const float4* p0 = (const float4*)(pp_bj + c0) + q4;
+                float4 acc = __ldcg(p0);
+                for (int r0 = 1; r0 < rsplit; r0 += 4) {
+                    float4 t[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (r0 + u < rsplit) t[u] = __ldcg((const float4*)((const float*)p0 + (size_t)(r0 + u) * d));
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (r0 + u < rsplit) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
+                }
+                *(float4*)(s_cs + 4 * q4) = acc;
+            }
+            if (blk + 1 < nblk) asm volatile("cp.async.wait_group 1;" ::: "memory");
+            else asm volatile("cp.async.wait_group 0;" ::: "memory");
+            __syncthreads();
+            const T* s_w = (const T*)(s_dyn4 + (blk & 1) * (wblk_bytes / 16));
+            if (g < groups) {           // four independent chains, then the tail: a fixed summation order
+                int cc = g;
+                for (; cc + 3 * groups < cw; cc += 4 * groups) {
+                    a0 = fmaf(s_cs[cc], to_f32(s_w[cc * n + i]), a0);
+                    a1 = fmaf(s_cs[cc + groups], to_f32(s_w[(cc + groups) * n + i]), a1);
+                    a2 = fmaf(s_cs[cc + 2 * groups], to_f32(s_w[(cc + 2 * groups) * n + i]), a2);
+                    a3 = fmaf(s_cs[cc + 3 * groups], to_f32(s_w[(cc + 3 * groups) * n + i]), a3);
+                }
+                for (; cc < cw; cc += groups) a0 = fmaf(s_cs[cc], to_f32(s_w[cc * n + i]), a0);
+            }
+            __syncthreads();
+        }
+        s_cs[tid] = (a0 + a1) + (a2 + a3);
+        __syncthreads();
+        if (tid < n) {
+            float sum = 0.f;
+            for (int q = 0; q < groups; ++q) sum += s_cs[q * n + tid];
+            scores[((size_t)bj * csplit + cpart) * n + tid] = sum;
+            __threadfence();
+        }
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            s_mine = (atomicAdd(&sample_ticket[b], 1) == m * csplit - 1);
+            if (s_mine) sample_ticket[b] = 0;
+        }
+        __syncthreads();
+        if (!s_mine) return;
+        __threadfence();
+        // ---- 3. this CTA completed sample b ----
+        select_sample((float*)s_dyn4, scores, csplit, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
+                      p_patch, offsets, ctl + 8, ctl + 1);
+    }
+}
+
+// Steps 2 and 3 as a kernel of their own (after a MODE 1 launch): grid B*m, one CTA per patch.  Thread t owns
+// columns t, t + 256, ...: it adds the row slices of pool_part for its column (fixed order), reads that column's
+// row of W_r (n consecutive elements) and accumulates one partial score per expert in registers; the CTA then
+// reduces the partials in a fixed order.  NMAX >= n bounds the register tile.
+template <typename T, int NMAX>
+__global__ void __launch_bounds__(kScoreThreads)
+route_patch_scores_kernel(const T* __restrict__ W_r, const float* __restrict__ pool_part, float* __restrict__ scores,
+                          int B, int Lv, int d, int n, int k, int m, int c, int l_p, int rsplit, int use_gate,
+                          int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
+                          float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
+                          int* __restrict__ ctl, int* __restrict__ sample_ticket) {
+    pdl_trigger();
+    pdl_wait();
+    constexpr int NT = kScoreThreads;
+    constexpr int V = Vec16<T>::N;
+    extern __shared__ float s_sel[];
+    __shared__ float s_red[NT / 32][NMAX];
+    __shared__ int s_mine;
+    const int bj = blockIdx.x, b = bj / m, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float* pp_bj = pool_part + (size_t)bj * rsplit * d;
+    const bool vec_rows = (n % V) == 0;           // a row of W_r is a whole number of 16-byte pieces
+    float acc[NMAX];
+#pragma unroll
+    for (int i = 0; i < NMAX; ++i) acc[i] = 0.f;
+    // four columns per round: every load of a round (row slices in batches of four, W_r rows) is issued before
+    // the first use, so a round costs one trip to L2 / HBM
+    for (int c0 = tid; c0 < d; c0 += 4 * NT) {
+        float p[4] = {0.f, 0.f, 0.f, 0.f};
+        uint4 wv[4][NMAX / V];
+        if (vec_rows) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int q = 0; q < NMAX / V; ++q)
+                    if (c0 + u * NT < d && q * V < n) wv[u][q] = *(const uint4*)(W_r + (size_t)(c0 + u * NT) * n + q * V);
+        }
+        for (int r0 = 0; r0 < rsplit; r0 += 4) {
+            float t[4][4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int r = 0; r < 4; ++r)
+                    t[u][r] = (c0 + u * NT < d && r0 + r < rsplit) ? __ldcg(pp_bj + (size_t)(r0 + r) * d + c0 + u * NT) : 0.f;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int r = 0; r < 4; ++r) p[u] += t[u][r];       // ascending slice order
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (c0 + u * NT >= d) continue;
+            if (vec_rows) {
+#pragma unroll
+                for (int q = 0; q < NMAX / V; ++q) {
+                    if (q * V < n) {
+                        float f[V];
+                        unpack16<T>(wv[u][q], f);
+#pragma unroll
+                        for (int v = 0; v < V; ++v) acc[q * V + v] = fmaf(p[u], f[v], acc[q * V + v]);
+                    }
+                }
+            } else {
+                const T* wrow = W_r + (size_t)(c0 + u * NT) * n;
+#pragma unroll
+                for (int i = 0; i < NMAX; ++i)
+                    if (i < n) acc[i] = fmaf(p[u], to_f32(wrow[i]), acc[i]);
+            }
         }
     }
 #pragma unroll
-    for (int v = 0; v < V; ++v) s_cs[tid * V + v] = cs[v];
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    __syncthreads();
-    for (int cc = tid; cc < cw; cc += kScoreThreads) {      // sum over the row threads, fixed order
-        float a = 0.f;
-        for (int q = 0; q < RT; ++q) a += s_cs[(q * CT + cc / V) * V + cc % V];
-        s_col[cc] = a;
+    for (int i = 0; i < NMAX; ++i) {
+        float v = acc[i];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+        if (lane == 0) s_red[warp][i] = v;
     }
-    __syncthreads();
-    // dot products with the n router columns: thread (group g, expert i) strides over the chunk's columns
-    const int groups = kScoreThreads / n;
-    const int i = tid % n, g = tid / n;
-    float a = 0.f;
-    if (g < groups)
-        for (int cc = g; cc < cw; cc += groups) a = fmaf(s_col[cc], to_f32(s_w[cc * n + i]), a);
-    s_cs[tid] = a;
     __syncthreads();
     if (tid < n) {
         float sum = 0.f;
-        for (int q = 0; q < groups; ++q) sum += s_cs[q * n + tid];
-        partial[((size_t)bj * nparts + part) * n + tid] = sum;
+        for (int q = 0; q < NT / 32; ++q) sum += s_red[q][tid];
+        scores[(size_t)bj * n + tid] = sum;
         __threadfence();
     }
-    // the CTA that completes sample b (all m * nparts partials written) runs its selection
-    __shared__ int s_mine;
     __syncthreads();
     if (tid == 0) {
         __threadfence();
-        const int done = atomicAdd(&sample_ticket[b], 1);
-        s_mine = (done == m * nparts - 1);
-        if (s_mine) sample_ticket[b] = 0;         // left at zero for the next call
+        s_mine = (atomicAdd(&sample_ticket[b], 1) == m - 1);
+        if (s_mine) sample_ticket[b] = 0;
     }
     __syncthreads();
     if (!s_mine) return;
     __threadfence();
-    select_sample((float*)s_w4, partial, nparts, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
-                  p_patch, offsets, ctl + 8, ctl + 1);
+    select_sample(s_sel, scores, 1, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch,
+                  offsets, ctl + 8, ctl + 1);
 }
 
-struct RouteWs { size_t tickets, partial, total; int nchunks, CT, rsplit, rows_per_cta; size_t smem; };
+struct RouteWs { size_t tickets, ptickets, scores, pool, total; int nchunks, CT, rsplit, rows_per_cta, wblk_bytes, csplit; size_t smem; bool two_kernels; };
 
 RouteWs route_ws(const Dims& D) {
     const int V = 16 / D.esize;
-    int CT = 64;
+    int CT = kScoreThreads;
     while (CT > 1 && (CT / 2) * V >= D.d) CT /= 2;
     const int nchunks = (D.d + CT * V - 1) / (CT * V);
     const int rows_per_cta = 32 * (kScoreThreads / CT);       // at most four 8-deep load batches per thread
     const int rsplit = (D.l_p + rows_per_cta - 1) / rows_per_cta;
-    WsCarver w;
-    w.take(kStatusBytes);
+    // The control block has a fixed size whatever the problem: status block, then the sample and patch tickets.
+    // Data starts behind it, so no problem shape ever writes data where another shape keeps its tickets, and a
+    // scratch area zeroed once serves calls of any shapes in any order.
     RouteWs r;
-    r.tickets = w.take((size_t)D.B * sizeof(int));            // inside the control block that is zeroed once
-    r.partial = w.take((size_t)D.B * D.m * nchunks * rsplit * D.n * sizeof(float));
+    r.tickets = kStatusBytes;
+    r.ptickets = r.tickets + (size_t)D.B * sizeof(int);
+    WsCarver w;
+    w.take(kControlBytes);
+    // a second launch pays off once step 1 moves enough bytes that it should do nothing but stream; its step-2
+    // CTAs each take a column range whose W_r rows fit one block
+    r.two_kernels = nchunks * rsplit > 1 && (size_t)D.B * D.L * D.d * D.esize >= ((size_t)64 << 20);
+    r.wblk_bytes = 16384;
+    r.csplit = 1;
+    r.scores = w.take((size_t)D.B * D.m * r.csplit * D.n * sizeof(float));
+    r.pool = w.take((size_t)D.B * D.m * rsplit * D.d * sizeof(float));
     r.rsplit = rsplit;
     r.rows_per_cta = rows_per_cta;
     r.total = w.off;
     r.nchunks = nchunks;
     r.CT = CT;
-    const size_t stage = (size_t)CT * 16 * D.n, sel = (size_t)D.n * D.m * sizeof(float);
-    r.smem = stage > sel ? stage : sel;
+    const size_t sel = (size_t)D.n * D.m * sizeof(float), wb = (r.two_kernels ? 1 : 2) * (size_t)r.wblk_bytes;
+    r.smem = sel > wb ? sel : wb;
     return r;
 }
 
-// Checks shared by uoe_route and uoe_route_static, then the launch.  `base` is the scratch (control block,
-// tickets, partials); its control block must have been zero when first used.
+// The launch shared by uoe_route and uoe_route_static.  `base` is the scratch (control block with the tickets,
+// scores, pooled sums); its control block must have been zero when first used.
 uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void* W_r, int32_t* expert_idx,
                         int32_t* patch_idx, float* gate, float* p_samp, float* p_patch, int32_t* expert_offsets,
                         char* base, const RouteWs& W, cudaStream_t stream, bool profile) {
     int* ctl = (int*)base;             // word 0 status (unused here), word 1 ticket, words 8.. expert loads
     int* tickets = (int*)(base + W.tickets);
-    float* partial = (float*)(base + W.partial);
+    int* ptickets = (int*)(base + W.ptickets);
+    float* scores = (float*)(base + W.scores);
+    float* pool = (float*)(base + W.pool);
     const int use_gate = (flags & UOE_FLAG_GATE) ? 1 : 0;
-    dim3 grid((unsigned)(D.B * D.m * W.nchunks * W.rsplit));
-    if (D.bf16) {
-        if (profile) {
-            ProfScope ps("route", stream);
-            launch_k(route_kernel<__nv_bfloat16>, grid, dim3(kScoreThreads), W.smem, stream, (const __nv_bfloat16*)x,
-                     (const __nv_bfloat16*)W_r, partial, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, W.nchunks,
-                     W.rsplit, W.rows_per_cta, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl,
-                     tickets);
-        } else {
-            launch_k(route_kernel<__nv_bfloat16>, grid, dim3(kScoreThreads), W.smem, stream, (const __nv_bfloat16*)x,
-                     (const __nv_bfloat16*)W_r, partial, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, W.nchunks,
-                     W.rsplit, W.rows_per_cta, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl,
-                     tickets);
-        }
-    } else {
-        ProfScope ps("route", stream);
-        launch_k(route_kernel<float>, grid, dim3(kScoreThreads), W.smem, stream, (const float*)x, (const float*)W_r,
-                 partial, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, W.nchunks, W.rsplit, W.rows_per_cta,
-                 use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, tickets);
+    dim3 grid((unsigned)(D.B * D.m * W.nchunks * W.rsplit)), grid2((unsigned)(D.B * D.m));
+#define UOE_ROUTE_ARGS(T) (const T*)x, (const T*)W_r, pool, scores, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, \
+        W.nchunks, W.rsplit, W.rows_per_cta, W.wblk_bytes, W.csplit, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, \
+        tickets, ptickets
+    cudaError_t e;
+    if (!W.two_kernels) {
+        ProfScope ps(profile ? "route" : nullptr, stream);
+        if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0>, grid, dim3(kScoreThreads), W.smem, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
+        else e = launch_k(route_kernel<float, 0>, grid, dim3(kScoreThreads), W.smem, stream, UOE_ROUTE_ARGS(float));
+        if (e != cudaSuccess) return UOE_ERR_CUDA;
+        UOE_LAUNCHED();
+        return UOE_OK;
     }
+    {
+        ProfScope ps(profile ? "route" : nullptr, stream);
+        if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 1>, grid, dim3(kScoreThreads), 0, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
+        else e = launch_k(route_kernel<float, 1>, grid, dim3(kScoreThreads), 0, stream, UOE_ROUTE_ARGS(float));
+    }
+    if (e != cudaSuccess) return UOE_ERR_CUDA;
+    UOE_LAUNCHED();
+    {
+        ProfScope ps(profile ? "route_select" : nullptr, stream);
+        const size_t sel = (size_t)D.n * D.m * sizeof(float);
+#define UOE_SCORE_ARGS(T) (const T*)W_r, pool, scores, D.B, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.rsplit, use_gate, expert_idx, \
+        patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, tickets
+#define UOE_SCORE_LAUNCH(T, NMAX) launch_k(route_patch_scores_kernel<T, NMAX>, grid2, dim3(kScoreThreads), sel, stream, UOE_SCORE_ARGS(T))
+        if (D.bf16) {
+            if (D.n <= 8) e = UOE_SCORE_LAUNCH(__nv_bfloat16, 8);
+            else if (D.n <= 16) e = UOE_SCORE_LAUNCH(__nv_bfloat16, 16);
+            else e = UOE_SCORE_LAUNCH(__nv_bfloat16, 32);
+        } else {
+            if (D.n <= 8) e = UOE_SCORE_LAUNCH(float, 8);
+            else if (D.n <= 16) e = UOE_SCORE_LAUNCH(float, 16);
+            else e = UOE_SCORE_LAUNCH(float, 32);
+        }
+#undef UOE_SCORE_LAUNCH
+#undef UOE_SCORE_ARGS
+    }
+#undef UOE_ROUTE_ARGS
+    if (e != cudaSuccess) return UOE_ERR_CUDA;
     UOE_LAUNCHED();
     return UOE_OK;
 }
@@ -311,10 +519,10 @@ uoe_status route_check(const uoe_problem* prob, Dims& D, RouteWs& W, const void*
     if (!x || !W_r || !expert_idx || !patch_idx || !gate || !p_samp || !p_patch || !expert_offsets)
         return UOE_ERR_INVALID_ARG;
     if (!aligned16(x) || !aligned16(W_r)) return UOE_ERR_INVALID_ARG;
-    if ((size_t)D.n * D.m * sizeof(float) > 32 * 1024) return UOE_ERR_UNSUPPORTED;   // gate values of a sample in shared memory
+    if ((size_t)D.n * D.m * sizeof(float) > 36 * 1024) return UOE_ERR_UNSUPPORTED;   // gate values of a sample in shared memory
     W = route_ws(D);
     if ((long long)D.B * D.m * W.nchunks * W.rsplit > 0x7fffffffll) return UOE_ERR_UNSUPPORTED;
-    if (W.tickets + (size_t)D.B * sizeof(int) > kControlBytes) return UOE_ERR_UNSUPPORTED;   // tickets sit in the zeroed block
+    if (W.ptickets + (size_t)D.B * D.m * sizeof(int) > kControlBytes) return UOE_ERR_UNSUPPORTED;   // tickets must fit the control block
     return UOE_OK;
 }
 
@@ -343,8 +551,8 @@ extern "C" uoe_status uoe_route(const uoe_problem* prob, const void* x, const vo
 // uoe_route_static: the same kernel with its scratch in a built-in device array
 // ------------------------------------------------------------------------------------------------
 
-// Scratch of uoe_route_static: the status block (ticket, expert loads) followed by the partial dot
-// products.  One copy per GPU that loads the library, held until the process exits.
+// Scratch of uoe_route_static: the control block (tickets, expert loads) followed by the scores and the pooled
+// column sums.  One copy per GPU that loads the library, held until the process exits.
 static __device__ __align__(256) unsigned char g_route_static_scratch[UOE_ROUTE_STATIC_SCRATCH_BYTES];
 
 namespace {
