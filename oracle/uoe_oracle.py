@@ -20,6 +20,8 @@ Functions and the passages they follow
   smha_forward     Eq. 27-30, 33-36 (SMHA), masks Eq. 41 and Fig. 4, decomposition Eq. 8-11
   mlp_backward     derivative of mlp_forward with the selection held constant (no paper text;
                    pinned by finite differences)
+  smha_backward    derivative of smha_forward with the selection held constant (no paper text;
+                   pinned by finite differences)
 
 Readings where the paper is silent or garbled are listed in the repository's design notes; the
 ones that matter here: the router is one linear map W_r[d, n] applied to the mean token of a
@@ -380,6 +382,116 @@ def mlp_backward(x, W1, W2, W_r, r: Routing, dy, act: str = "silu", residual: bo
                 dW_r += np.outer(pool[b, j], dl_p)
                 dx[b, j * l_p: j * l_p + cnt[j]] += (W_r @ dl_p)[None, :] / cnt[j]
     return dx, dW1, dW2, dW_r, dgate
+
+
+# ----------------------------------------------------------------------------------------------
+# SMHA backward (selection constant; gates differentiable when use_gate)
+# ----------------------------------------------------------------------------------------------
+
+def _gate_to_router_grads(x, W_r, r: Routing, dgate):
+    """Chain rule from d(loss)/d(gate[b,s,u]) through gate = P_samp[b,i] * P_patch[b,i,j] and the two
+    softmaxes (Eq. 14, 21) into W_r and x.  Returns (dW_r, dx_router)."""
+    B, L, d = x.shape
+    n = W_r.shape[1]
+    m, l_p, L_valid = r.m, r.l_p, r.L_valid
+    dW_r = np.zeros_like(W_r)
+    dxr = np.zeros_like(x)
+    p_samp, p_patch, pool, samp, cnt = router_probs(x, W_r, m, L_valid)
+    for b in range(B):
+        dP_samp = np.zeros(n)
+        dP_patch = np.zeros((n, m))
+        for s in range(r.expert_idx.shape[1]):
+            i = r.expert_idx[b, s]
+            for u in range(r.patch_idx.shape[2]):
+                j = r.patch_idx[b, s, u]
+                if j < 0:
+                    continue
+                dP_samp[i] += dgate[b, s, u] * p_patch[b, i, j]
+                dP_patch[i, j] += dgate[b, s, u] * p_samp[b, i]
+        dl_s = p_samp[b] * (dP_samp - np.dot(p_samp[b], dP_samp))          # softmax Jacobian, Eq. 21
+        dW_r += np.outer(samp[b], dl_s)
+        dxr[b, :L_valid] += (W_r @ dl_s)[None, :] / L_valid
+        for j in range(m):
+            if cnt[j] == 0:
+                continue
+            pj = p_patch[b, :, j]
+            dl_p = pj * (dP_patch[:, j] - np.dot(pj, dP_patch[:, j]))      # softmax Jacobian, Eq. 14
+            dW_r += np.outer(pool[b, j], dl_p)
+            dxr[b, j * l_p: j * l_p + cnt[j]] += (W_r @ dl_p)[None, :] / cnt[j]
+    return dW_r, dxr
+
+
+def smha_backward(x, Wq, Wk, Wv, Wo, W_r, r: Routing, dy, d_h: int, causal: bool, residual: bool = True,
+                  use_gate: bool = True):
+    """Gradients of sum(y * dy) for y = smha_forward(x, ...) with expert_idx / patch_idx frozen.
+
+    Per (sample b, chosen expert i), with h' the gathered tokens, P the masked softmax of Eq. 33 and
+    o = P v (Eq. 34), u' = o W^o_i (Eq. 35), y += gate * u' on the real query rows (Eq. 36):
+      du' = gate * dy (real query rows; pad query rows contribute nothing)
+      dW^o_i += o^T du',  do = du' W^o_i^T
+      dv = P^T do,  dP = do v^T,  dS = P * (dP - rowsum(dP * P)),  dq = dS k / sqrt(d_h),  dk = dS^T q / sqrt(d_h)
+      dW^{q,k,v}_i += h'^T d{q,k,v},  dh' = dq W^q_i^T + dk W^k_i^T + dv W^v_i^T, index-added into dx
+    Returns dx [B,L,d], dWq, dWk, dWv [n,d,d_g], dWo [n,d_g,d], dW_r [d,n], dgate [B,k,c].
+    """
+    B, L, d = x.shape
+    d_g = Wq.shape[2]
+    heads = d_g // d_h
+    l_p, L_valid = r.l_p, r.L_valid
+    dx = dy.copy() if residual else np.zeros_like(dy)
+    dWq, dWk, dWv, dWo = np.zeros_like(Wq), np.zeros_like(Wk), np.zeros_like(Wv), np.zeros_like(Wo)
+    dgate = np.zeros_like(r.gate)
+    full_causal = np.tril(np.ones((L, L), dtype=bool))
+    pad_mask = np.arange(L) < L_valid
+    for b in range(B):
+        for s in range(r.expert_idx.shape[1]):
+            i = r.expert_idx[b, s]
+            tok = gathered_tokens(r, b, s)
+            if len(tok) == 0:
+                continue
+            la = len(tok)
+            hp = x[b, tok]
+            q, kk, v = hp @ Wq[i], hp @ Wk[i], hp @ Wv[i]
+            keep = np.broadcast_to(pad_mask[tok][None, :], (la, la)).copy()
+            if causal:
+                keep &= full_causal[np.ix_(tok, tok)]
+            P = np.zeros((heads, la, la))
+            o = np.zeros((la, d_g))
+            for hd in range(heads):
+                sl = slice(hd * d_h, (hd + 1) * d_h)
+                sc = np.where(keep, (q[:, sl] @ kk[:, sl].T) / math.sqrt(d_h), -np.inf)
+                e = np.exp(sc - sc.max(axis=1, keepdims=True))
+                P[hd] = e / e.sum(axis=1, keepdims=True)
+                o[:, sl] = P[hd] @ v[:, sl]
+            up = o @ Wo[i]
+            dup = np.zeros((la, d))
+            row = 0
+            for u, j in enumerate(r.patch_idx[b, s]):
+                if j < 0:
+                    continue
+                t0, t1 = j * l_p, min((j + 1) * l_p, L_valid)
+                rows = slice(row, row + (t1 - t0))
+                dgate[b, s, u] = np.sum(dy[b, t0:t1] * up[rows])
+                dup[rows] = r.gate[b, s, u] * dy[b, t0:t1]
+                row += l_p
+            dWo[i] += o.T @ dup
+            do = dup @ Wo[i].T
+            dq, dk, dv = np.zeros_like(q), np.zeros_like(kk), np.zeros_like(v)
+            for hd in range(heads):
+                sl = slice(hd * d_h, (hd + 1) * d_h)
+                dv[:, sl] = P[hd].T @ do[:, sl]
+                dP = do[:, sl] @ v[:, sl].T
+                dS = P[hd] * (dP - np.sum(dP * P[hd], axis=1, keepdims=True))
+                dq[:, sl] = dS @ kk[:, sl] / math.sqrt(d_h)
+                dk[:, sl] = dS.T @ q[:, sl] / math.sqrt(d_h)
+            dWq[i] += hp.T @ dq
+            dWk[i] += hp.T @ dk
+            dWv[i] += hp.T @ dv
+            np.add.at(dx[b], tok, dq @ Wq[i].T + dk @ Wk[i].T + dv @ Wv[i].T)
+    dW_r = np.zeros_like(W_r)
+    if use_gate:
+        dW_r, dxr = _gate_to_router_grads(x, W_r, r, dgate)
+        dx += dxr
+    return dx, dWq, dWk, dWv, dWo, dW_r, dgate
 
 
 # ----------------------------------------------------------------------------------------------

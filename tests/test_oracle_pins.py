@@ -417,6 +417,81 @@ def test_backward_matches_finite_differences(act, L_valid, use_gate):
         assert np.all(dWr == 0.0)
 
 
+@pytest.mark.parametrize("causal,L_valid,use_gate,H", [(False, 24, True, 4), (True, 24, True, 4), (False, 21, True, 8),
+                                                        (True, 21, False, 4)])
+def test_smha_backward_matches_finite_differences(causal, L_valid, use_gate, H):
+    w = gen.tiny(B=2, L_valid=L_valid, d=8, H=H, d_h=2)
+    t = _inputs(w, ("att",))
+    x, Wq, Wk, Wv, Wo = t["x"], t["Wq"], t["Wk"], t["Wv"], t["Wo"]
+    Wr = _boost_router(t["Wra"], 10.0)
+    r = orc.route(x, Wr, w.k, w.m, w.c, L_valid=L_valid, use_gate=use_gate)
+    dy = gen.normal(9, 1, x.shape)
+    dy[:, L_valid:] = 0.0
+    dx, dWq, dWk, dWv, dWo, dWr, _ = orc.smha_backward(x, Wq, Wk, Wv, Wo, Wr, r, dy, w.d_h, causal, True, use_gate)
+
+    def loss(**a):
+        rr = orc.with_selection(a["x"], a["Wr"], r.expert_idx, r.patch_idx, w.m, L_valid, use_gate)
+        return float(np.sum(orc.smha_forward(a["x"], a["Wq"], a["Wk"], a["Wv"], a["Wo"], rr, w.d_h, causal) * dy))
+
+    base = dict(x=x, Wq=Wq, Wk=Wk, Wv=Wv, Wo=Wo, Wr=Wr)
+    grads = dict(x=dx, Wq=dWq, Wk=dWk, Wv=dWv, Wo=dWo, Wr=dWr)
+    eps = 1e-5
+    for si, which in enumerate(base):
+        for trial in range(2):
+            v = gen.normal(200 + trial, si, base[which].shape)
+            if which == "x":
+                v[:, L_valid:] = 0.0
+            ap, am = dict(base), dict(base)
+            ap[which] = base[which] + eps * v
+            am[which] = base[which] - eps * v
+            fd = (loss(**ap) - loss(**am)) / (2 * eps)
+            an = float(np.sum(grads[which] * v))
+            assert abs(fd - an) <= 2e-6 * max(1.0, abs(an)), (which, fd, an)
+    if not use_gate:
+        assert np.all(dWr == 0.0)
+
+
+def test_smha_backward_full_selection_equals_dense_attention_gradient():
+    """k = n, c = m, unit weights: the layer is textbook multi-head attention (Eq. 8-11), so its input gradient
+    must equal the gradient of that dense attention, derived here independently (per-head softmax backward)."""
+    w = gen.tiny(B=2, k=4, c=6, d=8, H=4, d_h=2)
+    t = _inputs(w, ("att",))
+    x = t["x"]
+    r = orc.route(x, t["Wra"], w.k, w.m, w.c, use_gate=False)
+    dy = gen.normal(13, 2, x.shape)
+    dx, dWq, dWk, dWv, dWo, dWr, _ = orc.smha_backward(x, t["Wq"], t["Wk"], t["Wv"], t["Wo"], t["Wra"], r, dy, w.d_h,
+                                                       causal=True, residual=False, use_gate=False)
+    WQ = np.concatenate(list(t["Wq"]), axis=1)
+    WK = np.concatenate(list(t["Wk"]), axis=1)
+    WV = np.concatenate(list(t["Wv"]), axis=1)
+    WO = np.concatenate(list(t["Wo"]), axis=0)
+    L = x.shape[1]
+    mask = np.tril(np.ones((L, L), dtype=bool))
+    dx_ref = np.zeros_like(x)
+    dWO = np.zeros_like(WO)
+    for b in range(x.shape[0]):
+        q, k_, v = x[b] @ WQ, x[b] @ WK, x[b] @ WV
+        do = dy[b] @ WO.T
+        dq, dk, dv = np.zeros_like(q), np.zeros_like(k_), np.zeros_like(v)
+        o = np.zeros_like(q)
+        for hd in range(w.H):
+            sl = slice(hd * w.d_h, (hd + 1) * w.d_h)
+            sc = np.where(mask, q[:, sl] @ k_[:, sl].T / np.sqrt(w.d_h), -np.inf)
+            P = np.exp(sc - sc.max(1, keepdims=True))
+            P /= P.sum(1, keepdims=True)
+            o[:, sl] = P @ v[:, sl]
+            dP = do[:, sl] @ v[:, sl].T
+            dS = P * (dP - (dP * P).sum(1, keepdims=True))
+            dv[:, sl] = P.T @ do[:, sl]
+            dq[:, sl] = dS @ k_[:, sl] / np.sqrt(w.d_h)
+            dk[:, sl] = dS.T @ q[:, sl] / np.sqrt(w.d_h)
+        dWO += o.T @ dy[b]
+        dx_ref[b] = dq @ WQ.T + dk @ WK.T + dv @ WV.T
+    assert np.allclose(dx, dx_ref, rtol=1e-10, atol=1e-12)
+    assert np.allclose(np.concatenate(list(dWo), axis=0), dWO, rtol=1e-10, atol=1e-12)
+    assert np.all(dWr == 0.0)
+
+
 # ----------------------------------------------------------------------------------------------
 # planted mistakes: the pins above must notice a wrong oracle
 # ----------------------------------------------------------------------------------------------
