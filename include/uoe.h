@@ -69,7 +69,7 @@ enum {
     UOE_FLAG_CAUSAL = 4        /* SMHA: shared lower-triangular mask over the gathered tokens (Fig. 4) */
 };
 
-typedef enum { UOE_OP_ROUTE = 0, UOE_OP_MLP_FWD = 1, UOE_OP_MLP_BWD = 2, UOE_OP_SMHA_FWD = 3 } uoe_op;
+typedef enum { UOE_OP_ROUTE = 0, UOE_OP_MLP_FWD = 1, UOE_OP_MLP_BWD = 2, UOE_OP_SMHA_FWD = 3, UOE_OP_SMHA_BWD = 4 } uoe_op;
 
 /* One Union-of-Experts block.  L must equal m * l_p; rows t >= L_valid of every sample are padding
  * (they take no part in routing means, are masked as attention keys (Eq. 41), and y = x there). */
@@ -165,6 +165,24 @@ uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, const void* 
                             const int32_t* expert_idx, const int32_t* patch_idx, const float* gate,
                             const int32_t* expert_offsets, void* y /* [B,L,d] */, float* lse,
                             void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * SMHA backward: gradients of sum(y * dy) for y = uoe_smha_forward(x, ...) with the selection (expert_idx,
+ * patch_idx) held constant.  The paper gives no backward text; this is the derivative of Eq. 28-30 and 33-36
+ * (masked softmax attention per chosen expert and head, projections, weighted index-add) and, with
+ * UOE_FLAG_GATE, of the gate through both softmaxes (Eq. 14, 21) into W_r and x.  Nothing saved by the
+ * forward is needed: q, k, v, the attention output and its log-sum-exp are recomputed inside.
+ *   dx [B,L,d] in prob->dtype; dWq, dWk, dWv [n,d,d_g], dWo [n,d_g,d], dW_r [d,n] in float32, overwritten.
+ * bfloat16 with 64-wide heads and d % 128 == 0 only (UOE_ERR_UNSUPPORTED otherwise).  All pointers except
+ * prob are device pointers.
+ */
+uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, const void* Wq, const void* Wk,
+                             const void* Wv, const void* Wo, const void* W_r,
+                             const int32_t* expert_idx, const int32_t* patch_idx, const float* gate,
+                             const int32_t* expert_offsets, const float* p_samp, const float* p_patch,
+                             const void* dy /* [B,L,d] */, void* dx /* [B,L,d] */,
+                             float* dWq, float* dWk, float* dWv, float* dWo, float* dW_r,
+                             void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
  * uoe_route without a workspace argument and without any allocation.  (The paper has no counterpart;

@@ -20,7 +20,7 @@ UOE_ROW_ALIGN = 128
 UOE_F32, UOE_BF16 = 0, 1
 ACTS = {"gelu_erf": 0, "gelu_tanh": 1, "silu": 2, "identity": 3}
 UOE_FLAG_RESIDUAL, UOE_FLAG_GATE, UOE_FLAG_CAUSAL = 1, 2, 4
-UOE_OP_ROUTE, UOE_OP_MLP_FWD, UOE_OP_MLP_BWD, UOE_OP_SMHA_FWD = 0, 1, 2, 3
+UOE_OP_ROUTE, UOE_OP_MLP_FWD, UOE_OP_MLP_BWD, UOE_OP_SMHA_FWD, UOE_OP_SMHA_BWD = 0, 1, 2, 3, 4
 
 
 class UoeError(RuntimeError):
@@ -96,6 +96,9 @@ def _load():
                                      f32p, vp, sz, vp]
     lib.uoe_smha_forward.restype = ctypes.c_int
     lib.uoe_smha_forward.argtypes = [pp, vp, vp, vp, vp, vp, i32p, i32p, f32p, i32p, vp, f32p, vp, sz, vp]
+    lib.uoe_smha_backward.restype = ctypes.c_int
+    lib.uoe_smha_backward.argtypes = [pp, vp, vp, vp, vp, vp, vp, i32p, i32p, f32p, i32p, f32p, f32p, vp, vp, f32p, f32p,
+                                      f32p, f32p, f32p, vp, sz, vp]
     lib.uoe_status_string.restype = ctypes.c_char_p
     lib.uoe_status_string.argtypes = [ctypes.c_int]
     lib.uoe_workspace_init.restype = ctypes.c_int
@@ -284,3 +287,26 @@ def uoe_smha_forward(prob: Problem, x, Wq, Wk, Wv, Wo, r: Routing, y=None, lse=N
     if check:
         _check(uoe_read_device_status(ws), "uoe_smha_forward (device)")
     return y
+
+
+def uoe_smha_backward(prob: Problem, x, Wq, Wk, Wv, Wo, W_r, r: Routing, dy, dx=None, dWq=None, dWk=None, dWv=None,
+                      dWo=None, dW_r=None, ws=None, check: bool = True):
+    for t in (x, Wq, Wk, Wv, Wo, W_r, dy):
+        _contig(t, prob.torch_dtype)
+    f32 = torch.float32
+    new = lambda like: torch.empty(like.shape, dtype=f32, device=x.device)
+    dx = dx if dx is not None else torch.empty_like(x)
+    dWq = dWq if dWq is not None else new(Wq)
+    dWk = dWk if dWk is not None else new(Wk)
+    dWv = dWv if dWv is not None else new(Wv)
+    dWo = dWo if dWo is not None else new(Wo)
+    dW_r = dW_r if dW_r is not None else new(W_r)
+    ws = ws if ws is not None else alloc_workspace(prob, UOE_OP_SMHA_BWD, x.device)
+    st = _lib.uoe_smha_backward(ctypes.byref(prob.c_struct()), _ptr(x), _ptr(Wq), _ptr(Wk), _ptr(Wv), _ptr(Wo), _ptr(W_r),
+                                _ptr(r.expert_idx), _ptr(r.patch_idx), _ptr(r.gate), _ptr(r.expert_offsets),
+                                _ptr(r.p_samp), _ptr(r.p_patch), _ptr(dy), _ptr(dx), _ptr(dWq), _ptr(dWk), _ptr(dWv),
+                                _ptr(dWo), _ptr(dW_r), _ptr(ws), ws.numel(), _stream())
+    _check(st, "uoe_smha_backward")
+    if check:
+        _check(uoe_read_device_status(ws), "uoe_smha_backward (device)")
+    return dx, dWq, dWk, dWv, dWo, dW_r

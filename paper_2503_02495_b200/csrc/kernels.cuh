@@ -8,6 +8,7 @@ size_t route_workspace_bytes(const Dims& D);
 size_t mlp_fwd_workspace_bytes(const Dims& D);
 size_t mlp_bwd_workspace_bytes(const Dims& D);
 size_t smha_fwd_workspace_bytes(const Dims& D);
+size_t smha_bwd_workspace_bytes(const Dims& D);
 
 // Layout of the routing plan inside a workspace: where each (sample, expert) pair's rows start and,
 // for every patch of every sample, which routed rows and gates feed it back (the inverse of Eq. 18).
@@ -114,6 +115,21 @@ inline int gemm_bf16_bn(int N) { return (N % 256 == 0) ? 256 : (N % 128 == 0 ? 1
 uoe_status launch_wgrad_bf16(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
                              long long rows_max, const char* label, int* status, cudaStream_t s);
 uoe_status launch_gemm_f32(const GemmArgs& g, cudaStream_t s);
+
+// Scratch of the router half of a backward pass (all float32).
+struct RouterBwdScratch {
+    float* G;       // [B*m, n]   gradient of the router logits per (sample, patch)
+    float* pool;    // [B*m, d]   sums of the real rows of each patch
+    float* rvec;    // [B*m, d]   W_r G: added to dx on every real token of the patch
+    float* dgate;   // [B,k,c]
+    float* wpart;   // partial sums of dW_r
+};
+size_t router_backward_scratch_bytes(const Dims& D);
+RouterBwdScratch router_backward_scratch(const Dims& D, char* base);
+// dgp: [rows, nt] float32, per-row partials of d(loss)/d(gate) (zero on rows that hold no real token).
+uoe_status launch_router_backward(const Dims& D, const void* x, const void* W_r, const int* expert_idx,
+                                  const int* patch_idx, const float* p_samp, const float* p_patch, const PlanPtrs& P,
+                                  const float* dgp, int nt, const RouterBwdScratch& rs, float* dW_r, cudaStream_t stream);
 uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s);
 
 }  // namespace uoe

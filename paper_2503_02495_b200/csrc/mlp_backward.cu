@@ -223,6 +223,77 @@ BwdWs bwd_ws(const Dims& D) {
 
 }  // namespace
 
+// Router half of a backward pass, shared by the UoME and SMHA backward: per-row partials of d(loss)/d(gate)
+// -> dgate per (sample, expert, patch) -> gradient of the router logits G (softmax Jacobians of Eq. 14 and 21)
+// -> dW_r (through the pooled token sums) and rvec, the vector every real token of a patch receives in dx.
+uoe_status launch_router_backward(const Dims& D, const void* x, const void* W_r, const int* expert_idx,
+                                  const int* patch_idx, const float* p_samp, const float* p_patch, const PlanPtrs& P,
+                                  const float* dgp, int nt, const RouterBwdScratch& rs, float* dW_r, cudaStream_t stream) {
+    if (!D.bf16) return UOE_ERR_UNSUPPORTED;
+    if ((size_t)2 * D.n * D.m * sizeof(float) > 40 * 1024) return UOE_ERR_UNSUPPORTED;
+    float *G = rs.G, *pool = rs.pool, *rvec = rs.rvec, *dgate = rs.dgate, *wpart = rs.wpart;
+    {
+        ProfScope ps("dgate", stream);
+        const int n_slabs = D.B * D.k * D.c;
+        launch_k(dgate_kernel, dim3((n_slabs + 3) / 4), dim3(128), 0, stream, dgp, nt, P.pair_row, patch_idx, n_slabs, D.c, D.m, D.l_p,
+                                                           dgate);
+    }
+    UOE_LAUNCHED();
+    {
+        ProfScope ps("router_bwd", stream);
+        launch_k(router_bwd_kernel, dim3(D.B), dim3(128), (size_t)2 * D.n * D.m * sizeof(float), stream, 
+            dgate, expert_idx, patch_idx, p_samp, p_patch, D.n, D.k, D.m, D.c, D.l_p, D.Lv, G);
+    }
+    UOE_LAUNCHED();
+    int CT = 64;
+    while (CT > 1 && (CT / 2) * 8 >= D.d) CT /= 2;
+    const int nchunks = (D.d + CT * 8 - 1) / (CT * 8);
+    dim3 grid((unsigned)(D.B * D.m * nchunks));
+    {
+        ProfScope ps("pool", stream);
+        launch_k(pool_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, stream, (const __nv_bfloat16*)x, pool, D.L, D.Lv, D.d,
+                                                                  D.m, D.l_p, CT, nchunks);
+    }
+    UOE_LAUNCHED();
+    {
+        ProfScope ps("dW_r", stream);
+        dim3 g2((D.d + kThreads - 1) / kThreads, kDwrSplit);
+        launch_k(dwr_partial_kernel, g2, dim3(kThreads), 0, stream, pool, G, wpart, D.B * D.m, D.d, D.n);
+    }
+    UOE_LAUNCHED();
+    {
+        ProfScope ps("dW_r_sum", stream);
+        const int total = D.d * D.n;
+        launch_k(dwr_sum_kernel, dim3((total + kThreads - 1) / kThreads), dim3(kThreads), 0, stream, wpart, dW_r, total);
+    }
+    UOE_LAUNCHED();
+    {
+        ProfScope ps("router_dx_vec", stream);
+        launch_k(rvec_kernel<__nv_bfloat16>, dim3(D.B * D.m), dim3(kThreads), 0, stream, (const __nv_bfloat16*)W_r, G, rvec, D.d, D.n);
+    }
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
+
+size_t router_backward_scratch_bytes(const Dims& D) {
+    return align_up((size_t)D.B * D.m * D.n * 4, 1024) + 2 * align_up((size_t)D.B * D.m * D.d * 4, 1024) +
+           align_up((size_t)D.B * D.k * D.c * 4, 1024) + align_up((size_t)kDwrSplit * D.d * D.n * 4, 1024);
+}
+
+RouterBwdScratch router_backward_scratch(const Dims& D, char* base) {
+    RouterBwdScratch r;
+    r.G = (float*)base;
+    base += align_up((size_t)D.B * D.m * D.n * 4, 1024);
+    r.pool = (float*)base;
+    base += align_up((size_t)D.B * D.m * D.d * 4, 1024);
+    r.rvec = (float*)base;
+    base += align_up((size_t)D.B * D.m * D.d * 4, 1024);
+    r.dgate = (float*)base;
+    base += align_up((size_t)D.B * D.k * D.c * 4, 1024);
+    r.wpart = (float*)base;
+    return r;
+}
+
 size_t mlp_bwd_workspace_bytes(const Dims& D) { return bwd_ws(D).total; }
 
 }  // namespace uoe
@@ -288,46 +359,9 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
     if (st != UOE_OK) return st;
 
     if (use_gate) {
-        {
-            ProfScope ps("dgate", stream);
-            const int n_slabs = D.B * D.k * D.c;
-            launch_k(dgate_kernel, dim3((n_slabs + 3) / 4), dim3(128), 0, stream, dgp, W.nt, P.pair_row, patch_idx, n_slabs, D.c, D.m, D.l_p,
-                                                               dgate);
-        }
-        UOE_LAUNCHED();
-        {
-            ProfScope ps("router_bwd", stream);
-            launch_k(router_bwd_kernel, dim3(D.B), dim3(128), (size_t)2 * D.n * D.m * sizeof(float), stream, 
-                dgate, expert_idx, patch_idx, p_samp, p_patch, D.n, D.k, D.m, D.c, D.l_p, D.Lv, G);
-        }
-        UOE_LAUNCHED();
-        int CT = 64;
-        while (CT > 1 && (CT / 2) * 8 >= D.d) CT /= 2;
-        const int nchunks = (D.d + CT * 8 - 1) / (CT * 8);
-        dim3 grid((unsigned)(D.B * D.m * nchunks));
-        {
-            ProfScope ps("pool", stream);
-            launch_k(pool_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, stream, (const __nv_bfloat16*)x, pool, D.L, D.Lv, D.d,
-                                                                      D.m, D.l_p, CT, nchunks);
-        }
-        UOE_LAUNCHED();
-        {
-            ProfScope ps("dW_r", stream);
-            dim3 g2((D.d + kThreads - 1) / kThreads, kDwrSplit);
-            launch_k(dwr_partial_kernel, g2, dim3(kThreads), 0, stream, pool, G, wpart, D.B * D.m, D.d, D.n);
-        }
-        UOE_LAUNCHED();
-        {
-            ProfScope ps("dW_r_sum", stream);
-            const int total = D.d * D.n;
-            launch_k(dwr_sum_kernel, dim3((total + kThreads - 1) / kThreads), dim3(kThreads), 0, stream, wpart, dW_r, total);
-        }
-        UOE_LAUNCHED();
-        {
-            ProfScope ps("router_dx_vec", stream);
-            launch_k(rvec_kernel<__nv_bfloat16>, dim3(D.B * D.m), dim3(kThreads), 0, stream, (const __nv_bfloat16*)W_r, G, rvec, D.d, D.n);
-        }
-        UOE_LAUNCHED();
+        RouterBwdScratch rs{G, pool, rvec, dgate, wpart};
+        st = launch_router_backward(D, x, W_r, expert_idx, patch_idx, p_samp, p_patch, P, dgp, W.nt, rs, dW_r, stream);
+        if (st != UOE_OK) return st;
     } else {
         UOE_CUDA_OK(cudaMemsetAsync(dW_r, 0, (size_t)D.d * D.n * sizeof(float), stream));
     }
