@@ -68,9 +68,19 @@ def work_table(w: gen.Workload):
     if w.H:
         dg = w.d_g
         att = 4 * w.l_a * w.l_a * dg * w.B * w.k
+        att = att // 2 if w.causal else att
         t["qkv_proj"] = dict(flops=6 * R * d * dg, bytes=(R * d + 3 * R * dg + 3 * n * d * dg) * s)
-        t["attention"] = dict(flops=att // 2 if w.causal else att, bytes=4 * R * dg * s)
+        t["attention"] = dict(flops=att, bytes=4 * R * dg * s)
         t["out_proj"] = dict(flops=2 * R * dg * d, bytes=(R * dg + R * d + n * dg * d) * s)
+    if w.H and w.backward:
+        # algorithmic work of the attention backward is five l_a x l_a contractions (dV, dP, dK, dQ and the
+        # rebuilt S); the dK/dV pass is credited with four of them, the dQ pass with one
+        t["attn_bwd_dkdv"] = dict(flops=2 * att, bytes=6 * R * dg * s)
+        t["attn_bwd_dq"] = dict(flops=att // 2, bytes=5 * R * dg * s)
+        t["bwd_do"] = dict(flops=2 * R * d * dg, bytes=(R * d + R * dg + n * dg * d) * s)
+        t["wgrad_Wo"] = dict(flops=2 * R * d * dg, bytes=(R * d + R * dg) * s + n * d * dg * 4)
+        t["wgrad_Wqkv"] = dict(flops=6 * R * d * dg, bytes=(R * d + 3 * R * dg) * s + 3 * n * d * dg * 4)
+        t["bwd_dx_att"] = dict(flops=6 * R * dg * d, bytes=(3 * R * dg + R * d + 3 * n * d * dg) * s)
     return t
 
 
@@ -83,6 +93,9 @@ def step_flops(w: gen.Workload) -> int:
         f += sum(t[k]["flops"] for k in ("bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2"))
     if w.H:
         f += t["qkv_proj"]["flops"] + t["attention"]["flops"] + t["out_proj"]["flops"]
+    if w.H and w.backward:
+        f += t["attn_bwd_dkdv"]["flops"] + t["attn_bwd_dq"]["flops"] + t["bwd_do"]["flops"] + t["wgrad_Wo"]["flops"] + \
+            t["wgrad_Wqkv"]["flops"] + t["bwd_dx_att"]["flops"]
     return f
 
 
@@ -111,14 +124,18 @@ def oracle_step(w: gen.Workload, h, B=None):
     t0 = time.perf_counter()
     cur = x
     if w.H:
-        r = orc.route(cur, h["Wr_att"].f64, w.k, w.m, w.c, L_valid=w.L_valid)
-        cur = orc.smha_forward(cur, h["Wq"].f64, h["Wk"].f64, h["Wv"].f64, h["Wo"].f64, r, w.d_h, w.causal)
+        r_att = orc.route(cur, h["Wr_att"].f64, w.k, w.m, w.c, L_valid=w.L_valid)
+        cur = orc.smha_forward(cur, h["Wq"].f64, h["Wk"].f64, h["Wv"].f64, h["Wo"].f64, r_att, w.d_h, w.causal)
     if w.d_ff:
         r = orc.route(cur, h["Wr_mlp"].f64, w.k, w.m, w.c, L_valid=w.L_valid)
         u = cur
         cur = orc.mlp_forward(u, h["W1"].f64, h["W2"].f64, r, w.act)
         if w.backward:
-            orc.mlp_backward(u, h["W1"].f64, h["W2"].f64, h["Wr_mlp"].f64, r, h["dy"].f64[:B], w.act)
+            g = orc.mlp_backward(u, h["W1"].f64, h["W2"].f64, h["Wr_mlp"].f64, r, h["dy"].f64[:B], w.act)[0]
+    elif w.backward:
+        g = h["dy"].f64[:B]
+    if w.H and w.backward:
+        orc.smha_backward(x, h["Wq"].f64, h["Wk"].f64, h["Wv"].f64, h["Wo"].f64, h["Wr_att"].f64, r_att, g, w.d_h, w.causal)
     return time.perf_counter() - t0
 
 
@@ -228,7 +245,7 @@ def base_line(w: gen.Workload, args, n_gpus: int):
         "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "stands_in_for": w.stands_in_for, "B": w.B, "L": w.L, "L_valid": w.L_valid,
                    "d": w.d, "n": w.n, "k": w.k, "m": w.m, "c": w.c, "d_ff": w.d_ff, "heads": w.H, "d_h": w.d_h,
-                   "causal": w.causal, "act": w.act, "blocks": ("smha+" if w.H else "") + ("uome" if w.d_ff else "") + ("+uome_backward" if w.backward else ""),
+                   "causal": w.causal, "act": w.act, "blocks": ("smha+" if w.H else "") + ("uome" if w.d_ff else "") + ("+backward" if w.backward else ""),
                    "parallelism": f"replicas x{n_gpus}" if n_gpus > 1 else "single gpu",
                    "l2": "flushed between timed steps (512 MB write)"},
     }
@@ -297,8 +314,14 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
             return blk.ra.gate
         out = blk.forward(xin)
         if w.backward:
-            blk.mlp_backward(xin, dy_dev)
-            return blk.dx
+            g = dy_dev
+            if w.d_ff:
+                blk.mlp_backward(blk.u if w.H else xin, g)
+                g = blk.dx
+            if w.H:
+                blk.smha_backward(xin, g)
+                g = blk.dh
+            return g
         return out
 
     def barrier():
@@ -381,7 +404,8 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
     return res
 
 
-TENSOR_KERNELS = ("gemm1_act", "gemm2", "qkv_proj", "out_proj", "attention", "bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2")
+TENSOR_KERNELS = ("gemm1_act", "gemm2", "qkv_proj", "out_proj", "attention", "bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2",
+                  "attn_bwd_dkdv", "attn_bwd_dq", "bwd_do", "bwd_dx_att", "wgrad_Wo", "wgrad_Wqkv")
 HBM_KERNELS = ("route", "gather", "combine", "pool")
 
 
@@ -486,6 +510,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (profiling on a smaller case)")
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing (profiling runs)")
+    ap.add_argument("--backward", action="store_true", help="add the backward of every half of the block to the step")
     ap.add_argument("--part", default="all", choices=["all", "route"], help="time only a part of the step (profiling runs)")
     ap.add_argument("--no-scale", action="store_true", help="do not add the scale workload's summary to the line")
     args = ap.parse_args()
@@ -495,6 +520,8 @@ def main():
     w = gen.WORKLOADS[args.workload]
     if args.B > 0:
         w = w.replace(B=args.B)
+    if args.backward:
+        w = w.replace(backward=True)
     if args.impl == "reference":
         run_reference(args, w, rank, world)
     else:

@@ -21,6 +21,12 @@ class UoEBlock:
             self.ra = B.alloc_routing(prob_att, device)
             self.ws_ra = B.alloc_workspace(prob_att, B.UOE_OP_ROUTE, device)
             self.ws_a = B.alloc_workspace(prob_att, B.UOE_OP_SMHA_FWD, device)
+            if backward:          # SMHA backward buffers (Eq. 27-36 differentiated)
+                f32 = torch.float32
+                self.ws_ab = B.alloc_workspace(prob_att, B.UOE_OP_SMHA_BWD, device)
+                self.dh = torch.empty_like(self.u)
+                self.dWa = {k: torch.empty(weights[k].shape, dtype=f32, device=device)
+                            for k in ("Wq", "Wk", "Wv", "Wo", "Wr_att")}
         if prob_mlp is not None:
             self.rm = B.alloc_routing(prob_mlp, device)
             self.ws_rm = B.alloc_workspace(prob_mlp, B.UOE_OP_ROUTE, device)
@@ -56,9 +62,16 @@ class UoEBlock:
         return B.uoe_mlp_backward(self.pm, h, w["W1"], w["W2"], w["Wr_mlp"], self.rm, self.saved_h, dy, dx=self.dx,
                                   dW1=self.dW1, dW2=self.dW2, dW_r=self.dWr, ws=self.ws_b, check=check)
 
+    def smha_backward(self, h: torch.Tensor, du: torch.Tensor, check: bool = False):
+        """Backward of the SMHA half for the routing of the last forward(h); du is the gradient w.r.t. its output."""
+        w, g = self.w, self.dWa
+        return B.uoe_smha_backward(self.pa, h, w["Wq"], w["Wk"], w["Wv"], w["Wo"], w["Wr_att"], self.ra, du, dx=self.dh,
+                                   dWq=g["Wq"], dWk=g["Wk"], dWv=g["Wv"], dWo=g["Wo"], dW_r=g["Wr_att"], ws=self.ws_ab,
+                                   check=check)
+
     def device_status(self) -> int:
         worst = 0
-        for name in ("ws_ra", "ws_a", "ws_rm", "ws_m", "ws_b"):
+        for name in ("ws_ra", "ws_a", "ws_rm", "ws_m", "ws_b", "ws_ab"):
             ws = getattr(self, name, None)
             if ws is not None:
                 worst = max(worst, B.uoe_read_device_status(ws))

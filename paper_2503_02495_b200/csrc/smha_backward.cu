@@ -254,7 +254,7 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
     }
     UOE_LAUNCHED();
     GemmArgs gx{dqkv, wcat, nullptr, dxg, nullptr, expert_offsets, D.n, 3 * D.d_g, D.d, UOE_ACT_IDENTITY, true, D.Rmax};
-    gx.label = "bwd_dx";
+    gx.label = "bwd_dx_att";
     st = launch_gemm_bf16(gx, status, stream);
     if (st != UOE_OK) return st;
     st = launch_wgrad_bf16(xg, dqkv, dwcat, expert_offsets, D.n, D.d, 3 * D.d_g, D.Rmax, "wgrad_Wqkv", status, stream);
