@@ -16,6 +16,9 @@ Functions and the passages they follow
   select           Eq. 17 (top-c patches, re-sorted), Eq. 22-23 (top-k experts, per-expert lists),
                    combined as in Fig. 3 / the "superposition" paragraph of Section III-B
   route            the two above + gate weights + buffer offsets
+  patch_expert_counts, dynamic_capacity   Eq. 15-16 (two-stage routing: c = largest number of patches any
+                   expert receives when every patch goes to its k best experts)
+  balance_loss     Eq. 42-44 (sequence-wise load-balancing loss over the patches of one sample)
   mlp_forward      Eq. 18-20 and Eq. 37-40 (UoME), decomposition Eq. 1-7
   smha_forward     Eq. 27-30, 33-36 (SMHA), masks Eq. 41 and Fig. 4, decomposition Eq. 8-11
   mlp_backward     derivative of mlp_forward with the selection held constant (no paper text;
@@ -149,9 +152,42 @@ def _top(values: np.ndarray, candidates: np.ndarray, count: int):
     return np.sort(take), margin
 
 
-def select(p_samp: np.ndarray, p_patch: np.ndarray, cnt: np.ndarray, k: int, c: int):
+def patch_expert_counts(p_patch_b: np.ndarray, cnt: np.ndarray, k: int) -> np.ndarray:
+    """Eq. 15 and the inner sum of Eq. 16 / Eq. 43 for one sample: every patch that holds a real token goes to
+    its k experts with the highest gate (ties: lower index); returns how many patches each expert receives."""
+    n, m = p_patch_b.shape
+    counts = np.zeros(n, dtype=np.int64)
+    for j in range(m):
+        if cnt[j] == 0:
+            continue
+        chosen, _ = _top(p_patch_b[:, j], np.arange(n), k)        # id'_j, Eq. 15
+        counts[chosen] += 1
+    return counts
+
+
+def dynamic_capacity(p_patch: np.ndarray, cnt: np.ndarray, k: int) -> np.ndarray:
+    """Eq. 16 per sample: c = max over experts of the number of patches routed to it in the first stage."""
+    return np.array([patch_expert_counts(p_patch[b], cnt, k).max() for b in range(p_patch.shape[0])], dtype=np.int64)
+
+
+def balance_loss(p_patch: np.ndarray, cnt: np.ndarray, k: int, alpha: float = 1.0) -> np.ndarray:
+    """Eq. 42-44 per sample, the routed units t being the sample's patches that hold a real token (l of them):
+    f_i = n / (k l) * #{t : expert i among the k best of t},  P_i = mean_t g_{i,t},  L = alpha * sum_i f_i P_i."""
+    B, n, m = p_patch.shape
+    elig = np.nonzero(cnt > 0)[0]
+    l = len(elig)
+    out = np.zeros(B)
+    for b in range(B):
+        f = n / (k * l) * patch_expert_counts(p_patch[b], cnt, k)        # Eq. 43
+        P = p_patch[b][:, elig].mean(axis=1)                               # Eq. 44
+        out[b] = alpha * float(np.sum(f * P))                              # Eq. 42
+    return out
+
+
+def select(p_samp: np.ndarray, p_patch: np.ndarray, cnt: np.ndarray, k: int, c: int, dynamic_c: bool = False):
     """Top-k experts per sample (Eq. 22), then top-c patches for each chosen expert (Eq. 17), indices
-    sorted ascending "to restore their original relative position"."""
+    sorted ascending "to restore their original relative position".  With dynamic_c the number of patches
+    per expert is the sample's own c of Eq. 16, capped by the given c (the width of the index array)."""
     B, n = p_samp.shape
     m = p_patch.shape[2]
     eligible = np.nonzero(cnt > 0)[0]
@@ -161,8 +197,9 @@ def select(p_samp: np.ndarray, p_patch: np.ndarray, cnt: np.ndarray, k: int, c: 
     p_margin = np.zeros((B, k))
     for b in range(B):
         expert_idx[b], e_margin[b] = _top(p_samp[b], np.arange(n), k)
+        c_b = min(c, int(patch_expert_counts(p_patch[b], cnt, k).max())) if dynamic_c else c
         for s, i in enumerate(expert_idx[b]):
-            take, p_margin[b, s] = _top(p_patch[b, i], eligible, min(c, len(eligible)))
+            take, p_margin[b, s] = _top(p_patch[b, i], eligible, min(c_b, len(eligible)))
             patch_idx[b, s, :len(take)] = take
     return expert_idx, patch_idx, e_margin, p_margin
 
@@ -196,12 +233,12 @@ def buffer_offsets(expert_idx: np.ndarray, n: int, rows_per_pair: int, row_align
 
 
 def route(x, W_r, k: int, m: int, c: int, L_valid: int | None = None, use_gate: bool = True,
-          row_align: int = 128) -> Routing:
+          row_align: int = 128, dynamic_c: bool = False) -> Routing:
     B, L, d = x.shape
     n = W_r.shape[1]
     L_valid = L if L_valid is None else L_valid
     p_samp, p_patch, _, _, cnt = router_probs(x, W_r, m, L_valid)
-    expert_idx, patch_idx, e_margin, p_margin = select(p_samp, p_patch, cnt, k, c)
+    expert_idx, patch_idx, e_margin, p_margin = select(p_samp, p_patch, cnt, k, c, dynamic_c)
     g = gates(p_samp, p_patch, expert_idx, patch_idx, use_gate)
     load, offsets = buffer_offsets(expert_idx, n, c * (L // m), row_align)
     return Routing(expert_idx, patch_idx, g, p_samp, p_patch, load, offsets, e_margin, p_margin,

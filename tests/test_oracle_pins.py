@@ -381,6 +381,68 @@ def test_array_oracle_equals_scalar_loops(L_valid, causal, act):
 
 
 # ----------------------------------------------------------------------------------------------
+# two-stage dynamic capacity (Eq. 15-16) and load-balancing loss (Eq. 42-44)
+# ----------------------------------------------------------------------------------------------
+
+def test_balance_loss_and_dynamic_capacity_worked_by_hand():
+    # n = 3 experts, k = 1, three patches; gate columns chosen by hand
+    p = np.array([[[0.7, 0.1, 0.5],
+                   [0.2, 0.6, 0.3],
+                   [0.1, 0.3, 0.2]]])                     # [B=1, n, m]
+    cnt = np.array([4, 4, 4])
+    counts = orc.patch_expert_counts(p[0], cnt, 1)
+    assert counts.tolist() == [2, 1, 0]                    # patches 0 and 2 -> expert 0, patch 1 -> expert 1
+    assert orc.dynamic_capacity(p, cnt, 1).tolist() == [2]
+    # f = n/(k l) * counts = [2, 1, 0];  P = row means = [1.3/3, 1.1/3, 0.6/3];  L = 2*1.3/3 + 1.1/3
+    assert orc.balance_loss(p, cnt, 1, alpha=1.0)[0] == pytest.approx((2 * 1.3 + 1.1) / 3, rel=1e-14)
+    assert orc.balance_loss(p, cnt, 1, alpha=0.01)[0] == pytest.approx(0.01 * (2 * 1.3 + 1.1) / 3, rel=1e-14)
+    # k = 2: patch 0 -> {0,1}, patch 1 -> {1,2}, patch 2 -> {0,1}: counts [2,3,1], c = 3
+    assert orc.patch_expert_counts(p[0], cnt, 2).tolist() == [2, 3, 1]
+    assert orc.dynamic_capacity(p, cnt, 2).tolist() == [3]
+
+
+def test_balance_loss_properties():
+    w = gen.tiny(B=4, n=5, k=2, m=6, c=3)
+    t = _inputs(w, ("mlp",))
+    Wr = _boost_router(gen.normal(3, 9, (w.d, w.n)), 2.0)
+    for L_valid in (24, 19):
+        p_samp, p_patch, _, _, cnt = orc.router_probs(t["x"], Wr, w.m, L_valid)
+        l = int((cnt > 0).sum())
+        for b in range(w.B):
+            counts = orc.patch_expert_counts(p_patch[b], cnt, w.k)
+            assert counts.sum() == w.k * l and counts.max() <= l       # every real patch picks exactly k experts
+        # sum_i f_i = n and sum_i P_i = 1, so a uniform gate gives exactly alpha (the loss's minimum over balanced loads)
+        uniform = np.full_like(p_patch, 1.0 / w.n)
+        assert np.allclose(orc.balance_loss(uniform, cnt, w.k, 2.5), 2.5, rtol=1e-13)
+        # all the mass on one expert for every patch: f = [n/k, ...] on k experts, P = e_0 -> alpha * n / k
+        one = np.zeros_like(p_patch)
+        one[:, 0, :] = 1.0
+        assert np.allclose(orc.balance_loss(one, cnt, w.k, 1.0), w.n / w.k, rtol=1e-13)
+        c_dyn = orc.dynamic_capacity(p_patch, cnt, w.k)
+        assert np.all(c_dyn >= -(-w.k * l // w.n)) and np.all(c_dyn <= l)   # pigeonhole bound and at most every patch
+
+
+def test_dynamic_capacity_limits_the_patches_per_expert():
+    w = gen.tiny(B=5, n=4, k=2, m=6, c=6)
+    t = _inputs(w, ("mlp",))
+    Wr = _boost_router(t["Wr"], 30.0)
+    r_fix = orc.route(t["x"], Wr, w.k, w.m, w.c)
+    r_dyn = orc.route(t["x"], Wr, w.k, w.m, w.c, dynamic_c=True)
+    _, p_patch, _, _, cnt = orc.router_probs(t["x"], Wr, w.m, 24)
+    c_dyn = orc.dynamic_capacity(p_patch, cnt, w.k)
+    assert np.array_equal(r_fix.expert_idx, r_dyn.expert_idx)
+    for b in range(w.B):
+        for s in range(w.k):
+            got = r_dyn.patch_idx[b, s]
+            assert (got >= 0).sum() == min(w.c, c_dyn[b])
+            # the dynamic selection is the head of the fixed one in gate order: same top patches, fewer of them
+            i = r_dyn.expert_idx[b, s]
+            best = np.argsort(-p_patch[b, i], kind="stable")[:(got >= 0).sum()]
+            assert sorted(best.tolist()) == got[got >= 0].tolist()
+    assert (c_dyn < w.c).any()          # the case really exercises a smaller capacity
+
+
+# ----------------------------------------------------------------------------------------------
 # backward: central finite differences with the selection frozen
 # ----------------------------------------------------------------------------------------------
 
