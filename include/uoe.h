@@ -66,7 +66,10 @@ typedef enum {
 enum {
     UOE_FLAG_RESIDUAL = 1,     /* y = x + sum(...) (the selective residual of Eq. 20); else y = sum(...) */
     UOE_FLAG_GATE = 2,         /* combine weight = P_samp[b,i] * P_patch[b,i,j]; else 1 (Eq. 20 literal) */
-    UOE_FLAG_CAUSAL = 4        /* SMHA: shared lower-triangular mask over the gathered tokens (Fig. 4) */
+    UOE_FLAG_CAUSAL = 4,       /* SMHA: shared lower-triangular mask over the gathered tokens (Fig. 4) */
+    UOE_FLAG_DYNAMIC_C = 8     /* uoe_route: two-stage routing (Eq. 15-16): every chosen expert of a sample takes
+                                  min(c, c_b) patches, c_b = the largest number of patches any expert receives when
+                                  each patch goes to its k best experts; the remaining slots are unused (-1) */
 };
 
 typedef enum { UOE_OP_ROUTE = 0, UOE_OP_MLP_FWD = 1, UOE_OP_MLP_BWD = 2, UOE_OP_SMHA_FWD = 3, UOE_OP_SMHA_BWD = 4 } uoe_op;
@@ -105,6 +108,7 @@ size_t uoe_workspace_bytes(const uoe_problem* prob, int op);
  *   expert_idx[b,:] = the k experts with the largest p_samp, ascending (ties: lower index)       (Eq. 22)
  *   patch_idx[b,s,:] = for the s-th chosen expert i, the min(c, #patches with a real token) patches
  *                      with the largest p_patch[b,i,:], ascending; unused slots are -1            (Eq. 17)
+ *                      (with UOE_FLAG_DYNAMIC_C also at most the sample's own capacity, Eq. 15-16)
  *   gate[b,s,u]     = p_samp[b,i] * p_patch[b,i,patch] with UOE_FLAG_GATE, else 1; 0 in unused slots
  *   expert_offsets  = row offsets of the per-expert regions (see "Routed buffers")               (Eq. 23)
  * All arguments except prob are device pointers.  x [B,L,d] and W_r [d,n] have prob->dtype;
@@ -114,6 +118,19 @@ uoe_status uoe_route(const uoe_problem* prob, const void* x, const void* W_r,
                      int32_t* expert_idx /* [B,k] */, int32_t* patch_idx /* [B,k,c] */,
                      float* gate /* [B,k,c] */, float* p_samp /* [B,n] */, float* p_patch /* [B,n,m] */,
                      int32_t* expert_offsets /* [n+1] */, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
+ * Load statistics of the patch gate (device pointers; p_patch [B,n,m] as written by uoe_route):
+ *   expert_count[b,i] = number of real patches of sample b that have expert i among their k best experts
+ *                       (Eq. 15; ties: lower index)                                       int32 [B,n], or NULL
+ *   c_dyn[b]          = max_i expert_count[b,i], the dynamic capacity of Eq. 16            int32 [B], or NULL
+ *   lb_loss[b]        = alpha * sum_i f_i P_i, the sequence-wise load-balancing loss of Eq. 42-44 taken over the
+ *                       sample's real patches: f_i = n/(k l) expert_count[b,i], P_i = mean gate of expert i
+ *                                                                                           float32 [B], or NULL
+ * Needs no workspace.
+ */
+uoe_status uoe_route_balance(const uoe_problem* prob, const float* p_patch, float alpha, float* lb_loss,
+                             int32_t* expert_count, int32_t* c_dyn, void* cuda_stream);
 
 /*
  * UoME forward (Eq. 37-40 with the index-select of Eq. 18 and the index-add of Eq. 20):

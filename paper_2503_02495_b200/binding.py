@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libuoe.so")
 UOE_ROW_ALIGN = 128
 UOE_F32, UOE_BF16 = 0, 1
 ACTS = {"gelu_erf": 0, "gelu_tanh": 1, "silu": 2, "identity": 3}
-UOE_FLAG_RESIDUAL, UOE_FLAG_GATE, UOE_FLAG_CAUSAL = 1, 2, 4
+UOE_FLAG_RESIDUAL, UOE_FLAG_GATE, UOE_FLAG_CAUSAL, UOE_FLAG_DYNAMIC_C = 1, 2, 4, 8
 UOE_OP_ROUTE, UOE_OP_MLP_FWD, UOE_OP_MLP_BWD, UOE_OP_SMHA_FWD, UOE_OP_SMHA_BWD = 0, 1, 2, 3, 4
 
 
@@ -54,10 +54,11 @@ class Problem:
     residual: bool = True
     gate: bool = True
     causal: bool = False
+    dynamic_c: bool = False
 
     def c_struct(self) -> _Problem:
         flags = (UOE_FLAG_RESIDUAL if self.residual else 0) | (UOE_FLAG_GATE if self.gate else 0) | \
-                (UOE_FLAG_CAUSAL if self.causal else 0)
+                (UOE_FLAG_CAUSAL if self.causal else 0) | (UOE_FLAG_DYNAMIC_C if self.dynamic_c else 0)
         return _Problem(self.B, self.L, self.L_valid, self.d, self.n, self.k, self.m, self.c, self.d_e, self.H,
                         self.d_h, UOE_BF16 if self.dtype == "bf16" else UOE_F32, ACTS[self.act], flags)
 
@@ -99,6 +100,8 @@ def _load():
     lib.uoe_smha_backward.restype = ctypes.c_int
     lib.uoe_smha_backward.argtypes = [pp, vp, vp, vp, vp, vp, vp, i32p, i32p, f32p, i32p, f32p, f32p, vp, vp, f32p, f32p,
                                       f32p, f32p, f32p, vp, sz, vp]
+    lib.uoe_route_balance.restype = ctypes.c_int
+    lib.uoe_route_balance.argtypes = [pp, f32p, ctypes.c_float, f32p, i32p, i32p, vp]
     lib.uoe_status_string.restype = ctypes.c_char_p
     lib.uoe_status_string.argtypes = [ctypes.c_int]
     lib.uoe_workspace_init.restype = ctypes.c_int
@@ -310,3 +313,16 @@ def uoe_smha_backward(prob: Problem, x, Wq, Wk, Wv, Wo, W_r, r: Routing, dy, dx=
     if check:
         _check(uoe_read_device_status(ws), "uoe_smha_backward (device)")
     return dx, dWq, dWk, dWv, dWo, dW_r
+
+
+def uoe_route_balance(prob: Problem, p_patch, alpha: float = 1.0):
+    """(lb_loss [B] float32, expert_count [B,n] int32, c_dyn [B] int32) for the patch gate written by uoe_route."""
+    _contig(p_patch, torch.float32)
+    dev = p_patch.device
+    lb = torch.empty(prob.B, dtype=torch.float32, device=dev)
+    cnt = torch.empty(prob.B, prob.n, dtype=torch.int32, device=dev)
+    cd = torch.empty(prob.B, dtype=torch.int32, device=dev)
+    st = _lib.uoe_route_balance(ctypes.byref(prob.c_struct()), _ptr(p_patch), ctypes.c_float(alpha), _ptr(lb), _ptr(cnt),
+                                _ptr(cd), _stream())
+    _check(st, "uoe_route_balance")
+    return lb, cnt, cd

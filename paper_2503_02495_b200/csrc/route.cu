@@ -18,15 +18,19 @@ constexpr int kScoreThreads = 256;
 
 // Selection for sample b by one CTA of kScoreThreads threads (all threads call).  pp: n*m floats of shared memory.
 __device__ void select_sample(float* pp, const float* __restrict__ partial, int nparts, int b, int B, int Lv, int n, int k,
-                              int m, int c, int l_p, int use_gate, int* __restrict__ expert_idx,
+                              int m, int c, int l_p, int sel_flags /* bit 0: gate weights, bit 1: dynamic capacity */,
+                              int* __restrict__ expert_idx,
                               int* __restrict__ patch_idx, float* __restrict__ gate, float* __restrict__ p_samp,
                               float* __restrict__ p_patch, int* __restrict__ offsets, int* __restrict__ load,
                               int* __restrict__ ticket) {
     constexpr int NT = kScoreThreads;
     __shared__ float ps[32];               // sample gate
     __shared__ int sel[32];                // chosen experts, ascending
+    __shared__ int cnts[32];               // Eq. 16: patches each expert receives in the first routing stage
     __shared__ int s_last;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int use_gate = sel_flags & 1, dynamic_c = (sel_flags >> 1) & 1;
+    if (tid < 32) cnts[tid] = 0;
     const int n_elig = (Lv + l_p - 1) / l_p;       // patches holding at least one real token (a prefix)
 
     for (int idx = tid; idx < n * m; idx += NT) {
@@ -58,6 +62,17 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
             pp[i * m + j] = pr;
             p_patch[((size_t)b * n + i) * m + j] = pr;
         }
+        if (dynamic_c && cnt > 0) {         // Eq. 15: this patch goes to its k best experts (ties: lower index)
+            for (int i = 0; i < n; ++i) {
+                const float v = pp[i * m + j];
+                int rank = 0;
+                for (int q = 0; q < n; ++q) {
+                    const float w = pp[q * m + j];
+                    rank += (w > v) || (w == v && q < i);
+                }
+                if (rank < k) atomicAdd(&cnts[i], 1);
+            }
+        }
     }
     if (warp == 0) {
         const float v = lane < n ? ps[lane] : -INFINITY;
@@ -86,7 +101,12 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
         }
     }
     __syncthreads();
-    const int take = min(c, n_elig);
+    int take = min(c, n_elig);
+    if (dynamic_c) {                        // Eq. 16: c = the largest first-stage count, capped by the slots available
+        int c_dyn = 0;
+        for (int i = 0; i < n; ++i) c_dyn = max(c_dyn, cnts[i]);
+        take = min(take, c_dyn);
+    }
     for (int s = warp; s < k; s += NT / 32) {       // Eq. 17 for the s-th chosen expert
         const int i = sel[s];
         const float* v_i = pp + i * m;
@@ -466,7 +486,7 @@ uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void
     int* ptickets = (int*)(base + W.ptickets);
     float* scores = (float*)(base + W.scores);
     float* pool = (float*)(base + W.pool);
-    const int use_gate = (flags & UOE_FLAG_GATE) ? 1 : 0;
+    const int use_gate = ((flags & UOE_FLAG_GATE) ? 1 : 0) | ((flags & UOE_FLAG_DYNAMIC_C) ? 2 : 0);     // selection flags
     dim3 grid((unsigned)(D.B * D.m * W.nchunks * W.rsplit)), grid2((unsigned)(D.B * D.m));
 #define UOE_ROUTE_ARGS(T) (const T*)x, (const T*)W_r, pool, scores, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, \
         W.nchunks, W.rsplit, W.rows_per_cta, W.wblk_bytes, W.csplit, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, \
@@ -545,6 +565,75 @@ extern "C" uoe_status uoe_route(const uoe_problem* prob, const void* x, const vo
     if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
     return route_launch(D, prob->flags, x, W_r, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, (char*)ws, W,
                         (cudaStream_t)cuda_stream, true);
+}
+
+// ------------------------------------------------------------------------------------------------
+// uoe_route_balance: Eq. 15-16 and 42-44 from the patch gate that uoe_route wrote
+// ------------------------------------------------------------------------------------------------
+namespace uoe {
+namespace {
+// grid B, 128 threads, dynamic shared memory n*m floats.
+__global__ void __launch_bounds__(128)
+balance_kernel(const float* __restrict__ p_patch, int Lv, int n, int k, int m, int l_p, float alpha,
+               float* __restrict__ lb_loss, int* __restrict__ expert_count, int* __restrict__ c_dyn) {
+    pdl_trigger();
+    pdl_wait();
+    extern __shared__ float pp[];          // [n][m]
+    __shared__ int cnts[32];
+    __shared__ float Pm[32];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int n_elig = (Lv + l_p - 1) / l_p;       // patches holding at least one real token (a prefix)
+    for (int idx = tid; idx < n * m; idx += 128) pp[idx] = p_patch[(size_t)b * n * m + idx];
+    if (tid < 32) cnts[tid] = 0;
+    __syncthreads();
+    for (int j = tid; j < n_elig; j += 128) {      // Eq. 15: patch j goes to its k best experts (ties: lower index)
+        for (int i = 0; i < n; ++i) {
+            const float v = pp[i * m + j];
+            int rank = 0;
+            for (int q = 0; q < n; ++q) {
+                const float w = pp[q * m + j];
+                rank += (w > v) || (w == v && q < i);
+            }
+            if (rank < k) atomicAdd(&cnts[i], 1);
+        }
+    }
+    if (tid < n) {                                  // Eq. 44: mean gate of expert i over the real patches, fixed order
+        float s = 0.f;
+        for (int j = 0; j < n_elig; ++j) s += pp[tid * m + j];
+        Pm[tid] = s / (float)n_elig;
+    }
+    __syncthreads();
+    if (tid < n && expert_count) expert_count[(size_t)b * n + tid] = cnts[tid];
+    if (tid == 0) {
+        int cmax = 0;
+        float loss = 0.f;
+        const float fs = (float)n / ((float)k * (float)n_elig);                       // Eq. 43
+        for (int i = 0; i < n; ++i) { cmax = max(cmax, cnts[i]); loss += fs * (float)cnts[i] * Pm[i]; }
+        if (c_dyn) c_dyn[b] = cmax;                                                     // Eq. 16
+        if (lb_loss) lb_loss[b] = alpha * loss;                                         // Eq. 42
+    }
+}
+}  // namespace
+}  // namespace uoe
+
+extern "C" uoe_status uoe_route_balance(const uoe_problem* prob, const float* p_patch, float alpha, float* lb_loss,
+                                        int32_t* expert_count, int32_t* c_dyn, void* cuda_stream) {
+    Dims D;
+    uoe_status st = make_dims(prob, D);
+    if (st != UOE_OK) return st;
+    if (!p_patch || (!lb_loss && !expert_count && !c_dyn)) return UOE_ERR_INVALID_ARG;
+    const size_t smem = (size_t)D.n * D.m * sizeof(float);
+    if (smem > 36 * 1024) return UOE_ERR_UNSUPPORTED;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    cudaError_t e;
+    {
+        ProfScope ps("route_balance", stream);
+        e = launch_k(balance_kernel, dim3(D.B), dim3(128), smem, stream, p_patch, D.Lv, D.n, D.k, D.m, D.l_p, alpha, lb_loss,
+                     expert_count, c_dyn);
+    }
+    if (e != cudaSuccess) return UOE_ERR_CUDA;
+    UOE_LAUNCHED();
+    return UOE_OK;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -83,3 +83,72 @@ def test_route_is_deterministic():
     b = uoe.uoe_route(prob, x, Wr)
     for f in ("expert_idx", "patch_idx", "gate", "p_samp", "p_patch", "expert_offsets"):
         assert torch.equal(getattr(a, f), getattr(b, f)), f
+
+
+# ------------------------------------------------------------------------------------------------
+# two-stage dynamic capacity (Eq. 15-16) and the load-balancing loss (Eq. 42-44)
+# ------------------------------------------------------------------------------------------------
+
+BAL_CASES = {
+    "tiny": (gen.tiny(B=5, n=4, k=2, m=6, c=6), 30.0),
+    "tiny_pad": (gen.tiny(B=4, n=5, k=2, m=6, c=4, L_valid=19), 30.0),
+    "wide_m": (gen.tiny(B=3, m=48, c=40, L=96, L_valid=91, d=40, n=5, k=3, d_ff=40), 40.0),
+    "cfg2": (gen.WORKLOADS["cfg2_lm"], 20.0),
+    "cfg4": (gen.WORKLOADS["cfg4_vit"], 20.0),
+}
+
+
+def _patch_counts(w):
+    return orc.patch_valid_counts(w.L, w.m, w.L_valid)
+
+
+@pytest.mark.parametrize("name", list(BAL_CASES))
+def test_route_balance_matches_oracle(name):
+    """Integers exact, the loss to float32 rounding: the oracle is given the gate values the GPU wrote, so both
+    sides rank the same numbers (ties: lower index on both)."""
+    import paper_2503_02495_b200 as uoe
+    w, scale = BAL_CASES[name]
+    x = gen.make_x(w)
+    Wr = gen.store(gen.make_router(w).f64 * scale, w.dtype)
+    prob = problem_of(w, "mlp")
+    r = uoe.uoe_route(prob, to_dev(x), to_dev(Wr))
+    lb, cnt, cd = uoe.uoe_route_balance(prob, r.p_patch, alpha=0.01)
+    pp = r.p_patch.cpu().numpy().astype(np.float64)
+    pc = _patch_counts(w)
+    ref_cnt = np.stack([orc.patch_expert_counts(pp[b], pc, w.k) for b in range(w.B)])
+    assert np.array_equal(cnt.cpu().numpy(), ref_cnt)
+    assert np.array_equal(cd.cpu().numpy(), orc.dynamic_capacity(pp, pc, w.k))
+    ref_lb = orc.balance_loss(pp, pc, w.k, alpha=0.01)
+    assert np.abs(lb.cpu().numpy() - ref_lb).max() <= 1e-5 * np.abs(ref_lb).max()
+
+
+@pytest.mark.parametrize("name", list(BAL_CASES))
+def test_route_with_dynamic_capacity_matches_oracle(name):
+    import paper_2503_02495_b200 as uoe
+    w, scale = BAL_CASES[name]
+    x = gen.make_x(w)
+    Wr = gen.store(gen.make_router(w).f64 * scale, w.dtype)
+    prob = problem_of(w, "mlp", dynamic_c=True)
+    r = uoe.uoe_route(prob, to_dev(x), to_dev(Wr))
+    # selection by the oracle on the probabilities the GPU wrote: every integer decision must agree exactly
+    ps = r.p_samp.cpu().numpy().astype(np.float64)
+    pp = r.p_patch.cpu().numpy().astype(np.float64)
+    pc = _patch_counts(w)
+    e_ref, p_ref, _, _ = orc.select(ps, pp, pc, w.k, w.c, dynamic_c=True)
+    assert np.array_equal(r.expert_idx.cpu().numpy(), e_ref)
+    assert np.array_equal(r.patch_idx.cpu().numpy(), p_ref)
+    c_dyn = orc.dynamic_capacity(pp, pc, w.k)
+    used = (r.patch_idx.cpu().numpy() >= 0).sum(axis=2)
+    n_elig = int((pc > 0).sum())
+    assert np.array_equal(used, np.minimum(np.minimum(c_dyn, w.c), n_elig)[:, None].repeat(w.k, 1))
+    g = r.gate.cpu().numpy()
+    assert np.all(g[r.patch_idx.cpu().numpy() < 0] == 0)
+    # and the layer runs on it: unused slots contribute nothing (compare with the oracle on the same routing)
+    if w.d_ff and w.dtype == "bf16":
+        W1, W2 = gen.make_mlp_weights(w)
+        pm = problem_of(w, "mlp", residual=False, dynamic_c=True)
+        y = uoe.uoe_mlp_forward(pm, to_dev(x), to_dev(W1), to_dev(W2), r)
+        ro = orc.with_selection(x.f64, Wr.f64, e_ref, p_ref, w.m, w.L_valid)
+        ref = orc.mlp_forward(x.f64, W1.f64, W2.f64, ro, w.act, residual=False)
+        got = y.detach().to(torch.float64).cpu().numpy()
+        assert np.abs(got - ref).max() <= 2e-2 * np.abs(ref).max()
