@@ -30,7 +30,9 @@ Readings where the paper is silent or garbled are listed in the repository's des
 ones that matter here: the router is one linear map W_r[d, n] applied to the mean token of a
 patch (patch gate) or of the sample (sample gate); the combine weight is
 P_samp[b,i] * P_patch[b,i,j] when gating is on, 1 otherwise (Eq. 20 literal); no activation
-after the second linear layer (Eq. 5-7, against the misprint in Eq. 39); RoPE is not applied.
+after the second linear layer (Eq. 5-7, against the misprint in Eq. 39); RoPE (Eq. 32; Eq. 31 is misprinted)
+is optional: the last d_r channels of every head of q and k are rotated in interleaved pairs by the
+token's position in its sample, base 10000 (the RoFormer form the paper cites).
 
 Parity unpinned: the *choice* of router form and gate formula cannot be pinned to the paper
 (it prints no worked example); everything else is pinned by tests/test_oracle_*.py.
@@ -310,8 +312,27 @@ def gathered_tokens(r: Routing, b: int, s: int) -> np.ndarray:
     return np.array(toks, dtype=np.int64)
 
 
+def rope(t: np.ndarray, pos: np.ndarray, d_h: int, d_r: int, inverse: bool = False) -> np.ndarray:
+    """Eq. 32: in every head of t [rows, heads*d_h] keep the first d_h - d_r channels (the constant part) and rotate
+    the last d_r in pairs (2i, 2i+1) by the angle pos * 10000^(-2i/d_r); `inverse` rotates back."""
+    if d_r == 0:
+        return t
+    out = t.copy()
+    theta = 10000.0 ** (-2.0 * np.arange(d_r // 2) / d_r)
+    ang = pos[:, None].astype(np.float64) * theta[None, :]
+    if inverse:
+        ang = -ang
+    cs, sn = np.cos(ang), np.sin(ang)
+    for hd in range(t.shape[1] // d_h):
+        c0 = hd * d_h + (d_h - d_r)
+        a, b = t[:, c0:c0 + d_r:2], t[:, c0 + 1:c0 + d_r:2]
+        out[:, c0:c0 + d_r:2] = a * cs - b * sn
+        out[:, c0 + 1:c0 + d_r:2] = a * sn + b * cs
+    return out
+
+
 def smha_forward(x, Wq, Wk, Wv, Wo, r: Routing, d_h: int, causal: bool, residual: bool = True,
-                 return_lse: bool = False):
+                 return_lse: bool = False, d_rope: int = 0):
     """Each attention expert i owns the column slice W^{q,k,v}_i [d, d_g] and the row slice W^o_i
     [d_g, d] (Eq. 8-11); d_g = (heads per expert) * d_h.  Expert i of sample b attends only over the
     tokens of its selected patches."""
@@ -330,6 +351,7 @@ def smha_forward(x, Wq, Wk, Wv, Wo, r: Routing, d_h: int, causal: bool, residual
                 continue
             hp = x[b, tok]                                   # h' (Eq. 27)
             q, kk, v = hp @ Wq[i], hp @ Wk[i], hp @ Wv[i]    # Eq. 28-30
+            q, kk = rope(q, tok, d_h, d_rope), rope(kk, tok, d_h, d_rope)      # Eq. 32, positions in the sample
             keep = np.broadcast_to(pad_mask[tok][None, :], (len(tok), len(tok))).copy()   # Eq. 41
             if causal:
                 keep &= full_causal[np.ix_(tok, tok)]        # the mask indexed on both axes (Fig. 4)
@@ -459,7 +481,7 @@ def _gate_to_router_grads(x, W_r, r: Routing, dgate):
 
 
 def smha_backward(x, Wq, Wk, Wv, Wo, W_r, r: Routing, dy, d_h: int, causal: bool, residual: bool = True,
-                  use_gate: bool = True):
+                  use_gate: bool = True, d_rope: int = 0):
     """Gradients of sum(y * dy) for y = smha_forward(x, ...) with expert_idx / patch_idx frozen.
 
     Per (sample b, chosen expert i), with h' the gathered tokens, P the masked softmax of Eq. 33 and
@@ -488,6 +510,7 @@ def smha_backward(x, Wq, Wk, Wv, Wo, W_r, r: Routing, dy, d_h: int, causal: bool
             la = len(tok)
             hp = x[b, tok]
             q, kk, v = hp @ Wq[i], hp @ Wk[i], hp @ Wv[i]
+            q, kk = rope(q, tok, d_h, d_rope), rope(kk, tok, d_h, d_rope)
             keep = np.broadcast_to(pad_mask[tok][None, :], (la, la)).copy()
             if causal:
                 keep &= full_causal[np.ix_(tok, tok)]
@@ -520,6 +543,8 @@ def smha_backward(x, Wq, Wk, Wv, Wo, W_r, r: Routing, dy, d_h: int, causal: bool
                 dS = P[hd] * (dP - np.sum(dP * P[hd], axis=1, keepdims=True))
                 dq[:, sl] = dS @ kk[:, sl] / math.sqrt(d_h)
                 dk[:, sl] = dS.T @ q[:, sl] / math.sqrt(d_h)
+            # a rotation is orthogonal: the gradient w.r.t. the unrotated q, k is the gradient rotated back
+            dq, dk = rope(dq, tok, d_h, d_rope, inverse=True), rope(dk, tok, d_h, d_rope, inverse=True)
             dWq[i] += hp.T @ dq
             dWk[i] += hp.T @ dk
             dWv[i] += hp.T @ dv

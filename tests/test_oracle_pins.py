@@ -554,6 +554,62 @@ def test_smha_backward_full_selection_equals_dense_attention_gradient():
     assert np.all(dWr == 0.0)
 
 
+def test_rope_is_a_rotation_by_relative_position():
+    """Eq. 32 against the complex form of rotary embeddings: with z_i = x_{2i} + j x_{2i+1}, RoPE multiplies z_i by
+    exp(j t theta_i), so <RoPE(q, t), RoPE(k, s)> = Re sum_i q_i conj(k_i) exp(j (t - s) theta_i) (a function of t - s
+    only), norms are kept, the constant part is untouched and the inverse undoes it."""
+    d_h, d_r = 8, 6
+    q = gen.normal(21, 0, (5, 2 * d_h))
+    k = gen.normal(21, 1, (5, 2 * d_h))
+    pos_q = np.array([0, 3, 7, 20, 21])
+    pos_k = np.array([5, 3, 9, 2, 40])
+    rq, rk = orc.rope(q, pos_q, d_h, d_r), orc.rope(k, pos_k, d_h, d_r)
+    theta = 10000.0 ** (-2.0 * np.arange(d_r // 2) / d_r)
+    for hd in range(2):
+        c0 = hd * d_h
+        assert np.array_equal(rq[:, c0:c0 + d_h - d_r], q[:, c0:c0 + d_h - d_r])
+        zq = q[:, c0 + d_h - d_r:c0 + d_h:2] + 1j * q[:, c0 + d_h - d_r + 1:c0 + d_h:2]
+        zk = k[:, c0 + d_h - d_r:c0 + d_h:2] + 1j * k[:, c0 + d_h - d_r + 1:c0 + d_h:2]
+        for a in range(5):
+            for b in range(5):
+                want = np.real(np.sum(zq[a] * np.conj(zk[b]) * np.exp(1j * (pos_q[a] - pos_k[b]) * theta)))
+                want += q[a, c0:c0 + d_h - d_r] @ k[b, c0:c0 + d_h - d_r]
+                got = rq[a, c0:c0 + d_h] @ rk[b, c0:c0 + d_h]
+                assert got == pytest.approx(want, rel=1e-12, abs=1e-12)
+    assert np.allclose(np.linalg.norm(rq, axis=1), np.linalg.norm(q, axis=1), rtol=1e-13)
+    assert np.allclose(orc.rope(rq, pos_q, d_h, d_r, inverse=True), q, rtol=1e-12, atol=1e-13)
+    assert orc.rope(q, pos_q, d_h, 0) is q
+
+
+def test_smha_with_rope_changes_the_output_and_backward_matches_finite_differences():
+    w = gen.tiny(B=2, L_valid=24, d=8, H=4, d_h=4)
+    t = _inputs(w, ("att",))
+    x, Wq, Wk, Wv, Wo = t["x"], t["Wq"], t["Wk"], t["Wv"], t["Wo"]
+    Wr = _boost_router(t["Wra"], 10.0)
+    r = orc.route(x, Wr, w.k, w.m, w.c)
+    y0 = orc.smha_forward(x, Wq, Wk, Wv, Wo, r, w.d_h, True, d_rope=0)
+    y1 = orc.smha_forward(x, Wq, Wk, Wv, Wo, r, w.d_h, True, d_rope=2)
+    assert not np.allclose(y0, y1)
+    # backward: finite differences with the rotary part on
+    dy = gen.normal(9, 1, x.shape)
+    dx, dWq, dWk, dWv, dWo, dWr, _ = orc.smha_backward(x, Wq, Wk, Wv, Wo, Wr, r, dy, w.d_h, True, True, True, d_rope=2)
+
+    def loss(**a):
+        rr = orc.with_selection(a["x"], a["Wr"], r.expert_idx, r.patch_idx, w.m, 24, True)
+        return float(np.sum(orc.smha_forward(a["x"], a["Wq"], a["Wk"], a["Wv"], a["Wo"], rr, w.d_h, True, d_rope=2) * dy))
+
+    base = dict(x=x, Wq=Wq, Wk=Wk, Wv=Wv, Wo=Wo, Wr=Wr)
+    grads = dict(x=dx, Wq=dWq, Wk=dWk, Wv=dWv, Wo=dWo, Wr=dWr)
+    for si, which in enumerate(base):
+        v = gen.normal(300, si, base[which].shape)
+        ap, am = dict(base), dict(base)
+        ap[which] = base[which] + 1e-5 * v
+        am[which] = base[which] - 1e-5 * v
+        fd = (loss(**ap) - loss(**am)) / 2e-5
+        an = float(np.sum(grads[which] * v))
+        assert abs(fd - an) <= 2e-6 * max(1.0, abs(an)), (which, fd, an)
+
+
 # ----------------------------------------------------------------------------------------------
 # planted mistakes: the pins above must notice a wrong oracle
 # ----------------------------------------------------------------------------------------------
