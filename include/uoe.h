@@ -91,6 +91,9 @@ typedef struct {
     int32_t dtype;    /* uoe_dtype */
     int32_t act;      /* uoe_act */
     uint32_t flags;   /* UOE_FLAG_* */
+    int32_t d_rope;   /* SMHA: rotary channels per head (Eq. 32), even, 0 <= d_rope <= d_h; 0 = no RoPE.  The last
+                         d_rope channels of every head of q and k are rotated in pairs (2i, 2i+1) by the angle
+                         t * 10000^(-2i/d_rope), t = the token's position in its sample */
 } uoe_problem;
 
 /* Upper bound on expert_offsets[n]: B*k*c*l_p rows plus per-expert padding.  Buffers indexed by routed
@@ -168,7 +171,7 @@ uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, const void* 
                             void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
- * SMHA forward (Eq. 27-30, 33-36; masks Eq. 41 and Fig. 4; RoPE of Eq. 32 not applied).
+ * SMHA forward (Eq. 27-30, 32-36; masks Eq. 41 and Fig. 4; RoPE of Eq. 32 when prob->d_rope > 0).
  * Attention expert i owns the column slices Wq/Wk/Wv[i] [d, d_g] and the row slice Wo[i] [d_g, d]
  * with d_g = (H/n)*d_h (Eq. 8-11).  For each sample b and chosen expert i the l_a gathered tokens
  * attend to each other per head: softmax(q k^T / sqrt(d_h) + mask) v, where pad tokens are masked as

@@ -32,7 +32,7 @@ class UoeError(RuntimeError):
 class _Problem(ctypes.Structure):
     _fields_ = [(f, ctypes.c_int32) for f in
                 ("B", "L", "L_valid", "d", "n", "k", "m", "c", "d_e", "H", "d_h", "dtype", "act")] + \
-               [("flags", ctypes.c_uint32)]
+               [("flags", ctypes.c_uint32), ("d_rope", ctypes.c_int32)]
 
 
 @dataclass
@@ -55,12 +55,13 @@ class Problem:
     gate: bool = True
     causal: bool = False
     dynamic_c: bool = False
+    d_rope: int = 0
 
     def c_struct(self) -> _Problem:
         flags = (UOE_FLAG_RESIDUAL if self.residual else 0) | (UOE_FLAG_GATE if self.gate else 0) | \
                 (UOE_FLAG_CAUSAL if self.causal else 0) | (UOE_FLAG_DYNAMIC_C if self.dynamic_c else 0)
         return _Problem(self.B, self.L, self.L_valid, self.d, self.n, self.k, self.m, self.c, self.d_e, self.H,
-                        self.d_h, UOE_BF16 if self.dtype == "bf16" else UOE_F32, ACTS[self.act], flags)
+                        self.d_h, UOE_BF16 if self.dtype == "bf16" else UOE_F32, ACTS[self.act], flags, self.d_rope)
 
     @property
     def torch_dtype(self):

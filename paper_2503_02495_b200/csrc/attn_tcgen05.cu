@@ -214,6 +214,53 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 
 }  // namespace
 
+// Rotary position embedding on the rotary part of q and k (Eq. 32): in every head the last d_r channels are rotated
+// in pairs (2i, 2i+1) by the angle t * 10000^(-2i/d_r), t = the token's position in its sample (so the score of a
+// query-key pair depends on their distance in the sample, whichever patches were selected); sign = -1 rotates
+// back (the backward of a rotation).  a, b: [rows, ld] bf16, rotated in place.  grid (pairs, chunks), one thread
+// per (row of the pair, head).
+namespace {
+__global__ void __launch_bounds__(256)
+rope_kernel(__nv_bfloat16* __restrict__ a, __nv_bfloat16* __restrict__ b, int ld, const int* __restrict__ pair_row,
+            const int* __restrict__ patch_idx, int c, int l_p, int l_a, int heads, int d_h, int d_r, float sign) {
+    pdl_trigger();
+    pdl_wait();
+    const int pair = blockIdx.x;
+    const int idx = blockIdx.y * 256 + threadIdx.x;
+    if (idx >= l_a * heads) return;
+    const int lr = idx / heads, head = idx % heads;
+    const int j = patch_idx[(size_t)pair * c + lr / l_p];
+    if (j < 0) return;                                   // unused slot: zero rows stay zero
+    const float t = (float)(j * l_p + lr % l_p);
+    const size_t off = (size_t)(pair_row[pair] + lr) * ld + head * d_h + (d_h - d_r);
+    uint32_t* pa = (uint32_t*)(a + off);                 // one 32-bit word = one rotated pair
+    uint32_t* pb = (uint32_t*)(b + off);
+    const float step = -2.0f * 13.287712379549449f / (float)d_r;      // log2(10000)
+    for (int i = 0; i < d_r / 2; ++i) {
+        float sn, cs;
+        sincosf(t * exp2f(step * (float)i), &sn, &cs);
+        sn *= sign;
+        const uint32_t wa = pa[i], wb = pb[i];
+        const float a0 = __uint_as_float(wa << 16), a1 = __uint_as_float(wa & 0xFFFF0000u);
+        const float b0 = __uint_as_float(wb << 16), b1 = __uint_as_float(wb & 0xFFFF0000u);
+        pa[i] = pack_bf16x2(a0 * cs - a1 * sn, a0 * sn + a1 * cs);
+        pb[i] = pack_bf16x2(b0 * cs - b1 * sn, b0 * sn + b1 * cs);
+    }
+}
+}  // namespace
+
+uoe_status launch_rope(const Dims& D, void* a, void* b, int ld, const int* pair_row, const int* patch_idx, bool inverse,
+                       cudaStream_t s) {
+    if (D.d_rope <= 0) return UOE_OK;
+    const int heads = D.d_g / D.d_h;
+    dim3 grid(D.B * D.k, (D.l_a * heads + 255) / 256);
+    ProfScope ps(inverse ? "rope_bwd" : "rope", s);
+    launch_k(rope_kernel, grid, dim3(256), 0, s, (__nv_bfloat16*)a, (__nv_bfloat16*)b, ld, pair_row, patch_idx, D.c, D.l_p,
+             D.l_a, heads, D.d_h, D.d_rope, inverse ? -1.0f : 1.0f);
+    UOE_LAUNCHED();
+    return UOE_OK;
+}
+
 // q, k, v, o: [rows_max, d_g] bf16 routed buffers.
 uoe_status launch_attention(const Dims& D, const void* q, const void* k, const void* v, void* o, float* lse,
                             const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s) {

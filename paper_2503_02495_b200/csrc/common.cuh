@@ -61,7 +61,7 @@ struct ProfScope {
 
 // Sizes derived from a problem (paper notation: l_p tokens per patch, l_a = c*l_p tokens per expert).
 struct Dims {
-    int B, L, Lv, d, n, k, m, c, l_p, l_a, d_e, H, d_h, d_g;
+    int B, L, Lv, d, n, k, m, c, l_p, l_a, d_e, H, d_h, d_g, d_rope;
     int esize;            // bytes per element of x / weights / y
     long long R;          // routed rows without padding = B*k*l_a
     long long Rmax;       // bound on expert_offsets[n]
@@ -78,9 +78,11 @@ inline uoe_status make_dims(const uoe_problem* p, Dims& D) {
     if (p->act < 0 || p->act > UOE_ACT_IDENTITY) return UOE_ERR_INVALID_ARG;
     if (p->d_e < 0 || p->H < 0 || p->d_h < 0) return UOE_ERR_INVALID_ARG;
     if (p->H > 0 && (p->H % p->n != 0 || p->d_h < 1)) return UOE_ERR_INVALID_ARG;
+    if (p->d_rope < 0 || p->d_rope % 2 != 0 || (p->d_rope > 0 && p->d_rope > p->d_h)) return UOE_ERR_INVALID_ARG;
     D.B = p->B; D.L = p->L; D.Lv = p->L_valid; D.d = p->d; D.n = p->n; D.k = p->k; D.m = p->m; D.c = p->c;
     D.l_p = p->L / p->m; D.l_a = p->c * D.l_p; D.d_e = p->d_e; D.H = p->H; D.d_h = p->d_h;
     D.d_g = p->H > 0 ? (p->H / p->n) * p->d_h : 0;
+    D.d_rope = p->d_rope;
     D.bf16 = p->dtype == UOE_BF16;
     D.esize = D.bf16 ? 2 : 4;
     D.R = (long long)p->B * p->k * D.l_a;

@@ -8,6 +8,9 @@ namespace uoe {
 uoe_status launch_attention(const Dims& D, const void* q, const void* k, const void* v, void* o, float* lse,
                             const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s);
 
+uoe_status launch_rope(const Dims& D, void* a, void* b, int ld, const int* pair_row, const int* patch_idx, bool inverse,
+                       cudaStream_t s);
+
 struct SmhaWs { size_t plan, xg, q, k, v, o, z, total; };
 
 static SmhaWs smha_ws(const Dims& D) {
@@ -68,6 +71,8 @@ extern "C" uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, c
     gq.label = "qkv_proj";
     gq.nmat = 3; gq.W1 = Wk; gq.W2 = Wv; gq.C1 = k; gq.C2 = v;
     st = launch_gemm_bf16(gq, status, stream);
+    if (st != UOE_OK) return st;
+    st = launch_rope(D, q, k, D.d_g, P.pair_row, patch_idx, false, stream);      // Eq. 32 (nothing if d_rope = 0)
     if (st != UOE_OK) return st;
     st = launch_attention(D, q, k, v, o, lse, P.pair_row, patch_idx, (prob->flags & UOE_FLAG_CAUSAL) != 0, status,
                           stream);

@@ -21,6 +21,9 @@ uoe_status launch_attention_backward(const Dims& D, const void* q, const void* k
                                      const int* pair_row, const int* patch_idx, bool causal, int* status,
                                      cudaStream_t s);
 
+uoe_status launch_rope(const Dims& D, void* a, void* b, int ld, const int* pair_row, const int* patch_idx, bool inverse,
+                       cudaStream_t s);
+
 namespace {
 
 constexpr int kThreads = 256;
@@ -221,6 +224,8 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
     gq.nmat = 3; gq.W1 = Wk; gq.W2 = Wv; gq.C1 = k; gq.C2 = v;
     st = launch_gemm_bf16(gq, status, stream);
     if (st != UOE_OK) return st;
+    st = launch_rope(D, q, k, D.d_g, P.pair_row, patch_idx, false, stream);      // Eq. 32 (nothing if d_rope = 0)
+    if (st != UOE_OK) return st;
     st = launch_attention(D, q, k, v, o, lse, P.pair_row, patch_idx, causal, status, stream);
     if (st != UOE_OK) return st;
 
@@ -244,6 +249,10 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
     __nv_bfloat16* dq = (__nv_bfloat16*)dqkv;
     st = launch_attention_backward(D, q, k, v, dout, lse, delta, dq, dq + D.d_g, dq + 2 * D.d_g, 3 * D.d_g, P.pair_row,
                                    patch_idx, causal, status, stream);
+    if (st != UOE_OK) return st;
+
+    // gradients w.r.t. the rotated q, k -> w.r.t. the projections: rotate back
+    st = launch_rope(D, dq, dq + D.d_g, 3 * D.d_g, P.pair_row, patch_idx, true, stream);
     if (st != UOE_OK) return st;
 
     // ---- projection backward: dx_g and the q/k/v weight gradients from the concatenated [dq dk dv] ----

@@ -38,13 +38,13 @@ CASES = {
 }
 
 
-def _run(w, residual, want_lse=False):
+def _run(w, residual, want_lse=False, d_rope=0):
     import paper_2503_02495_b200 as uoe
     x, Wr = gen.make_x(w), gen.make_router(w, "att")
     if not w.name.startswith("cfg"):
         Wr = gen.store(Wr.f64 * 20, w.dtype)
     Wq, Wk, Wv, Wo = gen.make_attn_weights(w)
-    prob = problem_of(w, "att", residual=residual)
+    prob = problem_of(w, "att", residual=residual, d_rope=d_rope)
     xd = to_dev(x)
     r = uoe.uoe_route(prob, xd, to_dev(Wr))
     lse = None
@@ -53,7 +53,7 @@ def _run(w, residual, want_lse=False):
     y = uoe.uoe_smha_forward(prob, xd, to_dev(Wq), to_dev(Wk), to_dev(Wv), to_dev(Wo), r, lse=lse)
     ro = orc.with_selection(x.f64, Wr.f64, r.expert_idx.cpu().numpy(), r.patch_idx.cpu().numpy(), w.m, w.L_valid)
     out = orc.smha_forward(x.f64, Wq.f64, Wk.f64, Wv.f64, Wo.f64, ro, w.d_h, w.causal, residual=residual,
-                           return_lse=want_lse)
+                           return_lse=want_lse, d_rope=d_rope)
     return to_f64(y), out, x.f64, r, ro, lse
 
 
@@ -73,6 +73,19 @@ def test_residual_output_matches_oracle(name):
     y, ref, x, r, ro, _ = _run(w, residual=True)
     assert rel_inf(y, ref) <= TOL
     assert np.array_equal(y[:, w.L_valid:], x[:, w.L_valid:])
+
+
+@pytest.mark.parametrize("name,d_rope", [("one_tile_causal", 64), ("pad", 32), ("three_tiles_causal_pad", 16),
+                                         ("two_heads_per_expert", 32), ("cfg3", 32), ("cfg4", 64)])
+def test_attention_with_rotary_embedding_matches_oracle(name, d_rope):
+    """Eq. 32: the last d_rope channels of every head of q and k rotated by the token's position in its sample."""
+    w = CASES[name]
+    y, ref, x, r, ro, _ = _run(w, residual=False, d_rope=d_rope)
+    y0, _, _, _, _, _ = _run(w, residual=False)
+    err = rel_inf(y, ref)
+    print(f"{name} d_rope={d_rope}: max|err|/max|ref| = {err:.3e}")
+    assert err <= TOL
+    assert rel_inf(y0, ref) > 5 * TOL or name.startswith("cfg")        # the rotation really changes the result
 
 
 def test_full_selection_equals_multihead_attention():

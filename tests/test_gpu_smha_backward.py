@@ -38,21 +38,21 @@ CASES = {
 }
 
 
-def _run(w, residual, use_gate=True):
+def _run(w, residual, use_gate=True, d_rope=0):
     import paper_2503_02495_b200 as uoe
     x, Wr = gen.make_x(w), gen.make_router(w, "att")
     if not w.name.startswith("cfg"):
         Wr = gen.store(Wr.f64 * 20, w.dtype)
     Wq, Wk, Wv, Wo = gen.make_attn_weights(w)
     dy = gen.make_dy(w)
-    prob = problem_of(w, "att", residual=residual, gate=use_gate)
+    prob = problem_of(w, "att", residual=residual, gate=use_gate, d_rope=d_rope)
     xd, Wrd = to_dev(x), to_dev(Wr)
     r = uoe.uoe_route(prob, xd, Wrd)
     got = uoe.uoe_smha_backward(prob, xd, to_dev(Wq), to_dev(Wk), to_dev(Wv), to_dev(Wo), Wrd, r, to_dev(dy))
     ro = orc.with_selection(x.f64, Wr.f64, r.expert_idx.cpu().numpy(), r.patch_idx.cpu().numpy(), w.m, w.L_valid,
                             use_gate)
     ref = orc.smha_backward(x.f64, Wq.f64, Wk.f64, Wv.f64, Wo.f64, Wr.f64, ro, dy.f64, w.d_h, w.causal, residual,
-                            use_gate)
+                            use_gate, d_rope=d_rope)
     return [to_f64(t) for t in got], ref
 
 
@@ -67,6 +67,16 @@ def test_smha_backward_matches_oracle(name, residual):
         assert np.isfinite(g).all(), nm
         err = rel_inf(g, r)
         print(f"{name} residual={residual} {nm}: {err:.3e}  (|ref|max {np.abs(r).max():.3e})")
+        assert err <= TOL, nm
+
+
+@pytest.mark.parametrize("name,d_rope", [("one_tile_causal", 64), ("pad", 32), ("three_tiles_causal_pad", 16),
+                                         ("lm_shape", 32)])
+def test_smha_backward_with_rotary_embedding_matches_oracle(name, d_rope):
+    got, ref = _run(CASES[name], False, d_rope=d_rope)
+    for nm, g, r in zip(NAMES, got, ref[:6]):
+        err = rel_inf(g, r)
+        print(f"{name} d_rope={d_rope} {nm}: {err:.3e}")
         assert err <= TOL, nm
 
 
