@@ -409,6 +409,23 @@ TENSOR_KERNELS = ("gemm1_act", "gemm2", "qkv_proj", "out_proj", "attention", "bw
 HBM_KERNELS = ("route", "gather", "combine", "pool")
 
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
+# (step_kernels_cfg2_lm.md, gemm_wgrad_cfg5_scale_B2.md, route_kernels_cfg5_scale.md).  Keyed by (workload, kernel
+# label); an entry is dropped when its kernel changes, and the line then reports null.  The scale entries were
+# captured at B=2 and scaled by 4: their traffic grows in proportion to the routed rows.
+NCU_TRAFFIC = {
+    ("cfg2_lm", "route"): 8.47e6,
+    ("cfg2_lm", "combine"): 25.18e6,
+    ("cfg2_lm", "qkv_proj"): 9.74e6,
+    ("cfg2_lm", "gemm1_act"): 10.24e6,
+    ("cfg2_lm", "gemm2"): 10.56e6,
+    ("cfg2_lm", "attention"): 6.35e6,
+    ("cfg2_lm", "out_proj"): 2.70e6,
+    ("cfg5_scale", "gemm2"): 4 * (92.4e6 + 86.0e6),
+    ("cfg5_scale", "bwd_dx"): 4 * (92.4e6 + 86.1e6),
+}
+
+
 def roofline_of(top, w: gen.Workload, peaks, peak_src):
     wk = work_table(w).get(top["kernel"], dict(flops=0, bytes=0))
     t_tensor = wk["flops"] / (peaks["bf16_tflops"] * 1e12)
@@ -417,7 +434,8 @@ def roofline_of(top, w: gen.Workload, peaks, peak_src):
         roof = {"bound": "tensor", "achieved": top["tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
     else:
         roof = {"bound": "hbm", "achieved": top["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": None, "kernel": top["kernel"],
+    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": NCU_TRAFFIC.get((w.name, top["kernel"])),
+                 "kernel": top["kernel"],
                  "avg_ms": top["avg_ms"], "share_of_kernel_time": top["share"], "peak_source": peak_src,
                  "algorithmic_flops": wk["flops"], "algorithmic_bytes": wk["bytes"]})
     return roof
