@@ -212,7 +212,7 @@ uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, const void*
  * synchronise the device or touch the allocator (a latency-critical serving loop, a plugin hosted by
  * a framework that owns all device memory and offers no way to request scratch, start-up code that
  * runs before the host application's memory pool exists).  Such a caller can pass its inputs and
- * outputs but has nowhere to get the extra buffer that uoe_route needs for its partial scores.
+ * outputs but has nowhere to get the extra buffer that uoe_route needs for its pooled sums, scores and tickets.
  *
  * Here that buffer is a fixed array of UOE_ROUTE_STATIC_SCRATCH_BYTES compiled into the library's
  * device image, so every GPU on which the library is loaded holds that many bytes until the process
@@ -223,10 +223,11 @@ uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, const void*
  *   - The first call on each device looks up the array's device address (a one-time set-up step, done
  *     with that device current).  Make that first call before starting any stream capture.
  *   - The function calls no cudaMalloc / cudaFree and no allocating library routine.
- *   - All calls on a device share the one array, which still holds what the previous call left; the
- *     counters that must start at zero are cleared on the stream at the start of every call.  Two calls
- *     whose kernels may overlap on the GPU (different streams, no ordering between them) race on the
- *     array and give wrong routing: order them, or use uoe_route with separate workspaces.
+ *   - All calls on a device share the one array.  It starts zeroed, and the kernels leave the counters that must
+ *     start at zero (completion tickets, expert loads) at zero again when a call finishes, whatever shapes the
+ *     calls have; the rest still holds what the previous call left and is overwritten before it is read.  Two calls
+ *     whose kernels may overlap on the GPU (different streams, no ordering between them) race on the array and
+ *     give wrong routing: order them, or use uoe_route with separate workspaces.
  *   - No device status word is kept for this variant (uoe_read_device_status does not apply).
  */
 #define UOE_ROUTE_STATIC_SCRATCH_BYTES (8 << 20)
