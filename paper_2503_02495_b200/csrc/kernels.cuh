@@ -112,8 +112,11 @@ inline int gemm_bf16_bn(int N) { return (N % 256 == 0) ? 256 : (N % 128 == 0 ? 1
 // Per-expert weight gradient over ragged row counts:  dW[e] [M, N] (float32, overwritten) =
 // sum over the rows r of expert e's region of  P[r, 0:M]^T  Q[r, 0:N]   (P [rows, M], Q [rows, N], bf16).
 // Rows of a region beyond its real rows must be zero in P or Q.
+// `part`: scratch of wgrad_scratch_bytes(n, M, N, rows_max) bytes for the split-K partial outputs (may be null when
+// that is 0; with null the contraction is never split).
+size_t wgrad_scratch_bytes(int n, int M, int N, long long rows_max);
 uoe_status launch_wgrad_bf16(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
-                             long long rows_max, const char* label, int* status, cudaStream_t s);
+                             long long rows_max, const char* label, int* status, cudaStream_t s, float* part = nullptr);
 uoe_status launch_gemm_f32(const GemmArgs& g, cudaStream_t s);
 
 // Scratch of the router half of a backward pass (all float32).

@@ -153,7 +153,7 @@ rvec_kernel(const T* __restrict__ W_r, const float* __restrict__ G, float* __res
 
 // dW_r[dd, i] = sum over (b, j) of pool[bj, dd] * G[bj, i] in two fixed-order stages: grid (d/256, S) partial sums
 // over S chunks of bj, then a sum over the chunks.
-constexpr int kDwrSplit = 16;
+constexpr int kDwrSplit = 64;
 __global__ void __launch_bounds__(kThreads)
 dwr_partial_kernel(const float* __restrict__ pool, const float* __restrict__ G, float* __restrict__ part, int BM, int d,
                    int n) {
@@ -197,7 +197,7 @@ dwr_sum_kernel(const float* __restrict__ part, float* __restrict__ dW_r, int tot
     dW_r[idx] = a;
 }
 
-struct BwdWs { size_t plan, dyg, xg, dh, ag, dxg, dgp, G, pool, rvec, dgate, wpart, total; int nt; };
+struct BwdWs { size_t plan, dyg, xg, dh, ag, dxg, dgp, G, pool, rvec, dgate, wpart, wgpart, total; int nt; };
 
 BwdWs bwd_ws(const Dims& D) {
     WsCarver w;
@@ -217,6 +217,10 @@ BwdWs bwd_ws(const Dims& D) {
     r.rvec = w.take((size_t)D.B * D.m * D.d * sizeof(float));
     r.dgate = w.take((size_t)D.B * D.k * D.c * sizeof(float));
     r.wpart = w.take((size_t)kDwrSplit * D.d * D.n * sizeof(float));
+    {   // split-K partials, sized for the larger of the two weight gradients
+        const size_t s1 = wgrad_scratch_bytes(D.n, D.d, D.d_e, D.Rmax), s2 = wgrad_scratch_bytes(D.n, D.d_e, D.d, D.Rmax);
+        r.wgpart = w.take((s1 > s2 ? s1 : s2) + 1024);
+    }
     r.total = w.off;
     return r;
 }
@@ -349,13 +353,15 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
     ga.bwd = true; ga.bwd_h = saved_h; ga.row_gate = P.row_gate; ga.row_valid = P.row_valid; ga.dg_part = dgp; ga.C1 = ag;
     st = launch_gemm_bf16(ga, status, stream);
     if (st != UOE_OK) return st;
-    st = launch_wgrad_bf16(ag, dyg, dW2, expert_offsets, D.n, D.d_e, D.d, D.Rmax, "wgrad_W2", status, stream);
+    st = launch_wgrad_bf16(ag, dyg, dW2, expert_offsets, D.n, D.d_e, D.d, D.Rmax, "wgrad_W2", status, stream,
+                           wgrad_scratch_bytes(D.n, D.d_e, D.d, D.Rmax) ? (float*)(base + W.wgpart) : nullptr);
     if (st != UOE_OK) return st;
     GemmArgs gx{dh, W1, nullptr, dxg, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, true, D.Rmax};
     gx.label = "bwd_dx";
     st = launch_gemm_bf16(gx, status, stream);
     if (st != UOE_OK) return st;
-    st = launch_wgrad_bf16(xg, dh, dW1, expert_offsets, D.n, D.d, D.d_e, D.Rmax, "wgrad_W1", status, stream);
+    st = launch_wgrad_bf16(xg, dh, dW1, expert_offsets, D.n, D.d, D.d_e, D.Rmax, "wgrad_W1", status, stream,
+                           wgrad_scratch_bytes(D.n, D.d, D.d_e, D.Rmax) ? (float*)(base + W.wgpart) : nullptr);
     if (st != UOE_OK) return st;
 
     if (use_gate) {

@@ -130,7 +130,7 @@ finalize_wgrads_kernel(const float* __restrict__ dWcat, const float* __restrict_
 }
 
 struct SmhaBwdWs {
-    size_t plan, xg, dyg, q, k, v, o, dout, og, dqkv, dxg, lse, delta, dgp, wcat, dwcat, dwot, router, total;
+    size_t plan, xg, dyg, q, k, v, o, dout, og, dqkv, dxg, lse, delta, dgp, wcat, dwcat, dwot, router, wgpart, total;
 };
 
 SmhaBwdWs smha_bwd_ws(const Dims& D) {
@@ -152,6 +152,10 @@ SmhaBwdWs smha_bwd_ws(const Dims& D) {
     r.dwcat = w.take((size_t)D.n * D.d * 3 * D.d_g * 4);
     r.dwot = w.take((size_t)D.n * D.d * D.d_g * 4);
     r.router = w.take(router_backward_scratch_bytes(D));
+    {   // split-K partials, sized for the larger of the two weight gradients
+        const size_t s1 = wgrad_scratch_bytes(D.n, D.d, 3 * D.d_g, D.Rmax), s2 = wgrad_scratch_bytes(D.n, D.d, D.d_g, D.Rmax);
+        r.wgpart = w.take((s1 > s2 ? s1 : s2) + 1024);
+    }
     r.total = w.off;
     return r;
 }
@@ -242,7 +246,8 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
                  (const float*)P.row_valid, delta, dgp, expert_offsets, D.n, heads, D.d_g);
     }
     UOE_LAUNCHED();
-    st = launch_wgrad_bf16(dyg, og, dwot, expert_offsets, D.n, D.d, D.d_g, D.Rmax, "wgrad_Wo", status, stream);
+    st = launch_wgrad_bf16(dyg, og, dwot, expert_offsets, D.n, D.d, D.d_g, D.Rmax, "wgrad_Wo", status, stream,
+                           wgrad_scratch_bytes(D.n, D.d, D.d_g, D.Rmax) ? (float*)(base + W.wgpart) : nullptr);
     if (st != UOE_OK) return st;
 
     // ---- attention backward ----
@@ -266,7 +271,8 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
     gx.label = "bwd_dx_att";
     st = launch_gemm_bf16(gx, status, stream);
     if (st != UOE_OK) return st;
-    st = launch_wgrad_bf16(xg, dqkv, dwcat, expert_offsets, D.n, D.d, 3 * D.d_g, D.Rmax, "wgrad_Wqkv", status, stream);
+    st = launch_wgrad_bf16(xg, dqkv, dwcat, expert_offsets, D.n, D.d, 3 * D.d_g, D.Rmax, "wgrad_Wqkv", status, stream,
+                           wgrad_scratch_bytes(D.n, D.d, 3 * D.d_g, D.Rmax) ? (float*)(base + W.wgpart) : nullptr);
     if (st != UOE_OK) return st;
     {
         ProfScope ps("finalize_wgrads", stream);

@@ -46,7 +46,7 @@ template <int BN, int MT>
 __global__ void __launch_bounds__(WCfg<BN, MT>::THREADS, 1)
 wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CUtensorMap tmQ,
              const __grid_constant__ CUtensorMap tmW, const int* __restrict__ offsets, int n, int M, int N,
-             int* status) {
+             int ksplit, int* status) {
     pdl_trigger();
     using Cf = WCfg<BN, MT>;
     extern __shared__ uint8_t smem_raw[];
@@ -74,7 +74,21 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
     constexpr int TM = MT * BM;
     const int m_tiles = M / TM, n_tiles = N / BN;
     const int per_expert = m_tiles * n_tiles;
-    const int total_tiles = n * per_expert;
+    const int total_tiles = n * per_expert * ksplit;
+    // tile -> expert, output tile, and the slice [kb_lo, kb_lo + kb_cnt) of the expert's 64-row K blocks that split
+    // `ks` of the contraction covers (ksplit = 1: all of them); split ks writes its own copy of the output
+    auto decode = [&](int tile, int& e, int& m0, int& n0, int& ks, int& kb_lo, int& kb_cnt) {
+        ks = tile % ksplit;
+        const int t2 = tile / ksplit;
+        e = t2 / per_expert;
+        const int rem = t2 % per_expert;
+        m0 = (rem / n_tiles) * TM;
+        n0 = (rem % n_tiles) * BN;
+        const int num_kb = (ctl->offs[e + 1] - ctl->offs[e]) / BK;
+        const int per = (num_kb + ksplit - 1) / ksplit;
+        kb_lo = ks * per;
+        kb_cnt = max(0, min(num_kb, kb_lo + per) - kb_lo);
+    };
 
     if (warp == 0) {
         // TMA producer: lane 0 runs the pipeline, the 64-wide boxes are issued one per lane
@@ -82,9 +96,9 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         uint32_t phase = 0, issued = 0, issued_parity = 0;
         bool stop = false;
         for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
-            const int e = tile / per_expert, rem = tile % per_expert;
-            const int m0 = (rem / n_tiles) * TM, n0 = (rem % n_tiles) * BN;
-            const int r0 = ctl->offs[e], num_kb = (ctl->offs[e + 1] - r0) / BK;
+            int e, m0, n0, ks, kb_lo, num_kb;
+            decode(tile, e, m0, n0, ks, kb_lo, num_kb);
+            const int r0 = ctl->offs[e] + kb_lo * BK;
             for (int kb = 0; kb < num_kb; ++kb) {
                 int ok = 1;
                 if (lane == 0) ok = (mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) && !*abort_flag) ? 1 : 0;
@@ -114,8 +128,8 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
             uint32_t phase = 0, acc_phase = 0;
             bool stop = false;
             for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
-                const int e = tile / per_expert;
-                const int num_kb = (ctl->offs[e + 1] - ctl->offs[e]) / BK;
+                int e, m0, n0, ks, kb_lo, num_kb;
+                decode(tile, e, m0, n0, ks, kb_lo, num_kb);
                 if (!mbar_wait(&ctl->tempty[acc], acc_phase ^ 1, abort_flag, status) || *abort_flag) break;
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
@@ -146,13 +160,12 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         int acc = 0;
         uint32_t acc_phase = 0;
         for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
-            const int e = tile / per_expert, rem = tile % per_expert;
-            const int m0 = (rem / n_tiles) * TM, n0 = (rem % n_tiles) * BN;
-            const int num_kb = (ctl->offs[e + 1] - ctl->offs[e]) / BK;
+            int e, m0, n0, ks, kb_lo, num_kb;
+            decode(tile, e, m0, n0, ks, kb_lo, num_kb);
             const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
             if (!__all_sync(0xffffffffu, ready)) break;
             tc_fence_after();
-            const int wrow0 = e * M + m0 + half * BM + quarter * 32;      // first row of this warp's piece in [n*M, N]
+            const int wrow0 = (ks * n + e) * M + m0 + half * BM + quarter * 32;   // first row of this warp's piece in [ksplit*n*M, N]
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (MT == 2 ? half * BN : acc * BN);
             uint8_t* stg = smem + Cf::STAGES * Cf::STAGE + 1024 + (warp - 2) * Cf::STG_BYTES;
 #pragma unroll 1
@@ -188,9 +201,24 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
     }
 }
 
+// dW = sum over the K splits of their partial outputs, ascending split order.  float4 pieces.
+__global__ void __launch_bounds__(256)
+wgrad_reduce_kernel(const float4* __restrict__ part, float4* __restrict__ dW, long long vecs, int ksplit) {
+    pdl_trigger();
+    pdl_wait();
+    for (long long q = (long long)blockIdx.x * 256 + threadIdx.x; q < vecs; q += (long long)gridDim.x * 256) {
+        float4 a = part[q];
+        for (int s = 1; s < ksplit; ++s) {
+            const float4 t = part[(long long)s * vecs + q];
+            a.x += t.x; a.y += t.y; a.z += t.z; a.w += t.w;
+        }
+        dW[q] = a;
+    }
+}
+
 template <int BN, int MT>
 uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
-                    long long rows_max, const char* label, int* status, cudaStream_t s) {
+                    long long rows_max, const char* label, int* status, cudaStream_t s, int ksplit, float* part) {
     using Cf = WCfg<BN, MT>;
     static bool attr_set = false;
     auto kern = wgrad_kernel<BN, MT>;
@@ -210,33 +238,59 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
         const uint64_t str[1] = {(uint64_t)N * 2};
         if (!make_tmap(&tmQ, Q, 2, dims, str, box)) return UOE_ERR_CUDA;
     }
-    CUtensorMap tmW;      // dW as [n*M, N] float32, written in [32 x 32] pieces
+    CUtensorMap tmW;      // the output (or the per-split partial outputs) as [ksplit*n*M, N] float32, [32 x 32] pieces
     {
-        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)n * M};
+        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)ksplit * n * M};
         const uint64_t str[1] = {(uint64_t)N * 4};
         const uint32_t wbox[2] = {32, 32};
-        if (!make_tmap(&tmW, dW, 2, dims, str, wbox, CU_TENSOR_MAP_DATA_TYPE_FLOAT32)) return UOE_ERR_CUDA;
+        if (!make_tmap(&tmW, ksplit > 1 ? part : dW, 2, dims, str, wbox, CU_TENSOR_MAP_DATA_TYPE_FLOAT32)) return UOE_ERR_CUDA;
     }
-    const long long tiles = (long long)n * (M / (MT * BM)) * (N / BN);
+    const long long tiles = (long long)n * (M / (MT * BM)) * (N / BN) * ksplit;
     int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     ProfScope ps(label, s);
-    launch_k(kern, grid, dim3(Cf::THREADS), Cf::SMEM, s, tmP, tmQ, tmW, offsets, n, M, N, status);
+    launch_k(kern, grid, dim3(Cf::THREADS), Cf::SMEM, s, tmP, tmQ, tmW, offsets, n, M, N, ksplit, status);
     UOE_LAUNCHED();
+    if (ksplit > 1) {
+        const long long vecs = (long long)n * M * N / 4;
+        launch_k(wgrad_reduce_kernel, dim3((unsigned)((vecs + 255) / 256 < 1184 ? (vecs + 255) / 256 : 1184)), dim3(256), 0, s,
+                 (const float4*)part, (float4*)dW, vecs, ksplit);
+        UOE_LAUNCHED();
+    }
     return UOE_OK;
 }
 
 }  // namespace
 
+// How many ways the contraction is split: weight gradients with few output tiles (small M x N per expert) leave most
+// SMs idle and give each busy one a long serial K loop, so their rows are split across CTAs into partial outputs
+// that a second kernel adds in a fixed order.  1 = no split.
+int wgrad_ksplit(int n, int M, int N, long long rows_max) {
+    const int bn = gemm_bf16_bn(N);
+    const long long tiles = (long long)n * (M / BM) * (N / bn);
+    if (tiles < 1 || n < 1 || tiles >= sm_count()) return 1;      // (shapes the kernel does not cover are refused later)
+    long long ks = (2ll * sm_count() + tiles - 1) / tiles;
+    const long long avg_kb = rows_max / ((long long)n * BK);        // 64-row K blocks per expert on average
+    if (ks > avg_kb / 4) ks = avg_kb / 4;                            // at least four K blocks per split
+    if (ks > 32) ks = 32;
+    return ks < 2 ? 1 : (int)ks;
+}
+
+size_t wgrad_scratch_bytes(int n, int M, int N, long long rows_max) {
+    const int ks = wgrad_ksplit(n, M, N, rows_max);
+    return ks > 1 ? (size_t)ks * n * M * N * sizeof(float) : 0;
+}
+
 uoe_status launch_wgrad_bf16(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
-                             long long rows_max, const char* label, int* status, cudaStream_t s) {
+                             long long rows_max, const char* label, int* status, cudaStream_t s, float* part) {
     if (M % BM != 0 || N % 64 != 0 || n > 32) return UOE_ERR_UNSUPPORTED;
     const int bn = gemm_bf16_bn(N);
+    const int ks = part ? wgrad_ksplit(n, M, N, rows_max) : 1;
     // 256-row output tiles when the weight matrices are large enough to keep every SM busy with them
     if (bn == 256 && M % 256 == 0 && (long long)n * (M / 256) * (N / 256) >= 2 * sm_count())
-        return launch_w<256, 2>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
-    if (bn == 256) return launch_w<256, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
-    if (bn == 128) return launch_w<128, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
-    return launch_w<64, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s);
+        return launch_w<256, 2>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, 1, nullptr);
+    if (bn == 256) return launch_w<256, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, ks, part);
+    if (bn == 128) return launch_w<128, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, ks, part);
+    return launch_w<64, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, ks, part);
 }
 
 }  // namespace uoe
