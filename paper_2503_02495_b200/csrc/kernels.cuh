@@ -115,8 +115,19 @@ inline int gemm_bf16_bn(int N) { return (N % 256 == 0) ? 256 : (N % 128 == 0 ? 1
 // `part`: scratch of wgrad_scratch_bytes(n, M, N, rows_max) bytes for the split-K partial outputs (may be null when
 // that is 0; with null the contraction is never split).
 size_t wgrad_scratch_bytes(int n, int M, int N, long long rows_max);
+// Gathered operands (Eq. 18 inside the weight-gradient contraction): with gather_p (gather_q) the pointer P (Q) is
+// the source tensor [Bm patches, l_p, M (N)] and routed row r is row r % l_p of patch src_patch[r / l_p]
+// (-1 = zero rows).  Needs every 64-row K block to be whole slabs inside whole patches, with regions (multiples of
+// 128 rows) starting on patch boundaries:
+inline bool wgrad_can_gather(int l_p) { return l_p >= 16 && 128 % l_p == 0; }
+struct WgradGather {
+    bool gather_p = false, gather_q = false;
+    const int* src_patch = nullptr;
+    int l_p = 64, Bm = 0;
+};
 uoe_status launch_wgrad_bf16(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
-                             long long rows_max, const char* label, int* status, cudaStream_t s, float* part = nullptr);
+                             long long rows_max, const char* label, int* status, cudaStream_t s, float* part = nullptr,
+                             const WgradGather& g = WgradGather());
 uoe_status launch_gemm_f32(const GemmArgs& g, cudaStream_t s);
 
 // Scratch of the router half of a backward pass (all float32).

@@ -206,8 +206,9 @@ BwdWs bwd_ws(const Dims& D) {
     r.nt = D.d_e / gemm_bf16_bn(D.d_e > 0 ? D.d_e : 64);
     if (r.nt < 1) r.nt = 1;
     r.plan = w.take(plan_bytes(D, true));
-    r.dyg = w.take((size_t)D.Rmax * D.d * D.esize);
-    r.xg = w.take((size_t)D.Rmax * D.d * D.esize);
+    const bool fused = can_fuse_gather(D) && wgrad_can_gather(D.l_p);      // dy and x gathered inside the consumers' TMA loads
+    r.dyg = fused ? 0 : w.take((size_t)D.Rmax * D.d * D.esize);
+    r.xg = fused ? 0 : w.take((size_t)D.Rmax * D.d * D.esize);
     r.dh = w.take((size_t)D.Rmax * D.d_e * D.esize);
     r.ag = w.take((size_t)D.Rmax * D.d_e * D.esize);
     r.dxg = w.take((size_t)D.Rmax * D.d * D.esize);
@@ -343,25 +344,35 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
 
     st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream, use_gate);
     if (st != UOE_OK) return st;
-    st = launch_gather(D, dy, patch_idx, expert_offsets, P, dyg, stream);
-    if (st != UOE_OK) return st;
-    st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
-    if (st != UOE_OK) return st;
+    // Eq. 18 for dy and x: either inside the TMA loads of the kernels that consume them, or as routed copies
+    const bool fused = can_fuse_gather(D) && wgrad_can_gather(D.l_p);
+    if (!fused) {
+        st = launch_gather(D, dy, patch_idx, expert_offsets, P, dyg, stream);
+        if (st != UOE_OK) return st;
+        st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
+        if (st != UOE_OK) return st;
+    }
+    WgradGather gq, gp;          // dW2 = ag^T dy_g (Q gathered), dW1 = x_g^T dh (P gathered)
+    if (fused) {
+        gq.gather_q = true; gq.src_patch = P.src_patch; gq.l_p = D.l_p; gq.Bm = D.B * D.m;
+        gp.gather_p = true; gp.src_patch = P.src_patch; gp.l_p = D.l_p; gp.Bm = D.B * D.m;
+    }
 
     GemmArgs ga{dyg, W2, nullptr, dh, nullptr, expert_offsets, D.n, D.d, D.d_e, prob->act, true, D.Rmax};
     ga.label = "bwd_da_dh";
     ga.bwd = true; ga.bwd_h = saved_h; ga.row_gate = P.row_gate; ga.row_valid = P.row_valid; ga.dg_part = dgp; ga.C1 = ag;
+    if (fused) { ga.gather_x = dy; ga.src_patch = P.src_patch; ga.l_p = D.l_p; ga.Bm = D.B * D.m; }
     st = launch_gemm_bf16(ga, status, stream);
     if (st != UOE_OK) return st;
-    st = launch_wgrad_bf16(ag, dyg, dW2, expert_offsets, D.n, D.d_e, D.d, D.Rmax, "wgrad_W2", status, stream,
-                           wgrad_scratch_bytes(D.n, D.d_e, D.d, D.Rmax) ? (float*)(base + W.wgpart) : nullptr);
+    st = launch_wgrad_bf16(ag, fused ? dy : dyg, dW2, expert_offsets, D.n, D.d_e, D.d, D.Rmax, "wgrad_W2", status, stream,
+                           wgrad_scratch_bytes(D.n, D.d_e, D.d, D.Rmax) ? (float*)(base + W.wgpart) : nullptr, gq);
     if (st != UOE_OK) return st;
     GemmArgs gx{dh, W1, nullptr, dxg, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, true, D.Rmax};
     gx.label = "bwd_dx";
     st = launch_gemm_bf16(gx, status, stream);
     if (st != UOE_OK) return st;
-    st = launch_wgrad_bf16(xg, dh, dW1, expert_offsets, D.n, D.d, D.d_e, D.Rmax, "wgrad_W1", status, stream,
-                           wgrad_scratch_bytes(D.n, D.d, D.d_e, D.Rmax) ? (float*)(base + W.wgpart) : nullptr);
+    st = launch_wgrad_bf16(fused ? x : xg, dh, dW1, expert_offsets, D.n, D.d, D.d_e, D.Rmax, "wgrad_W1", status, stream,
+                           wgrad_scratch_bytes(D.n, D.d, D.d_e, D.Rmax) ? (float*)(base + W.wgpart) : nullptr, gp);
     if (st != UOE_OK) return st;
 
     if (use_gate) {

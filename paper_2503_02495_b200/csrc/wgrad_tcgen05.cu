@@ -46,7 +46,7 @@ template <int BN, int MT>
 __global__ void __launch_bounds__(WCfg<BN, MT>::THREADS, 1)
 wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CUtensorMap tmQ,
              const __grid_constant__ CUtensorMap tmW, const int* __restrict__ offsets, int n, int M, int N,
-             int ksplit, int* status) {
+             int ksplit, int* status, int gather_p, int gather_q, const int* __restrict__ src_patch, int l_p, int Bm) {
     pdl_trigger();
     using Cf = WCfg<BN, MT>;
     extern __shared__ uint8_t smem_raw[];
@@ -95,6 +95,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         int stage = 0;
         uint32_t phase = 0, issued = 0, issued_parity = 0;
         bool stop = false;
+        const int sub_rows = (gather_p || gather_q) ? min(l_p, BK) : BK, nsub = BK / sub_rows;
         for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
             int e, m0, n0, ks, kb_lo, num_kb;
             decode(tile, e, m0, n0, ks, kb_lo, num_kb);
@@ -108,10 +109,35 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
                 uint8_t* sb = sa + Cf::A_BYTES;
                 if (lane == 0) mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
                 __syncwarp();
-                if (lane < TM / 64)
-                    tma_load_2d(sa + lane * 8192, &tmP, m0 + lane * 64, r0 + kb * BK, &ctl->full[stage]);
-                else if (lane >= 16 && lane < 16 + BN / 64)
-                    tma_load_2d(sb + (lane - 16) * 8192, &tmQ, n0 + (lane - 16) * 64, r0 + kb * BK, &ctl->full[stage]);
+                // a gathered operand (Eq. 18 inside the contraction) comes from the source tensor [Bm patches, l_p, cols]:
+                // the 64 routed rows of a K block are 64 / sub_rows slabs of sub_rows rows, each inside one patch
+                const int row = r0 + kb * BK;
+                if (lane < 16) {
+                    const int cnt = (TM / 64) * (gather_p ? nsub : 1);
+                    if (lane < cnt) {
+                        if (gather_p) {
+                            const int cb = lane / nsub, sub = lane % nsub, rr = row + sub * sub_rows;
+                            int src = src_patch[rr / l_p];
+                            if (src < 0) src = Bm;                    // out of range: zero-filled box
+                            tma_load_3d(sa + cb * 8192 + sub * sub_rows * 128, &tmP, m0 + cb * 64, rr % l_p, src, &ctl->full[stage]);
+                        } else {
+                            tma_load_2d(sa + lane * 8192, &tmP, m0 + lane * 64, row, &ctl->full[stage]);
+                        }
+                    }
+                } else {
+                    const int l2 = lane - 16;
+                    const int cnt = (BN / 64) * (gather_q ? nsub : 1);
+                    if (l2 < cnt) {
+                        if (gather_q) {
+                            const int cb = l2 / nsub, sub = l2 % nsub, rr = row + sub * sub_rows;
+                            int src = src_patch[rr / l_p];
+                            if (src < 0) src = Bm;
+                            tma_load_3d(sb + cb * 8192 + sub * sub_rows * 128, &tmQ, n0 + cb * 64, rr % l_p, src, &ctl->full[stage]);
+                        } else {
+                            tma_load_2d(sb + l2 * 8192, &tmQ, n0 + l2 * 64, row, &ctl->full[stage]);
+                        }
+                    }
+                }
                 issued |= 1u << stage;
                 issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
                 if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
@@ -218,7 +244,8 @@ wgrad_reduce_kernel(const float4* __restrict__ part, float4* __restrict__ dW, lo
 
 template <int BN, int MT>
 uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
-                    long long rows_max, const char* label, int* status, cudaStream_t s, int ksplit, float* part) {
+                    long long rows_max, const char* label, int* status, cudaStream_t s, int ksplit, float* part,
+                    const WgradGather& g) {
     using Cf = WCfg<BN, MT>;
     static bool attr_set = false;
     auto kern = wgrad_kernel<BN, MT>;
@@ -228,12 +255,21 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
     }
     CUtensorMap tmP, tmQ;
     const uint32_t box[2] = {64, BK};
-    {
+    const uint32_t gbox[3] = {64, (uint32_t)(g.l_p < BK ? g.l_p : BK), 1};
+    if (g.gather_p) {      // P rows come from the source tensor [Bm patches, l_p, M]
+        const uint64_t dims[3] = {(uint64_t)M, (uint64_t)g.l_p, (uint64_t)g.Bm};
+        const uint64_t str[2] = {(uint64_t)M * 2, (uint64_t)M * 2 * g.l_p};
+        if (!make_tmap(&tmP, P, 3, dims, str, gbox)) return UOE_ERR_CUDA;
+    } else {
         const uint64_t dims[2] = {(uint64_t)M, (uint64_t)rows_max};
         const uint64_t str[1] = {(uint64_t)M * 2};
         if (!make_tmap(&tmP, P, 2, dims, str, box)) return UOE_ERR_CUDA;
     }
-    {
+    if (g.gather_q) {
+        const uint64_t dims[3] = {(uint64_t)N, (uint64_t)g.l_p, (uint64_t)g.Bm};
+        const uint64_t str[2] = {(uint64_t)N * 2, (uint64_t)N * 2 * g.l_p};
+        if (!make_tmap(&tmQ, Q, 3, dims, str, gbox)) return UOE_ERR_CUDA;
+    } else {
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)rows_max};
         const uint64_t str[1] = {(uint64_t)N * 2};
         if (!make_tmap(&tmQ, Q, 2, dims, str, box)) return UOE_ERR_CUDA;
@@ -248,7 +284,8 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
     const long long tiles = (long long)n * (M / (MT * BM)) * (N / BN) * ksplit;
     int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     ProfScope ps(label, s);
-    launch_k(kern, grid, dim3(Cf::THREADS), Cf::SMEM, s, tmP, tmQ, tmW, offsets, n, M, N, ksplit, status);
+    launch_k(kern, grid, dim3(Cf::THREADS), Cf::SMEM, s, tmP, tmQ, tmW, offsets, n, M, N, ksplit, status, g.gather_p ? 1 : 0,
+             g.gather_q ? 1 : 0, g.src_patch, g.l_p, g.Bm);
     UOE_LAUNCHED();
     if (ksplit > 1) {
         const long long vecs = (long long)n * M * N / 4;
@@ -281,16 +318,18 @@ size_t wgrad_scratch_bytes(int n, int M, int N, long long rows_max) {
 }
 
 uoe_status launch_wgrad_bf16(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
-                             long long rows_max, const char* label, int* status, cudaStream_t s, float* part) {
+                             long long rows_max, const char* label, int* status, cudaStream_t s, float* part,
+                             const WgradGather& g) {
     if (M % BM != 0 || N % 64 != 0 || n > 32) return UOE_ERR_UNSUPPORTED;
+    if ((g.gather_p || g.gather_q) && (!g.src_patch || !wgrad_can_gather(g.l_p))) return UOE_ERR_INVALID_ARG;
     const int bn = gemm_bf16_bn(N);
     const int ks = part ? wgrad_ksplit(n, M, N, rows_max) : 1;
     // 256-row output tiles when the weight matrices are large enough to keep every SM busy with them
     if (bn == 256 && M % 256 == 0 && (long long)n * (M / 256) * (N / 256) >= 2 * sm_count())
-        return launch_w<256, 2>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, 1, nullptr);
-    if (bn == 256) return launch_w<256, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, ks, part);
-    if (bn == 128) return launch_w<128, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, ks, part);
-    return launch_w<64, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, ks, part);
+        return launch_w<256, 2>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, 1, nullptr, g);
+    if (bn == 256) return launch_w<256, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, ks, part, g);
+    if (bn == 128) return launch_w<128, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, ks, part, g);
+    return launch_w<64, 1>(P, Q, dW, offsets, n, M, N, rows_max, label, status, s, ks, part, g);
 }
 
 }  // namespace uoe
