@@ -140,8 +140,9 @@ SmhaBwdWs smha_bwd_ws(const Dims& D) {
     const int heads = D.d_g > 0 ? D.d_g / 64 : 1;
     const size_t rg = (size_t)D.Rmax * D.d_g * D.esize;
     r.plan = w.take(plan_bytes(D, true));
-    r.xg = w.take((size_t)D.Rmax * D.d * D.esize);
-    r.dyg = w.take((size_t)D.Rmax * D.d * D.esize);
+    const bool fused = can_fuse_gather(D) && wgrad_can_gather(D.l_p);      // x and dy gathered inside the consumers' TMA loads
+    r.xg = fused ? 0 : w.take((size_t)D.Rmax * D.d * D.esize);
+    r.dyg = fused ? 0 : w.take((size_t)D.Rmax * D.d * D.esize);
     r.q = w.take(rg); r.k = w.take(rg); r.v = w.take(rg); r.o = w.take(rg); r.dout = w.take(rg); r.og = w.take(rg);
     r.dqkv = w.take(3 * rg);
     r.dxg = w.take((size_t)D.Rmax * D.d * D.esize);
@@ -208,10 +209,17 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
 
     st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream, use_gate, v, rowb);
     if (st != UOE_OK) return st;
-    st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
-    if (st != UOE_OK) return st;
-    st = launch_gather(D, dy, patch_idx, expert_offsets, P, dyg, stream);
-    if (st != UOE_OK) return st;
+    // Eq. 18 for x and dy: either inside the TMA loads of the kernels that consume them, or as routed copies
+    const bool fused = can_fuse_gather(D) && wgrad_can_gather(D.l_p);
+    WgradGather gp;
+    if (fused) {
+        gp.gather_p = true; gp.src_patch = P.src_patch; gp.l_p = D.l_p; gp.Bm = D.B * D.m;
+    } else {
+        st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
+        if (st != UOE_OK) return st;
+        st = launch_gather(D, dy, patch_idx, expert_offsets, P, dyg, stream);
+        if (st != UOE_OK) return st;
+    }
     {
         ProfScope ps("zero_pad_rows", stream);
         launch_k(zero_pad_rows_kernel, dim3(D.n + 1, 16), dim3(kThreads), 0, stream, (uint4*)q, (uint4*)k, (uint4*)dout,
@@ -224,6 +232,7 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
 
     // ---- forward recomputation (Eq. 28-34) ----
     GemmArgs gq{xg, Wq, nullptr, q, nullptr, expert_offsets, D.n, D.d, D.d_g, UOE_ACT_IDENTITY, false, D.Rmax};
+    if (fused) { gq.gather_x = x; gq.src_patch = P.src_patch; gq.l_p = D.l_p; gq.Bm = D.B * D.m; }
     gq.label = "qkv_proj";
     gq.nmat = 3; gq.W1 = Wk; gq.W2 = Wv; gq.C1 = k; gq.C2 = v;
     st = launch_gemm_bf16(gq, status, stream);
@@ -235,6 +244,7 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
 
     // ---- out-projection backward ----
     GemmArgs gd{dyg, Wo, nullptr, dout, nullptr, expert_offsets, D.n, D.d, D.d_g, UOE_ACT_IDENTITY, true, D.Rmax};
+    if (fused) { gd.gather_x = dy; gd.src_patch = P.src_patch; gd.l_p = D.l_p; gd.Bm = D.B * D.m; }
     gd.label = "bwd_do";
     st = launch_gemm_bf16(gd, status, stream);
     if (st != UOE_OK) return st;
@@ -246,8 +256,8 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
                  (const float*)P.row_valid, delta, dgp, expert_offsets, D.n, heads, D.d_g);
     }
     UOE_LAUNCHED();
-    st = launch_wgrad_bf16(dyg, og, dwot, expert_offsets, D.n, D.d, D.d_g, D.Rmax, "wgrad_Wo", status, stream,
-                           wgrad_scratch_bytes(D.n, D.d, D.d_g, D.Rmax) ? (float*)(base + W.wgpart) : nullptr);
+    st = launch_wgrad_bf16(fused ? dy : dyg, og, dwot, expert_offsets, D.n, D.d, D.d_g, D.Rmax, "wgrad_Wo", status, stream,
+                           wgrad_scratch_bytes(D.n, D.d, D.d_g, D.Rmax) ? (float*)(base + W.wgpart) : nullptr, gp);
     if (st != UOE_OK) return st;
 
     // ---- attention backward ----
@@ -271,8 +281,8 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
     gx.label = "bwd_dx_att";
     st = launch_gemm_bf16(gx, status, stream);
     if (st != UOE_OK) return st;
-    st = launch_wgrad_bf16(xg, dqkv, dwcat, expert_offsets, D.n, D.d, 3 * D.d_g, D.Rmax, "wgrad_Wqkv", status, stream,
-                           wgrad_scratch_bytes(D.n, D.d, 3 * D.d_g, D.Rmax) ? (float*)(base + W.wgpart) : nullptr);
+    st = launch_wgrad_bf16(fused ? x : xg, dqkv, dwcat, expert_offsets, D.n, D.d, 3 * D.d_g, D.Rmax, "wgrad_Wqkv", status, stream,
+                           wgrad_scratch_bytes(D.n, D.d, 3 * D.d_g, D.Rmax) ? (float*)(base + W.wgpart) : nullptr, gp);
     if (st != UOE_OK) return st;
     {
         ProfScope ps("finalize_wgrads", stream);
