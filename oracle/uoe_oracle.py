@@ -19,6 +19,7 @@ Functions and the passages they follow
   patch_expert_counts, dynamic_capacity   Eq. 15-16 (two-stage routing: c = largest number of patches any
                    expert receives when every patch goes to its k best experts)
   balance_loss     Eq. 42-44 (sequence-wise load-balancing loss over the patches of one sample)
+  balance_loss_backward   its gradient w.r.t. x and W_r (through P_i; pinned by finite differences)
   mlp_forward      Eq. 18-20 and Eq. 37-40 (UoME), decomposition Eq. 1-7
   smha_forward     Eq. 27-30, 33-36 (SMHA), masks Eq. 41 and Fig. 4, decomposition Eq. 8-11
   mlp_backward     derivative of mlp_forward with the selection held constant (no paper text;
@@ -184,6 +185,32 @@ def balance_loss(p_patch: np.ndarray, cnt: np.ndarray, k: int, alpha: float = 1.
         P = p_patch[b][:, elig].mean(axis=1)                               # Eq. 44
         out[b] = alpha * float(np.sum(f * P))                              # Eq. 42
     return out
+
+
+def balance_loss_backward(x: np.ndarray, W_r: np.ndarray, m: int, L_valid: int, k: int, alpha: float,
+                          dloss: np.ndarray):
+    """Gradient of sum_b dloss[b] * L_b (Eq. 42-44) with respect to x and W_r.  f_i (Eq. 43) counts top-k memberships
+    and is piecewise constant, so the gradient flows through P_i (Eq. 44) only:
+    dL_b/dg_{i,t} = alpha f_i / l on the real patches, then the softmax Jacobian of Eq. 14 and the mean-pooled
+    linear router of Eq. 13."""
+    B, L, d = x.shape
+    n = W_r.shape[1]
+    l_p = L // m
+    p_samp, p_patch, pool, samp, cnt = router_probs(x, W_r, m, L_valid)
+    l = int((cnt > 0).sum())
+    dx = np.zeros_like(x)
+    dW_r = np.zeros_like(W_r)
+    for b in range(B):
+        f = n / (k * l) * patch_expert_counts(p_patch[b], cnt, k)
+        for j in range(m):
+            if cnt[j] == 0:
+                continue
+            dg = dloss[b] * alpha * f / l                                  # d/dg_{:,j}
+            pj = p_patch[b, :, j]
+            dlogit = pj * (dg - np.dot(pj, dg))                            # softmax Jacobian, Eq. 14
+            dW_r += np.outer(pool[b, j], dlogit)
+            dx[b, j * l_p: j * l_p + cnt[j]] += (W_r @ dlogit)[None, :] / cnt[j]
+    return dx, dW_r
 
 
 def select(p_samp: np.ndarray, p_patch: np.ndarray, cnt: np.ndarray, k: int, c: int, dynamic_c: bool = False):

@@ -442,6 +442,32 @@ def test_dynamic_capacity_limits_the_patches_per_expert():
     assert (c_dyn < w.c).any()          # the case really exercises a smaller capacity
 
 
+@pytest.mark.parametrize("L_valid", [24, 19])
+def test_balance_loss_backward_matches_finite_differences(L_valid):
+    w = gen.tiny(B=3, n=5, k=2, m=6, c=3, d=8)
+    x = gen.make_x(w).f64
+    Wr = gen.normal(5, 4, (w.d, w.n)) * 0.8
+    dloss = np.array([0.5, -1.25, 2.0])
+    alpha = 0.3
+    dx, dWr = orc.balance_loss_backward(x, Wr, w.m, L_valid, w.k, alpha, dloss)
+
+    def loss(x_, Wr_):
+        _, pp, _, _, cnt = orc.router_probs(x_, Wr_, w.m, L_valid)
+        return float(np.dot(dloss, orc.balance_loss(pp, cnt, w.k, alpha)))
+
+    eps = 1e-6
+    for which, grad, arr in (("x", dx, x), ("Wr", dWr, Wr)):
+        for trial in range(3):
+            v = gen.normal(400 + trial, 0 if which == "x" else 1, arr.shape)
+            if which == "x":
+                v[:, L_valid:] = 0.0
+            fd = (loss(x + eps * v, Wr) - loss(x - eps * v, Wr)) / (2 * eps) if which == "x" else \
+                (loss(x, Wr + eps * v) - loss(x, Wr - eps * v)) / (2 * eps)
+            an = float(np.sum(grad * v))
+            assert abs(fd - an) <= 1e-6 * max(1.0, abs(an)), (which, fd, an)
+    assert np.all(dx[:, L_valid:] == 0.0)
+
+
 # ----------------------------------------------------------------------------------------------
 # backward: central finite differences with the selection frozen
 # ----------------------------------------------------------------------------------------------
