@@ -72,7 +72,8 @@ enum {
                                   each patch goes to its k best experts; the remaining slots are unused (-1) */
 };
 
-typedef enum { UOE_OP_ROUTE = 0, UOE_OP_MLP_FWD = 1, UOE_OP_MLP_BWD = 2, UOE_OP_SMHA_FWD = 3, UOE_OP_SMHA_BWD = 4 } uoe_op;
+typedef enum { UOE_OP_ROUTE = 0, UOE_OP_MLP_FWD = 1, UOE_OP_MLP_BWD = 2, UOE_OP_SMHA_FWD = 3, UOE_OP_SMHA_BWD = 4,
+               UOE_OP_BALANCE_BWD = 5 } uoe_op;
 
 /* One Union-of-Experts block.  L must equal m * l_p; rows t >= L_valid of every sample are padding
  * (they take no part in routing means, are masked as attention keys (Eq. 41), and y = x there). */
@@ -134,6 +135,18 @@ uoe_status uoe_route(const uoe_problem* prob, const void* x, const void* W_r,
  */
 uoe_status uoe_route_balance(const uoe_problem* prob, const float* p_patch, float alpha, float* lb_loss,
                              int32_t* expert_count, int32_t* c_dyn, void* cuda_stream);
+
+/*
+ * Gradient of sum_b dloss[b] * lb_loss[b] (the loss of uoe_route_balance, Eq. 42-44) with respect to x and W_r.
+ * f_i counts top-k memberships and is piecewise constant, so the gradient flows through P_i only: through the patch
+ * softmax (Eq. 14) and the mean-pooled linear router (Eq. 13).  The paper gives no backward text.
+ *   dx [B,L,d] in prob->dtype and dW_r [d,n] float32 are overwritten (add them to the layer's own gradients);
+ *   dloss [B] float32; p_patch [B,n,m] as written by uoe_route for the same x and W_r.  bfloat16 only.
+ * Workspace: uoe_workspace_bytes(prob, UOE_OP_BALANCE_BWD).  All pointers except prob are device pointers.
+ */
+uoe_status uoe_route_balance_backward(const uoe_problem* prob, const void* x, const void* W_r, const float* p_patch,
+                                      float alpha, const float* dloss, void* dx, float* dW_r,
+                                      void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
  * UoME forward (Eq. 37-40 with the index-select of Eq. 18 and the index-add of Eq. 20):

@@ -21,6 +21,7 @@ UOE_F32, UOE_BF16 = 0, 1
 ACTS = {"gelu_erf": 0, "gelu_tanh": 1, "silu": 2, "identity": 3}
 UOE_FLAG_RESIDUAL, UOE_FLAG_GATE, UOE_FLAG_CAUSAL, UOE_FLAG_DYNAMIC_C = 1, 2, 4, 8
 UOE_OP_ROUTE, UOE_OP_MLP_FWD, UOE_OP_MLP_BWD, UOE_OP_SMHA_FWD, UOE_OP_SMHA_BWD = 0, 1, 2, 3, 4
+UOE_OP_BALANCE_BWD = 5
 
 
 class UoeError(RuntimeError):
@@ -103,6 +104,8 @@ def _load():
                                       f32p, f32p, f32p, vp, sz, vp]
     lib.uoe_route_balance.restype = ctypes.c_int
     lib.uoe_route_balance.argtypes = [pp, f32p, ctypes.c_float, f32p, i32p, i32p, vp]
+    lib.uoe_route_balance_backward.restype = ctypes.c_int
+    lib.uoe_route_balance_backward.argtypes = [pp, vp, vp, f32p, ctypes.c_float, f32p, vp, f32p, vp, sz, vp]
     lib.uoe_status_string.restype = ctypes.c_char_p
     lib.uoe_status_string.argtypes = [ctypes.c_int]
     lib.uoe_workspace_init.restype = ctypes.c_int
@@ -327,3 +330,19 @@ def uoe_route_balance(prob: Problem, p_patch, alpha: float = 1.0):
                                 _ptr(cd), _stream())
     _check(st, "uoe_route_balance")
     return lb, cnt, cd
+
+
+def uoe_route_balance_backward(prob: Problem, x, W_r, p_patch, alpha: float, dloss, ws=None):
+    """(dx [B,L,d], dW_r [d,n] float32): gradient of sum(dloss * lb_loss) with respect to x and W_r."""
+    _contig(x, prob.torch_dtype)
+    _contig(W_r, prob.torch_dtype)
+    _contig(p_patch, torch.float32)
+    _contig(dloss, torch.float32)
+    dx = torch.empty_like(x)
+    dW_r = torch.empty(W_r.shape, dtype=torch.float32, device=x.device)
+    ws = ws if ws is not None else alloc_workspace(prob, UOE_OP_BALANCE_BWD, x.device)
+    st = _lib.uoe_route_balance_backward(ctypes.byref(prob.c_struct()), _ptr(x), _ptr(W_r), _ptr(p_patch),
+                                         ctypes.c_float(alpha), _ptr(dloss), _ptr(dx), _ptr(dW_r), _ptr(ws), ws.numel(),
+                                         _stream())
+    _check(st, "uoe_route_balance_backward")
+    return dx, dW_r

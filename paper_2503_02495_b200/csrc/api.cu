@@ -58,6 +58,7 @@ extern "C" size_t uoe_workspace_bytes(const uoe_problem* prob, int op) {
         case UOE_OP_MLP_BWD: return D.d_e > 0 ? mlp_bwd_workspace_bytes(D) : 0;
         case UOE_OP_SMHA_FWD: return D.H > 0 ? smha_fwd_workspace_bytes(D) : 0;
         case UOE_OP_SMHA_BWD: return D.H > 0 ? smha_bwd_workspace_bytes(D) : 0;
+        case UOE_OP_BALANCE_BWD: return balance_bwd_workspace_bytes(D);
         default: return 0;
     }
 }

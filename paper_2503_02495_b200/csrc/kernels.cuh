@@ -9,6 +9,7 @@ size_t mlp_fwd_workspace_bytes(const Dims& D);
 size_t mlp_bwd_workspace_bytes(const Dims& D);
 size_t smha_fwd_workspace_bytes(const Dims& D);
 size_t smha_bwd_workspace_bytes(const Dims& D);
+size_t balance_bwd_workspace_bytes(const Dims& D);
 
 // Layout of the routing plan inside a workspace: where each (sample, expert) pair's rows start and,
 // for every patch of every sample, which routed rows and gates feed it back (the inverse of Eq. 18).

@@ -197,6 +197,61 @@ dwr_sum_kernel(const float* __restrict__ part, float* __restrict__ dW_r, int tot
     dW_r[idx] = a;
 }
 
+// Gradient of the load-balancing loss (Eq. 42-44) with respect to the router logits.  grid B, 128 threads, dynamic
+// shared memory n*m floats.  f_i (Eq. 43) is piecewise constant, so only P_i (Eq. 44) carries a gradient:
+//   dL_b/dg_{i,j} = alpha f_i / l on the real patches;  G[b,j,i] = softmax Jacobian (Eq. 14) of that, / cnt_j.
+__global__ void __launch_bounds__(128)
+balance_bwd_kernel(const float* __restrict__ p_patch, const float* __restrict__ dloss, int Lv, int n, int k, int m,
+                   int l_p, float alpha, float* __restrict__ G) {
+    pdl_trigger();
+    pdl_wait();
+    extern __shared__ float pp[];          // [n][m]
+    __shared__ int cnts[32];
+    const int b = blockIdx.x, tid = threadIdx.x;
+    const int n_elig = (Lv + l_p - 1) / l_p;
+    for (int idx = tid; idx < n * m; idx += 128) pp[idx] = p_patch[(size_t)b * n * m + idx];
+    if (tid < 32) cnts[tid] = 0;
+    __syncthreads();
+    for (int j = tid; j < n_elig; j += 128) {      // Eq. 15 / 43: patch j counts for its k best experts
+        for (int i = 0; i < n; ++i) {
+            const float v = pp[i * m + j];
+            int rank = 0;
+            for (int q = 0; q < n; ++q) {
+                const float w = pp[q * m + j];
+                rank += (w > v) || (w == v && q < i);
+            }
+            if (rank < k) atomicAdd(&cnts[i], 1);
+        }
+    }
+    __syncthreads();
+    const float scale = dloss[b] * alpha * (float)n / ((float)k * (float)n_elig * (float)n_elig);     // dloss alpha (n / k l) / l
+    for (int j = tid; j < m; j += 128) {
+        const int cnt = max(0, min(l_p, Lv - j * l_p));
+        float dot = 0.f;
+        for (int i = 0; i < n; ++i) dot += pp[i * m + j] * scale * (float)cnts[i];
+        for (int i = 0; i < n; ++i) {
+            const float dl = pp[i * m + j] * (scale * (float)cnts[i] - dot);
+            G[((size_t)b * m + j) * n + i] = cnt > 0 ? dl / (float)cnt : 0.f;
+        }
+    }
+}
+
+// dx[b, t, :] = rvec[b, patch of t, :] on real tokens, 0 on pad tokens (bf16).  grid B*m, 256 threads.
+__global__ void __launch_bounds__(kThreads)
+spread_rvec_kernel(const float* __restrict__ rvec, __nv_bfloat16* __restrict__ dx, int L, int Lv, int d, int m, int l_p) {
+    pdl_trigger();
+    pdl_wait();
+    const int bj = blockIdx.x, b = bj / m, j = bj % m;
+    const int vpr = d / 8;
+    for (int idx = threadIdx.x; idx < l_p * vpr; idx += kThreads) {
+        const int r = idx / vpr, cv = idx % vpr, t = j * l_p + r;
+        float f[8];
+#pragma unroll
+        for (int v = 0; v < 8; ++v) f[v] = t < Lv ? rvec[(size_t)bj * d + cv * 8 + v] : 0.f;
+        st_stream16(dx + ((size_t)b * L + t) * d + (size_t)cv * 8, pack16<__nv_bfloat16>(f));
+    }
+}
+
 struct BwdWs { size_t plan, dyg, xg, dh, ag, dxg, dgp, G, pool, rvec, dgate, wpart, wgpart, total; int nt; };
 
 BwdWs bwd_ws(const Dims& D) {
@@ -384,4 +439,64 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
     }
     // dx = dy (selective residual) + the routed input gradients (the gate is already inside dh) + router term
     return launch_combine(D, dy, dxg, P, residual, false, dx, stream, use_gate ? rvec : nullptr);
+}
+
+
+namespace uoe {
+size_t balance_bwd_workspace_bytes(const Dims& D) { return kStatusBytes + router_backward_scratch_bytes(D); }
+}  // namespace uoe
+
+extern "C" uoe_status uoe_route_balance_backward(const uoe_problem* prob, const void* x, const void* W_r,
+                                                 const float* p_patch, float alpha, const float* dloss, void* dx,
+                                                 float* dW_r, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Dims D;
+    uoe_status st = make_dims(prob, D);
+    if (st != UOE_OK) return st;
+    if (!x || !W_r || !p_patch || !dloss || !dx || !dW_r || !ws) return UOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(dx) || !aligned16(ws)) return UOE_ERR_INVALID_ARG;
+    if (!D.bf16) return UOE_ERR_UNSUPPORTED;
+    if ((size_t)D.n * D.m * sizeof(float) > 36 * 1024) return UOE_ERR_UNSUPPORTED;
+    if (ws_bytes < balance_bwd_workspace_bytes(D)) return UOE_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const RouterBwdScratch rs = router_backward_scratch(D, (char*)ws + kStatusBytes);
+    {
+        ProfScope ps("balance_bwd", stream);
+        launch_k(balance_bwd_kernel, dim3(D.B), dim3(128), (size_t)D.n * D.m * sizeof(float), stream, p_patch, dloss, D.Lv, D.n,
+                 D.k, D.m, D.l_p, alpha, rs.G);
+    }
+    UOE_LAUNCHED();
+    int CT = 64;
+    while (CT > 1 && (CT / 2) * 8 >= D.d) CT /= 2;
+    const int nchunks = (D.d + CT * 8 - 1) / (CT * 8);
+    {
+        ProfScope ps("pool", stream);
+        launch_k(pool_kernel<__nv_bfloat16>, dim3((unsigned)(D.B * D.m * nchunks)), dim3(kThreads), 0, stream,
+                 (const __nv_bfloat16*)x, rs.pool, D.L, D.Lv, D.d, D.m, D.l_p, CT, nchunks);
+    }
+    UOE_LAUNCHED();
+    {
+        ProfScope ps("dW_r", stream);
+        launch_k(dwr_partial_kernel, dim3((D.d + kThreads - 1) / kThreads, kDwrSplit), dim3(kThreads), 0, stream, (const float*)rs.pool,
+                 (const float*)rs.G, rs.wpart, D.B * D.m, D.d, D.n);
+    }
+    UOE_LAUNCHED();
+    {
+        ProfScope ps("dW_r_sum", stream);
+        const int total = D.d * D.n;
+        launch_k(dwr_sum_kernel, dim3((total + kThreads - 1) / kThreads), dim3(kThreads), 0, stream, (const float*)rs.wpart, dW_r, total);
+    }
+    UOE_LAUNCHED();
+    {
+        ProfScope ps("router_dx_vec", stream);
+        launch_k(rvec_kernel<__nv_bfloat16>, dim3(D.B * D.m), dim3(kThreads), 0, stream, (const __nv_bfloat16*)W_r, (const float*)rs.G,
+                 rs.rvec, D.d, D.n);
+    }
+    UOE_LAUNCHED();
+    {
+        ProfScope ps("spread_rvec", stream);
+        launch_k(spread_rvec_kernel, dim3(D.B * D.m), dim3(kThreads), 0, stream, (const float*)rs.rvec, (__nv_bfloat16*)dx, D.L, D.Lv,
+                 D.d, D.m, D.l_p);
+    }
+    UOE_LAUNCHED();
+    return UOE_OK;
 }

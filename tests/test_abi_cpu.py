@@ -72,6 +72,9 @@ def test_every_entry_point_validates_on_the_host(uoe):
     assert lib.uoe_smha_backward(ctypes.byref(att), *([None] * 20), sz0, None) == 1
     assert lib.uoe_route_static(ctypes.byref(mlp), *([None] * 8), None) == 1
     assert lib.uoe_route_balance(ctypes.byref(mlp), None, ctypes.c_float(1.0), None, None, None, None) == 1
+    lib.uoe_route_balance_backward.restype = ctypes.c_int
+    assert lib.uoe_route_balance_backward(ctypes.byref(mlp), None, None, None, ctypes.c_float(1.0), None, None, None, None,
+                                          sz0, None) == 1
     assert lib.uoe_workspace_init(None, sz0, None) == 1
     assert lib.uoe_read_device_status(None, None) == 1
     # a problem that is itself invalid is refused whatever the pointers are

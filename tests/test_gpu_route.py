@@ -152,3 +152,27 @@ def test_route_with_dynamic_capacity_matches_oracle(name):
         ref = orc.mlp_forward(x.f64, W1.f64, W2.f64, ro, w.act, residual=False)
         got = y.detach().to(torch.float64).cpu().numpy()
         assert np.abs(got - ref).max() <= 2e-2 * np.abs(ref).max()
+
+
+@pytest.mark.parametrize("name", ["tiny_pad", "cfg2", "cfg4"])
+def test_route_balance_backward_matches_oracle(name):
+    """Gradient of sum(dloss * lb_loss) w.r.t. x and W_r: bf16 inputs, fp32 arithmetic; the oracle recomputes the
+    gate in float64 from the same stored inputs.  Tolerance 2e-2 * max|ref| as for the other bf16 gradients (dx is
+    stored in bf16)."""
+    import paper_2503_02495_b200 as uoe
+    w, scale = BAL_CASES[name]
+    if w.dtype != "bf16":
+        w = w.replace(dtype="bf16", d=64)
+    x = gen.make_x(w)
+    Wr = gen.store(gen.make_router(w).f64 * scale, w.dtype)
+    prob = problem_of(w, "mlp")
+    xd, Wrd = to_dev(x), to_dev(Wr)
+    r = uoe.uoe_route(prob, xd, Wrd)
+    dloss = gen.normal(77, 0, (w.B,))
+    dl = torch.from_numpy(dloss.astype(np.float32)).cuda()
+    dx, dWr = uoe.uoe_route_balance_backward(prob, xd, Wrd, r.p_patch, 0.05, dl)
+    ref_dx, ref_dWr = orc.balance_loss_backward(x.f64, Wr.f64, w.m, w.L_valid, w.k, 0.05, dloss.astype(np.float32).astype(np.float64))
+    got_dx = dx.detach().to(torch.float64).cpu().numpy()
+    assert np.abs(got_dx - ref_dx).max() <= 2e-2 * np.abs(ref_dx).max()
+    assert np.abs(dWr.cpu().numpy() - ref_dWr).max() <= 2e-2 * np.abs(ref_dWr).max()
+    assert np.all(got_dx[:, w.L_valid:] == 0)
