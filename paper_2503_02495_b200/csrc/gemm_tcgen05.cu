@@ -35,9 +35,10 @@ template <int BN, int MT> struct Cfg {
     static constexpr int A_BYTES = MT * A_BLOCK_BYTES;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (MT == 2) ? 3 : ((BN == 256) ? 4 : (BN == 128 ? 6 : 8));
+    static constexpr int STAGES = (MT == 2) ? 3 : ((BN == 256) ? 4 : (BN == 192 ? 5 : (BN == 128 ? 6 : 8)));
     static constexpr int NACC = (MT == 2) ? 1 : 2;                 // accumulator sets in TMEM
-    static constexpr int TMEM_COLS = 2 * BN;                       // MT=1: two sets; MT=2: one set of two blocks
+    static constexpr int ACC_STRIDE = (BN == 192) ? 256 : BN;      // TMEM columns between the two accumulator sets
+    static constexpr int TMEM_COLS = 2 * ACC_STRIDE;               // MT=1: two sets; MT=2: one set of two blocks
     static constexpr int EPI_WARPS = 4 * MT;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
     static constexpr int STG_BYTES = 32 * 128;                     // one epilogue warp's staging piece
@@ -103,8 +104,12 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const uint32_t tmem_base = ctl->tmem_base;
 
     // tile index -> (row tile, matrix, column tile); the matrices share the A tile, so they are adjacent
-    const int n_tiles_mat = N / BN;
-    const int n_tiles = n_tiles_mat * nmat;
+    // BN = 192 is the "three 64-wide matrices side by side" tile: the B stage holds one 64-column box of each of the
+    // three weight tensors and the three 64-column pieces of the accumulator go to the three outputs, so the A tile is
+    // loaded once for q, k and v
+    constexpr bool SIDE3 = BN == 192;
+    const int n_tiles_mat = SIDE3 ? 1 : N / BN;
+    const int n_tiles = SIDE3 ? 1 : n_tiles_mat * nmat;
     const int num_kb = K / BK;
     const int total_tiles = ctl->tstart[n] * n_tiles;
 
@@ -124,6 +129,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         uint32_t issued = 0, issued_parity = 0;      // per stage: a load is in flight with this parity
         bool stop = false;
         constexpr int nbox_b = B_KMAJOR ? 1 : BN / 64;
+        const CUtensorMap* tmB_lane = lane == 0 ? &tmB0 : (lane == 1 ? &tmB1 : &tmB2);
         for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
             int e, row0, blocks;
             locate(tile / n_tiles, e, row0, blocks);
@@ -150,7 +156,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     else tma_load_2d(sa + lane * A_BLOCK_BYTES, &tmA, kb * BK, row0 + lane * BM, &ctl->full[stage]);
                 }
                 if (lane < nbox_b) {
-                    if (B_KMAJOR) tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
+                    if (SIDE3) tma_load_3d(sb + lane * 8192, tmB_lane, 0, kb * BK, e, &ctl->full[stage]);
+                    else if (B_KMAJOR) tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
                     else tma_load_3d(sb + lane * 8192, tmB, col0 + lane * 64, kb * BK, e, &ctl->full[stage]);
                 }
                 issued |= 1u << stage;
@@ -174,7 +181,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 locate(tile / n_tiles, e, row0, blocks);
                 if (!mbar_wait(&ctl->tempty[acc], acc_phase ^ 1, abort_flag, status) || *abort_flag) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + acc * BN;        // MT=2: acc is always 0, block h at column h*BN
+                const uint32_t d_tmem = tmem_base + acc * Cf::ACC_STRIDE;        // MT=2: acc is always 0, block h at column h*BN
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&ctl->full[stage], phase, abort_flag, status) || *abort_flag) { stop = true; break; }
                     tc_fence_after();
@@ -232,7 +239,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (half < blocks) {
                 const int wrow0 = row0 + half * BM + quarter * 32;       // first row of this warp's piece
                 const size_t row = (size_t)wrow0 + lane;
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (MT == 2 ? half * BN : acc * BN);
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (MT == 2 ? half * BN : acc * Cf::ACC_STRIDE);
                 if constexpr (BWD) {
                     const float rg = row_gate[row], rv = row_valid[row];
                     float dsum = 0.f;
@@ -273,7 +280,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         for (int q = 0; q < 64; ++q) f[q] = __uint_as_float(v[q]);
                         if (pre) stage_store(f, &tmPre, col0 + g * 64, wrow0);
                         act_apply_n<64>(f, act);
-                        stage_store(f, tmC, col0 + g * 64, wrow0);
+                        if (SIDE3) stage_store(f, g == 0 ? &tmC0 : (g == 1 ? &tmC1 : &tmC2), 0, wrow0);
+                        else stage_store(f, tmC, col0 + g * 64, wrow0);
                     }
                 }
             }
@@ -340,7 +348,7 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
             if (!make_tmap(&tmC[q], Cs[q], 2, dims, str, box)) return UOE_ERR_CUDA;
         if (!make_tmap(&tmPre, g.pre ? g.pre : g.C, 2, dims, str, box)) return UOE_ERR_CUDA;
     }
-    long long max_tiles = ((g.rows_max / BM + MT - 1) / MT + g.n) * (g.N / BN) * nmat;
+    long long max_tiles = ((g.rows_max / BM + MT - 1) / MT + g.n) * (BN == 192 ? 1 : (g.N / BN) * nmat);
     int grid = (int)(max_tiles < sm_count() ? max_tiles : sm_count());
     if (grid < 1) grid = 1;
     ProfScope ps(g.label, s);
@@ -380,6 +388,7 @@ uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s) {
             return UOE_ERR_INVALID_ARG;
         return dispatch<true, true>(g, status, s);
     }
+    if (g.nmat == 3 && g.N == 64 && !g.b_kmajor && !g.pre) return launch_one<192, false, false, 1>(g, status, s);
     if (g.b_kmajor) return dispatch<true, false>(g, status, s);
     return dispatch<false, false>(g, status, s);
 }

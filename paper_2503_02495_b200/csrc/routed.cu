@@ -42,9 +42,18 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
         s_pi[idx] = pj;
         s_g[idx] = gate[(size_t)b * k * c + idx];
     }
-    for (int idx = tid; idx < b * k; idx += 128) {          // choices of the samples before b, per expert
-        const int e = expert_idx[idx];
-        if (e >= 0 && e < n) atomicAdd(&hist[e], 1);
+    {   // choices of the samples before b, per expert: lane i of each warp counts expert i through ballots
+        int acc = 0;
+        const int lane = tid & 31;
+        for (int i0 = 0; i0 < b * k; i0 += 128) {
+            const int idx = i0 + tid;
+            const int e = idx < b * k ? expert_idx[idx] : -1;
+            for (int i = 0; i < n; ++i) {
+                const unsigned msk = __ballot_sync(0xffffffffu, e == i);
+                if (lane == i) acc += __popc(msk);
+            }
+        }
+        if (lane < n && acc) atomicAdd(&hist[lane], acc);
     }
     __syncthreads();
     if (tid < k) {
