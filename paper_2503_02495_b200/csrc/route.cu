@@ -16,14 +16,14 @@ namespace {
 
 constexpr int kScoreThreads = 256;
 
-// Selection for sample b by one CTA of kScoreThreads threads (all threads call).  pp: n*m floats of shared memory.
+// Selection for sample b by one CTA of NT threads (all threads call).  pp: n*m floats of shared memory.
+template <int NT>
 __device__ void select_sample(float* pp, const float* __restrict__ partial, int nparts, int b, int B, int Lv, int n, int k,
                               int m, int c, int l_p, int sel_flags /* bit 0: gate weights, bit 1: dynamic capacity */,
                               int* __restrict__ expert_idx,
                               int* __restrict__ patch_idx, float* __restrict__ gate, float* __restrict__ p_samp,
                               float* __restrict__ p_patch, int* __restrict__ offsets, int* __restrict__ load,
                               int* __restrict__ ticket) {
-    constexpr int NT = kScoreThreads;
     __shared__ float ps[32];               // sample gate
     __shared__ int sel[32];                // chosen experts, ascending
     __shared__ int cnts[32];               // Eq. 16: patches each expert receives in the first routing stage
@@ -173,8 +173,8 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
 // where step 1 should be nothing but streaming.
 // Dynamic shared memory: max(n*m floats for step 3, the blocks of W_r rows for step 2).
 
-template <typename T, int MODE>
-__global__ void __launch_bounds__(kScoreThreads, MODE == 1 ? 6 : 5)
+template <typename T, int MODE, int NT>
+__global__ void __launch_bounds__(NT, NT == 64 ? 16 : (MODE == 1 ? 6 : 5))
 route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ pool_part,
              float* __restrict__ scores, int B, int L, int Lv, int d, int n, int k, int m, int c, int l_p, int CT,
              int nchunks, int rsplit, int rows_per_cta, int wblk_bytes, int csplit, int use_gate,
@@ -185,7 +185,6 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
     pdl_trigger();
     pdl_wait();
     constexpr int V = Vec16<T>::N;
-    constexpr int NT = kScoreThreads;
     extern __shared__ uint4 s_dyn4[];
     __shared__ __align__(16) float s_cs[NT * V];                    // column sums across row threads; later pooled columns, dot partials
     __shared__ int s_mine;
@@ -341,7 +340,7 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
         if (!s_mine) return;
         __threadfence();
         // ---- 3. this CTA completed sample b ----
-        select_sample((float*)s_dyn4, scores, csplit, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
+        select_sample<NT>((float*)s_dyn4, scores, csplit, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
                       p_patch, offsets, ctl + 8, ctl + 1);
     }
 }
@@ -438,11 +437,11 @@ route_patch_scores_kernel(const T* __restrict__ W_r, const float* __restrict__ p
     __syncthreads();
     if (!s_mine) return;
     __threadfence();
-    select_sample(s_sel, scores, 1, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch,
+    select_sample<kScoreThreads>(s_sel, scores, 1, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch,
                   offsets, ctl + 8, ctl + 1);
 }
 
-struct RouteWs { size_t tickets, ptickets, scores, pool, total; int nchunks, CT, rsplit, rows_per_cta, wblk_bytes, csplit; size_t smem; bool two_kernels; };
+struct RouteWs { size_t tickets, ptickets, scores, pool, total; int nchunks, CT, rsplit, rows_per_cta, wblk_bytes, csplit; size_t smem; bool two_kernels, small_ctas; };
 
 RouteWs route_ws(const Dims& D) {
     const int V = 16 / D.esize;
@@ -471,7 +470,17 @@ RouteWs route_ws(const Dims& D) {
     r.total = w.off;
     r.nchunks = nchunks;
     r.CT = CT;
-    const size_t sel = (size_t)D.n * D.m * sizeof(float), wb = (r.two_kernels ? 1 : 2) * (size_t)r.wblk_bytes;
+    const size_t sel = (size_t)D.n * D.m * sizeof(float);
+    size_t wb = (r.two_kernels ? 1 : 2) * (size_t)r.wblk_bytes;
+    // Many small patches (a patch is one CTA's work and a few KB): 64-thread CTAs with exactly the shared memory they
+    // need, so that all of them are resident at once and the per-CTA chain (loads, dots, ticket) is paid once.
+    r.small_ctas = !r.two_kernels && nchunks == 1 && rsplit == 1 && D.d <= 64 * V && D.l_p <= 32 &&
+                   (size_t)D.d * D.n * D.esize <= (size_t)r.wblk_bytes && (long long)D.B * D.m >= 1024;
+    if (r.small_ctas) {
+        r.CT = 64;
+        r.rows_per_cta = D.l_p;
+        wb = ((size_t)D.d * D.n * D.esize + 15) / 16 * 16;
+    }
     r.smem = sel > wb ? sel : wb;
     return r;
 }
@@ -494,16 +503,21 @@ uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void
     cudaError_t e;
     if (!W.two_kernels) {
         ProfScope ps(profile ? "route" : nullptr, stream);
-        if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0>, grid, dim3(kScoreThreads), W.smem, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
-        else e = launch_k(route_kernel<float, 0>, grid, dim3(kScoreThreads), W.smem, stream, UOE_ROUTE_ARGS(float));
+        if (W.small_ctas) {
+            if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0, 64>, grid, dim3(64), W.smem, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
+            else e = launch_k(route_kernel<float, 0, 64>, grid, dim3(64), W.smem, stream, UOE_ROUTE_ARGS(float));
+        } else {
+            if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0, kScoreThreads>, grid, dim3(kScoreThreads), W.smem, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
+            else e = launch_k(route_kernel<float, 0, kScoreThreads>, grid, dim3(kScoreThreads), W.smem, stream, UOE_ROUTE_ARGS(float));
+        }
         if (e != cudaSuccess) return UOE_ERR_CUDA;
         UOE_LAUNCHED();
         return UOE_OK;
     }
     {
         ProfScope ps(profile ? "route" : nullptr, stream);
-        if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 1>, grid, dim3(kScoreThreads), 0, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
-        else e = launch_k(route_kernel<float, 1>, grid, dim3(kScoreThreads), 0, stream, UOE_ROUTE_ARGS(float));
+        if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 1, kScoreThreads>, grid, dim3(kScoreThreads), 0, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
+        else e = launch_k(route_kernel<float, 1, kScoreThreads>, grid, dim3(kScoreThreads), 0, stream, UOE_ROUTE_ARGS(float));
     }
     if (e != cudaSuccess) return UOE_ERR_CUDA;
     UOE_LAUNCHED();
