@@ -31,15 +31,17 @@ using namespace tc;
 constexpr int BM = 128, BK = 64;
 constexpr int A_BLOCK_BYTES = BM * BK * 2;     // 16 KB per 128-row block
 
-template <int BN, int MT> struct Cfg {
+template <int BN, int MT, bool BWD = false> struct Cfg {
     static constexpr int A_BYTES = MT * A_BLOCK_BYTES;
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (MT == 2) ? 3 : ((BN == 256) ? 4 : (BN == 192 ? 5 : (BN == 128 ? 6 : 8)));
+    static constexpr int STAGES = (MT == 2) ? 3 : ((BN == 256 || BN == 192) ? 4 : (BN == 128 ? 6 : 8));
     static constexpr int NACC = (MT == 2) ? 1 : 2;                 // accumulator sets in TMEM
     static constexpr int ACC_STRIDE = (BN == 192) ? 256 : BN;      // TMEM columns between the two accumulator sets
     static constexpr int TMEM_COLS = 2 * ACC_STRIDE;               // MT=1: two sets; MT=2: one set of two blocks
-    static constexpr int EPI_WARPS = 4 * MT;
+    // eight epilogue warps: with 256-row tiles one per (row block, TMEM lane quarter); with 128-row tiles two per lane
+    // quarter, each draining half of the columns (the long backward epilogue keeps four: its registers would not fit)
+    static constexpr int EPI_WARPS = (MT == 2 || !BWD) ? 8 : 4;
     static constexpr int THREADS = 64 + 32 * EPI_WARPS;
     static constexpr int STG_BYTES = 32 * 128;                     // one epilogue warp's staging piece
     static constexpr int SMEM = STAGES * STAGE + 1024 /*align slack*/ + 1024 /*barriers, offsets*/ + EPI_WARPS * STG_BYTES;
@@ -54,7 +56,7 @@ struct Ctl {                       // lives behind the stage ring
 };
 
 template <int BN, bool B_KMAJOR, bool BWD, int MT>
-__global__ void __launch_bounds__(Cfg<BN, MT>::THREADS, 1)
+__global__ void __launch_bounds__(Cfg<BN, MT, BWD>::THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
                  __nv_bfloat16* __restrict__ C0, __nv_bfloat16* __restrict__ C1, __nv_bfloat16* __restrict__ C2,
@@ -65,7 +67,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                  const __grid_constant__ CUtensorMap tmC2, const __grid_constant__ CUtensorMap tmPre) {
     pdl_trigger();
-    using Cf = Cfg<BN, MT>;
+    using Cf = Cfg<BN, MT, BWD>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     Ctl* ctl = (Ctl*)(smem + Cf::STAGES * Cf::STAGE);
@@ -79,6 +81,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         fence_barrier_init();
         prefetch_tmap(&tmA);
         prefetch_tmap(&tmB0);
+        prefetch_tmap(&tmX);
+        prefetch_tmap(&tmC0);
+        if (nmat > 1 || BN == 192) { prefetch_tmap(&tmB1); prefetch_tmap(&tmB2); prefetch_tmap(&tmC1); prefetch_tmap(&tmC2); }
+        if (BWD) prefetch_tmap(&tmC1);
     }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
     pdl_wait();                     // everything above touches only this CTA's own resources
@@ -206,9 +212,15 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
         }
     } else {
-        // ---------------- epilogue: warp w drains 128-row block (w-2)/4, TMEM lane quarter w % 4 ----------------
+        // ---------------- epilogue: warp w drains TMEM lane quarter w % 4 of 128-row block (w-2)/4 (256-row tiles) or,
+        // with 128-row tiles and eight warps, of column half (w-2)/4 ----------------
         const int quarter = warp & 3;
-        const int half = (warp - 2) >> 2;
+        const int wsel = (warp - 2) >> 2;
+        const int half = MT == 2 ? wsel : 0;                  // 128-row block this warp drains
+        constexpr int G = BN / 64;                            // 64-column groups of the accumulator
+        constexpr bool SPLIT_COLS = MT == 1 && Cf::EPI_WARPS == 8;
+        const int g_lo = SPLIT_COLS ? wsel * ((G + 1) / 2) : 0;
+        const int g_hi = SPLIT_COLS ? min(G, g_lo + (G + 1) / 2) : G;
         int acc = 0;
         uint32_t acc_phase = 0;
         auto pack8 = [](const float* f) {
@@ -270,7 +282,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     dg_part[row * n_tiles_mat + (col0 / BN)] = rv * dsum;
                 } else {
 #pragma unroll 1
-                    for (int g = 0; g < BN / 64; ++g) {
+                    for (int g = g_lo; g < g_hi; ++g) {
                         uint32_t v[64];
                         tmem_ld32(taddr + g * 64, v);
                         tmem_ld32(taddr + g * 64 + 32, v + 32);
@@ -301,7 +313,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
 template <int BN, bool B_KMAJOR, bool BWD, int MT>
 uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
-    using Cf = Cfg<BN, MT>;
+    using Cf = Cfg<BN, MT, BWD>;
     static bool attr_set = false;
     auto kern = gemm_bf16_kernel<BN, B_KMAJOR, BWD, MT>;
     if (!attr_set) {
