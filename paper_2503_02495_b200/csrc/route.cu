@@ -47,22 +47,37 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
         ps[tid] = s / (float)Lv;
     }
     __syncthreads();
-    for (int j = tid; j < m; j += NT) {     // Eq. 14: softmax over the experts of patch j
+    // Eq. 14: softmax over the experts of every patch.  The exponentials and divisions run one element per thread; the
+    // per-patch maximum and sum (ascending expert order) one patch per thread.
+    __shared__ float colstat[1024];         // per patch: maximum, then sum
+    for (int idx = tid; idx < n * m; idx += NT) {
+        const int j = idx % m;
         const int cnt = max(0, min(l_p, Lv - j * l_p));
+        pp[idx] = cnt > 0 ? pp[idx] / (float)cnt : 0.f;
+    }
+    __syncthreads();
+    for (int j = tid; j < m; j += NT) {
         float mx = -INFINITY;
-        for (int i = 0; i < n; ++i) {
-            const float v = cnt > 0 ? pp[i * m + j] / (float)cnt : 0.f;
-            pp[i * m + j] = v;
-            mx = fmaxf(mx, v);
-        }
+        for (int i = 0; i < n; ++i) mx = fmaxf(mx, pp[i * m + j]);
+        colstat[j] = mx;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < n * m; idx += NT) pp[idx] = expf(pp[idx] - colstat[idx % m]);
+    __syncthreads();
+    for (int j = tid; j < m; j += NT) {
         float sum = 0.f;
-        for (int i = 0; i < n; ++i) { const float e = expf(pp[i * m + j] - mx); pp[i * m + j] = e; sum += e; }
-        for (int i = 0; i < n; ++i) {
-            const float pr = pp[i * m + j] / sum;
-            pp[i * m + j] = pr;
-            p_patch[((size_t)b * n + i) * m + j] = pr;
-        }
-        if (dynamic_c && cnt > 0) {         // Eq. 15: this patch goes to its k best experts (ties: lower index)
+        for (int i = 0; i < n; ++i) sum += pp[i * m + j];
+        colstat[j] = sum;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < n * m; idx += NT) {
+        const float pr = pp[idx] / colstat[idx % m];
+        pp[idx] = pr;
+        p_patch[(size_t)b * n * m + idx] = pr;
+    }
+    __syncthreads();
+    if (dynamic_c) {                        // Eq. 15: every real patch goes to its k best experts (ties: lower index)
+        for (int j = tid; j < n_elig; j += NT) {
             for (int i = 0; i < n; ++i) {
                 const float v = pp[i * m + j];
                 int rank = 0;
