@@ -153,7 +153,13 @@ rvec_kernel(const T* __restrict__ W_r, const float* __restrict__ G, float* __res
 
 // dW_r[dd, i] = sum over (b, j) of pool[bj, dd] * G[bj, i] in two fixed-order stages: grid (d/256, S) partial sums
 // over S chunks of bj, then a sum over the chunks.
-constexpr int kDwrSplit = 64;
+constexpr int kDwrSplit = 64;            // most splits (sizes the partial buffer)
+// splits actually used: enough (column block, split) CTAs for two per SM, no more (every split writes d*n partials)
+inline int dwr_split(int d) {
+    const int col_blocks = (d + kThreads - 1) / kThreads;
+    int s = (2 * 148 + col_blocks - 1) / col_blocks;
+    return s < 4 ? 4 : (s > kDwrSplit ? kDwrSplit : s);
+}
 __global__ void __launch_bounds__(kThreads)
 dwr_partial_kernel(const float* __restrict__ pool, const float* __restrict__ G, float* __restrict__ part, int BM, int d,
                    int n) {
@@ -161,7 +167,7 @@ dwr_partial_kernel(const float* __restrict__ pool, const float* __restrict__ G, 
     pdl_wait();
     __shared__ float sG[64 * 32];
     const int dd = blockIdx.x * kThreads + threadIdx.x;
-    const int per = (BM + kDwrSplit - 1) / kDwrSplit;
+    const int per = (BM + (int)gridDim.y - 1) / (int)gridDim.y;
     const int lo = blockIdx.y * per, hi = min(BM, lo + per);
     float acc[32];
 #pragma unroll
@@ -187,13 +193,13 @@ dwr_partial_kernel(const float* __restrict__ pool, const float* __restrict__ G, 
     }
 }
 __global__ void __launch_bounds__(kThreads)
-dwr_sum_kernel(const float* __restrict__ part, float* __restrict__ dW_r, int total) {
+dwr_sum_kernel(const float* __restrict__ part, float* __restrict__ dW_r, int total, int nsplit) {
     pdl_trigger();
     pdl_wait();
     const int idx = blockIdx.x * kThreads + threadIdx.x;
     if (idx >= total) return;
     float a = 0.f;
-    for (int s = 0; s < kDwrSplit; ++s) a += part[(size_t)s * total + idx];
+    for (int s = 0; s < nsplit; ++s) a += part[(size_t)s * total + idx];
     dW_r[idx] = a;
 }
 
@@ -317,14 +323,14 @@ uoe_status launch_router_backward(const Dims& D, const void* x, const void* W_r,
     UOE_LAUNCHED();
     {
         ProfScope ps("dW_r", stream);
-        dim3 g2((D.d + kThreads - 1) / kThreads, kDwrSplit);
+        dim3 g2((D.d + kThreads - 1) / kThreads, dwr_split(D.d));
         launch_k(dwr_partial_kernel, g2, dim3(kThreads), 0, stream, pool, G, wpart, D.B * D.m, D.d, D.n);
     }
     UOE_LAUNCHED();
     {
         ProfScope ps("dW_r_sum", stream);
         const int total = D.d * D.n;
-        launch_k(dwr_sum_kernel, dim3((total + kThreads - 1) / kThreads), dim3(kThreads), 0, stream, wpart, dW_r, total);
+        launch_k(dwr_sum_kernel, dim3((total + kThreads - 1) / kThreads), dim3(kThreads), 0, stream, wpart, dW_r, total, dwr_split(D.d));
     }
     UOE_LAUNCHED();
     {
@@ -476,14 +482,14 @@ extern "C" uoe_status uoe_route_balance_backward(const uoe_problem* prob, const 
     UOE_LAUNCHED();
     {
         ProfScope ps("dW_r", stream);
-        launch_k(dwr_partial_kernel, dim3((D.d + kThreads - 1) / kThreads, kDwrSplit), dim3(kThreads), 0, stream, (const float*)rs.pool,
+        launch_k(dwr_partial_kernel, dim3((D.d + kThreads - 1) / kThreads, dwr_split(D.d)), dim3(kThreads), 0, stream, (const float*)rs.pool,
                  (const float*)rs.G, rs.wpart, D.B * D.m, D.d, D.n);
     }
     UOE_LAUNCHED();
     {
         ProfScope ps("dW_r_sum", stream);
         const int total = D.d * D.n;
-        launch_k(dwr_sum_kernel, dim3((total + kThreads - 1) / kThreads), dim3(kThreads), 0, stream, (const float*)rs.wpart, dW_r, total);
+        launch_k(dwr_sum_kernel, dim3((total + kThreads - 1) / kThreads), dim3(kThreads), 0, stream, (const float*)rs.wpart, dW_r, total, dwr_split(D.d));
     }
     UOE_LAUNCHED();
     {
