@@ -52,7 +52,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     const int qt = blockIdx.x, head = blockIdx.y, pair = blockIdx.z;
     const int q0 = qt * TQ;
 
-    if (warp == 0) tmem_alloc(&ctl->tmem_base, 256);       // S: columns [0,128), O_t: [128,192)
+    if (warp == 0) tmem_alloc(&ctl->tmem_base, 512);       // S: two buffers, columns [0,128) and [128,256); O_t: [256,320)
     pdl_wait();                                             // from here on: data written by earlier kernels
     const int row_base = pair_row[pair];
     if (tid == 0) {
@@ -105,12 +105,12 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 
     for (int it = 0; it < n_kv; ++it) {
         const int st = it & 1;
-        // ---- S = Q K^T ----
-        if (tid == 0) {
-            if (it == 0) ok = mbar_wait(&ctl->bar_q, 0, abort_flag, status);
-            ok = mbar_wait(&ctl->bar_kv[st], (it >> 1) & 1, abort_flag, status) && ok;
+        // ---- S = Q K^T (issued here for the first tile only; later tiles are issued behind the previous P V) ----
+        if (tid == 0 && it == 0) {
+            ok = mbar_wait(&ctl->bar_q, 0, abort_flag, status);
+            ok = mbar_wait(&ctl->bar_kv[0], 0, abort_flag, status) && ok;
             tc_fence_after();
-            const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + st * TILE_BYTES);
+            const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK);
 #pragma unroll
             for (int ks = 0; ks < DH / 16; ++ks)
                 mma_bf16(tmem_base, smem_desc(qa + ks * 32, 16, 1024), smem_desc(ka + ks * 32, 16, 1024), idesc_s, ks != 0);
@@ -124,7 +124,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         const int kv0 = it * TK;
         float s_row[TK];
 #pragma unroll
-        for (int ch = 0; ch < TK / 32; ++ch) tmem_ld32(t_lane + ch * 32, (uint32_t*)(s_row + ch * 32));
+        for (int ch = 0; ch < TK / 32; ++ch) tmem_ld32(t_lane + (it & 1) * 128 + ch * 32, (uint32_t*)(s_row + ch * 32));
         tmem_ld_wait();
         float m_new = m_run;
 #pragma unroll
@@ -157,15 +157,26 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         tc_fence_before();
         __syncthreads();
 
-        // ---- O_t = P V ----
+        // ---- O_t = P V, and behind it S of the next tile into the other S buffer (it runs under the O update) ----
         if (tid == 0) {
             tc_fence_after();
             const uint32_t pa = smem_u32(sP), va = smem_u32(sV + st * TILE_BYTES);
 #pragma unroll
             for (int ks = 0; ks < TK / 16; ++ks)
-                mma_bf16(tmem_base + 128, smem_desc(pa + (ks >> 2) * TILE_BYTES + (ks & 3) * 32, 16, 1024),
+                mma_bf16(tmem_base + 256, smem_desc(pa + (ks >> 2) * TILE_BYTES + (ks & 3) * 32, 16, 1024),
                          smem_desc(va + ks * 2048, 8192, 1024), idesc_o, ks != 0);
             mma_commit(&ctl->bar_o);
+            if (it + 1 < n_kv) {
+                const int ns = (it + 1) & 1;
+                ok = mbar_wait(&ctl->bar_kv[ns], ((it + 1) >> 1) & 1, abort_flag, status) && ok;
+                tc_fence_after();
+                const uint32_t qa = smem_u32(sQ), ka = smem_u32(sK + ns * TILE_BYTES);
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ++ks)
+                    mma_bf16(tmem_base + ns * 128, smem_desc(qa + ks * 32, 16, 1024), smem_desc(ka + ks * 32, 16, 1024), idesc_s,
+                             ks != 0);
+                mma_commit(&ctl->bar_s);
+            }
         }
         ok = mbar_wait(&ctl->bar_o, it & 1, abort_flag, status);
         if (!__all_sync(0xffffffffu, ok && !*abort_flag)) break;
@@ -177,8 +188,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
         {
             float o_t[DH];
-            tmem_ld32(t_lane + 128, (uint32_t*)o_t);
-            tmem_ld32(t_lane + 160, (uint32_t*)(o_t + 32));
+            tmem_ld32(t_lane + 256, (uint32_t*)o_t);
+            tmem_ld32(t_lane + 288, (uint32_t*)(o_t + 32));
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < DH; ++i) o_acc[i] = o_acc[i] * alpha + o_t[i];
@@ -208,7 +219,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     __syncthreads();
     if (warp == 0) {
         __syncwarp();
-        tmem_dealloc(tmem_base, 256);
+        tmem_dealloc(tmem_base, 512);
     }
 }
 

@@ -192,7 +192,7 @@ template <typename T, int MODE, int NT>
 __global__ void __launch_bounds__(NT, NT == 64 ? 16 : (MODE == 1 ? 6 : 5))
 route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ pool_part,
              float* __restrict__ scores, int B, int L, int Lv, int d, int n, int k, int m, int c, int l_p, int CT,
-             int nchunks, int rsplit, int rows_per_cta, int wblk_bytes, int csplit, int use_gate,
+             int nchunks, int rsplit, int rows_per_cta, int wblk_bytes, int use_gate,
              int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
              float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
              int* __restrict__ ctl /* word 1: ticket, words 8..: expert loads */, int* __restrict__ sample_ticket /* [B] */,
@@ -206,7 +206,6 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
     const int tid = threadIdx.x;
     const int nparts = nchunks * rsplit;
     const int bj = blockIdx.x / nparts;
-    const int cpart = 0;
     const int b = bj / m, j = bj % m;
 
     // step 2 set-up (used by the CTA that completes a patch)
@@ -214,8 +213,7 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
     const int i = tid % n, g = tid / n;
     int cb = (wblk_bytes / (n * (int)sizeof(T))) / V * V;
     cb = min(cb, NT * V);
-    const int cols_per_part = ((d + csplit - 1) / csplit + V - 1) / V * V;
-    const int col_lo = cpart * cols_per_part, col_hi = min(d, col_lo + cols_per_part);
+    const int col_lo = 0, col_hi = d;
     const int nblk = col_hi > col_lo ? (col_hi - col_lo + cb - 1) / cb : 0;
     const float* pp_bj = pool_part + (size_t)bj * rsplit * d;
     auto stage_w = [&](int blk) {
@@ -300,7 +298,7 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
     }
 
     if constexpr (MODE != 1) {
-        // ---- 2. scores[bj, cpart, :] = pooled columns . W_r over this CTA's column range, W_r rows staged block
+        // ---- 2. scores[bj, :] = pooled columns . W_r, W_r rows staged block
         //         by block in shared memory (double-buffered when the range takes more than one block) ----
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
         if (!direct && nblk > 0) stage_w(0);
@@ -342,20 +340,20 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
         if (tid < n) {
             float sum = 0.f;
             for (int q = 0; q < groups; ++q) sum += s_cs[q * n + tid];
-            scores[((size_t)bj * csplit + cpart) * n + tid] = sum;
+            scores[(size_t)bj * n + tid] = sum;
             __threadfence();
         }
         __syncthreads();
         if (tid == 0) {
             __threadfence();
-            s_mine = (atomicAdd(&sample_ticket[b], 1) == m * csplit - 1);
+            s_mine = (atomicAdd(&sample_ticket[b], 1) == m - 1);
             if (s_mine) sample_ticket[b] = 0;
         }
         __syncthreads();
         if (!s_mine) return;
         __threadfence();
         // ---- 3. this CTA completed sample b ----
-        select_sample<NT>((float*)s_dyn4, scores, csplit, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
+        select_sample<NT>((float*)s_dyn4, scores, 1, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
                       p_patch, offsets, ctl + 8, ctl + 1);
     }
 }
@@ -456,7 +454,7 @@ route_patch_scores_kernel(const T* __restrict__ W_r, const float* __restrict__ p
                   offsets, ctl + 8, ctl + 1);
 }
 
-struct RouteWs { size_t tickets, ptickets, scores, pool, total; int nchunks, CT, rsplit, rows_per_cta, wblk_bytes, csplit; size_t smem; bool two_kernels, small_ctas; };
+struct RouteWs { size_t tickets, ptickets, scores, pool, total; int nchunks, CT, rsplit, rows_per_cta, wblk_bytes; size_t smem; bool two_kernels, small_ctas; };
 
 RouteWs route_ws(const Dims& D) {
     const int V = 16 / D.esize;
@@ -477,8 +475,7 @@ RouteWs route_ws(const Dims& D) {
     // CTAs each take a column range whose W_r rows fit one block
     r.two_kernels = nchunks * rsplit > 1 && (size_t)D.B * D.L * D.d * D.esize >= ((size_t)64 << 20);
     r.wblk_bytes = 16384;
-    r.csplit = 1;
-    r.scores = w.take((size_t)D.B * D.m * r.csplit * D.n * sizeof(float));
+    r.scores = w.take((size_t)D.B * D.m * D.n * sizeof(float));
     r.pool = w.take((size_t)D.B * D.m * rsplit * D.d * sizeof(float));
     r.rsplit = rsplit;
     r.rows_per_cta = rows_per_cta;
@@ -513,7 +510,7 @@ uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void
     const int use_gate = ((flags & UOE_FLAG_GATE) ? 1 : 0) | ((flags & UOE_FLAG_DYNAMIC_C) ? 2 : 0);     // selection flags
     dim3 grid((unsigned)(D.B * D.m * W.nchunks * W.rsplit)), grid2((unsigned)(D.B * D.m));
 #define UOE_ROUTE_ARGS(T) (const T*)x, (const T*)W_r, pool, scores, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, \
-        W.nchunks, W.rsplit, W.rows_per_cta, W.wblk_bytes, W.csplit, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, \
+        W.nchunks, W.rsplit, W.rows_per_cta, W.wblk_bytes, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, \
         tickets, ptickets
     cudaError_t e;
     if (!W.two_kernels) {
