@@ -25,18 +25,27 @@ constexpr int TQ = 128, TK = 128, DH = 64;
 constexpr int kAttnThreads = 128;
 constexpr int TILE_BYTES = 128 * DH * 2;          // 16 KB: a [128 x 64] bf16 tile
 constexpr int ATTN_SMEM = TILE_BYTES * (1 + 2 + 2 + 2) + 1024 + 256;
+constexpr int kFuseMaxD = 512;                               // fused output projection: z tile [128 x d] fp32 fills TMEM
+constexpr int ATTN_SMEM_FUSED = ATTN_SMEM + 1024 + kFuseMaxD * DH * 2;      // + the expert's W^o slice [64 x d] behind the control block
 
 struct AttnCtl {
-    uint64_t bar_q, bar_kv[2], bar_s, bar_o;
+    uint64_t bar_q, bar_kv[2], bar_s, bar_o, bar_w, bar_z;
     uint32_t tmem_base;
     int abort_flag;
 };
 
+// FUSE_O (one head per expert, d <= 512): the output projection of Eq. 35 runs in the same CTA.  The expert's W^o
+// slice [64 x d] is fetched by TMA at kernel start; after the last key tile the normalised o tile goes to shared
+// memory (bf16, swizzled, in place of Q), z = o W^o_i [128 x d] is accumulated over the whole of TMEM (S and O_t are
+// no longer needed) and written to Z instead of o to O.
+template <bool FUSE_O>
 __global__ void __launch_bounds__(kAttnThreads)
 attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
             const __grid_constant__ CUtensorMap tmV, __nv_bfloat16* __restrict__ O, float* __restrict__ lse,
             const int* __restrict__ pair_row, const int* __restrict__ patch_idx, int c, int l_p, int Lv, int l_a,
-            int d_g, int heads, int causal, float scale_log2, int* status) {
+            int d_g, int heads, int causal, float scale_log2, int* status,
+            const __grid_constant__ CUtensorMap tmWo, const int* __restrict__ expert_idx, __nv_bfloat16* __restrict__ Z,
+            int d) {
     pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -45,6 +54,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     uint8_t* sV = sK + 2 * TILE_BYTES;             // 2 stages
     uint8_t* sP = sV + 2 * TILE_BYTES;             // [128 x 128] bf16 as two [128 x 64] swizzled halves
     AttnCtl* ctl = (AttnCtl*)(sP + 2 * TILE_BYTES);
+    uint8_t* sW = sP + 2 * TILE_BYTES + 1024;       // FUSE_O: W^o slice as d/64 boxes of [64 x 64], 8 KB each
     volatile int* abort_flag = &ctl->abort_flag;
     __shared__ int s_nvalid;
 
@@ -61,6 +71,8 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         mbar_init(&ctl->bar_kv[1], 1);
         mbar_init(&ctl->bar_s, 1);
         mbar_init(&ctl->bar_o, 1);
+        mbar_init(&ctl->bar_w, 1);
+        mbar_init(&ctl->bar_z, 1);
         ctl->abort_flag = 0;
         fence_barrier_init();
         // real keys of this pair: sum over its slots of the real tokens in the slot's patch
@@ -89,6 +101,11 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             mbar_arrive_expect_tx(&ctl->bar_kv[t], 2 * TILE_BYTES);
             tma_load_2d(sK + t * TILE_BYTES, &tmK, col_h, row_base + t * TK, &ctl->bar_kv[t]);
             tma_load_2d(sV + t * TILE_BYTES, &tmV, col_h, row_base + t * TK, &ctl->bar_kv[t]);
+        }
+        if (FUSE_O) {                        // the expert's W^o slice, needed only after the last key tile
+            const int e = expert_idx[pair];
+            mbar_arrive_expect_tx(&ctl->bar_w, (uint32_t)d * DH * 2);
+            for (int nb = 0; nb < d / 64; ++nb) tma_load_3d(sW + nb * 8192, &tmWo, nb * 64, 0, e, &ctl->bar_w);
         }
     }
 
@@ -197,23 +214,90 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         tc_fence_before();                   // S and O_t are read; the next iteration may overwrite them
     }
 
-    if (qrow < l_a && !*abort_flag) {
-        const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
-        __nv_bfloat16* out = O + (size_t)(row_base + qrow) * d_g + col_h;
+    const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
+    if (lse && qrow < l_a && !*abort_flag) lse[(size_t)(row_base + qrow) * heads + head] = (m_run + log2f(l_run)) * 0.69314718055994531f;
+    if (!FUSE_O) {
+        if (qrow < l_a && !*abort_flag) {
+            __nv_bfloat16* out = O + (size_t)(row_base + qrow) * d_g + col_h;
 #pragma unroll
-        for (int ch = 0; ch < DH / 8; ++ch) {
-            uint4 w;
-            w.x = pack_bf16x2(o_acc[ch * 8 + 0] * inv, o_acc[ch * 8 + 1] * inv);
-            w.y = pack_bf16x2(o_acc[ch * 8 + 2] * inv, o_acc[ch * 8 + 3] * inv);
-            w.z = pack_bf16x2(o_acc[ch * 8 + 4] * inv, o_acc[ch * 8 + 5] * inv);
-            w.w = pack_bf16x2(o_acc[ch * 8 + 6] * inv, o_acc[ch * 8 + 7] * inv);
-            ((uint4*)out)[ch] = w;
+            for (int ch = 0; ch < DH / 8; ++ch) {
+                uint4 w;
+                w.x = pack_bf16x2(o_acc[ch * 8 + 0] * inv, o_acc[ch * 8 + 1] * inv);
+                w.y = pack_bf16x2(o_acc[ch * 8 + 2] * inv, o_acc[ch * 8 + 3] * inv);
+                w.z = pack_bf16x2(o_acc[ch * 8 + 4] * inv, o_acc[ch * 8 + 5] * inv);
+                w.w = pack_bf16x2(o_acc[ch * 8 + 6] * inv, o_acc[ch * 8 + 7] * inv);
+                ((uint4*)out)[ch] = w;
+            }
         }
-        if (lse) lse[(size_t)(row_base + qrow) * heads + head] = (m_run + log2f(l_run)) * 0.69314718055994531f;
+    } else {
+        // ---- z = o W^o_i (Eq. 35): o tile -> shared memory (in place of Q), one MMA group over all of TMEM ----
+        const int trow = warp * 32 + lane;
+        {
+            const int sw = trow & 7;
+#pragma unroll
+            for (int ch = 0; ch < DH / 8; ++ch) {
+                uint4 w;
+                w.x = pack_bf16x2(o_acc[ch * 8 + 0] * inv, o_acc[ch * 8 + 1] * inv);
+                w.y = pack_bf16x2(o_acc[ch * 8 + 2] * inv, o_acc[ch * 8 + 3] * inv);
+                w.z = pack_bf16x2(o_acc[ch * 8 + 4] * inv, o_acc[ch * 8 + 5] * inv);
+                w.w = pack_bf16x2(o_acc[ch * 8 + 6] * inv, o_acc[ch * 8 + 7] * inv);
+                *(uint4*)(sQ + trow * 128 + ((ch ^ sw) << 4)) = w;
+            }
+        }
+        fence_async_smem();
+        tc_fence_before();
+        __syncthreads();
+        if (tid == 0 && !*abort_flag) {
+            ok = mbar_wait(&ctl->bar_w, 0, abort_flag, status);
+            tc_fence_after();
+            const uint32_t oa = smem_u32(sQ), wa = smem_u32(sW);
+            for (int n0 = 0; n0 < d; n0 += 256) {            // up to 256 output columns per MMA
+                const int nn = min(256, d - n0);
+                const uint32_t idesc_z = instr_desc_bf16(TQ, nn, false, true);
+#pragma unroll
+                for (int ks = 0; ks < DH / 16; ++ks)
+                    mma_bf16(tmem_base + n0, smem_desc(oa + ks * 32, 16, 1024), smem_desc(wa + (n0 / 64) * 8192 + ks * 2048, 8192, 1024),
+                             idesc_z, ks != 0);
+            }
+            mma_commit(&ctl->bar_z);
+        }
+        ok = mbar_wait(&ctl->bar_z, 0, abort_flag, status);
+        if (__all_sync(0xffffffffu, ok && !*abort_flag)) {
+            tc_fence_after();
+            // each warp stages its [32 rows x 64 columns] piece in shared memory (in place of P) and writes it out with
+            // eight lanes per row, so that every store instruction covers whole 128-byte row segments
+            uint8_t* stg = sP + warp * 4096;
+            const int wrow0 = q0 + warp * 32;                     // first query row of this warp's piece
+#pragma unroll 1
+            for (int g = 0; g < d / 64; ++g) {
+                float zf[64];
+                tmem_ld32(t_lane + g * 64, (uint32_t*)zf);
+                tmem_ld32(t_lane + g * 64 + 32, (uint32_t*)(zf + 32));
+                tmem_ld_wait();
+                __syncwarp();                                     // the previous piece has been read back
+#pragma unroll
+                for (int ch = 0; ch < 8; ++ch) {
+                    uint4 w;
+                    w.x = pack_bf16x2(zf[ch * 8 + 0], zf[ch * 8 + 1]); w.y = pack_bf16x2(zf[ch * 8 + 2], zf[ch * 8 + 3]);
+                    w.z = pack_bf16x2(zf[ch * 8 + 4], zf[ch * 8 + 5]); w.w = pack_bf16x2(zf[ch * 8 + 6], zf[ch * 8 + 7]);
+                    *(uint4*)(stg + lane * 128 + ((ch ^ (lane & 7)) << 4)) = w;
+                }
+                __syncwarp();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int r = i * 4 + (lane >> 3), ch = lane & 7;
+                    if (wrow0 + r < l_a) {
+                        const uint4 w = *(const uint4*)(stg + r * 128 + ((ch ^ (r & 7)) << 4));
+                        *(uint4*)(Z + (size_t)(row_base + wrow0 + r) * d + g * 64 + ch * 8) = w;
+                    }
+                }
+            }
+        }
     }
     if (tid == 0 && *abort_flag) {           // let copies that may still be in flight land (bounded)
         mbar_wait(&ctl->bar_q, 0, abort_flag, status);
         for (int t = 0; t < 2 && t < n_kv; ++t) mbar_try_wait(&ctl->bar_kv[t], 0);
+        if (FUSE_O) mbar_wait(&ctl->bar_w, 0, abort_flag, status);
     }
     tc_fence_before();
     __syncthreads();
@@ -272,16 +356,23 @@ uoe_status launch_rope(const Dims& D, void* a, void* b, int ld, const int* pair_
     return UOE_OK;
 }
 
-// q, k, v, o: [rows_max, d_g] bf16 routed buffers.
+// q, k, v, o: [rows_max, d_g] bf16 routed buffers.  If Wo is not null (one head per expert, d <= 512, d % 64 == 0)
+// the output projection is fused: o is not written and z [rows_max, d] receives o W^o_i of every routed row.
+bool attention_can_fuse_out(const Dims& D) { return D.d_g == DH && D.d <= kFuseMaxD && D.d % 64 == 0; }
+
 uoe_status launch_attention(const Dims& D, const void* q, const void* k, const void* v, void* o, float* lse,
-                            const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s) {
+                            const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s,
+                            const void* Wo, const int* expert_idx, void* z) {
     if (D.d_h != DH) return UOE_ERR_UNSUPPORTED;
+    const bool fuse = Wo != nullptr;
+    if (fuse && (!attention_can_fuse_out(D) || !expert_idx || !z)) return UOE_ERR_INVALID_ARG;
     static bool attr_set = false;
     if (!attr_set) {
-        UOE_CUDA_OK(cudaFuncSetAttribute(attn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM));
+        UOE_CUDA_OK(cudaFuncSetAttribute(attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM));
+        UOE_CUDA_OK(cudaFuncSetAttribute(attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM_FUSED));
         attr_set = true;
     }
-    CUtensorMap tm[3];
+    CUtensorMap tm[3], tmWo;
     const void* ptrs[3] = {q, k, v};
     for (int i = 0; i < 3; ++i) {
         const uint64_t dims[2] = {(uint64_t)D.d_g, (uint64_t)D.Rmax};
@@ -289,13 +380,25 @@ uoe_status launch_attention(const Dims& D, const void* q, const void* k, const v
         const uint32_t box[2] = {DH, 128};
         if (!make_tmap(&tm[i], ptrs[i], 2, dims, str, box)) return UOE_ERR_CUDA;
     }
+    tmWo = tm[0];
+    if (fuse) {       // W^o [n, d_g, d]: boxes of 64 output columns x 64 contraction rows of one expert
+        const uint64_t dims[3] = {(uint64_t)D.d, (uint64_t)D.d_g, (uint64_t)D.n};
+        const uint64_t str[2] = {(uint64_t)D.d * 2, (uint64_t)D.d * D.d_g * 2};
+        const uint32_t box[3] = {64, DH, 1};
+        if (!make_tmap(&tmWo, Wo, 3, dims, str, box)) return UOE_ERR_CUDA;
+    }
     const int heads = D.d_g / DH;
     dim3 grid((D.l_a + TQ - 1) / TQ, heads, D.B * D.k);
     const float scale_log2 = 1.4426950408889634f / sqrtf((float)D.d_h);
     ProfScope ps("attention", s);
-    launch_k(attn_kernel, grid, dim3(kAttnThreads), ATTN_SMEM, s, tm[0], tm[1], tm[2], (__nv_bfloat16*)o, lse, pair_row, patch_idx,
-                                                      D.c, D.l_p, D.Lv, D.l_a, D.d_g, heads, causal ? 1 : 0,
-                                                      scale_log2, status);
+    if (fuse)
+        launch_k(attn_kernel<true>, grid, dim3(kAttnThreads), ATTN_SMEM_FUSED, s, tm[0], tm[1], tm[2], (__nv_bfloat16*)o, lse, pair_row,
+                 patch_idx, D.c, D.l_p, D.Lv, D.l_a, D.d_g, heads, causal ? 1 : 0, scale_log2, status, tmWo, expert_idx,
+                 (__nv_bfloat16*)z, D.d);
+    else
+        launch_k(attn_kernel<false>, grid, dim3(kAttnThreads), ATTN_SMEM, s, tm[0], tm[1], tm[2], (__nv_bfloat16*)o, lse, pair_row,
+                 patch_idx, D.c, D.l_p, D.Lv, D.l_a, D.d_g, heads, causal ? 1 : 0, scale_log2, status, tmWo, (const int*)nullptr,
+                 (__nv_bfloat16*)nullptr, D.d);
     UOE_LAUNCHED();
     return UOE_OK;
 }

@@ -6,7 +6,9 @@
 namespace uoe {
 
 uoe_status launch_attention(const Dims& D, const void* q, const void* k, const void* v, void* o, float* lse,
-                            const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s);
+                            const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s,
+                            const void* Wo = nullptr, const int* expert_idx = nullptr, void* z = nullptr);
+bool attention_can_fuse_out(const Dims& D);
 
 uoe_status launch_rope(const Dims& D, void* a, void* b, int ld, const int* pair_row, const int* patch_idx, bool inverse,
                        cudaStream_t s);
@@ -74,13 +76,18 @@ extern "C" uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, c
     if (st != UOE_OK) return st;
     st = launch_rope(D, q, k, D.d_g, P.pair_row, patch_idx, false, stream);      // Eq. 32 (nothing if d_rope = 0)
     if (st != UOE_OK) return st;
-    st = launch_attention(D, q, k, v, o, lse, P.pair_row, patch_idx, (prob->flags & UOE_FLAG_CAUSAL) != 0, status,
-                          stream);
-    if (st != UOE_OK) return st;
-    GemmArgs go{o, Wo, nullptr, z, nullptr, expert_offsets, D.n, D.d_g, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
-    go.label = "out_proj";
-    st = launch_gemm_bf16(go, status, stream);
-    if (st != UOE_OK) return st;
+    const bool causal = (prob->flags & UOE_FLAG_CAUSAL) != 0;
+    if (attention_can_fuse_out(D)) {          // Eq. 33-35 in one kernel: attention and the expert's output projection
+        st = launch_attention(D, q, k, v, o, lse, P.pair_row, patch_idx, causal, status, stream, Wo, expert_idx, z);
+        if (st != UOE_OK) return st;
+    } else {
+        st = launch_attention(D, q, k, v, o, lse, P.pair_row, patch_idx, causal, status, stream);
+        if (st != UOE_OK) return st;
+        GemmArgs go{o, Wo, nullptr, z, nullptr, expert_offsets, D.n, D.d_g, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
+        go.label = "out_proj";
+        st = launch_gemm_bf16(go, status, stream);
+        if (st != UOE_OK) return st;
+    }
     return launch_combine(D, x, z, P, (prob->flags & UOE_FLAG_RESIDUAL) != 0, (prob->flags & UOE_FLAG_GATE) != 0, y,
                           stream);
 }

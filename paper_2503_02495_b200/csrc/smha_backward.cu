@@ -15,7 +15,9 @@
 namespace uoe {
 
 uoe_status launch_attention(const Dims& D, const void* q, const void* k, const void* v, void* o, float* lse,
-                            const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s);
+                            const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s,
+                            const void* Wo = nullptr, const int* expert_idx = nullptr, void* z = nullptr);
+bool attention_can_fuse_out(const Dims& D);
 uoe_status launch_attention_backward(const Dims& D, const void* q, const void* k, const void* v, const void* dout,
                                      const float* lse, const float* delta, void* dq, void* dk, void* dv, int ld_out,
                                      const int* pair_row, const int* patch_idx, bool causal, int* status,
