@@ -8,7 +8,8 @@
 //   softmax        one query row per thread (TMEM lane = row): running max / sum in registers,
 //                  P rounded to bf16 and written to shared memory in the 128B-swizzled K-major layout
 //   O_t = P V      tcgen05.mma 128x64x128, V as the MN-major operand, fresh TMEM accumulator,
-//                  then O = alpha * O + O_t in registers
+//                  then O = alpha * O + O_t in registers; S of the next key tile is issued right behind
+//                  P V into a second TMEM buffer, so it runs under this update
 // Masks: the real keys of a pair are a prefix of its gathered order (patches ascending, pad tokens at
 // the end of the sample), so key c is kept iff c < n_valid, and with the causal flag iff also
 // c <= query row (the shared lower triangle of Fig. 4).

@@ -1,11 +1,13 @@
-// uoe_route: router scoring (Eq. 13-14, 21) and fused top-k expert / top-c patch selection
-// (Eq. 17, 22-23) in ONE kernel:
-//   every CTA streams one (patch, column chunk, row slice) of x (16-byte loads) and leaves the partial dot
-//   products  sum_{t} x[t, chunk] . W_r[chunk, i];  it then takes a ticket of its sample, and the CTA that
-//   completes a sample runs that sample's selection: fixed-order sum of the partials, both softmaxes,
-//   rank-based selection with warp ballots, gates.  The CTA that completes the last sample turns the
-//   per-expert loads into row offsets.  Tickets and loads are reset by their last user, so a workspace
-//   whose control block was zeroed once (uoe_workspace_init) serves any number of calls.
+// uoe_route: router scoring (Eq. 13-14, 21) and fused top-k expert / top-c patch selection (Eq. 17, 22-23).
+//   Every CTA streams one (patch, column chunk, row slice) of x with 16-byte loads and sums its rows per column.
+//   The CTA that completes a patch (a ticket per patch; none when the patch is one CTA's work) multiplies the
+//   pooled columns by W_r; the CTA that completes a sample (a ticket per sample) runs that sample's selection:
+//   both softmaxes, rank-based selection with warp ballots, gates; the CTA that completes the last sample turns
+//   the per-expert loads into row offsets.  One kernel for small inputs (64-thread CTAs when the patches are
+//   many and tiny); for large inputs a first kernel that only streams and a second with one CTA per patch.
+//   Tickets and loads are reset by their last user, so a scratch area whose control block was zeroed once
+//   (uoe_workspace_init, or the static array of uoe_route_static) serves any number of calls of any shapes.
+// Also here: uoe_route_balance (Eq. 15-16, 42-44) and uoe_route_static.
 #include "kernels.cuh"
 
 namespace uoe {

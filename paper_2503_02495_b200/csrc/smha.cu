@@ -1,6 +1,7 @@
-// uoe_smha_forward: SMHA forward (Eq. 27-30, 33-36) as plan -> gather (Eq. 27) -> grouped q/k/v
-// projections in one launch (Eq. 28-30) -> attention over each pair's gathered tokens (Eq. 33-34)
-// -> grouped output projection (Eq. 35) -> weighted combine (Eq. 36).
+// uoe_smha_forward: SMHA forward (Eq. 27-30, 32-36) as plan -> grouped q/k/v projections in one launch,
+// gathering x inside the TMA loads (Eq. 27-30) -> optional RoPE (Eq. 32) -> attention over each pair's
+// gathered tokens with the expert's output projection in the same kernel (Eq. 33-35; a separate grouped GEMM
+// when an expert has several heads or d > 512) -> weighted combine (Eq. 36).
 #include "kernels.cuh"
 
 namespace uoe {
