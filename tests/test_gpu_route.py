@@ -16,6 +16,9 @@ CASES = {
     "tiny_full": gen.tiny(k=4, c=6),
     "tiny_bf16": gen.tiny(dtype="bf16", d=64, B=7),
     "wide_m": gen.tiny(B=3, m=48, c=20, L=96, L_valid=91, d=40, n=5, k=3, d_ff=40),
+    # more than a thousand tiny patches: the 64-thread-CTA variant of the router (float32 and bfloat16)
+    "many_small_f32": gen.tiny(B=200, L=24, L_valid=22, m=6, c=3, d=48, n=4, k=2, d_ff=48),
+    "many_small_bf16": gen.tiny(B=180, L=96, L_valid=96, m=6, c=2, d=128, n=5, k=3, d_ff=40, dtype="bf16"),
     "cfg1": gen.WORKLOADS["cfg1_small_f32"],
     "cfg2": gen.WORKLOADS["cfg2_lm"],
     "cfg3": gen.WORKLOADS["cfg3_long"],
@@ -31,7 +34,7 @@ def test_route_matches_oracle(name, use_gate):
     if name.startswith("cfg") and not use_gate:
         pytest.skip("gate-off variant covered by the small cases")
     x, Wr = gen.make_x(w), gen.make_router(w)
-    scale = 40.0 if name.startswith("tiny") or name == "wide_m" else 1.0
+    scale = 40.0 if name.startswith("tiny") or name.startswith("many") or name == "wide_m" else 1.0
     Wr = gen.store(Wr.f64 * scale, w.dtype)
     prob = problem_of(w, "mlp", gate=use_gate)
     r = uoe.uoe_route(prob, to_dev(x), to_dev(Wr))
