@@ -419,8 +419,7 @@ NCU_TRAFFIC = {
     ("cfg2_lm", "qkv_proj"): 9.73e6,
     ("cfg2_lm", "gemm1_act"): 10.23e6,
     ("cfg2_lm", "gemm2"): 10.55e6,
-    ("cfg2_lm", "attention"): 6.35e6,
-    ("cfg2_lm", "out_proj"): 2.69e6,
+    ("cfg2_lm", "attention"): 6.89e6,
     ("cfg5_scale", "gemm2"): 4 * (92.3e6 + 86.2e6),
     ("cfg5_scale", "bwd_dx"): 4 * (92.3e6 + 86.5e6),
     ("cfg5_scale", "route"): 268.4e6 + 16.8e6,
