@@ -104,3 +104,27 @@ def test_smha_backward_unsupported_shapes():
     with pytest.raises(uoe.UoeError) as ei:
         uoe.uoe_smha_backward(prob, x, Wq, Wk, Wv, Wo, Wr, r, x)
     assert ei.value.status == 2
+
+
+def test_smha_forward_and_backward_on_dynamic_capacity_routing():
+    """Two-stage routing (Eq. 15-16) leaves unused slots (-1) at the end of a pair's patch list: zero rows in the routed
+    buffers, no keys, no gradient.  Forward and backward must match the oracle on the same routing."""
+    import paper_2503_02495_b200 as uoe
+    w = _w(B=4, L=512, L_valid=490, m=8, c=8, n=4, k=2, H=4, causal=True)
+    x, Wr = gen.make_x(w), gen.store(gen.make_router(w, "att").f64 * 30, w.dtype)
+    Wq, Wk, Wv, Wo = gen.make_attn_weights(w)
+    dy = gen.make_dy(w)
+    prob = problem_of(w, "att", residual=False, dynamic_c=True)
+    xd, Wrd = to_dev(x), to_dev(Wr)
+    r = uoe.uoe_route(prob, xd, Wrd)
+    p_idx = r.patch_idx.cpu().numpy()
+    assert (p_idx < 0).any() and (p_idx >= 0).any()          # the case really has unused slots
+    wd = [to_dev(t) for t in (Wq, Wk, Wv, Wo)]
+    y = uoe.uoe_smha_forward(prob, xd, *wd, r)
+    got = uoe.uoe_smha_backward(prob, xd, *wd, Wrd, r, to_dev(dy))
+    ro = orc.with_selection(x.f64, Wr.f64, r.expert_idx.cpu().numpy(), p_idx, w.m, w.L_valid)
+    ref_y = orc.smha_forward(x.f64, Wq.f64, Wk.f64, Wv.f64, Wo.f64, ro, w.d_h, True, residual=False)
+    assert rel_inf(to_f64(y), ref_y) <= TOL
+    ref = orc.smha_backward(x.f64, Wq.f64, Wk.f64, Wv.f64, Wo.f64, Wr.f64, ro, dy.f64, w.d_h, True, False, True)
+    for nm, g, rr in zip(NAMES, got, ref[:6]):
+        assert rel_inf(to_f64(g), rr) <= TOL, nm
