@@ -5,11 +5,13 @@
 // One CTA per (128-query tile, head, pair).  q, k, v are rows of the routed buffers [rows, d_g] (bf16),
 // so the pair's tokens are contiguous.  Per 128-key tile:
 //   S = Q K^T      tcgen05.mma 128x128x64, both operands K-major from TMA, accumulator in TMEM
-//   softmax        one query row per thread (TMEM lane = row): running max / sum in registers,
-//                  P rounded to bf16 and written to shared memory in the 128B-swizzled K-major layout
+//   softmax        two threads per query row (TMEM lane = row; warps 0-3 take keys 0-63 of the tile, warps 4-7
+//                  keys 64-127): tile maxima exchanged through shared memory, running max in both threads,
+//                  each keeps the sum of its own half; P rounded to bf16 and written to shared memory in the
+//                  128B-swizzled K-major layout (each thread's half is one [128 x 64] operand tile)
 //   O_t = P V      tcgen05.mma 128x64x128, V as the MN-major operand, fresh TMEM accumulator,
-//                  then O = alpha * O + O_t in registers; S of the next key tile is issued right behind
-//                  P V into a second TMEM buffer, so it runs under this update
+//                  then O = alpha * O + O_t in registers, 32 of the 64 channels per thread; S of the next key
+//                  tile is issued right behind P V into a second TMEM buffer, so it runs under this update
 // Masks: the real keys of a pair are a prefix of its gathered order (patches ascending, pad tokens at
 // the end of the sample), so key c is kept iff c < n_valid, and with the causal flag iff also
 // c <= query row (the shared lower triangle of Fig. 4).
@@ -23,7 +25,7 @@ namespace {
 using namespace tc;
 
 constexpr int TQ = 128, TK = 128, DH = 64;
-constexpr int kAttnThreads = 128;
+constexpr int kAttnThreads = 256;
 constexpr int TILE_BYTES = 128 * DH * 2;          // 16 KB: a [128 x 64] bf16 tile
 constexpr int ATTN_SMEM = TILE_BYTES * (1 + 2 + 2 + 2) + 1024 + 256;
 constexpr int kFuseMaxD = 512;                               // fused output projection: z tile [128 x d] fp32 fills TMEM
@@ -58,6 +60,7 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
     uint8_t* sW = sP + 2 * TILE_BYTES + 1024;       // FUSE_O: W^o slice as d/64 boxes of [64 x 64], 8 KB each
     volatile int* abort_flag = &ctl->abort_flag;
     __shared__ int s_nvalid;
+    __shared__ float s_xch[2][TQ];               // per row: the two half-tile maxima, later the two half sums
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int qt = blockIdx.x, head = blockIdx.y, pair = blockIdx.z;
@@ -112,13 +115,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
 
     constexpr uint32_t idesc_s = instr_desc_bf16(TQ, TK, false, false);
     constexpr uint32_t idesc_o = instr_desc_bf16(TQ, DH, false, true);
-    const int qrow = q0 + warp * 32 + lane;                // query index inside the pair (TMEM lane)
-    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const int quarter = warp & 3, hsel = warp >> 2;        // TMEM lane quarter of this warp; which half of the keys / channels
+    const int trow = quarter * 32 + lane;                  // row of the tile (TMEM lane)
+    const int qrow = q0 + trow;                            // query index inside the pair
+    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    constexpr int HK = TK / 2, HD = DH / 2;
 
-    float o_acc[DH];
+    float o_acc[HD];
 #pragma unroll
-    for (int i = 0; i < DH; ++i) o_acc[i] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f;
+    for (int i = 0; i < HD; ++i) o_acc[i] = 0.f;
+    float m_run = -INFINITY, l_run = 0.f;                  // l_run: sum over this thread's half of the keys
     bool ok = true;
 
     for (int it = 0; it < n_kv; ++it) {
@@ -139,35 +145,38 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         tc_fence_after();
 
         // ---- online softmax for this row ----
-        const int kv0 = it * TK;
-        float s_row[TK];
+        const int kv0 = it * TK + hsel * HK;
+        float s_row[HK];
 #pragma unroll
-        for (int ch = 0; ch < TK / 32; ++ch) tmem_ld32(t_lane + (it & 1) * 128 + ch * 32, (uint32_t*)(s_row + ch * 32));
+        for (int ch = 0; ch < HK / 32; ++ch)
+            tmem_ld32(t_lane + (it & 1) * 128 + hsel * HK + ch * 32, (uint32_t*)(s_row + ch * 32));
         tmem_ld_wait();
         float m_new = m_run;
 #pragma unroll
-        for (int j = 0; j < TK; ++j) {
+        for (int j = 0; j < HK; ++j) {
             const int col = kv0 + j;
             const bool keep = col < n_valid && col < l_a && (!causal || col <= qrow);
             s_row[j] = keep ? s_row[j] * scale_log2 : -INFINITY;
             m_new = fmaxf(m_new, s_row[j]);
         }
+        s_xch[hsel][trow] = m_new;            // read by the row's other thread; rewritten only after the next barrier
+        __syncthreads();
+        m_new = fmaxf(m_new, s_xch[hsel ^ 1][trow]);
         // a row with no kept key so far keeps m = -inf; exp2(-inf - (-inf)) is avoided by the guard
         const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
         const float alpha = exp2f(m_run - m_use);
         float l_add = 0.f;
-        uint8_t* prow = sP + (size_t)(warp * 32 + lane) * 128;
-        const int sw = (warp * 32 + lane) & 7;
+        uint8_t* prow = sP + hsel * TILE_BYTES + (size_t)trow * 128;
+        const int sw = trow & 7;
 #pragma unroll
-        for (int ch = 0; ch < TK / 8; ++ch) {                 // 16-byte chunks of 8 bf16
+        for (int ch = 0; ch < HK / 8; ++ch) {                 // 16-byte chunks of 8 bf16
             float p[8];
 #pragma unroll
             for (int q = 0; q < 8; ++q) { p[q] = exp2f(s_row[ch * 8 + q] - m_use); l_add += p[q]; }
             uint4 w;
             w.x = pack_bf16x2(p[0], p[1]); w.y = pack_bf16x2(p[2], p[3]);
             w.z = pack_bf16x2(p[4], p[5]); w.w = pack_bf16x2(p[6], p[7]);
-            const int half = ch >> 3, cc = ch & 7;
-            *(uint4*)(prow + half * TILE_BYTES + ((cc ^ sw) << 4)) = w;
+            *(uint4*)(prow + ((ch ^ sw) << 4)) = w;
         }
         l_run = l_run * alpha + l_add;
         m_run = m_new;
@@ -205,23 +214,25 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
             tma_load_2d(sV + st * TILE_BYTES, &tmV, col_h, row_base + (it + 2) * TK, &ctl->bar_kv[st]);
         }
         {
-            float o_t[DH];
-            tmem_ld32(t_lane + 256, (uint32_t*)o_t);
-            tmem_ld32(t_lane + 288, (uint32_t*)(o_t + 32));
+            float o_t[HD];
+            tmem_ld32(t_lane + 256 + hsel * HD, (uint32_t*)o_t);
             tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < DH; ++i) o_acc[i] = o_acc[i] * alpha + o_t[i];
+            for (int i = 0; i < HD; ++i) o_acc[i] = o_acc[i] * alpha + o_t[i];
         }
         tc_fence_before();                   // S and O_t are read; the next iteration may overwrite them
     }
 
+    s_xch[hsel][trow] = l_run;                // the last read of the maxima lies before the last P barrier
+    __syncthreads();
+    l_run += s_xch[hsel ^ 1][trow];
     const float inv = l_run > 0.f ? 1.0f / l_run : 0.f;
-    if (lse && qrow < l_a && !*abort_flag) lse[(size_t)(row_base + qrow) * heads + head] = (m_run + log2f(l_run)) * 0.69314718055994531f;
+    if (lse && hsel == 0 && qrow < l_a && !*abort_flag) lse[(size_t)(row_base + qrow) * heads + head] = (m_run + log2f(l_run)) * 0.69314718055994531f;
     if (!FUSE_O) {
         if (qrow < l_a && !*abort_flag) {
-            __nv_bfloat16* out = O + (size_t)(row_base + qrow) * d_g + col_h;
+            __nv_bfloat16* out = O + (size_t)(row_base + qrow) * d_g + col_h + hsel * HD;
 #pragma unroll
-            for (int ch = 0; ch < DH / 8; ++ch) {
+            for (int ch = 0; ch < HD / 8; ++ch) {
                 uint4 w;
                 w.x = pack_bf16x2(o_acc[ch * 8 + 0] * inv, o_acc[ch * 8 + 1] * inv);
                 w.y = pack_bf16x2(o_acc[ch * 8 + 2] * inv, o_acc[ch * 8 + 3] * inv);
@@ -232,17 +243,16 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         }
     } else {
         // ---- z = o W^o_i (Eq. 35): o tile -> shared memory (in place of Q), one MMA group over all of TMEM ----
-        const int trow = warp * 32 + lane;
         {
             const int sw = trow & 7;
 #pragma unroll
-            for (int ch = 0; ch < DH / 8; ++ch) {
+            for (int ch = 0; ch < HD / 8; ++ch) {
                 uint4 w;
                 w.x = pack_bf16x2(o_acc[ch * 8 + 0] * inv, o_acc[ch * 8 + 1] * inv);
                 w.y = pack_bf16x2(o_acc[ch * 8 + 2] * inv, o_acc[ch * 8 + 3] * inv);
                 w.z = pack_bf16x2(o_acc[ch * 8 + 4] * inv, o_acc[ch * 8 + 5] * inv);
                 w.w = pack_bf16x2(o_acc[ch * 8 + 6] * inv, o_acc[ch * 8 + 7] * inv);
-                *(uint4*)(sQ + trow * 128 + ((ch ^ sw) << 4)) = w;
+                *(uint4*)(sQ + trow * 128 + (((hsel * (HD / 8) + ch) ^ sw) << 4)) = w;
             }
         }
         fence_async_smem();
@@ -265,12 +275,13 @@ attn_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUt
         ok = mbar_wait(&ctl->bar_z, 0, abort_flag, status);
         if (__all_sync(0xffffffffu, ok && !*abort_flag)) {
             tc_fence_after();
-            // each warp stages its [32 rows x 64 columns] piece in shared memory (in place of P) and writes it out with
-            // eight lanes per row, so that every store instruction covers whole 128-byte row segments
+            // each warp stages a [32 rows x 64 columns] piece in shared memory (in place of P) and writes it out with
+            // eight lanes per row, so that every store instruction covers whole 128-byte row segments; the two warps
+            // of a lane quarter take alternate 64-column groups
             uint8_t* stg = sP + warp * 4096;
-            const int wrow0 = q0 + warp * 32;                     // first query row of this warp's piece
+            const int wrow0 = q0 + quarter * 32;                  // first query row of this warp's piece
 #pragma unroll 1
-            for (int g = 0; g < d / 64; ++g) {
+            for (int g = hsel; g < d / 64; g += 2) {
                 float zf[64];
                 tmem_ld32(t_lane + g * 64, (uint32_t*)zf);
                 tmem_ld32(t_lane + g * 64 + 32, (uint32_t*)(zf + 32));
