@@ -17,6 +17,11 @@
 //           per flop, which is what bounds the ring at large K (the ring holds ~1 us of MMA work against an
 //           L2/HBM latency of the same order); one accumulator set, drained by eight epilogue warps.
 //           A 256-row unit at the end of an expert region may hold a single 128-row block ("half tile").
+//   PAIR    256-row tiles worked by a cluster of two CTAs (tcgen05 cta_group::2): CTA r of the pair loads row block r
+//           of A and half r of the B tile's columns, the even CTA issues 256 x BN x 16 MMAs that read both CTAs'
+//           shared memory and write 128 rows into each CTA's TMEM.  Operand bytes per flop as with MT = 2, but each
+//           CTA keeps two accumulator sets, so the epilogue runs under the next main loop; one barrier round covers
+//           128 columns of K.  Used for the backward epilogue, which is too long to leave exposed.
 // The A operand is either a routed buffer (2-D tensor map) or gathered on the fly from x, one TMA box per
 // source patch (Eq. 18 inside the GEMM).
 #include "kernels.cuh"
@@ -31,11 +36,15 @@ using namespace tc;
 constexpr int BM = 128, BK = 64;
 constexpr int A_BLOCK_BYTES = BM * BK * 2;     // 16 KB per 128-row block
 
-template <int BN, int MT, bool BWD = false> struct Cfg {
+template <int BN, int MT, bool BWD = false, bool PAIR = false> struct Cfg {
+    static_assert(!PAIR || (MT == 1 && BN == 256), "CTA pairs: 128 rows and half of a 256-column B tile per CTA");
+    static constexpr int UNIT = PAIR ? 2 : MT;                     // 128-row blocks per row tile
     static constexpr int A_BYTES = MT * A_BLOCK_BYTES;
-    static constexpr int B_BYTES = BN * BK * 2;
-    static constexpr int STAGE = A_BYTES + B_BYTES;
-    static constexpr int STAGES = (MT == 2) ? 3 : ((BN == 256 || BN == 192) ? 4 : (BN == 128 ? 6 : 8));
+    static constexpr int B_BYTES = (PAIR ? BN / 2 : BN) * BK * 2;  // per CTA
+    static constexpr int KSUB = PAIR ? 2 : 1;                      // 64-wide K blocks per stage (one barrier round)
+    static constexpr int SUB = A_BYTES + B_BYTES;
+    static constexpr int STAGE = KSUB * SUB;
+    static constexpr int STAGES = PAIR ? 3 : (MT == 2) ? 3 : ((BN == 256 || BN == 192) ? 4 : (BN == 128 ? 6 : 8));
     static constexpr int NACC = (MT == 2) ? 1 : 2;                 // accumulator sets in TMEM
     static constexpr int ACC_STRIDE = (BN == 192) ? 256 : BN;      // TMEM columns between the two accumulator sets
     static constexpr int TMEM_COLS = 2 * ACC_STRIDE;               // MT=1: two sets; MT=2: one set of two blocks
@@ -55,8 +64,8 @@ struct Ctl {                       // lives behind the stage ring
     int tstart[34];                // first row tile of each expert (prefix sum), tstart[n] = number of row tiles
 };
 
-template <int BN, bool B_KMAJOR, bool BWD, int MT>
-__global__ void __launch_bounds__(Cfg<BN, MT, BWD>::THREADS, 1)
+template <int BN, bool B_KMAJOR, bool BWD, int MT, bool PAIR>
+__global__ void __launch_bounds__(Cfg<BN, MT, BWD, PAIR>::THREADS, 1)
 gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB0,
                  const __grid_constant__ CUtensorMap tmB1, const __grid_constant__ CUtensorMap tmB2,
                  __nv_bfloat16* __restrict__ C0, __nv_bfloat16* __restrict__ C1, __nv_bfloat16* __restrict__ C2,
@@ -67,16 +76,20 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                  const __grid_constant__ CUtensorMap tmC2, const __grid_constant__ CUtensorMap tmPre) {
     pdl_trigger();
-    using Cf = Cfg<BN, MT, BWD>;
+    using Cf = Cfg<BN, MT, BWD, PAIR>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     Ctl* ctl = (Ctl*)(smem + Cf::STAGES * Cf::STAGE);
     volatile int* abort_flag = &ctl->abort_flag;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int rank = PAIR ? (int)cluster_ctarank() : 0;            // CTA of the pair; rank 0 issues the MMAs
+    const int worker = PAIR ? blockIdx.x >> 1 : blockIdx.x;        // index of this CTA (pair) among the tile walkers
+    const int workers = PAIR ? gridDim.x >> 1 : gridDim.x;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < Cf::STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 32 * Cf::EPI_WARPS); }
+        // (pairs: the epilogue threads of both CTAs arrive on rank 0's barrier)
+        for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], (PAIR ? 2 : 1) * 32 * Cf::EPI_WARPS); }
         ctl->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmA);
@@ -86,14 +99,17 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (nmat > 1 || BN == 192) { prefetch_tmap(&tmB1); prefetch_tmap(&tmB2); prefetch_tmap(&tmC1); prefetch_tmap(&tmC2); }
         if (BWD) prefetch_tmap(&tmC1);
     }
-    if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
+    if (warp == 1) {
+        if constexpr (PAIR) tmem_alloc_pair(&ctl->tmem_base, Cf::TMEM_COLS);
+        else tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
+    }
     pdl_wait();                     // everything above touches only this CTA's own resources
     if (warp == 2) {                // offsets and the row-tile prefix over experts (n <= 31 here)
         int o = 0;
         if (lane <= n) o = offsets[lane];
         const int o1 = __shfl_down_sync(0xffffffffu, o, 1);
         const int blocks = lane < n ? (o1 - o) / BM : 0;
-        const int tiles = (blocks + MT - 1) / MT;
+        const int tiles = (blocks + Cf::UNIT - 1) / Cf::UNIT;
         int incl = tiles;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -106,6 +122,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_sync_all();     // the other CTA's barriers exist before anything arrives on them
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
 
@@ -116,7 +133,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     constexpr bool SIDE3 = BN == 192;
     const int n_tiles_mat = SIDE3 ? 1 : N / BN;
     const int n_tiles = SIDE3 ? 1 : n_tiles_mat * nmat;
-    const int num_kb = K / BK;
+    const int num_kb = K / (BK * Cf::KSUB);
     const int total_tiles = ctl->tstart[n] * n_tiles;
 
     // row tile -> expert, first row, number of 128-row blocks it holds
@@ -124,8 +141,8 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         e = 0;
         while (e + 1 < n && row_tile >= ctl->tstart[e + 1]) ++e;
         const int i = row_tile - ctl->tstart[e];
-        row0 = ctl->offs[e] + i * (MT * BM);
-        blocks = min(MT, (ctl->offs[e + 1] - row0) / BM);
+        row0 = ctl->offs[e] + i * (Cf::UNIT * BM);
+        blocks = min(Cf::UNIT, (ctl->offs[e + 1] - row0) / BM);
     };
 
     if (warp == 0) {
@@ -134,20 +151,24 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         uint32_t phase = 0;
         uint32_t issued = 0, issued_parity = 0;      // per stage: a load is in flight with this parity
         bool stop = false;
-        constexpr int nbox_b = B_KMAJOR ? 1 : BN / 64;
+        constexpr int BN_CTA = PAIR ? BN / 2 : BN;              // B columns this CTA loads
+        constexpr int nbox_b = B_KMAJOR ? 1 : BN_CTA / 64;
         const CUtensorMap* tmB_lane = lane == 0 ? &tmB0 : (lane == 1 ? &tmB1 : &tmB2);
-        for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+        for (int tile = worker; tile < total_tiles && !stop; tile += workers) {
             int e, row0, blocks;
             locate(tile / n_tiles, e, row0, blocks);
             const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
             const CUtensorMap* tmB = mat == 0 ? &tmB0 : (mat == 1 ? &tmB1 : &tmB2);
-            const int nbox_a = src_patch ? blocks * (BM / l_p) : blocks;      // <= 32
+            // pairs: this CTA loads row block `rank` (none if the tile holds one block: its MMA rows are never stored)
+            const int my_blocks = PAIR ? (rank < blocks ? 1 : 0) : blocks;
+            const int arow0 = row0 + rank * BM;
+            const int nbox_a = src_patch ? my_blocks * (BM / l_p) : my_blocks;  // <= 32
             int my_src = 0;                                                     // source patch of this lane's box
             if (src_patch && lane < nbox_a) {
-                my_src = src_patch[row0 / l_p + lane];
+                my_src = src_patch[arow0 / l_p + lane];
                 if (my_src < 0) my_src = Bm;                                    // out of range: zero-filled box
             }
-            const uint32_t stage_bytes = blocks * A_BLOCK_BYTES + Cf::B_BYTES;
+            const uint32_t stage_bytes = Cf::KSUB * (blocks * A_BLOCK_BYTES + (PAIR ? 2 : 1) * Cf::B_BYTES);   // both CTAs' bytes
             for (int kb = 0; kb < num_kb; ++kb) {
                 int ok = 1;
                 if (lane == 0) ok = (mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) && !*abort_flag) ? 1 : 0;
@@ -155,34 +176,53 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (!ok) { stop = true; break; }
                 uint8_t* sa = smem + stage * Cf::STAGE;
                 uint8_t* sb = sa + Cf::A_BYTES;
-                if (lane == 0) mbar_arrive_expect_tx(&ctl->full[stage], stage_bytes);
+                if (lane == 0 && rank == 0) mbar_arrive_expect_tx(&ctl->full[stage], stage_bytes);
                 __syncwarp();
-                if (lane < nbox_a) {
-                    if (src_patch) tma_load_3d(sa + lane * l_p * 128, &tmX, kb * BK, 0, my_src, &ctl->full[stage]);
-                    else tma_load_2d(sa + lane * A_BLOCK_BYTES, &tmA, kb * BK, row0 + lane * BM, &ctl->full[stage]);
-                }
-                if (lane < nbox_b) {
-                    if (SIDE3) tma_load_3d(sb + lane * 8192, tmB_lane, 0, kb * BK, e, &ctl->full[stage]);
-                    else if (B_KMAJOR) tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
-                    else tma_load_3d(sb + lane * 8192, tmB, col0 + lane * 64, kb * BK, e, &ctl->full[stage]);
+                if constexpr (PAIR) {
+                    const uint32_t full0 = map_to_cta(&ctl->full[stage], 0);    // rank 0's barrier counts both CTAs' bytes
+                    const int bcol0 = col0 + rank * BN_CTA;
+#pragma unroll
+                    for (int j = 0; j < Cf::KSUB; ++j) {
+                        const int k0 = (kb * Cf::KSUB + j) * BK;
+                        uint8_t* sa_j = sa + j * Cf::SUB;
+                        uint8_t* sb_j = sa_j + Cf::A_BYTES;
+                        if (lane < nbox_a) {
+                            if (src_patch) tma_load_3d_pair(sa_j + lane * l_p * 128, &tmX, k0, 0, my_src, full0);
+                            else tma_load_2d_pair(sa_j, &tmA, k0, arow0, full0);
+                        }
+                        if (lane < nbox_b) {
+                            if (B_KMAJOR) tma_load_3d_pair(sb_j, tmB, k0, bcol0, e, full0);
+                            else tma_load_3d_pair(sb_j + lane * 8192, tmB, bcol0 + lane * 64, k0, e, full0);
+                        }
+                    }
+                } else {
+                    if (lane < nbox_a) {
+                        if (src_patch) tma_load_3d(sa + lane * l_p * 128, &tmX, kb * BK, 0, my_src, &ctl->full[stage]);
+                        else tma_load_2d(sa + lane * A_BLOCK_BYTES, &tmA, kb * BK, row0 + lane * BM, &ctl->full[stage]);
+                    }
+                    if (lane < nbox_b) {
+                        if (SIDE3) tma_load_3d(sb + lane * 8192, tmB_lane, 0, kb * BK, e, &ctl->full[stage]);
+                        else if (B_KMAJOR) tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
+                        else tma_load_3d(sb + lane * 8192, tmB, col0 + lane * 64, kb * BK, e, &ctl->full[stage]);
+                    }
                 }
                 issued |= 1u << stage;
                 issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
                 if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
             }
         }
-        if (lane == 0 && *abort_flag) {      // let this CTA's own copies land before it exits
+        if (lane == 0 && rank == 0 && *abort_flag) {      // let the copies counted by this CTA's barriers land before it exits
             for (int s = 0; s < Cf::STAGES; ++s)
                 if (issued & (1u << s)) mbar_wait(&ctl->full[s], (issued_parity >> s) & 1, abort_flag, status);
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        if (lane == 0 && rank == 0) {
             // ---------------- MMA issuer ----------------
-            constexpr uint32_t idesc = instr_desc_bf16(BM, BN, false, !B_KMAJOR);
+            constexpr uint32_t idesc = instr_desc_bf16(PAIR ? 2 * BM : BM, BN, false, !B_KMAJOR);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool stop = false;
-            for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+            for (int tile = worker; tile < total_tiles && !stop; tile += workers) {
                 int e, row0, blocks;
                 locate(tile / n_tiles, e, row0, blocks);
                 if (!mbar_wait(&ctl->tempty[acc], acc_phase ^ 1, abort_flag, status) || *abort_flag) break;
@@ -191,23 +231,30 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 for (int kb = 0; kb < num_kb; ++kb) {
                     if (!mbar_wait(&ctl->full[stage], phase, abort_flag, status) || *abort_flag) { stop = true; break; }
                     tc_fence_after();
-                    const uint32_t sa = smem_u32(smem + stage * Cf::STAGE);
-                    const uint32_t sb = sa + Cf::A_BYTES;
 #pragma unroll
-                    for (int ks = 0; ks < BK / 16; ++ks) {
-                        const uint64_t bd = B_KMAJOR ? smem_desc(sb + ks * 32, 16, 1024)
-                                                     : smem_desc(sb + ks * 2048, 8192, 1024);
+                    for (int ks = 0; ks < Cf::KSUB * (BK / 16); ++ks) {
+                        const uint32_t sa = smem_u32(smem + stage * Cf::STAGE + (ks / (BK / 16)) * Cf::SUB);
+                        const uint32_t sb = sa + Cf::A_BYTES;
+                        const int kq = ks % (BK / 16);
+                        const uint64_t bd = B_KMAJOR ? smem_desc(sb + kq * 32, 16, 1024)
+                                                     : smem_desc(sb + kq * 2048, 8192, 1024);
+                        if constexpr (PAIR) {
+                            mma_bf16_pair(d_tmem, smem_desc(sa + kq * 32, 16, 1024), bd, idesc, (kb | ks) != 0);
+                        } else {
 #pragma unroll
-                        for (int h = 0; h < MT; ++h)
-                            if (h < blocks)
-                                mma_bf16(d_tmem + h * BN, smem_desc(sa + h * A_BLOCK_BYTES + ks * 32, 16, 1024), bd, idesc,
-                                         (kb | ks) != 0);
+                            for (int h = 0; h < MT; ++h)
+                                if (h < blocks)
+                                    mma_bf16(d_tmem + h * BN, smem_desc(sa + h * A_BLOCK_BYTES + kq * 32, 16, 1024), bd, idesc,
+                                             (kb | ks) != 0);
+                        }
                     }
-                    mma_commit(&ctl->empty[stage]);
+                    if constexpr (PAIR) mma_commit_pair(&ctl->empty[stage]);       // frees the stage in both CTAs
+                    else mma_commit(&ctl->empty[stage]);
                     if (++stage == Cf::STAGES) { stage = 0; phase ^= 1; }
                 }
                 if (stop) break;
-                mma_commit(&ctl->tfull[acc]);
+                if constexpr (PAIR) mma_commit_pair(&ctl->tfull[acc]);
+                else mma_commit(&ctl->tfull[acc]);
                 if (++acc == Cf::NACC) { acc = 0; acc_phase ^= 1; }
             }
         }
@@ -216,7 +263,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         // with 128-row tiles and eight warps, of column half (w-2)/4 ----------------
         const int quarter = warp & 3;
         const int wsel = (warp - 2) >> 2;
-        const int half = MT == 2 ? wsel : 0;                  // 128-row block this warp drains
+        const int half = PAIR ? rank : (MT == 2 ? wsel : 0);  // 128-row block this warp drains
         constexpr int G = BN / 64;                            // 64-column groups of the accumulator
         constexpr bool SPLIT_COLS = MT == 1 && Cf::EPI_WARPS == 8;
         const int g_lo = SPLIT_COLS ? wsel * ((G + 1) / 2) : 0;
@@ -240,7 +287,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             __syncwarp();
             if (lane == 0) { tma_store_2d(tm, stg, c0, r0); bulk_commit(); }
         };
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        for (int tile = worker; tile < total_tiles; tile += workers) {
             int e, row0, blocks;
             locate(tile / n_tiles, e, row0, blocks);
             const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
@@ -298,26 +345,36 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 }
             }
             tc_fence_before();
-            mbar_arrive(&ctl->tempty[acc]);
+            if constexpr (PAIR) mbar_arrive_cluster(map_to_cta(&ctl->tempty[acc], 0));
+            else mbar_arrive(&ctl->tempty[acc]);
             if (++acc == Cf::NACC) { acc = 0; acc_phase ^= 1; }
         }
     }
     if (warp >= 2 && lane == 0) bulk_wait_all();       // this warp's tensor stores are complete
     tc_fence_before();
     __syncthreads();
+    // pairs: neither CTA leaves (or gives up its TMEM) while the other may still arrive on its barriers or its MMAs
+    // may still read this CTA's shared memory
+    if constexpr (PAIR) cluster_sync_all();
     if (warp == 1) {
         __syncwarp();
-        tmem_dealloc(tmem_base, Cf::TMEM_COLS);
+        if constexpr (PAIR) tmem_dealloc_pair(tmem_base, Cf::TMEM_COLS);
+        else tmem_dealloc(tmem_base, Cf::TMEM_COLS);
     }
 }
 
-template <int BN, bool B_KMAJOR, bool BWD, int MT>
+template <int BN, bool B_KMAJOR, bool BWD, int MT, bool PAIR = false>
 uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
-    using Cf = Cfg<BN, MT, BWD>;
+    using Cf = Cfg<BN, MT, BWD, PAIR>;
     static bool attr_set = false;
-    auto kern = gemm_bf16_kernel<BN, B_KMAJOR, BWD, MT>;
+    static int max_pairs = 0;          // CTA pairs that can be resident at once
+    auto kern = gemm_bf16_kernel<BN, B_KMAJOR, BWD, MT, PAIR>;
     if (!attr_set) {
         UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
+        if (PAIR) {
+            UOE_CUDA_OK(max_resident_pairs(kern, Cf::THREADS, Cf::SMEM, &max_pairs));
+            if (max_pairs < 1) return UOE_ERR_CUDA;
+        }
         attr_set = true;
     }
     CUtensorMap tmA, tmB[3], tmX;
@@ -340,7 +397,7 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
         if (B_KMAJOR) {       // W [n, N, K]
             const uint64_t dims[3] = {(uint64_t)g.K, (uint64_t)g.N, (uint64_t)g.n};
             const uint64_t str[2] = {(uint64_t)g.K * 2, (uint64_t)g.K * g.N * 2};
-            const uint32_t box[3] = {BK, BN, 1};
+            const uint32_t box[3] = {BK, PAIR ? BN / 2 : BN, 1};
             if (!make_tmap(&tmB[q], Ws[q], 3, dims, str, box)) return UOE_ERR_CUDA;
         } else {              // W [n, K, N]
             const uint64_t dims[3] = {(uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.n};
@@ -360,11 +417,17 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
             if (!make_tmap(&tmC[q], Cs[q], 2, dims, str, box)) return UOE_ERR_CUDA;
         if (!make_tmap(&tmPre, g.pre ? g.pre : g.C, 2, dims, str, box)) return UOE_ERR_CUDA;
     }
-    long long max_tiles = ((g.rows_max / BM + MT - 1) / MT + g.n) * (BN == 192 ? 1 : (g.N / BN) * nmat);
-    int grid = (int)(max_tiles < sm_count() ? max_tiles : sm_count());
+    long long max_tiles = ((g.rows_max / BM + Cf::UNIT - 1) / Cf::UNIT + g.n) * (BN == 192 ? 1 : (g.N / BN) * nmat);
+    const int walkers = PAIR ? max_pairs : sm_count();
+    int grid = (int)(max_tiles < walkers ? max_tiles : walkers);
     if (grid < 1) grid = 1;
+    if (PAIR) grid *= 2;
     ProfScope ps(g.label, s);
-    launch_k(kern, grid, dim3(Cf::THREADS), Cf::SMEM, s, tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
+    auto launch = [&](auto... a) {
+        if constexpr (PAIR) return launch_k_pairs(a...);
+        else return launch_k(a...);
+    };
+    launch(kern, dim3(grid), dim3(Cf::THREADS), (size_t)Cf::SMEM, s, tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
                                              (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
                                              nmat, g.act, status, (const __nv_bfloat16*)g.bwd_h, g.row_gate, g.row_valid,
                                              g.dg_part, tmX, g.gather_x ? g.src_patch : nullptr, g.l_p, g.Bm, tmC[0],
@@ -379,7 +442,11 @@ uoe_status dispatch(const GemmArgs& g, int* status, cudaStream_t s) {
     // 256-row tiles pay off when every SM still gets several of them and the K loop is long enough to be
     // bound by operand delivery rather than by the prologue
     const long long tiles256 = (g.rows_max / 256) * (g.N / 256);
-    // (the backward epilogue is long: it stays on 128-row tiles, where it overlaps the next tile's main loop)
+    // the backward epilogue is long: it stays on 128-row accumulators, whose drain overlaps the next tile's main loop,
+    // and takes its 256-row tiles from CTA pairs when there are enough of them for every pair of SMs
+    if constexpr (BWD) {
+        if (bn == 256 && g.K % 128 == 0 && tiles256 >= 2 * sm_count()) return launch_one<256, B_KMAJOR, BWD, 1, true>(g, status, s);
+    }
     if constexpr (!BWD) {
         if (bn == 256 && g.K >= 1024 && tiles256 >= 2 * sm_count()) return launch_one<256, B_KMAJOR, BWD, 2>(g, status, s);
     }
