@@ -410,18 +410,21 @@ HBM_KERNELS = ("route", "gather", "combine", "pool")
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (step_kernels_cfg2_lm.md, gemm_wgrad_cfg5_scale_B2.md, route_kernels_cfg5_scale.md).  Keyed by (workload, kernel
-# label); an entry is dropped when its kernel changes, and the line then reports null.  The scale entries were
-# captured at B=2 and scaled by 4: their traffic grows in proportion to the routed rows.
+# (step_kernels_cfg2_lm.md, launches_gemm_cfg5_scale_B4.md, route_kernels_cfg5_scale.md).  Keyed by (workload, kernel
+# label); an entry is dropped when its kernel changes, and the line then reports null.  The scale workload's GEMM
+# entries were captured at B=4 and scaled by 2 (the part that is weight reads does not grow with B, so they are upper
+# estimates); its route entry was captured at full size.
 NCU_TRAFFIC = {
     ("cfg2_lm", "route"): 8.47e6,
     ("cfg2_lm", "combine"): 25.18e6,
     ("cfg2_lm", "qkv_proj"): 9.73e6,
     ("cfg2_lm", "gemm1_act"): 10.23e6,
     ("cfg2_lm", "gemm2"): 10.55e6,
-    ("cfg2_lm", "attention"): 6.89e6,
-    ("cfg5_scale", "gemm2"): 4 * (92.3e6 + 86.2e6),
-    ("cfg5_scale", "bwd_dx"): 4 * (92.3e6 + 86.5e6),
+    ("cfg2_lm", "attention"): 6.88e6,
+    ("cfg5_scale", "gemm1_act"): 2 * (351.9e6 + 105.7e6),
+    ("cfg5_scale", "gemm2"): 2 * (176.2e6 + 220.0e6),
+    ("cfg5_scale", "bwd_da_dh"): 2 * (442.7e6 + 113.8e6),
+    ("cfg5_scale", "bwd_dx"): 2 * (176.3e6 + 220.6e6),
     ("cfg5_scale", "route"): 268.4e6 + 16.8e6,
 }
 
