@@ -10,9 +10,9 @@
 //   DQ = false  CTA = (key tile j, head, pair): K_j, V_j stay in shared memory, the query tiles stream through;
 //               dV_j += P^T dO_i and dK_j += dS^T Q_i accumulate in TMEM over i
 //   DQ = true   CTA = (query tile i, head, pair): Q_i, dO_i stay, the key tiles stream; dQ_i += dS K_j
-// Per streamed tile:  S = Q K^T and dP = dO V^T (tcgen05.mma 128x128x64 each, accumulators in TMEM), then one
-// query row per thread (TMEM lane = row) forms P and dS in 32-column pieces, rounds them to bf16 and writes
-// them to shared memory in the 128B-swizzled layout, where they are the A operands of the second MMAs (read
+// Per streamed tile:  S = Q K^T and dP = dO V^T (tcgen05.mma 128x128x64 each, accumulators in TMEM), then two
+// threads per query row (TMEM lane = row; warps 0-3 take keys 0-63 of the tile, warps 4-7 keys 64-127) form P and
+// dS in 32-column pieces, round them to bf16 and write them to shared memory in the 128B-swizzled layout, where they are the A operands of the second MMAs (read
 // K-major for dQ, MN-major, i.e. transposed, for dV / dK).
 // Masks as in the forward kernel: key c is kept iff c < n_valid (real keys are a prefix of the gathered order)
 // and, with the causal flag, c <= query row; query rows >= l_a of a tile belong to the next pair and are dropped.
@@ -26,7 +26,7 @@ namespace {
 using namespace tc;
 
 constexpr int T = 128, DH = 64;
-constexpr int kThreads = 128;
+constexpr int kThreads = 256;
 constexpr int TILE_BYTES = T * DH * 2;            // 16 KB: a [128 x 64] bf16 tile
 constexpr int SQ_BYTES = 2 * TILE_BYTES;          // a [128 x 128] bf16 matrix as two swizzled halves
 
@@ -115,8 +115,9 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     constexpr uint32_t idesc_s = instr_desc_bf16(T, T, false, false);        // S, dP: both operands K-major
     constexpr uint32_t idesc_q = instr_desc_bf16(T, DH, false, true);        // dQ = dS K: A K-major, B MN-major
     constexpr uint32_t idesc_t = instr_desc_bf16(T, DH, true, true);         // dV = P^T dO, dK = dS^T Q: both MN-major
-    const int trow = warp * 32 + lane;                                       // TMEM lane = row inside the tile
-    const uint32_t t_lane = tmem_base + ((uint32_t)(warp * 32) << 16);
+    const int quarter = warp & 3, hsel = warp >> 2;                          // TMEM lane quarter; half of the keys / channels
+    const int trow = quarter * 32 + lane;                                    // TMEM lane = row inside the tile
+    const uint32_t t_lane = tmem_base + ((uint32_t)(quarter * 32) << 16);
     bool ok = true;
 
     float my_lse2 = 0.f, my_delta = 0.f;
@@ -171,7 +172,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
         const int kv0 = k_tile * T;
         const int sw = trow & 7;
 #pragma unroll 1
-        for (int ch = 0; ch < T / 32; ++ch) {
+        for (int ch = 2 * hsel; ch < 2 * hsel + 2; ++ch) {
             float s_v[32], dp_v[32];
             tmem_ld32(t_lane + ch * 32, (uint32_t*)s_v);
             tmem_ld32(t_lane + 128 + ch * 32, (uint32_t*)dp_v);
@@ -237,21 +238,20 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     const int orow = tile * T + trow;
     {
-        float acc[DH];
+        float acc[DH / 2];                                   // this thread's 32 of the row's 64 channels
 #pragma unroll 1
         for (int which = 0; which < (DQ ? 1 : 2); ++which) {
             if (have) {                                      // warp-uniform
-                tmem_ld32(t_lane + 256 + which * 64, (uint32_t*)acc);
-                tmem_ld32(t_lane + 256 + which * 64 + 32, (uint32_t*)(acc + 32));
+                tmem_ld32(t_lane + 256 + which * 64 + hsel * 32, (uint32_t*)acc);
                 tmem_ld_wait();
             } else {
 #pragma unroll
-                for (int i = 0; i < DH; ++i) acc[i] = 0.f;
+                for (int i = 0; i < DH / 2; ++i) acc[i] = 0.f;
             }
             if (orow < l_a) {
-                __nv_bfloat16* out = (which == 0 ? out0 : out1) + (size_t)(row_base + orow) * ld_out + col_h;
+                __nv_bfloat16* out = (which == 0 ? out0 : out1) + (size_t)(row_base + orow) * ld_out + col_h + hsel * 32;
 #pragma unroll
-                for (int ch = 0; ch < DH / 8; ++ch) {
+                for (int ch = 0; ch < DH / 16; ++ch) {
                     uint4 w;
                     w.x = pack_bf16x2(acc[ch * 8 + 0], acc[ch * 8 + 1]); w.y = pack_bf16x2(acc[ch * 8 + 2], acc[ch * 8 + 3]);
                     w.z = pack_bf16x2(acc[ch * 8 + 4], acc[ch * 8 + 5]); w.w = pack_bf16x2(acc[ch * 8 + 6], acc[ch * 8 + 7]);
