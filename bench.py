@@ -59,6 +59,8 @@ def work_table(w: gen.Workload):
         de = w.d_e
         t["gemm1_act"] = dict(flops=2 * R * d * de, bytes=(R * d + R * de + n * d * de) * s)
         t["gemm2"] = dict(flops=2 * R * de * d, bytes=(R * de + R * d + n * d * de) * s)
+        # both GEMMs in one kernel (narrow experts): the hidden tile is neither written nor read back
+        t["mlp_fused"] = dict(flops=4 * R * d * de, bytes=(2 * R * d + 2 * n * d * de) * s)
     if w.d_ff and w.backward:
         de = w.d_e
         for name in ("bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2"):
@@ -404,7 +406,7 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
     return res
 
 
-TENSOR_KERNELS = ("gemm1_act", "gemm2", "qkv_proj", "out_proj", "attention", "bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2",
+TENSOR_KERNELS = ("gemm1_act", "gemm2", "mlp_fused", "qkv_proj", "out_proj", "attention", "bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2",
                   "attn_bwd_dkdv", "attn_bwd_dq", "bwd_do", "bwd_dx_att", "wgrad_Wo", "wgrad_Wqkv")
 HBM_KERNELS = ("route", "gather", "combine", "pool")
 

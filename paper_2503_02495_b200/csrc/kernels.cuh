@@ -147,4 +147,12 @@ uoe_status launch_router_backward(const Dims& D, const void* x, const void* W_r,
                                   const float* dgp, int nt, const RouterBwdScratch& rs, float* dW_r, cudaStream_t stream);
 uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s);
 
+// Eq. 38-39 in one kernel for narrow experts (bf16, d_e = 256, d <= 512): z = phi(A W1[e]) W2[e] with the hidden tile
+// kept on chip.  A [rows, d] is a routed buffer, or gathered from gather_x through src_patch as in GemmArgs;
+// pre (optional) [rows, 256] receives the pre-activation.
+bool mlp_can_fuse(const Dims& D);
+uoe_status launch_mlp_fused(const Dims& D, const void* A, const void* W1, const void* W2, void* z, void* pre,
+                            const int* offsets, int act, const void* gather_x, const int* src_patch, int* status,
+                            cudaStream_t s);
+
 }  // namespace uoe

@@ -1,5 +1,6 @@
 // uoe_mlp_forward: UoME forward (Eq. 37-40) as plan -> gather (Eq. 18) -> grouped GEMM1 + phi (Eq. 38)
-// -> grouped GEMM2 (Eq. 39) -> weighted combine (Eq. 20 / 40).
+// -> grouped GEMM2 (Eq. 39) -> weighted combine (Eq. 20 / 40).  On the bf16 path the gather happens inside the
+// first GEMM's loads, and for narrow experts (d_e = 256, d <= 512) both GEMMs are one kernel.
 #include "kernels.cuh"
 
 namespace uoe {
@@ -61,7 +62,11 @@ extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, co
     GemmArgs g2{a, W2, b2, z, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
     g1.label = "gemm1_act";
     g2.label = "gemm2";
-    if (D.bf16) {
+    if (mlp_can_fuse(D) && !b1 && !b2) {      // narrow experts: both GEMMs in one kernel, the hidden tile stays on chip
+        st = launch_mlp_fused(D, xg, W1, W2, z, saved_h, expert_offsets, prob->act, fused ? x : nullptr, P.src_patch, status,
+                              stream);
+        if (st != UOE_OK) return st;
+    } else if (D.bf16) {
         st = launch_gemm_bf16(g1, status, stream);
         if (st != UOE_OK) return st;
         st = launch_gemm_bf16(g2, status, stream);

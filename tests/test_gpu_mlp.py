@@ -29,6 +29,14 @@ CASES = {
                          act="gelu_erf"),
     # long K and many row tiles: the 256-row tile variant, with regions of 3*load 128-row blocks (half tiles)
     "tall_tiles": gen.tiny(B=40, L=1152, L_valid=1152, m=9, c=3, d=1024, n=4, k=2, d_ff=4096, dtype="bf16", w_std=0.02),
+    # narrow experts (d_e = 256): both GEMMs in one kernel; 64 output columns, a ragged second output half, pad
+    # tokens, and a patch length the GEMM cannot gather by itself (routed copy of x as the A operand)
+    "fused_d64": gen.tiny(B=3, L=96, L_valid=96, m=6, c=3, d=64, n=2, k=1, d_ff=512, dtype="bf16", w_std=0.05),
+    "fused_d192_pad": gen.tiny(B=5, L=112, L_valid=100, m=7, c=4, d=192, n=3, k=2, d_ff=768, dtype="bf16", w_std=0.05,
+                               act="gelu_erf"),
+    "fused_d448": gen.tiny(B=4, L=256, L_valid=250, m=8, c=5, d=448, n=4, k=3, d_ff=1024, dtype="bf16", w_std=0.04,
+                           act="gelu_tanh"),
+    "fused_copy_a": gen.tiny(B=4, L=120, L_valid=115, m=10, c=4, d=128, n=2, k=2, d_ff=512, dtype="bf16", w_std=0.05),
     "cfg2": gen.WORKLOADS["cfg2_lm"],
     "cfg3": gen.WORKLOADS["cfg3_long"],
     "cfg4": gen.WORKLOADS["cfg4_vit"],
