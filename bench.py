@@ -420,8 +420,7 @@ NCU_TRAFFIC = {
     ("cfg2_lm", "route"): 8.47e6,
     ("cfg2_lm", "combine"): 25.18e6,
     ("cfg2_lm", "qkv_proj"): 9.73e6,
-    ("cfg2_lm", "gemm1_act"): 10.23e6,
-    ("cfg2_lm", "gemm2"): 10.55e6,
+    ("cfg2_lm", "mlp_fused"): 12.34e6,
     ("cfg2_lm", "attention"): 6.88e6,
     ("cfg5_scale", "gemm1_act"): 2 * (351.9e6 + 105.7e6),
     ("cfg5_scale", "gemm2"): 2 * (176.2e6 + 220.0e6),
