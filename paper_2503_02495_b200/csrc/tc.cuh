@@ -141,7 +141,7 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 // One MMA of the pair covers 256 rows: CTA r of the cluster holds rows [128 r, 128 r + 128) of A and columns
 // [N/2 r, N/2 r + N/2) of B in its own shared memory, at the same offsets in both CTAs, and receives its 128 rows
 // of D (all N columns) in its own TMEM.  The even CTA (rank 0) issues the MMAs; its mbarriers collect the TMA
-// bytes of both CTAs, and its commits arrive on the barrier at the same offset in both CTAs.
+// bytes of both CTAs, and its commits arrive on the barrier at the same offset in each of the two CTAs.
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -187,10 +187,13 @@ __device__ __forceinline__ void mma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, 
         "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         :: "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"((uint32_t)accumulate) : "memory");
 }
-// one arrival on the barrier at this offset in both CTAs when all MMAs issued so far by this thread have completed
+// one arrival on the barrier at this offset in each CTA of the pair when all MMAs issued so far by this thread have
+// completed (two commits, one per CTA: the second names the other CTA's barrier by its cluster address)
 __device__ __forceinline__ void mma_commit_pair(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 :: "r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 :: "r"(map_to_cta(bar, 0)) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 :: "r"(map_to_cta(bar, 1)) : "memory");
 }
 
 // ---- descriptors ------------------------------------------------------------------------------
