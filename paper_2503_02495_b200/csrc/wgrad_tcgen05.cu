@@ -8,6 +8,9 @@
 // TMEM accumulator are the same as in the forward grouped GEMM.  The output is float32 and overwritten
 // (each epilogue warp stages [32 rows x 32 columns] in swizzled shared memory and issues one TMA tensor
 // store); an expert with no rows gets zeros.
+// A tile's cost is its expert's row count, so the tile list is ordered by descending row count and dealt to the
+// CTAs in a snake (wave w goes 0..G-1 if w is even, G-1..0 if odd): every CTA gets nearly the same number of K
+// steps whatever the load skew, with a fixed assignment (no atomics, deterministic).
 #include "kernels.cuh"
 #include "tc.cuh"
 #include "tmap.cuh"
@@ -40,6 +43,7 @@ struct WCtl {
     uint32_t tmem_base;
     int abort_flag;
     int offs[34];
+    int perm[32];                  // experts by descending row count
 };
 
 template <int BN, int MT>
@@ -65,7 +69,17 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
     }
     if (warp == 1) tmem_alloc(&ctl->tmem_base, Cf::TMEM_COLS);
     pdl_wait();                     // everything above touches only this CTA's own resources
-    if (threadIdx.x >= 64 && threadIdx.x < 64 + n + 1) ctl->offs[threadIdx.x - 64] = offsets[threadIdx.x - 64];
+    if (warp == 2) {               // offsets, and the experts ranked by row count (n <= 32)
+        const int o = offsets[min(lane, n)], o1 = offsets[min(lane + 1, n)];
+        const int rows = lane < n ? o1 - o : -1;
+        int rank = 0;
+        for (int j = 0; j < n; ++j) {
+            const int rj = __shfl_sync(0xffffffffu, rows, j);
+            rank += (rj > rows || (rj == rows && j < lane)) ? 1 : 0;
+        }
+        if (lane < n) { ctl->offs[lane] = o; ctl->perm[rank] = lane; }
+        if (lane == n - 1) ctl->offs[n] = o1;
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -80,7 +94,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
     auto decode = [&](int tile, int& e, int& m0, int& n0, int& ks, int& kb_lo, int& kb_cnt) {
         ks = tile % ksplit;
         const int t2 = tile / ksplit;
-        e = t2 / per_expert;
+        e = ctl->perm[t2 / per_expert];
         const int rem = t2 % per_expert;
         m0 = (rem / n_tiles) * TM;
         n0 = (rem % n_tiles) * BN;
@@ -90,13 +104,20 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         kb_cnt = max(0, min(num_kb, kb_lo + per) - kb_lo);
     };
 
+    // the tile this CTA works in wave `wave` of the snake
+    auto snake_tile = [&](int wave) {
+        return wave * (int)gridDim.x + ((wave & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x);
+    };
+
     if (warp == 0) {
         // TMA producer: lane 0 runs the pipeline, the 64-wide boxes are issued one per lane
         int stage = 0;
         uint32_t phase = 0, issued = 0, issued_parity = 0;
         bool stop = false;
         const int sub_rows = (gather_p || gather_q) ? min(l_p, BK) : BK, nsub = BK / sub_rows;
-        for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+        for (int wave = 0; wave * (int)gridDim.x < total_tiles && !stop; ++wave) {
+            const int tile = snake_tile(wave);
+            if (tile >= total_tiles) continue;
             int e, m0, n0, ks, kb_lo, num_kb;
             decode(tile, e, m0, n0, ks, kb_lo, num_kb);
             const int r0 = ctl->offs[e] + kb_lo * BK;
@@ -153,7 +174,9 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool stop = false;
-            for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+            for (int wave = 0; wave * (int)gridDim.x < total_tiles && !stop; ++wave) {
+                const int tile = snake_tile(wave);
+                if (tile >= total_tiles) continue;
                 int e, m0, n0, ks, kb_lo, num_kb;
                 decode(tile, e, m0, n0, ks, kb_lo, num_kb);
                 if (!mbar_wait(&ctl->tempty[acc], acc_phase ^ 1, abort_flag, status) || *abort_flag) break;
@@ -185,7 +208,9 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         const int half = (warp - 2) >> 2;
         int acc = 0;
         uint32_t acc_phase = 0;
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        for (int wave = 0; wave * (int)gridDim.x < total_tiles; ++wave) {
+            const int tile = snake_tile(wave);
+            if (tile >= total_tiles) continue;
             int e, m0, n0, ks, kb_lo, num_kb;
             decode(tile, e, m0, n0, ks, kb_lo, num_kb);
             const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
