@@ -13,7 +13,7 @@ static MlpFwdWs mlp_fwd_ws(const Dims& D) {
     MlpFwdWs r;
     r.plan = w.take(plan_bytes(D));
     r.xg = can_fuse_gather(D) ? 0 : w.take((size_t)D.Rmax * D.d * D.esize);     // the GEMM gathers x itself
-    r.a = w.take((size_t)D.Rmax * D.d_e * D.esize);
+    r.a = mlp_can_fuse(D) ? 0 : w.take((size_t)D.Rmax * D.d_e * D.esize);          // the fused kernel keeps the hidden tile on chip
     r.z = w.take((size_t)D.Rmax * D.d * D.esize);
     r.total = w.off;
     return r;
@@ -62,7 +62,7 @@ extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, co
     GemmArgs g2{a, W2, b2, z, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
     g1.label = "gemm1_act";
     g2.label = "gemm2";
-    if (mlp_can_fuse(D) && !b1 && !b2) {      // narrow experts: both GEMMs in one kernel, the hidden tile stays on chip
+    if (mlp_can_fuse(D)) {                    // (bf16: no biases, checked above)      // narrow experts: both GEMMs in one kernel, the hidden tile stays on chip
         st = launch_mlp_fused(D, xg, W1, W2, z, saved_h, expert_offsets, prob->act, fused ? x : nullptr, P.src_patch, status,
                               stream);
         if (st != UOE_OK) return st;
