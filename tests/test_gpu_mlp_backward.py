@@ -29,6 +29,10 @@ CASES = {
     "full": _w(k=4, c=6),
     "wide": _w(B=3, d=256, d_ff=1024, n=4, k=3, L=256, L_valid=250, m=8, c=5),
     "skewed": _w(B=9, n=5, k=2, d_ff=640),
+    # narrow experts (d_e = 256): the forward is the one-kernel MLP, which also writes the saved pre-activation;
+    # 384 and 512 output columns take two output halves, with pad tokens and a ragged second half
+    "fused_fwd_d384_pad": _w(B=6, L=224, L_valid=197, m=14, c=7, d=384, n=3, k=2, d_ff=768),
+    "fused_fwd_d512": _w(B=4, L=256, L_valid=256, m=8, c=4, d=512, n=4, k=2, d_ff=1024, act="gelu_tanh"),
     # long K and many row tiles: 256-row GEMM tiles with half tiles at the region ends
     "tall_tiles": _w(B=40, L=1152, L_valid=1152, m=9, c=3, d=1024, n=4, k=2, d_ff=4096, w_std=0.02),
 }
