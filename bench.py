@@ -296,7 +296,7 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
 
     import paper_2503_02495_b200 as uoe
     from paper_2503_02495_b200.block import UoEBlock
-    from tests.helpers import problem_of, to_dev
+    from paper_2503_02495_b200.workload import problem_of, to_dev
 
     h = host_inputs(w)
     wd = {k: to_dev(v, dev) for k, v in h.items() if k not in ("x", "dy")}

@@ -22,6 +22,10 @@
  *     call clears it on its own (a clear on the stream would sit between the kernels of
  *     consecutive calls and stop them from overlapping).  A new workspace is prepared once with
  *     uoe_workspace_init; uoe_read_device_status clears the word after reporting an anomaly.
+ *   - Devices and threads.  A process may use the library on several devices; kernel attributes and cached
+ *     device properties are set up per device by the first call that needs them there.  That first call per
+ *     device (of each entry point, uoe_route_static included) is not thread-safe; afterwards calls from several
+ *     threads are safe as long as they use distinct workspaces.  uoe_profile_* is never thread-safe.
  *   - Element type: `dtype` selects float32 or bfloat16 storage for x, weights and y.  Products are
  *     accumulated in float32.  Routing probabilities and gates are always float32.
  *
@@ -76,7 +80,11 @@ typedef enum { UOE_OP_ROUTE = 0, UOE_OP_MLP_FWD = 1, UOE_OP_MLP_BWD = 2, UOE_OP_
                UOE_OP_BALANCE_BWD = 5 } uoe_op;
 
 /* One Union-of-Experts block.  L must equal m * l_p; rows t >= L_valid of every sample are padding
- * (they take no part in routing means, are masked as attention keys (Eq. 41), and y = x there). */
+ * (they take no part in routing means, are masked as attention keys (Eq. 41), and y = x there).
+ * Padding rows of x and dy must hold finite values (zeros by convention): whole patches travel through the
+ * tensor-core kernels, where a padding row is neutralised by a zero weight or a zero probability, and
+ * 0 * Inf or 0 * NaN would spread into the real rows of the same expert (weight gradients, attention outputs).
+ * A buffer padded from uninitialised memory must be zero-filled first. */
 typedef struct {
     int32_t B;        /* samples */
     int32_t L;        /* tokens per sample, padded: L = m * l_p */

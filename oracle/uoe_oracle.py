@@ -215,7 +215,7 @@ def balance_loss_backward(x: np.ndarray, W_r: np.ndarray, m: int, L_valid: int, 
 
 def select(p_samp: np.ndarray, p_patch: np.ndarray, cnt: np.ndarray, k: int, c: int, dynamic_c: bool = False):
     """Top-k experts per sample (Eq. 22), then top-c patches for each chosen expert (Eq. 17), indices
-    sorted ascending "to restore their original relative position".  With dynamic_c the number of patches
+    re-sorted ascending (text below Eq. 17).  With dynamic_c the number of patches
     per expert is the sample's own c of Eq. 16, capped by the given c (the width of the index array)."""
     B, n = p_samp.shape
     m = p_patch.shape[2]

@@ -281,12 +281,13 @@ uoe_status launch_attention_backward(const Dims& D, const void* q, const void* k
                                      const int* pair_row, const int* patch_idx, bool causal, int* status,
                                      cudaStream_t s) {
     if (D.d_h != DH) return UOE_ERR_UNSUPPORTED;
-    static bool attr_set = false;
-    if (!attr_set) {
-        UOE_CUDA_OK(cudaFuncSetAttribute(attn_bwd_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, BCfg<false>::SMEM));
-        UOE_CUDA_OK(cudaFuncSetAttribute(attn_bwd_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, BCfg<true>::SMEM));
-        attr_set = true;
+    static DeviceOnce once_kv, once_q;
+    {
+        uoe_status st = smem_opt_in(once_kv, attn_bwd_kernel<false>, BCfg<false>::SMEM);
+        if (st == UOE_OK) st = smem_opt_in(once_q, attn_bwd_kernel<true>, BCfg<true>::SMEM);
+        if (st != UOE_OK) return st;
     }
+    if ((long long)D.B * D.k > 65535) return UOE_ERR_UNSUPPORTED;      // pairs ride on grid.z
     CUtensorMap tm[4];
     const void* ptrs[4] = {q, k, v, dout};
     for (int i = 0; i < 4; ++i) {

@@ -376,13 +376,14 @@ uoe_status launch_attention(const Dims& D, const void* q, const void* k, const v
                             const int* pair_row, const int* patch_idx, bool causal, int* status, cudaStream_t s,
                             const void* Wo, const int* expert_idx, void* z) {
     if (D.d_h != DH) return UOE_ERR_UNSUPPORTED;
+    if ((long long)D.B * D.k > 65535) return UOE_ERR_UNSUPPORTED;      // pairs ride on grid.z
     const bool fuse = Wo != nullptr;
     if (fuse && (!attention_can_fuse_out(D) || !expert_idx || !z)) return UOE_ERR_INVALID_ARG;
-    static bool attr_set = false;
-    if (!attr_set) {
-        UOE_CUDA_OK(cudaFuncSetAttribute(attn_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM));
-        UOE_CUDA_OK(cudaFuncSetAttribute(attn_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATTN_SMEM_FUSED));
-        attr_set = true;
+    static DeviceOnce once_plain, once_fused;
+    {
+        uoe_status st = smem_opt_in(once_plain, attn_kernel<false>, ATTN_SMEM);
+        if (st == UOE_OK) st = smem_opt_in(once_fused, attn_kernel<true>, ATTN_SMEM_FUSED);
+        if (st != UOE_OK) return st;
     }
     CUtensorMap tm[3], tmWo;
     const void* ptrs[3] = {q, k, v};

@@ -7,6 +7,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "device_once.h"
 #include "uoe.h"
 
 namespace uoe {
@@ -30,6 +31,26 @@ extern long long g_launch_count;   // kernels enqueued by this process (reported
     } while (0)
 
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Ordinal of the current device, or -1 (no device, or an ordinal beyond the per-device tables).
+inline int current_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+
+// Opt-in of `kern` to `bytes` of dynamic shared memory, done once on every device the kernel is launched on
+// (the attribute belongs to the device's copy of the function).
+template <typename K>
+inline uoe_status smem_opt_in(DeviceOnce& once, K kern, int bytes) {
+    const int dev = current_device();
+    if (dev < 0) return UOE_ERR_CUDA;
+    if (once.needs(dev)) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return UOE_ERR_CUDA;
+        once.mark(dev);
+    }
+    return UOE_OK;
+}
 
 // Every kernel is launched with programmatic stream serialization allowed: the next kernel in the stream may
 // be scheduled, and run up to its pdl_wait(), while this one is still executing, which hides launch and

@@ -366,16 +366,23 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 template <int BN, bool B_KMAJOR, bool BWD, int MT, bool PAIR = false>
 uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     using Cf = Cfg<BN, MT, BWD, PAIR>;
-    static bool attr_set = false;
-    static int max_pairs = 0;          // CTA pairs that can be resident at once
+    static DeviceOnce once;
+    static DeviceValue pairs_cache;    // CTA pairs that can be resident at once, per device
     auto kern = gemm_bf16_kernel<BN, B_KMAJOR, BWD, MT, PAIR>;
-    if (!attr_set) {
-        UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
-        if (PAIR) {
-            UOE_CUDA_OK(max_resident_pairs(kern, Cf::THREADS, Cf::SMEM, &max_pairs));
-            if (max_pairs < 1) return UOE_ERR_CUDA;
+    {
+        const uoe_status st = smem_opt_in(once, kern, Cf::SMEM);
+        if (st != UOE_OK) return st;
+    }
+    int max_pairs = 0;
+    if (PAIR) {
+        const int dev = current_device();
+        if (!pairs_cache.has(dev)) {
+            int v = 0;
+            UOE_CUDA_OK(max_resident_pairs(kern, Cf::THREADS, Cf::SMEM, &v));
+            if (v < 1) return UOE_ERR_CUDA;
+            pairs_cache.set(dev, v);
         }
-        attr_set = true;
+        max_pairs = pairs_cache.get(dev);
     }
     CUtensorMap tmA, tmB[3], tmX;
     if (g.gather_x) {     // x as [Bm patches, l_p rows, K]; the 2-D map of A is unused

@@ -304,10 +304,10 @@ uoe_status launch_mlp_fused(const Dims& D, const void* A, const void* W1, const 
                             cudaStream_t s) {
     if (!mlp_can_fuse(D) || D.Rmax % BM != 0) return UOE_ERR_UNSUPPORTED;
     if (gather_x && (!src_patch || D.l_p < 8 || D.l_p % 8 != 0 || BM % D.l_p != 0)) return UOE_ERR_INVALID_ARG;
-    static bool attr_set = false;
-    if (!attr_set) {
-        UOE_CUDA_OK(cudaFuncSetAttribute(mlp_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM));
-        attr_set = true;
+    static DeviceOnce once;
+    {
+        const uoe_status st = smem_opt_in(once, mlp_fused_kernel, SMEM);
+        if (st != UOE_OK) return st;
     }
     CUtensorMap tmA, tmX, tmW1, tmW2, tmZ;
     if (gather_x) {       // x as [Bm patches, l_p rows, d]

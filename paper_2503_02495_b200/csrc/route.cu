@@ -673,7 +673,6 @@ extern "C" uoe_status uoe_route_balance(const uoe_problem* prob, const float* p_
 static __device__ __align__(256) unsigned char g_route_static_scratch[UOE_ROUTE_STATIC_SCRATCH_BYTES];
 
 namespace {
-constexpr int kMaxDevices = 64;
 unsigned char* g_route_static_ptr[kMaxDevices] = {};    // device address of the array, per device
 
 // In host code `g_route_static_scratch` is only a handle; the address a kernel can use comes from

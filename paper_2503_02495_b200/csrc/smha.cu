@@ -51,6 +51,7 @@ extern "C" uoe_status uoe_smha_forward(const uoe_problem* prob, const void* x, c
         !aligned16(ws))
         return UOE_ERR_INVALID_ARG;
     if (!D.bf16 || D.d_h != 64) return UOE_ERR_UNSUPPORTED;     // tensor-core path: bf16, 64-wide heads
+    if ((long long)D.B * D.k > 65535) return UOE_ERR_UNSUPPORTED;  // the attention grid carries the pairs on its z axis
     const SmhaWs W = smha_ws(D);
     if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)cuda_stream;

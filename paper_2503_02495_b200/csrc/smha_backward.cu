@@ -189,6 +189,7 @@ extern "C" uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, 
         if (!aligned16(p)) return UOE_ERR_INVALID_ARG;
     // tensor-core path only: bf16, 64-wide heads, model width that tiles the 128-row weight-gradient MMA
     if (!D.bf16 || D.d_h != 64 || D.d % 128 != 0) return UOE_ERR_UNSUPPORTED;
+    if ((long long)D.B * D.k > 65535) return UOE_ERR_UNSUPPORTED;  // the attention grids carry the pairs on their z axis
     const SmhaBwdWs W = smha_bwd_ws(D);
     if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
     cudaStream_t stream = (cudaStream_t)cuda_stream;

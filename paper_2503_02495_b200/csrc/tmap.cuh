@@ -36,13 +36,16 @@ inline bool make_tmap(CUtensorMap* out, const void* base, int rank, const uint64
     return r == CUDA_SUCCESS;
 }
 
+// SM count of the current device (cached per device).
 inline int sm_count() {
-    static int n = []() {
-        int dev = 0, v = 148;
-        if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-        return v > 0 ? v : 148;
-    }();
-    return n;
+    static DeviceValue cache;
+    const int dev = current_device();
+    if (cache.has(dev)) return cache.get(dev);
+    int v = 148;
+    if (dev >= 0) cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+    if (v <= 0) v = 148;
+    if (dev >= 0) cache.set(dev, v);
+    return v;
 }
 
 }  // namespace uoe

@@ -272,11 +272,11 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
                     long long rows_max, const char* label, int* status, cudaStream_t s, int ksplit, float* part,
                     const WgradGather& g) {
     using Cf = WCfg<BN, MT>;
-    static bool attr_set = false;
+    static DeviceOnce once;
     auto kern = wgrad_kernel<BN, MT>;
-    if (!attr_set) {
-        UOE_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cf::SMEM));
-        attr_set = true;
+    {
+        const uoe_status st = smem_opt_in(once, kern, Cf::SMEM);
+        if (st != UOE_OK) return st;
     }
     CUtensorMap tmP, tmQ;
     const uint32_t box[2] = {64, BK};

@@ -7,24 +7,18 @@ import torch
 import uoe_inputs as gen
 
 
-def to_dev(st: gen.Stored, device="cuda") -> torch.Tensor:
-    if st.dtype == "f32":
-        return torch.from_numpy(np.ascontiguousarray(st.raw)).to(device)
-    return torch.from_numpy(np.ascontiguousarray(st.raw).view(np.int16)).to(device).view(torch.bfloat16)
-
-
 def to_f64(t: torch.Tensor) -> np.ndarray:
     return t.detach().to(torch.float64).cpu().numpy()
 
 
-def problem_of(w: gen.Workload, block: str = "mlp", **kw):
-    import paper_2503_02495_b200 as uoe
-    base = dict(B=w.B, L=w.L, L_valid=w.L_valid, d=w.d, n=w.n, k=w.k, m=w.m, c=w.c,
-                d_e=w.d_e if block == "mlp" else 0, H=w.H if block == "att" else 0,
-                d_h=w.d_h if block == "att" else 0, dtype=w.dtype, act=w.act, residual=True, gate=True,
-                causal=w.causal if block == "att" else False)
-    base.update(kw)
-    return uoe.Problem(**base)
+def to_dev(st, device="cuda"):
+    from paper_2503_02495_b200.workload import to_dev as f
+    return f(st, device)
+
+
+def problem_of(w, block: str = "mlp", **kw):
+    from paper_2503_02495_b200.workload import problem_of as f
+    return f(w, block, **kw)
 
 
 def check_routing(r_gpu, r_or, margin_tol=1e-5):

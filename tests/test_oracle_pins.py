@@ -194,6 +194,39 @@ def test_uome_full_selection_with_gates_scales_hidden_blocks():
     assert np.allclose(y - t["x"], hidden @ A_O, rtol=1e-12, atol=1e-13)
 
 
+def test_uome_full_selection_with_biases_equals_dense_mlp_with_bias():
+    # the bias branch (the in-place bias of the batched product, Section III-D.2): at k=n, c=m with unit weights the
+    # layer is the dense MLP whose first bias is the concatenation of the experts' b1 and whose second bias is the
+    # SUM of the experts' b2 (every expert adds its own b2 to every token it serves, Eq. 5-7)
+    w = gen.tiny(k=4, c=6, act="gelu_erf")
+    t = _inputs(w, ("mlp",))
+    b1 = gen.normal(500, 1, (w.n, w.d_e), 0.5)
+    b2 = gen.normal(500, 2, (w.n, w.d), 0.5)
+    r = orc.route(t["x"], t["Wr"], w.k, w.m, w.c, use_gate=False)
+    y = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, "gelu_erf", b1=b1, b2=b2)
+    A_I = np.concatenate(list(t["W1"]), axis=1)
+    A_O = np.concatenate(list(t["W2"]), axis=0)
+    dense = orc.act_fn(t["x"] @ A_I + b1.reshape(-1), "gelu_erf") @ A_O + b2.sum(axis=0)
+    assert np.allclose(y - t["x"], dense, rtol=1e-12, atol=1e-13)
+    # a dropped or misplaced bias is visible at this size
+    y_nob = orc.mlp_forward(t["x"], t["W1"], t["W2"], r, "gelu_erf")
+    assert np.abs(y - y_nob).max() > 0.1
+    # partial selection: a token served by q experts receives q second-layer biases, scaled by their gates
+    w2 = gen.tiny(act="identity")
+    t2 = _inputs(w2, ("mlp",))
+    r2 = orc.route(t2["x"], _boost_router(t2["Wr"]), w2.k, w2.m, w2.c)
+    zero = np.zeros_like(t2["W1"])
+    b2s = gen.normal(500, 3, (w2.n, w2.d), 1.0)
+    y2 = orc.mlp_forward(t2["x"], zero, t2["W2"], r2, "identity", b1=np.zeros((w2.n, w2.d_e)), b2=b2s, residual=False)
+    for b in range(w2.B):
+        want = np.zeros((w2.L, w2.d))
+        for s, i in enumerate(r2.expert_idx[b]):
+            for u, j in enumerate(r2.patch_idx[b, s]):
+                if j >= 0:
+                    want[j * w2.l_p:(j + 1) * w2.l_p] += r2.gate[b, s, u] * b2s[i]
+        assert np.allclose(y2[b], want, rtol=1e-12, atol=1e-14)
+
+
 def _textbook_mha(x, WI_q, WI_k, WI_v, WO, heads, d_h, causal, L_valid):
     """Plain multi-head attention on one sample, written independently of the oracle."""
     L = x.shape[0]
@@ -224,6 +257,33 @@ def test_smha_full_selection_equals_multihead_attention(causal, H, L_valid):
         ref = _textbook_mha(t["x"][b], cat(t["Wq"]), cat(t["Wk"]), cat(t["Wv"]), WO, H, w.d_h, causal, L_valid)
         assert np.allclose((y - t["x"])[b, :L_valid], ref[:L_valid], rtol=1e-11, atol=1e-12)
         assert np.array_equal(y[b, L_valid:], t["x"][b, L_valid:])
+
+
+@pytest.mark.parametrize("causal,L_valid", [(False, 24), (True, 24), (False, 21)])
+def test_smha_log_sum_exp_output_is_the_textbook_one(causal, L_valid):
+    # return_lse: per (sample, chosen expert, head) the natural log of the sum over kept keys of exp(q.k / sqrt(d_h)),
+    # written here from the definition with scalar loops over the gathered tokens
+    w = gen.tiny(B=2, causal=causal, L_valid=L_valid, H=8)
+    t = _inputs(w, ("att",))
+    r = orc.route(t["x"], _boost_router(t["Wra"]), w.k, w.m, w.c, L_valid=L_valid)
+    y, lse = orc.smha_forward(t["x"], t["Wq"], t["Wk"], t["Wv"], t["Wo"], r, w.d_h, causal, return_lse=True)
+    assert np.array_equal(y, orc.smha_forward(t["x"], t["Wq"], t["Wk"], t["Wv"], t["Wo"], r, w.d_h, causal))
+    heads = w.d_g // w.d_h
+    assert len(lse) == w.B * w.k * heads
+    for b in range(w.B):
+        for s, i in enumerate(r.expert_idx[b]):
+            tok = orc.gathered_tokens(r, b, s)
+            q, kk = t["x"][b, tok] @ t["Wq"][i], t["x"][b, tok] @ t["Wk"][i]
+            for hd in range(heads):
+                sl = slice(hd * w.d_h, (hd + 1) * w.d_h)
+                got = lse[(b, s, hd)]
+                assert got.shape == (len(tok),)
+                for a in range(len(tok)):
+                    tot = 0.0
+                    for bb in range(len(tok)):
+                        if tok[bb] < L_valid and (not causal or bb <= a):
+                            tot += math.exp(float(q[a, sl] @ kk[bb, sl]) / math.sqrt(w.d_h))
+                    assert abs(got[a] - math.log(tot)) <= 1e-12 * max(1.0, abs(math.log(tot)))
 
 
 def test_fig4_mask_identity_and_its_negative():
@@ -653,11 +713,20 @@ def test_planted_mistakes_are_caught(monkeypatch):
         return np.allclose(y - t["x"], dense, rtol=1e-12, atol=1e-13)
 
     assert dense_ok()
-    # (1) activation also after the second layer (the misprint in Eq. 39)
+    # (1a) the activation applied twice to the hidden layer
     real_act = orc.act_fn
     monkeypatch.setattr(orc, "act_fn", lambda h, a: real_act(real_act(h, a), a))
     assert not dense_ok()
     monkeypatch.setattr(orc, "act_fn", real_act)
+    # (1b) an activation after the second layer of every expert (the misprint in Eq. 39): the sum of the per-expert
+    # phi(z_i) is not the dense layer (Eq. 5-7 put phi, if any, after the sum)
+    y_phi = t["x"].copy()
+    for b in range(w.B):
+        for s, i in enumerate(r.expert_idx[b]):
+            for j in r.patch_idx[b, s]:
+                rows = slice(j * w.l_p, (j + 1) * w.l_p)
+                y_phi[b, rows] += orc.act_fn(orc.act_fn(t["x"][b, rows] @ t["W1"][i], "silu") @ t["W2"][i], "silu")
+    assert not np.allclose(y_phi - t["x"], dense, rtol=1e-9, atol=1e-10)
     # (2) experts' weight slices swapped between layers
     y = orc.mlp_forward(t["x"], t["W1"], t["W2"][::-1], r, "silu")
     assert not np.allclose(y - t["x"], dense, rtol=1e-9, atol=1e-10)
