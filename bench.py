@@ -1,14 +1,19 @@
-"""Benchmark of the UoE routed hot path: one step = one forward pass of a whole UoE block
-(router -> SMHA -> router -> UoME; a block without attention or without MLP skips that half; the scale
-workload adds the UoME backward) over one batch of seeded synthetic input.
+"""Benchmark of the UoE routed hot path.  One step = one pass of the whole hot path over one batch of seeded
+synthetic input: router -> SMHA -> router -> UoME for a block workload (a block without attention or without MLP
+skips that half), router -> UoME forward -> UoME backward for the scale workload.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2_lm] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg5_scale] [--impl ours|reference]
 
-Prints ONE JSON line (rank 0).  `value` is tokens/s with inputs resident in HBM; `e2e` is the same metric
-through the public API with host buffers (pinned host -> device copy of x and device -> host copy of the
-result inside the timed region).  L2 is flushed between timed steps (a 512 MB write), and every step is
-timed with its own pair of CUDA events on the launching stream.  `--impl reference` times the float64
-CPU oracle on the same workload.
+Prints ONE JSON line (rank 0).  The top-level keys describe the largest single-GPU workload (cfg5_scale); with one
+GPU the line also carries, under "workloads", one block per other workload (language-model, long-sequence, image and
+the small float32 shape) measured with the same protocol: step time, tokens/s, TFLOP/s, roofline of the dominant
+kernel, the oracle's CPU time on a bounded sample, and parity statistics against the oracle (max error over
+tolerance, near-tie index mismatches).  `value` is tokens/s with inputs resident in HBM; `e2e` is the same metric
+through the public API with host buffers (pinned host -> device copies of the step's inputs and a device -> host
+copy of its result inside the timed region).  Small workloads: L2 is flushed between timed steps (a 512 MB write)
+and every step has its own pair of CUDA events; the scale workload streams far more than L2 per step and is timed
+back to back, once for K steps and once for at least a second ("sustained", against the sustained peak).
+`--impl reference` times the float64 CPU oracle on a bounded sample of the same workload.
 """
 from __future__ import annotations
 
@@ -240,16 +245,24 @@ class ClockSampler:
 # arms
 # ------------------------------------------------------------------------------------------------
 
-def base_line(w: gen.Workload, args, n_gpus: int):
+TOP_WORKLOAD = "cfg5_scale"          # the largest single-GPU workload: the one the headline line sits on
+ALL_WORKLOADS = ("cfg1_small_f32", "cfg2_lm", "cfg3_long", "cfg4_vit", "cfg5_scale")
+L2_BYTES = 126 << 20
+
+
+def config_of(w: gen.Workload, n_gpus: int, l2: str):
+    return {"workload": w.name, "stands_in_for": w.stands_in_for, "B": w.B, "L": w.L, "L_valid": w.L_valid,
+            "d": w.d, "n": w.n, "k": w.k, "m": w.m, "c": w.c, "d_ff": w.d_ff, "heads": w.H, "d_h": w.d_h,
+            "causal": w.causal, "act": w.act,
+            "blocks": ("smha+" if w.H else "") + ("uome" if w.d_ff else "") + ("+backward" if w.backward else ""),
+            "parallelism": f"replicas x{n_gpus}" if n_gpus > 1 else "single gpu", "l2": l2}
+
+
+def base_line(w: gen.Workload, args, n_gpus: int, l2: str = "flushed between timed steps (512 MB write)"):
     return {
         "metric": "UoME+SMHA layer tokens/s", "unit": "tokens/s", "n_gpus": n_gpus, "steps": args.steps,
         "warmup": args.warmup, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": w.dtype, "data": "synthetic",
-        "config": {"workload": w.name, "stands_in_for": w.stands_in_for, "B": w.B, "L": w.L, "L_valid": w.L_valid,
-                   "d": w.d, "n": w.n, "k": w.k, "m": w.m, "c": w.c, "d_ff": w.d_ff, "heads": w.H, "d_h": w.d_h,
-                   "causal": w.causal, "act": w.act, "blocks": ("smha+" if w.H else "") + ("uome" if w.d_ff else "") + ("+backward" if w.backward else ""),
-                   "parallelism": f"replicas x{n_gpus}" if n_gpus > 1 else "single gpu",
-                   "l2": "flushed between timed steps (512 MB write)"},
+        "dtype": w.dtype, "data": "synthetic", "config": config_of(w, n_gpus, l2),
     }
 
 
@@ -269,6 +282,25 @@ def job_throughput(w: gen.Workload, world: int, ms_per_step: float) -> float:
     return w.B * w.L_valid * world / (ms_per_step * 1e-3)
 
 
+def inputs_exceed_l2(w: gen.Workload) -> bool:
+    """True when one step streams far more than the L2 holds, so that no step finds its inputs cached."""
+    s = 2 if w.dtype == "bf16" else 4
+    return w.B * w.L * w.d * s >= 2 * L2_BYTES
+
+
+def cpu_baseline_of(w: gen.Workload, h, budget_s: float = 6.0, max_steps: int = 10):
+    """The oracle as it stands, timed on the host cores on the first Bs samples of the workload."""
+    Bs = cpu_sample_B(w)
+    oracle_step(w, h, Bs)                                   # first call pays imports and page faults
+    ts, t_begin = [], time.perf_counter()
+    while len(ts) < 2 or (time.perf_counter() - t_begin < budget_s and len(ts) < max_steps):
+        ts.append(oracle_step(w, h, Bs))
+    sec = sum(ts) / len(ts)
+    return {"value": Bs * w.L_valid / sec, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
+            "sec_per_step": sec, "tflops": step_flops(w) * Bs / w.B / sec / 1e12,
+            "sample": f"first {Bs} of {w.B} samples, whole step ({config_of(w, 1, '')['blocks']}), {len(ts)} steps"}
+
+
 def run_reference(args, w: gen.Workload, rank: int, world: int):
     if rank != 0:
         return
@@ -279,19 +311,102 @@ def run_reference(args, w: gen.Workload, rank: int, world: int):
     ts = [oracle_step(w, h, Bs) for _ in range(args.steps)]
     sec = sum(ts) / len(ts)
     tok_s = Bs * w.L_valid / sec
-    line = base_line(w, args, 1)
+    line = base_line(w, args, 1, "not applicable (CPU)")
     line.update({"impl": "reference", "value": tok_s, "ms_per_step": sec * 1e3, "dtype": "f64", "n_gpus": world,
                  "tflops": step_flops(w) * Bs / w.B / sec / 1e12,
                  "cpu_baseline": {"value": tok_s, "unit": "tokens/s", "cores": blas_threads(), "kind": "oracle",
-                                  "sample": f"first {Bs} of {w.B} samples, whole block, {args.steps} steps"},
+                                  "sample": f"first {Bs} of {w.B} samples, whole step, {args.steps} steps"},
                  "e2e": {"value": tok_s, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
                  "gpu_launches": 0})
     print(json.dumps(line), flush=True)
 
 
-def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int, with_e2e: bool):
-    """Times `steps` steps of workload w on this rank's GPU.  Returns a dict with the per-step milliseconds
-    (device events, L2 flushed between steps), launches, clocks, per-kernel records and the e2e time."""
+# ------------------------------------------------------------------------------------------------
+# parity of the launch configuration that is timed, on a bounded sample the oracle can afford
+# ------------------------------------------------------------------------------------------------
+
+def parity_of(w: gen.Workload, h, wd, x_dev, dy_dev, dev):
+    """Runs every half of the block once more through the C ABI (expert terms: residual off) and compares the first
+    Bs samples with the float64 oracle fed the same stored inputs.  Returns max error over tolerance per output,
+    routing-probability errors and the near-tie index mismatch counts."""
+    import torch
+
+    import paper_2503_02495_b200 as uoe
+    from oracle import uoe_oracle as orc
+    from paper_2503_02495_b200.workload import problem_of
+
+    tol = 2e-2 if w.dtype == "bf16" else 1e-4
+    Bs = min(cpu_sample_B(w), 64)
+    f64 = lambda t: t.detach().to(torch.float64).cpu().numpy()
+    rel = lambda got, ref: float(np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-300))
+    out = {"tolerance": tol, "sample": f"first {Bs} of {w.B} samples", "outputs": {}, "routing": {}}
+    worst = 0.0
+
+    def routing_stats(tag, r_gpu, x64, Wr64):
+        ro = orc.route(x64, Wr64, w.k, w.m, w.c, L_valid=w.L_valid)
+        e_gpu, p_gpu = r_gpu.expert_idx[:Bs].cpu().numpy(), r_gpu.patch_idx[:Bs].cpu().numpy()
+        near_e = near_p = hard = 0
+        for b in range(Bs):
+            if not np.array_equal(e_gpu[b], ro.expert_idx[b]):
+                near_e += 1
+                hard += ro.expert_margin[b] > 1e-5
+                continue
+            for s in range(w.k):
+                if not np.array_equal(p_gpu[b, s], ro.patch_idx[b, s]):
+                    near_p += 1
+                    hard += ro.patch_margin[b, s] > 1e-5
+        out["routing"][tag] = {
+            "p_samp_max_abs_err": float(np.abs(r_gpu.p_samp[:Bs].cpu().numpy() - ro.p_samp).max()),
+            "p_patch_max_abs_err": float(np.abs(r_gpu.p_patch[:Bs].cpu().numpy() - ro.p_patch).max()),
+            "near_tie_expert_set_mismatches": int(near_e), "near_tie_patch_set_mismatches": int(near_p),
+            "mismatches_outside_1e-5_margin": int(hard)}
+        return e_gpu, p_gpu, int(hard)
+
+    cur, cur64 = x_dev, h["x"].f64[:Bs]
+    hard_total = 0
+    if w.H:
+        pa = problem_of(w, "att")
+        r = uoe.uoe_route(pa, cur, wd["Wr_att"])
+        e_gpu, p_gpu, hard = routing_stats("smha", r, cur64, h["Wr_att"].f64)
+        hard_total += hard
+        z = uoe.uoe_smha_forward(problem_of(w, "att", residual=False), cur, wd["Wq"], wd["Wk"], wd["Wv"], wd["Wo"], r)
+        ro = orc.with_selection(cur64, h["Wr_att"].f64, e_gpu, p_gpu, w.m, w.L_valid)
+        ref = orc.smha_forward(cur64, h["Wq"].f64, h["Wk"].f64, h["Wv"].f64, h["Wo"].f64, ro, w.d_h, w.causal, residual=False)
+        out["outputs"]["smha_expert_term"] = rel(f64(z[:Bs]), ref) / tol
+        cur = uoe.uoe_smha_forward(pa, cur, wd["Wq"], wd["Wk"], wd["Wv"], wd["Wo"], r)
+        cur64 = f64(cur[:Bs])              # the UoME half is checked on the bits the GPU feeds it
+    if w.d_ff:
+        pm = problem_of(w, "mlp")
+        r = uoe.uoe_route(pm, cur, wd["Wr_mlp"])
+        e_gpu, p_gpu, hard = routing_stats("uome", r, cur64, h["Wr_mlp"].f64)
+        hard_total += hard
+        pm0 = problem_of(w, "mlp", residual=False)
+        sh = uoe.alloc_saved_h(pm0, dev) if w.backward else None
+        z = uoe.uoe_mlp_forward(pm0, cur, wd["W1"], wd["W2"], r, saved_h=sh)
+        ro = orc.with_selection(cur64, h["Wr_mlp"].f64, e_gpu, p_gpu, w.m, w.L_valid)
+        ref = orc.mlp_forward(cur64, h["W1"].f64, h["W2"].f64, ro, w.act, residual=False)
+        out["outputs"]["uome_expert_term"] = rel(f64(z[:Bs]), ref) / tol
+        if w.backward:
+            dx = uoe.uoe_mlp_backward(pm0, cur, wd["W1"], wd["W2"], wd["Wr_mlp"], r, sh, dy_dev)[0]
+            dref = orc.mlp_backward(cur64, h["W1"].f64, h["W2"].f64, h["Wr_mlp"].f64, ro, h["dy"].f64[:Bs], w.act,
+                                    residual=False)[0]
+            out["outputs"]["uome_dx_expert_term"] = rel(f64(dx[:Bs]), dref) / tol
+            out["note"] = "dW1, dW2, dW_r need every sample: checked at full size in tests/test_gpu_scale.py"
+            del dx, sh
+    worst = max(out["outputs"].values()) if out["outputs"] else 0.0
+    out["max_err_over_tol"] = worst
+    out["ok"] = bool(worst <= 1.0 and hard_total == 0)
+    return out
+
+
+# ------------------------------------------------------------------------------------------------
+# measurement of one workload on this rank's GPU
+# ------------------------------------------------------------------------------------------------
+
+def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int, with_e2e: bool, with_parity: bool = False,
+                sustain_s: float = 0.0):
+    """Times `steps` steps of workload w on this rank's GPU.  Returns a dict with the step time (device events),
+    launches, clocks, per-kernel records, the e2e time and, on request, the parity block and a sustained run."""
     import torch
 
     import paper_2503_02495_b200 as uoe
@@ -304,10 +419,11 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
     dy_dev = to_dev(h["dy"], dev) if w.backward else None
     blk = UoEBlock(problem_of(w, "att") if w.H else None, problem_of(w, "mlp") if w.d_ff else None, wd, dev,
                    backward=w.backward)
-    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    big = inputs_exceed_l2(w)
+    flush = None if big else torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     stream = torch.cuda.current_stream()
 
-    def step(xin):
+    def step(xin, dyin=None):
         if args.part == "route":          # the router alone (profiling): one uoe_route call on the block's input
             if blk.pm is not None:
                 uoe.uoe_route(blk.pm, xin, wd["Wr_mlp"], out=blk.rm, ws=blk.ws_rm, check=False)
@@ -316,7 +432,7 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
             return blk.ra.gate
         out = blk.forward(xin)
         if w.backward:
-            g = dy_dev
+            g = dy_dev if dyin is None else dyin
             if w.d_ff:
                 blk.mlp_backward(blk.u if w.H else xin, g)
                 g = blk.dx
@@ -332,60 +448,105 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
             dist.barrier()
         torch.cuda.synchronize()
 
+    def check_status(where):
+        st = blk.device_status()
+        if st != 0:
+            raise RuntimeError(f"device status after {where}: " + uoe.status_string(st))
+
     for _ in range(max(warmup, 3)):
         step(x_dev)
     torch.cuda.synchronize()
-    st = blk.device_status()
-    if st != 0:
-        raise RuntimeError("device status after warm-up: " + uoe.status_string(st))
+    check_status("warm-up")
 
-    # ---- timed region: K steps, each with its own event pair, L2 flushed in between ----
+    # ---- timed region: K steps.  Small inputs: each step has its own event pair and L2 is flushed in between.
+    #      Inputs far larger than L2: the K steps run back to back inside one event pair. ----
     sampler = ClockSampler(dev.index or 0)
     sampler.start()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     barrier()
     launches0 = uoe.uoe_launch_count()
-    for e0, e1 in ev:
-        flush.zero_()
+    if big:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        step(x_dev)
+        for _ in range(steps):
+            step(x_dev)
         e1.record(stream)
-    barrier()
+        barrier()
+        ms = [e0.elapsed_time(e1) / steps]
+    else:
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        for e0, e1 in ev:
+            flush.zero_()
+            e0.record(stream)
+            step(x_dev)
+            e1.record(stream)
+        barrier()
+        ms = [e0.elapsed_time(e1) for e0, e1 in ev]
     launches = uoe.uoe_launch_count() - launches0
     clocks = sampler.stop()
-    ms = [e0.elapsed_time(e1) for e0, e1 in ev]
-    res = {"ms_step": sum(ms) / len(ms), "ms_min": min(ms), "launches": int(launches), "clocks": clocks, "host": h}
+    check_status("the timed region")
+    res = {"ms_step": sum(ms) / len(ms), "ms_min": min(ms), "launches": int(launches), "clocks": clocks, "host": h,
+           "l2": "inputs far larger than L2 (x alone is %d MB): steps run back to back, no flush" % (w.B * w.L * w.d * 2 >> 20)
+                 if big else "flushed between timed steps (512 MB write)"}
 
-    # ---- end to end through the public API with host buffers ----
+    # ---- a run long enough for the power cap to settle (same step, back to back, one event pair) ----
+    if sustain_s > 0 and big:
+        n_sus = max(steps, int(sustain_s * 1e3 / res["ms_step"]) + 1)
+        sampler = ClockSampler(dev.index or 0, period_s=0.02)
+        sampler.start()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n_sus):
+            step(x_dev)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        res["sustained"] = {"steps": n_sus, "seconds": e0.elapsed_time(e1) * 1e-3, "ms_per_step": e0.elapsed_time(e1) / n_sus,
+                            "clocks": sampler.stop()}
+        check_status("the sustained run")
+
+    # ---- end to end through the public API with host buffers: inputs (x, and dy when the step has a backward) from
+    #      pinned host memory, the step's result back to pinned host memory, all inside the timed region ----
     if with_e2e:
-        x_host = h["x"].raw
-        x_pin = torch.from_numpy(np.ascontiguousarray(x_host).view(np.int16 if w.dtype == "bf16" else np.float32)).pin_memory()
+        npdt = np.int16 if w.dtype == "bf16" else np.float32
+        pin = lambda st: torch.from_numpy(np.ascontiguousarray(st.raw).view(npdt)).pin_memory()
+        x_pin = pin(h["x"])
         x_in = torch.empty_like(x_dev)
+        dy_pin = pin(h["dy"]) if w.backward else None
+        dy_in = torch.empty_like(dy_dev) if w.backward else None
         y_pin = torch.empty(x_pin.shape, dtype=x_pin.dtype).pin_memory()
         e2e_t = []
-        for i in range(steps + 2):
-            flush.zero_()
+        n_e2e = min(steps, 20) + 2
+        for i in range(n_e2e):
+            if flush is not None:
+                flush.zero_()
             torch.cuda.synchronize()
             t0 = time.perf_counter()
             x_in.view(x_pin.dtype).copy_(x_pin, non_blocking=True)
-            out = step(x_in)
+            if w.backward:
+                dy_in.view(dy_pin.dtype).copy_(dy_pin, non_blocking=True)
+            out = step(x_in, dy_in)
             if out.shape == x_in.shape:
                 y_pin.copy_(out.view(x_pin.dtype), non_blocking=True)
             torch.cuda.synchronize()
             if i >= 2:
                 e2e_t.append(time.perf_counter() - t0)
         res["e2e_ms"] = sum(e2e_t) / len(e2e_t) * 1e3
-        res["h2d"] = int(x_pin.numel() * x_pin.element_size())
+        res["e2e_steps"] = len(e2e_t)
+        res["h2d"] = int(x_pin.numel() * x_pin.element_size()) * (2 if w.backward else 1)
         res["d2h"] = int(y_pin.numel() * y_pin.element_size())
+        check_status("the end-to-end loop")
+        del x_pin, y_pin, x_in, dy_pin, dy_in
 
     # ---- per-kernel durations (separate pass: the event pairs would perturb the timed region) ----
     steps_prof = min(steps, 20)
     uoe.uoe_profile_enable(True)
     for _ in range(steps_prof):
-        flush.zero_()
+        if flush is not None:
+            flush.zero_()
         step(x_dev)
     torch.cuda.synchronize()
     uoe.uoe_profile_enable(False)
+    check_status("the per-kernel pass")
     per = {}
     for name, t in uoe.uoe_profile_records():
         per.setdefault(name, []).append(t)
@@ -401,6 +562,15 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
                      "gbs": wk["bytes"] / avg / 1e6 if avg > 0 else 0.0})
     kern.sort(key=lambda r: -r["share"])
     res["kernels"] = kern
+    # the whole router call (all of its kernels), for the HBM figure of Eq. 13-14, 21
+    route_labels = [n for n in per if n in ("route", "route_select")]
+    t_route = sum(sum(per[n]) for n in route_labels) / steps_prof
+    n_route = (1 if w.H else 0) + (1 if w.d_ff else 0)
+    if t_route > 0 and n_route:
+        res["route_call"] = {"ms": t_route / n_route, "gbs": work["route"]["bytes"] / (t_route / n_route) / 1e6,
+                             "kernels": sorted(route_labels)}
+    if with_parity:
+        res["parity"] = parity_of(w, h, wd, x_dev, dy_dev, dev)
     del blk, flush
     torch.cuda.empty_cache()
     return res
@@ -411,38 +581,86 @@ TENSOR_KERNELS = ("gemm1_act", "gemm2", "mlp_fused", "qkv_proj", "out_proj", "at
 HBM_KERNELS = ("route", "gather", "combine", "pool")
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/
-# (step_kernels_cfg2_lm.md, launches_gemm_cfg5_scale_B4.md, route_kernels_cfg5_scale.md).  Keyed by (workload, kernel
-# label); an entry is dropped when its kernel changes, and the line then reports null.  The scale workload's GEMM
-# entries were captured at B=4 and scaled by 2 (the part that is weight reads does not grow with B, so they are upper
-# estimates); its route entry was captured at full size.
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under profiles/.  Every
+# entry names the source file of its kernel and that file's SHA-1 at the time of the capture: when the file has
+# changed since, the line reports null instead of a stale figure.  (workload, kernel label) ->
+# (bytes per launch at the benchmark's size, source file, sha1 prefix, profiles/ summary)
 NCU_TRAFFIC = {
-    ("cfg2_lm", "route"): 8.47e6,
-    ("cfg2_lm", "combine"): 25.18e6,
-    ("cfg2_lm", "qkv_proj"): 9.73e6,
-    ("cfg2_lm", "mlp_fused"): 12.34e6,
-    ("cfg2_lm", "attention"): 6.88e6,
-    ("cfg5_scale", "gemm1_act"): 2 * (351.9e6 + 105.7e6),
-    ("cfg5_scale", "gemm2"): 2 * (176.2e6 + 220.0e6),
-    ("cfg5_scale", "bwd_da_dh"): 2 * (442.7e6 + 113.8e6),
-    ("cfg5_scale", "bwd_dx"): 2 * (176.3e6 + 220.6e6),
-    ("cfg5_scale", "route"): 268.4e6 + 16.8e6,
 }
 
 
-def roofline_of(top, w: gen.Workload, peaks, peak_src):
+def traffic_of(workload: str, kernel: str):
+    ent = NCU_TRAFFIC.get((workload, kernel))
+    if ent is None:
+        return None
+    import hashlib
+    nbytes, src, sha, _summary = ent
+    try:
+        cur = hashlib.sha1(open(os.path.join(ROOT, "paper_2503_02495_b200", "csrc", src), "rb").read()).hexdigest()
+    except OSError:
+        return None
+    return nbytes if cur.startswith(sha) else None
+
+
+def roofline_of(top, w: gen.Workload, peaks, peak_src, sustained: bool = False):
     wk = work_table(w).get(top["kernel"], dict(flops=0, bytes=0))
-    t_tensor = wk["flops"] / (peaks["bf16_tflops"] * 1e12)
+    tpeak = peaks["bf16_tflops_sustained"] if sustained else peaks["bf16_tflops"]
+    t_tensor = wk["flops"] / (tpeak * 1e12)
     t_hbm = wk["bytes"] / (peaks["hbm_gbs"] * 1e9)
     if t_tensor >= t_hbm and wk["flops"] > 0:
-        roof = {"bound": "tensor", "achieved": top["tflops"], "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
+        roof = {"bound": "tensor", "achieved": top["tflops"], "peak": tpeak, "unit": "TFLOP/s"}
     else:
         roof = {"bound": "hbm", "achieved": top["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s"}
-    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": NCU_TRAFFIC.get((w.name, top["kernel"])),
+    roof.update({"frac": roof["achieved"] / roof["peak"], "traffic": traffic_of(w.name, top["kernel"]),
                  "kernel": top["kernel"],
-                 "avg_ms": top["avg_ms"], "share_of_kernel_time": top["share"], "peak_source": peak_src,
+                 "avg_ms": top["avg_ms"], "share_of_kernel_time": top["share"],
+                 "peak_source": peak_src + (" (sustained figure)" if sustained else " (burst figure)"),
                  "algorithmic_flops": wk["flops"], "algorithmic_bytes": wk["bytes"]})
     return roof
+
+
+def block_of(w: gen.Workload, m, peaks, peak_src, world: int, ms_step: float, e2e_ms, args):
+    """Everything reported for one workload, from one measure_gpu result."""
+    flops = step_flops(w)
+    kern = m["kernels"]
+    k_by = {r["kernel"]: r for r in kern}
+    tens = [k_by[n] for n in TENSOR_KERNELS if n in k_by]
+    wt = work_table(w)
+    tf_sum = sum(wt[r["kernel"]]["flops"] for r in tens)
+    tm_sum = sum(r["avg_ms"] * r["launches_per_step"] for r in tens)
+    blk = {
+        "config": config_of(w, world, m["l2"]),
+        "steps": args.steps, "ms_per_step": ms_step, "ms_per_step_min": m["ms_min"],
+        "tokens_per_s": job_throughput(w, world, ms_step),
+        "routed_rows_per_s": w.R * world / (ms_step * 1e-3),
+        "tflops": flops * world / (ms_step * 1e-3) / 1e12,
+        "frac_of_bf16_peak": flops / (ms_step * 1e-3) / 1e12 / peaks["bf16_tflops"],
+        "algorithmic_gflop_per_step": flops / 1e9,
+        "gpu_launches": m["launches"], "clocks": m["clocks"],
+        "roofline": roofline_of(kern[0], w, peaks, peak_src),
+        "tensor_kernels": {"tflops": tf_sum / tm_sum / 1e9, "frac_of_bf16_peak": tf_sum / tm_sum / 1e9 / peaks["bf16_tflops"]}
+                          if tm_sum > 0 and w.dtype == "bf16" else None,
+        "hbm_kernels": {n: {"gbs": k_by[n]["gbs"], "frac_of_hbm_peak": k_by[n]["gbs"] / peaks["hbm_gbs"]}
+                        for n in HBM_KERNELS if n in k_by and n != "route"},
+        "kernels": [{kk: (round(vv, 5) if isinstance(vv, float) else vv) for kk, vv in r.items()} for r in kern],
+    }
+    if "route_call" in m:
+        rc = m["route_call"]
+        blk["hbm_kernels"]["uoe_route (whole call)"] = {"ms": rc["ms"], "gbs": rc["gbs"], "frac_of_hbm_peak": rc["gbs"] / peaks["hbm_gbs"],
+                                                         "kernels": rc["kernels"]}
+    if e2e_ms is not None:
+        blk["e2e"] = {"value": w.B * w.L_valid * world / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
+                      "steps": m.get("e2e_steps"), "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"]}
+    if "sustained" in m:
+        s = m["sustained"]
+        tf = flops / (s["ms_per_step"] * 1e-3) / 1e12
+        blk["sustained"] = {"steps": s["steps"], "seconds": s["seconds"], "ms_per_step": s["ms_per_step"],
+                            "tokens_per_s": w.B * w.L_valid / (s["ms_per_step"] * 1e-3), "tflops": tf,
+                            "frac_of_bf16_sustained_peak": tf / peaks["bf16_tflops_sustained"],
+                            "frac_of_bf16_burst_peak": tf / peaks["bf16_tflops"], "clocks": s["clocks"]}
+    if "parity" in m:
+        blk["parity"] = m["parity"]
+    return blk
 
 
 def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
@@ -454,7 +672,9 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
 
-    m = measure_gpu(args, w, dev, world, args.steps, args.warmup, True)
+    solo = world == 1 and args.part == "all"
+    m = measure_gpu(args, w, dev, world, args.steps, args.warmup, True, with_parity=solo and not args.skip_cpu_baseline,
+                    sustain_s=1.2 if solo else 0.0)
     ms_step, e2e_ms = max_over_ranks([m["ms_step"], m["e2e_ms"]], world, dev)
     if rank != 0:
         if world > 1:
@@ -462,62 +682,37 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
         return
 
     peaks, peak_src = load_peaks()
-    tokens = w.B * w.L_valid * world
-    flops = step_flops(w) * world
-    kern = m["kernels"]
-    roof = roofline_of(kern[0], w, peaks, peak_src)
-
-    # ---- CPU baseline: the oracle as it stands, on a bounded sample ----
-    h = m["host"]
-    Bs = cpu_sample_B(w)
-    ts = []
+    top = block_of(w, m, peaks, peak_src, world, ms_step, e2e_ms, args)
     if not args.skip_cpu_baseline:
-        oracle_step(w, h, Bs)
-        t_begin = time.perf_counter()
-        while len(ts) < 3 or (time.perf_counter() - t_begin < 8.0 and len(ts) < 20):
-            ts.append(oracle_step(w, h, Bs))
-    cpu_sec = sum(ts) / len(ts) if ts else float("nan")
+        top["cpu_baseline"] = cpu_baseline_of(w, m["host"])
+    del m
 
-    line = base_line(w, args, world)
-    line.update({
-        "value": job_throughput(w, world, ms_step), "ms_per_step": ms_step, "ms_per_step_min": m["ms_min"],
-        "tflops": flops / (ms_step * 1e-3) / 1e12,
-        "frac_of_bf16_peak": flops / (ms_step * 1e-3) / 1e12 / (peaks["bf16_tflops"] * world),
-        "e2e": {"value": tokens / (e2e_ms * 1e-3), "unit": "tokens/s", "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": m["h2d"], "d2h_bytes_per_step": m["d2h"]},
-        "gpu_launches": m["launches"],
-        "clocks": m["clocks"],
-        "roofline": roof,
-        "kernels": kern,
-        "cpu_baseline": {"value": (Bs * w.L_valid / cpu_sec) if ts else None, "unit": "tokens/s", "cores": blas_threads(),
-                         "kind": "oracle", "sec_per_step": cpu_sec if ts else None,
-                         "sample": f"first {Bs} of {w.B} samples, whole block, {len(ts)} steps"},
-    })
-    del m, h
+    line = base_line(w, args, world, top["config"]["l2"])
+    line.update({"value": top["tokens_per_s"], "ms_per_step": ms_step, "ms_per_step_min": top["ms_per_step_min"],
+                 "tflops": top["tflops"], "frac_of_bf16_peak": top["frac_of_bf16_peak"],
+                 "e2e": top["e2e"], "gpu_launches": top["gpu_launches"], "clocks": top["clocks"],
+                 "roofline": top["roofline"],
+                 "cpu_baseline": top.get("cpu_baseline", {"value": None, "unit": "tokens/s", "cores": blas_threads(),
+                                                          "kind": "oracle", "sample": "skipped"})})
+    for key in ("sustained", "parity", "tensor_kernels", "hbm_kernels", "kernels", "routed_rows_per_s", "algorithmic_gflop_per_step"):
+        if key in top:
+            line[key] = top[key]
 
-    # ---- the large MLP workload (forward + backward), where the tensor-core and HBM targets are quoted ----
-    if world == 1 and not args.no_scale and w.name != "cfg5_scale" and args.B == 0:
-        ws = gen.WORKLOADS["cfg5_scale"]
-        ms5 = measure_gpu(args, ws, dev, 1, 10, 3, False)
-        k5 = {r["kernel"]: r for r in ms5["kernels"]}
-        tens = [k5[n] for n in TENSOR_KERNELS if n in k5]
-        wt = work_table(ws)
-        tf_sum = sum(wt[r["kernel"]]["flops"] for r in tens)
-        tm_sum = sum(r["avg_ms"] * r["launches_per_step"] for r in tens)
-        line["scale_workload"] = {
-            "workload": ws.name, "blocks": "uome forward + backward", "B": ws.B, "L": ws.L, "d": ws.d, "d_ff": ws.d_ff,
-            "n": ws.n, "k": ws.k, "m": ws.m, "c": ws.c, "steps": 10,
-            "ms_per_step": ms5["ms_step"], "tokens_per_s": ws.B * ws.L_valid / (ms5["ms_step"] * 1e-3),
-            "tflops": step_flops(ws) / (ms5["ms_step"] * 1e-3) / 1e12,
-            "frac_of_bf16_peak": step_flops(ws) / (ms5["ms_step"] * 1e-3) / 1e12 / peaks["bf16_tflops"],
-            "grouped_gemm_tflops": tf_sum / tm_sum / 1e9 if tm_sum > 0 else None,
-            "grouped_gemm_frac_of_bf16_peak": tf_sum / tm_sum / 1e9 / peaks["bf16_tflops"] if tm_sum > 0 else None,
-            "hbm_kernels": {n: {"gbs": k5[n]["gbs"], "frac_of_hbm_peak": k5[n]["gbs"] / peaks["hbm_gbs"]}
-                            for n in HBM_KERNELS if n in k5},
-            "gpu_launches": ms5["launches"], "clocks": ms5["clocks"],
-            "roofline": roofline_of(ms5["kernels"][0], ws, peaks, peak_src),
-            "kernels": [{kk: (round(vv, 5) if isinstance(vv, float) else vv) for kk, vv in r.items()} for r in ms5["kernels"]],
-        }
+    # ---- the other workloads (language-model, long-sequence, image and the small float32 shapes), same protocol ----
+    if solo and not args.no_others and args.B == 0 and not args.backward:
+        others = {}
+        for name in ALL_WORKLOADS:
+            if name == w.name:
+                continue
+            wo = gen.WORKLOADS[name]
+            mo = measure_gpu(args, wo, dev, 1, args.steps, args.warmup, True, with_parity=not args.skip_cpu_baseline,
+                             sustain_s=1.2)
+            bo = block_of(wo, mo, peaks, peak_src, 1, mo["ms_step"], mo["e2e_ms"], args)
+            if not args.skip_cpu_baseline:
+                bo["cpu_baseline"] = cpu_baseline_of(wo, mo["host"], budget_s=4.0)
+            del mo
+            others[name] = bo
+        line["workloads"] = others
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -526,15 +721,16 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="cfg2_lm", choices=sorted(gen.WORKLOADS))
+    ap.add_argument("--workload", default=TOP_WORKLOAD, choices=sorted(gen.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--B", type=int, default=0, help="override the workload's batch size (profiling on a smaller case)")
-    ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing (profiling runs)")
+    ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing and the parity block (profiling runs)")
     ap.add_argument("--backward", action="store_true", help="add the backward of every half of the block to the step")
     ap.add_argument("--part", default="all", choices=["all", "route"], help="time only a part of the step (profiling runs)")
-    ap.add_argument("--no-scale", action="store_true", help="do not add the scale workload's summary to the line")
+    ap.add_argument("--no-others", "--no-scale", dest="no_others", action="store_true",
+                    help="only the selected workload: do not add the other workloads' blocks to the line")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
