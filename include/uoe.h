@@ -225,6 +225,43 @@ uoe_status uoe_smha_backward(const uoe_problem* prob, const void* x, const void*
                              float* dWq, float* dWk, float* dWv, float* dWo, float* dW_r,
                              void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Device arrays written by a router (shapes as for uoe_route).  A set is complete or absent as a whole. */
+typedef struct {
+    int32_t* expert_idx;      /* [B,k] */
+    int32_t* patch_idx;       /* [B,k,c] */
+    float* gate;              /* [B,k,c] */
+    float* p_samp;            /* [B,n] */
+    float* p_patch;           /* [B,n,m] */
+    int32_t* expert_offsets;  /* [n+1] */
+} uoe_routing;
+
+/*
+ * One UoE transformer block in one call (Section III-C, Fig. 2): selective attention over attention experts
+ * followed by the MLP experts, each half with its own router,
+ *     u = uoe_smha_forward(att, x, ...) with the routing of uoe_route(att, x, Wr_att),
+ *     y = uoe_mlp_forward (mlp, u, ...) with the routing of uoe_route(mlp, u, Wr_mlp),
+ * and the same results as that sequence of calls (Eq. 27-36, then Eq. 37-40; routing Eq. 12-17, 21-23).  Either
+ * half may be left out by passing NULL for its problem (then its weights are ignored and y is the other half's
+ * output; with only the MLP half, x is its input).  One workspace of uoe_block_workspace_bytes(att, mlp) bytes,
+ * prepared once with uoe_workspace_init, serves the whole call: the routers share their scratch, write their
+ * routing plans themselves, and the routed buffers of the two halves share memory, so a block costs fewer
+ * launches and less memory than the four separate calls.
+ *   att, mlp   host pointers; both describe the same B, L, L_valid, d and dtype (n, k, m, c may differ).
+ *   x [B,L,d]; Wr_att, Wr_mlp [d,n]; Wq, Wk, Wv [n,d,d_g]; Wo [n,d_g,d]; W1 [n,d,d_e]; W2 [n,d_e,d]   device, inputs.
+ *   r_att, r_mlp   host pointers to sets of device arrays that receive each router's outputs (for a later
+ *              backward call), or NULL to keep them inside the workspace.
+ *   u [B,L,d]  device, output of the attention half; required when both halves are present; distinct from x and y.
+ *   y [B,L,d]  device, output of the block.
+ *   saved_h    as for uoe_mlp_forward, or NULL.     lse   as for uoe_smha_forward, or NULL.
+ * Biases are not supported here.  Errors as for the separate calls; nothing is launched when an argument is rejected.
+ */
+size_t uoe_block_workspace_bytes(const uoe_problem* att, const uoe_problem* mlp);
+uoe_status uoe_block_forward(const uoe_problem* att, const uoe_problem* mlp, const void* x,
+                             const void* Wr_att, const void* Wq, const void* Wk, const void* Wv, const void* Wo,
+                             const void* Wr_mlp, const void* W1, const void* W2,
+                             const uoe_routing* r_att, const uoe_routing* r_mlp, void* u, void* y,
+                             void* saved_h, float* lse, void* ws, size_t ws_bytes, void* cuda_stream);
+
 /*
  * uoe_route without a workspace argument and without any allocation.  (The paper has no counterpart;
  * this exists for callers that cannot hand the library device memory of their own.)

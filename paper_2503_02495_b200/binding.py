@@ -30,6 +30,10 @@ class UoeError(RuntimeError):
         super().__init__(f"{where}: {status_string(status)} (status {status})")
 
 
+class _Routing(ctypes.Structure):
+    _fields_ = [(f, ctypes.c_void_p) for f in ("expert_idx", "patch_idx", "gate", "p_samp", "p_patch", "expert_offsets")]
+
+
 class _Problem(ctypes.Structure):
     _fields_ = [(f, ctypes.c_int32) for f in
                 ("B", "L", "L_valid", "d", "n", "k", "m", "c", "d_e", "H", "d_h", "dtype", "act")] + \
@@ -106,6 +110,10 @@ def _load():
     lib.uoe_route_balance.argtypes = [pp, f32p, ctypes.c_float, f32p, i32p, i32p, vp]
     lib.uoe_route_balance_backward.restype = ctypes.c_int
     lib.uoe_route_balance_backward.argtypes = [pp, vp, vp, f32p, ctypes.c_float, f32p, vp, f32p, vp, sz, vp]
+    lib.uoe_block_workspace_bytes.restype = sz
+    lib.uoe_block_workspace_bytes.argtypes = [pp, pp]
+    lib.uoe_block_forward.restype = ctypes.c_int
+    lib.uoe_block_forward.argtypes = [pp, pp] + [vp] * 9 + [ctypes.POINTER(_Routing)] * 2 + [vp, vp, vp, f32p, vp, sz, vp]
     lib.uoe_status_string.restype = ctypes.c_char_p
     lib.uoe_status_string.argtypes = [ctypes.c_int]
     lib.uoe_workspace_init.restype = ctypes.c_int
@@ -346,3 +354,49 @@ def uoe_route_balance_backward(prob: Problem, x, W_r, p_patch, alpha: float, dlo
                                          _stream())
     _check(st, "uoe_route_balance_backward")
     return dx, dW_r
+
+
+def uoe_block_workspace_bytes(att: Problem | None, mlp: Problem | None) -> int:
+    pa = ctypes.byref(att.c_struct()) if att is not None else None
+    pm = ctypes.byref(mlp.c_struct()) if mlp is not None else None
+    return int(_lib.uoe_block_workspace_bytes(pa, pm))
+
+
+def alloc_block_workspace(att: Problem | None, mlp: Problem | None, device="cuda") -> torch.Tensor:
+    nbytes = uoe_block_workspace_bytes(att, mlp)
+    if nbytes == 0:
+        raise UoeError(1, "uoe_block_workspace_bytes")
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    with torch.cuda.device(ws.device):
+        _check(_lib.uoe_workspace_init(_ptr(ws), nbytes, _stream()), "uoe_workspace_init")
+    return ws
+
+
+def _routing_struct(r: Routing | None):
+    if r is None:
+        return None
+    return ctypes.byref(_Routing(*(t.data_ptr() for t in (r.expert_idx, r.patch_idx, r.gate, r.p_samp, r.p_patch,
+                                                          r.expert_offsets))))
+
+
+def uoe_block_forward(att: Problem | None, mlp: Problem | None, x, weights: dict, r_att: Routing | None = None,
+                      r_mlp: Routing | None = None, u=None, y=None, saved_h=None, lse=None, ws=None, check: bool = True):
+    """One UoE block (SMHA half, then UoME half; either may be None) through the single C entry point.
+    `weights` holds Wr_att, Wq, Wk, Wv, Wo and / or Wr_mlp, W1, W2.  Returns y (and fills u, r_att, r_mlp when given)."""
+    p0 = att or mlp
+    _contig(x, p0.torch_dtype)
+    g = lambda name: _contig(weights.get(name), p0.torch_dtype)
+    y = y if y is not None else torch.empty_like(x)
+    if att is not None and mlp is not None and u is None:
+        u = torch.empty_like(x)
+    ws = ws if ws is not None else alloc_block_workspace(att, mlp, x.device)
+    pa = ctypes.byref(att.c_struct()) if att is not None else None
+    pm = ctypes.byref(mlp.c_struct()) if mlp is not None else None
+    st = _lib.uoe_block_forward(pa, pm, _ptr(x), _ptr(g("Wr_att")), _ptr(g("Wq")), _ptr(g("Wk")), _ptr(g("Wv")),
+                                _ptr(g("Wo")), _ptr(g("Wr_mlp")), _ptr(g("W1")), _ptr(g("W2")), _routing_struct(r_att),
+                                _routing_struct(r_mlp), _ptr(u), _ptr(y), _ptr(saved_h), _ptr(lse), _ptr(ws), ws.numel(),
+                                _stream())
+    _check(st, "uoe_block_forward")
+    if check:
+        _check(uoe_read_device_status(ws), "uoe_block_forward (device)")
+    return y

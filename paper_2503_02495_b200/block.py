@@ -1,4 +1,5 @@
-"""One UoE transformer block as a sequence of C-ABI calls with preallocated buffers.
+"""One UoE transformer block with preallocated buffers: the forward is the single C entry point
+uoe_block_forward, the backward the per-half entry points.
 
 u = SMHA(h) (router, Eq. 27-36), out = UoME(u) (router, Eq. 37-40): each sub-block has its own router,
 as in Section III-C.  Nothing is computed here; the class only owns device buffers and issues the calls.
@@ -17,10 +18,10 @@ class UoEBlock:
         p0 = prob_att or prob_mlp
         self.u = torch.empty(p0.B, p0.L, p0.d, dtype=p0.torch_dtype, device=device)
         self.out = torch.empty_like(self.u)
+        self.ws_blk = B.alloc_block_workspace(prob_att, prob_mlp, device)
         if prob_att is not None:
             self.ra = B.alloc_routing(prob_att, device)
             self.ws_ra = B.alloc_workspace(prob_att, B.UOE_OP_ROUTE, device)
-            self.ws_a = B.alloc_workspace(prob_att, B.UOE_OP_SMHA_FWD, device)
             if backward:          # SMHA backward buffers (Eq. 27-36 differentiated)
                 f32 = torch.float32
                 self.ws_ab = B.alloc_workspace(prob_att, B.UOE_OP_SMHA_BWD, device)
@@ -30,7 +31,6 @@ class UoEBlock:
         if prob_mlp is not None:
             self.rm = B.alloc_routing(prob_mlp, device)
             self.ws_rm = B.alloc_workspace(prob_mlp, B.UOE_OP_ROUTE, device)
-            self.ws_m = B.alloc_workspace(prob_mlp, B.UOE_OP_MLP_FWD, device)
             self.saved_h = B.alloc_saved_h(prob_mlp, device) if (save_h or backward) else None
             self.backward = backward
             if backward:          # UoME backward buffers (Eq. 38-40 differentiated)
@@ -42,19 +42,11 @@ class UoEBlock:
                 self.dWr = torch.empty(weights["Wr_mlp"].shape, dtype=f32, device=device)
 
     def forward(self, h: torch.Tensor, check: bool = False) -> torch.Tensor:
-        w = self.w
-        cur = h
-        if self.pa is not None:
-            B.uoe_route(self.pa, cur, w["Wr_att"], out=self.ra, ws=self.ws_ra, check=check)
-            B.uoe_smha_forward(self.pa, cur, w["Wq"], w["Wk"], w["Wv"], w["Wo"], self.ra, y=self.u, ws=self.ws_a,
-                               check=check)
-            cur = self.u
-        if self.pm is not None:
-            B.uoe_route(self.pm, cur, w["Wr_mlp"], out=self.rm, ws=self.ws_rm, check=check)
-            B.uoe_mlp_forward(self.pm, cur, w["W1"], w["W2"], self.rm, y=self.out, saved_h=self.saved_h,
-                              ws=self.ws_m, check=check)
-            cur = self.out
-        return cur
+        """The whole block through uoe_block_forward; the routing of both halves is kept for the backward."""
+        both = self.pa is not None and self.pm is not None
+        return B.uoe_block_forward(self.pa, self.pm, h, self.w, r_att=getattr(self, "ra", None),
+                                   r_mlp=getattr(self, "rm", None), u=self.u if both else None, y=self.out,
+                                   saved_h=getattr(self, "saved_h", None), ws=self.ws_blk, check=check)
 
     def mlp_backward(self, h: torch.Tensor, dy: torch.Tensor, check: bool = False):
         """Backward of the UoME half for the routing and saved pre-activations of the last forward(h)."""
@@ -71,7 +63,7 @@ class UoEBlock:
 
     def device_status(self) -> int:
         worst = 0
-        for name in ("ws_ra", "ws_a", "ws_rm", "ws_m", "ws_b", "ws_ab"):
+        for name in ("ws_blk", "ws_ra", "ws_rm", "ws_b", "ws_ab"):
             ws = getattr(self, name, None)
             if ws is not None:
                 worst = max(worst, B.uoe_read_device_status(ws))

@@ -72,7 +72,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  __nv_bfloat16* __restrict__ pre, const int* __restrict__ offsets,
                  int n, int K, int N, int nmat, int act, int* status, const __nv_bfloat16* __restrict__ bwd_h,
                  const float* __restrict__ row_gate, const float* __restrict__ row_valid, float* __restrict__ dg_part,
-                 const __grid_constant__ CUtensorMap tmX, const int* __restrict__ src_patch, int l_p, int Bm,
+                 const __grid_constant__ CUtensorMap tmX, const SrcMap smap, int l_p, int Bm,
                  const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                  const __grid_constant__ CUtensorMap tmC2, const __grid_constant__ CUtensorMap tmPre) {
     pdl_trigger();
@@ -162,12 +162,10 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // pairs: this CTA loads row block `rank` (none if the tile holds one block: its MMA rows are never stored)
             const int my_blocks = PAIR ? (rank < blocks ? 1 : 0) : blocks;
             const int arow0 = row0 + rank * BM;
-            const int nbox_a = src_patch ? my_blocks * (BM / l_p) : my_blocks;  // <= 32
+            const bool gathered = smap.on();
+            const int nbox_a = gathered ? my_blocks * (BM / l_p) : my_blocks;   // <= 32
             int my_src = 0;                                                     // source patch of this lane's box
-            if (src_patch && lane < nbox_a) {
-                my_src = src_patch[arow0 / l_p + lane];
-                if (my_src < 0) my_src = Bm;                                    // out of range: zero-filled box
-            }
+            if (gathered && lane < nbox_a) my_src = src_of(smap, arow0 + lane * l_p, e, ctl->offs[e], Bm);
             const uint32_t stage_bytes = Cf::KSUB * (blocks * A_BLOCK_BYTES + (PAIR ? 2 : 1) * Cf::B_BYTES);   // both CTAs' bytes
             for (int kb = 0; kb < num_kb; ++kb) {
                 int ok = 1;
@@ -187,7 +185,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         uint8_t* sa_j = sa + j * Cf::SUB;
                         uint8_t* sb_j = sa_j + Cf::A_BYTES;
                         if (lane < nbox_a) {
-                            if (src_patch) tma_load_3d_pair(sa_j + lane * l_p * 128, &tmX, k0, 0, my_src, full0);
+                            if (gathered) tma_load_3d_pair(sa_j + lane * l_p * 128, &tmX, k0, 0, my_src, full0);
                             else tma_load_2d_pair(sa_j, &tmA, k0, arow0, full0);
                         }
                         if (lane < nbox_b) {
@@ -197,7 +195,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                 } else {
                     if (lane < nbox_a) {
-                        if (src_patch) tma_load_3d(sa + lane * l_p * 128, &tmX, kb * BK, 0, my_src, &ctl->full[stage]);
+                        if (gathered) tma_load_3d(sa + lane * l_p * 128, &tmX, kb * BK, 0, my_src, &ctl->full[stage]);
                         else tma_load_2d(sa + lane * A_BLOCK_BYTES, &tmA, kb * BK, row0 + lane * BM, &ctl->full[stage]);
                     }
                     if (lane < nbox_b) {
@@ -429,6 +427,11 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     int grid = (int)(max_tiles < walkers ? max_tiles : walkers);
     if (grid < 1) grid = 1;
     if (PAIR) grid *= 2;
+    SrcMap smap;          // how the rows of a gathered A are found
+    if (g.gather_x) {
+        if (g.map.on()) smap = g.map;
+        else { smap.src_patch = g.src_patch; smap.l_p = g.l_p; }
+    }
     ProfScope ps(g.label, s);
     auto launch = [&](auto... a) {
         if constexpr (PAIR) return launch_k_pairs(a...);
@@ -437,7 +440,7 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     launch(kern, dim3(grid), dim3(Cf::THREADS), (size_t)Cf::SMEM, s, tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
                                              (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
                                              nmat, g.act, status, (const __nv_bfloat16*)g.bwd_h, g.row_gate, g.row_valid,
-                                             g.dg_part, tmX, g.gather_x ? g.src_patch : nullptr, g.l_p, g.Bm, tmC[0],
+                                             g.dg_part, tmX, smap, g.l_p, g.Bm, tmC[0],
                                              tmC[1], tmC[2], tmPre);
     UOE_LAUNCHED();
     return UOE_OK;
@@ -467,7 +470,7 @@ uoe_status dispatch(const GemmArgs& g, int* status, cudaStream_t s) {
 uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s) {
     if (g.K % BK != 0 || g.N % 64 != 0 || g.bias || g.nmat > 3) return UOE_ERR_UNSUPPORTED;
     if (g.nmat > 1 && g.pre) return UOE_ERR_UNSUPPORTED;
-    if (g.gather_x && (!g.src_patch || g.l_p < 8 || g.l_p % 8 != 0 || BM % g.l_p != 0)) return UOE_ERR_INVALID_ARG;
+    if (g.gather_x && ((!g.src_patch && !g.map.on()) || g.l_p < 8 || g.l_p % 8 != 0 || BM % g.l_p != 0)) return UOE_ERR_INVALID_ARG;
     if (g.rows_max % BM != 0 || g.n > 31) return UOE_ERR_UNSUPPORTED;
     if (g.bwd) {          // backward epilogue: weights are read K-major ([n, N, K])
         if (!g.b_kmajor || !g.bwd_h || !g.row_gate || !g.row_valid || !g.dg_part || !g.C1 || g.nmat > 1)

@@ -14,14 +14,40 @@ size_t balance_bwd_workspace_bytes(const Dims& D);
 // Layout of the routing plan inside a workspace: where each (sample, expert) pair's rows start and,
 // for every patch of every sample, which routed rows and gates feed it back (the inverse of Eq. 18).
 struct PlanPtrs {
-    int* pair_row;     // [B,k]    first routed row of (b, s)
-    int* inv_row;      // [B,m,k]  first routed row of patch j in slot s, or -1
-    float* inv_gate;   // [B,m,k]
-    int* expert_end;   // [n]      first padding row of expert i's region
-    float* row_gate;   // [Rmax]   backward only: combine weight of each routed row (0 on pad-token rows and unused slots)
-    float* row_valid;  // [Rmax]   backward only: 1 on rows that hold a real token, else 0
-    int* src_patch;    // [Rmax/l_p] source patch (b*m + j) of every l_p-row block of the routed buffers, -1 = zero rows
+    int* pair_row = nullptr;     // [B,k]    first routed row of (b, s)
+    int* inv_row = nullptr;      // [B,m,k]  first routed row of patch j in slot s, or -1; when the router wrote the plan:
+                                 //          the row's offset from pair_row[b,s] (inv_relative)
+    float* inv_gate = nullptr;   // [B,m,k]
+    int* expert_end = nullptr;   // [n]      first padding row of expert i's region
+    float* row_gate = nullptr;   // [Rmax]   backward only: combine weight of each routed row (0 on pad-token rows and unused slots)
+    float* row_valid = nullptr;  // [Rmax]   backward only: 1 on rows that hold a real token, else 0
+    int* src_patch = nullptr;    // [Rmax/l_p] source patch (b*m + j) of every l_p-row block of the routed buffers, -1 = zero rows
+    int* slot_pair = nullptr;    // [n,B]    plan written by the router kernel: pair (b*k + s) of the q-th sample in expert i's
+                                 //          region (it replaces src_patch, which that plan does not fill)
+    unsigned* sample_mask = nullptr;   // [B]  plan written by the router kernel: chosen experts of every sample as a bit set
+    bool inv_relative = false;   // inv_row holds offsets from pair_row (plan written by the router kernel)
+    // plan written by the router kernel only: a routed buffer whose first rows past the last expert region are
+    // zero-filled (up to 128 of them, as many as a 128-row tile that starts inside the last region can reach)
+    uint4* tail = nullptr;
+    long long tail_row_vecs = 0, rows_max = 0;
 };
+
+// Device arrays that uoe_route writes (shapes as in uoe.h).
+struct RoutingPtrs {
+    int* expert_idx = nullptr;
+    int* patch_idx = nullptr;
+    float* gate = nullptr;
+    float* p_samp = nullptr;
+    float* p_patch = nullptr;
+    int* expert_offsets = nullptr;
+};
+
+// uoe_route on a scratch area laid out as route_workspace_bytes describes (its control block zeroed once).  With
+// `plan` the routing plan is written by the same kernels (inv_row relative to pair_row), so no plan kernel is needed;
+// route_can_plan says whether the problem allows that.
+bool route_can_plan(const Dims& D);
+uoe_status route_run(const uoe_problem* prob, const void* x, const void* W_r, const RoutingPtrs& r, char* scratch,
+                     cudaStream_t stream, const PlanPtrs* plan);
 // Gathering through the GEMM's own TMA loads needs whole patches inside a 128-row tile, 8-row swizzle groups
 // and 64-column K steps.
 inline bool can_fuse_gather(const Dims& D) {
@@ -29,7 +55,8 @@ inline bool can_fuse_gather(const Dims& D) {
 }
 inline size_t plan_bytes(const Dims& D, bool with_rows = false) {
     return align_up((size_t)D.B * D.k * 4, 1024) + 2 * align_up((size_t)D.B * D.m * D.k * 4, 1024) + 1024 +
-           (with_rows ? 2 * align_up((size_t)D.Rmax * 4, 1024) : 0) + align_up((size_t)(D.Rmax / D.l_p + 1) * 4, 1024);
+           (with_rows ? 2 * align_up((size_t)D.Rmax * 4, 1024) : 0) + align_up((size_t)(D.Rmax / D.l_p + 1) * 4, 1024) +
+           align_up((size_t)D.n * D.B * 4, 1024) + align_up((size_t)D.B * 4, 1024);
 }
 inline PlanPtrs plan_ptrs(const Dims& D, char* base, bool with_rows = false) {
     PlanPtrs p;
@@ -46,8 +73,51 @@ inline PlanPtrs plan_ptrs(const Dims& D, char* base, bool with_rows = false) {
     p.row_valid = with_rows ? (float*)base : nullptr;
     base += with_rows ? align_up((size_t)D.Rmax * 4, 1024) : 0;
     p.src_patch = (int*)base;
+    base += align_up((size_t)(D.Rmax / D.l_p + 1) * 4, 1024);
+    p.slot_pair = (int*)base;
+    base += align_up((size_t)D.n * D.B * 4, 1024);
+    p.sample_mask = (unsigned*)base;
     return p;
 }
+
+// Where the rows of a gathered operand come from (Eq. 18 inside a kernel's own loads): either the table that the
+// plan kernel writes (src_patch[row / l_p]) or, with the plan the router kernel writes, derived per row block from the
+// pair that owns the block (slot_pair) and that pair's selected patches (patch_idx).
+struct SrcMap {
+    const int* src_patch = nullptr;
+    const int* slot_pair = nullptr;    // [n,B]
+    const int* patch_idx = nullptr;    // [B,k,c]
+    const int* expert_end = nullptr;   // [n]
+    int B = 0, k = 0, c = 0, m = 0, l_p = 0;
+    __host__ __device__ bool on() const { return src_patch != nullptr || slot_pair != nullptr; }
+};
+inline SrcMap src_map_of(const Dims& D, const PlanPtrs& P, const int* patch_idx) {
+    SrcMap g;
+    if (P.inv_relative) { g.slot_pair = P.slot_pair; g.patch_idx = patch_idx; g.expert_end = P.expert_end; }
+    else g.src_patch = P.src_patch;
+    g.B = D.B; g.k = D.k; g.c = D.c; g.m = D.m; g.l_p = D.l_p;
+    return g;
+}
+#ifdef __CUDACC__
+// Source patch (index into the [Bm patches] view of the source tensor) of the l_p-row block that starts at routed row
+// r inside the region of expert e (first row off_e); Bm (out of range: the loads return zeros) for padding rows and
+// unused slots.
+__device__ __forceinline__ int src_of(const SrcMap& g, int r, int e, int off_e, int Bm) {
+    int src;
+    if (g.src_patch) {
+        src = g.src_patch[r / g.l_p];
+    } else {
+        src = -1;
+        if (r < g.expert_end[e]) {
+            const int rel = r - off_e, l_a = g.c * g.l_p;
+            const int pair = g.slot_pair[(size_t)e * g.B + rel / l_a];
+            const int pj = g.patch_idx[(size_t)pair * g.c + (rel % l_a) / g.l_p];
+            if (pj >= 0 && pj < g.m) src = (pair / g.k) * g.m + pj;
+        }
+    }
+    return src < 0 ? Bm : src;
+}
+#endif
 
 // use_gate only matters for the per-row arrays of the backward (row_gate = gate or 1).
 // If tail is not null, rows [offsets[n], Rmax) of tail (rows of tail_row_bytes) are zero-filled.
@@ -100,6 +170,7 @@ struct GemmArgs {
     const void* gather_x = nullptr;
     const int* src_patch = nullptr;
     int l_p = 0, Bm = 0;
+    SrcMap map;             // if map.on(): used instead of src_patch (the router-written plan has no src_patch table)
     bool bwd = false;
     const void* bwd_h = nullptr;
     const float* row_gate = nullptr;
@@ -152,7 +223,27 @@ uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s);
 // pre (optional) [rows, 256] receives the pre-activation.
 bool mlp_can_fuse(const Dims& D);
 uoe_status launch_mlp_fused(const Dims& D, const void* A, const void* W1, const void* W2, void* z, void* pre,
-                            const int* offsets, int act, const void* gather_x, const int* src_patch, int* status,
+                            const int* offsets, int act, const void* gather_x, const SrcMap& map, int* status,
                             cudaStream_t s);
+
+// ---- forward halves behind the routing plan (shared by the per-half entry points and the block entry) ----
+struct MlpFwdBufs { void* xg; void* a; void* z; };
+struct SmhaFwdBufs { void *xg, *q, *k, *v, *o, *z; };
+struct SmhaFwdOffsets { size_t xg, q, k, v, o, z; };
+// bytes of the routed buffers of a forward half and their offsets (0 for a buffer the path does not need)
+size_t mlp_fwd_buffer_bytes(const Dims& D, size_t* xg, size_t* a, size_t* z);
+size_t smha_fwd_buffer_bytes(const Dims& D, SmhaFwdOffsets* o);
+uoe_status mlp_forward_check(const uoe_problem* prob, Dims& D, const void* x, const void* W1, const void* W2,
+                             const void* b1, const void* b2, const void* y, const void* saved_h);
+uoe_status mlp_forward_run(const Dims& D, const uoe_problem* prob, const void* x, const void* W1, const void* W2,
+                           const void* b1, const void* b2, const int* patch_idx, const int* expert_offsets,
+                           const PlanPtrs& P, const MlpFwdBufs& bufs, void* y, void* saved_h, int* status,
+                           cudaStream_t stream);
+uoe_status smha_forward_check(const uoe_problem* prob, Dims& D, const void* x, const void* Wq, const void* Wk,
+                              const void* Wv, const void* Wo, const void* y);
+uoe_status smha_forward_run(const Dims& D, const uoe_problem* prob, const void* x, const void* Wq, const void* Wk,
+                            const void* Wv, const void* Wo, const int* expert_idx, const int* patch_idx,
+                            const int* expert_offsets, const PlanPtrs& P, const SmhaFwdBufs& bufs, void* y, float* lse,
+                            int* status, cudaStream_t stream);
 
 }  // namespace uoe

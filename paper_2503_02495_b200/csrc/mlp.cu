@@ -21,36 +21,24 @@ static MlpFwdWs mlp_fwd_ws(const Dims& D) {
 
 size_t mlp_fwd_workspace_bytes(const Dims& D) { return mlp_fwd_ws(D).total; }
 
+size_t mlp_fwd_buffer_bytes(const Dims& D, size_t* xg, size_t* a, size_t* z) {
+    WsCarver w;
+    *xg = can_fuse_gather(D) ? 0 : w.take((size_t)D.Rmax * D.d * D.esize);
+    *a = mlp_can_fuse(D) ? 0 : w.take((size_t)D.Rmax * D.d_e * D.esize);
+    *z = w.take((size_t)D.Rmax * D.d * D.esize);
+    return w.off;
+}
+
 }  // namespace uoe
 
-using namespace uoe;
-
-extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, const void* W1, const void* W2,
-                                      const void* b1, const void* b2, const int32_t* expert_idx,
-                                      const int32_t* patch_idx, const float* gate, const int32_t* expert_offsets,
-                                      void* y, void* saved_h, void* ws, size_t ws_bytes, void* cuda_stream) {
-    Dims D;
-    uoe_status st = make_dims(prob, D);
-    if (st != UOE_OK) return st;
-    if (!x || !W1 || !W2 || !expert_idx || !patch_idx || !gate || !expert_offsets || !y || !ws) return UOE_ERR_INVALID_ARG;
-    if (D.d_e < 1) return UOE_ERR_INVALID_ARG;
-    if (!aligned16(x) || !aligned16(W1) || !aligned16(W2) || !aligned16(y) || !aligned16(ws) ||
-        (saved_h && !aligned16(saved_h)))
-        return UOE_ERR_INVALID_ARG;
-    if ((D.d_e * D.esize) % 16 != 0) return UOE_ERR_UNSUPPORTED;
-    if (D.bf16 && (b1 || b2)) return UOE_ERR_UNSUPPORTED;
-    const MlpFwdWs W = mlp_fwd_ws(D);
-    if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
-    cudaStream_t stream = (cudaStream_t)cuda_stream;
-    char* base = (char*)ws;
-    int* status = (int*)base;
-    const PlanPtrs P = plan_ptrs(D, base + W.plan);
-    void* xg = base + W.xg;
-    void* a = base + W.a;
-    void* z = base + W.z;
-
-    st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream);
-    if (st != UOE_OK) return st;
+// Everything of the UoME forward behind the routing plan: gather (unless the GEMM gathers), the two grouped GEMMs
+// (or the one fused kernel), combine.
+uoe_status uoe::mlp_forward_run(const Dims& D, const uoe_problem* prob, const void* x, const void* W1, const void* W2,
+                                const void* b1, const void* b2, const int* patch_idx, const int* expert_offsets,
+                                const PlanPtrs& P, const MlpFwdBufs& bufs, void* y, void* saved_h, int* status,
+                                cudaStream_t stream) {
+    uoe_status st;
+    void *xg = bufs.xg, *a = bufs.a, *z = bufs.z;
     const bool fused = can_fuse_gather(D);
     if (!fused) {
         st = launch_gather(D, x, patch_idx, expert_offsets, P, xg, stream);
@@ -58,12 +46,13 @@ extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, co
     }
 
     GemmArgs g1{xg, W1, b1, a, saved_h, expert_offsets, D.n, D.d, D.d_e, prob->act, false, D.Rmax};
-    if (fused) { g1.gather_x = x; g1.src_patch = P.src_patch; g1.l_p = D.l_p; g1.Bm = D.B * D.m; }
+    const SrcMap map = src_map_of(D, P, patch_idx);
+    if (fused) { g1.gather_x = x; g1.map = map; g1.l_p = D.l_p; g1.Bm = D.B * D.m; }
     GemmArgs g2{a, W2, b2, z, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
     g1.label = "gemm1_act";
     g2.label = "gemm2";
-    if (mlp_can_fuse(D)) {                    // (bf16: no biases, checked above)      // narrow experts: both GEMMs in one kernel, the hidden tile stays on chip
-        st = launch_mlp_fused(D, xg, W1, W2, z, saved_h, expert_offsets, prob->act, fused ? x : nullptr, P.src_patch, status,
+    if (mlp_can_fuse(D)) {                    // (bf16: no biases)      narrow experts: both GEMMs in one kernel, the hidden tile stays on chip
+        st = launch_mlp_fused(D, xg, W1, W2, z, saved_h, expert_offsets, prob->act, fused ? x : nullptr, map, status,
                               stream);
         if (st != UOE_OK) return st;
     } else if (D.bf16) {
@@ -79,4 +68,39 @@ extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, co
     }
     return launch_combine(D, x, z, P, (prob->flags & UOE_FLAG_RESIDUAL) != 0, (prob->flags & UOE_FLAG_GATE) != 0, y,
                           stream);
+}
+
+uoe_status uoe::mlp_forward_check(const uoe_problem* prob, Dims& D, const void* x, const void* W1, const void* W2,
+                                  const void* b1, const void* b2, const void* y, const void* saved_h) {
+    uoe_status st = make_dims(prob, D);
+    if (st != UOE_OK) return st;
+    if (!x || !W1 || !W2 || !y) return UOE_ERR_INVALID_ARG;
+    if (D.d_e < 1) return UOE_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(W1) || !aligned16(W2) || !aligned16(y) || (saved_h && !aligned16(saved_h)))
+        return UOE_ERR_INVALID_ARG;
+    if ((D.d_e * D.esize) % 16 != 0) return UOE_ERR_UNSUPPORTED;
+    if (D.bf16 && (b1 || b2)) return UOE_ERR_UNSUPPORTED;
+    return UOE_OK;
+}
+
+using namespace uoe;
+
+extern "C" uoe_status uoe_mlp_forward(const uoe_problem* prob, const void* x, const void* W1, const void* W2,
+                                      const void* b1, const void* b2, const int32_t* expert_idx,
+                                      const int32_t* patch_idx, const float* gate, const int32_t* expert_offsets,
+                                      void* y, void* saved_h, void* ws, size_t ws_bytes, void* cuda_stream) {
+    Dims D;
+    uoe_status st = mlp_forward_check(prob, D, x, W1, W2, b1, b2, y, saved_h);
+    if (st != UOE_OK) return st;
+    if (!expert_idx || !patch_idx || !gate || !expert_offsets || !ws || !aligned16(ws)) return UOE_ERR_INVALID_ARG;
+    const MlpFwdWs W = mlp_fwd_ws(D);
+    if (ws_bytes < W.total) return UOE_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    char* base = (char*)ws;
+    int* status = (int*)base;
+    const PlanPtrs P = plan_ptrs(D, base + W.plan);
+    st = launch_plan(D, expert_idx, patch_idx, gate, expert_offsets, P, status, stream);
+    if (st != UOE_OK) return st;
+    const MlpFwdBufs bufs{base + W.xg, base + W.a, base + W.z};
+    return mlp_forward_run(D, prob, x, W1, W2, b1, b2, patch_idx, expert_offsets, P, bufs, y, saved_h, status, stream);
 }

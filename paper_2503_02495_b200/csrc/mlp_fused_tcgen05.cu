@@ -48,7 +48,7 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW2,
                  const __grid_constant__ CUtensorMap tmZ, __nv_bfloat16* __restrict__ pre,
                  const int* __restrict__ offsets, int n, int d, int act, int* status,
-                 const int* __restrict__ src_patch, int l_p, int Bm) {
+                 const SrcMap smap, int l_p, int Bm) {
     pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -125,18 +125,16 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
             int e, row0;
             locate(tile, e, row0);
-            const int nbox_a = src_patch ? BM / l_p : 1;                        // <= 16
+            const bool gathered = smap.on();
+            const int nbox_a = gathered ? BM / l_p : 1;                         // <= 16
             int my_src = 0;
-            if (src_patch && lane < nbox_a) {
-                my_src = src_patch[row0 / l_p + lane];
-                if (my_src < 0) my_src = Bm;                                    // out of range: zero-filled box
-            }
+            if (gathered && lane < nbox_a) my_src = src_of(smap, row0 + lane * l_p, e, ctl->offs[e], Bm);   // Bm: zero-filled box
             for (int kb = 0; kb < kb1 && !stop; ++kb) {
                 if (!acquire(STAGE)) { stop = true; break; }
                 uint8_t* sa = smem + stage * STAGE;
                 uint8_t* sb = sa + A_BYTES;
                 if (lane < nbox_a) {
-                    if (src_patch) tma_load_3d(sa + lane * l_p * 128, &tmX, kb * BK, 0, my_src, &ctl->full[stage]);
+                    if (gathered) tma_load_3d(sa + lane * l_p * 128, &tmX, kb * BK, 0, my_src, &ctl->full[stage]);
                     else tma_load_2d(sa, &tmA, kb * BK, row0, &ctl->full[stage]);
                 }
                 if (lane >= 16 && lane < 20)
@@ -300,10 +298,10 @@ bool mlp_can_fuse(const Dims& D) { return D.bf16 && D.d_e == DE && D.d % 64 == 0
 // A: routed rows [rows_max, d] (or gathered from gather_x through src_patch), W1 [n, d, 256], W2 [n, 256, d],
 // z [rows_max, d]; pre (optional) [rows_max, 256] receives the pre-activation.
 uoe_status launch_mlp_fused(const Dims& D, const void* A, const void* W1, const void* W2, void* z, void* pre,
-                            const int* offsets, int act, const void* gather_x, const int* src_patch, int* status,
+                            const int* offsets, int act, const void* gather_x, const SrcMap& map, int* status,
                             cudaStream_t s) {
     if (!mlp_can_fuse(D) || D.Rmax % BM != 0) return UOE_ERR_UNSUPPORTED;
-    if (gather_x && (!src_patch || D.l_p < 8 || D.l_p % 8 != 0 || BM % D.l_p != 0)) return UOE_ERR_INVALID_ARG;
+    if (gather_x && (!map.on() || D.l_p < 8 || D.l_p % 8 != 0 || BM % D.l_p != 0)) return UOE_ERR_INVALID_ARG;
     static DeviceOnce once;
     {
         const uoe_status st = smem_opt_in(once, mlp_fused_kernel, SMEM);
@@ -343,7 +341,7 @@ uoe_status launch_mlp_fused(const Dims& D, const void* A, const void* W1, const 
     if (grid < 1) grid = 1;
     ProfScope ps("mlp_fused", s);
     launch_k(mlp_fused_kernel, dim3(grid), dim3(THREADS), (size_t)SMEM, s, tmA, tmX, tmW1, tmW2, tmZ, (__nv_bfloat16*)pre, offsets,
-             D.n, D.d, act, status, gather_x ? src_patch : (const int*)nullptr, D.l_p, (int)(D.B * D.m));
+             D.n, D.d, act, status, gather_x ? map : SrcMap(), D.l_p, (int)(D.B * D.m));
     UOE_LAUNCHED();
     return UOE_OK;
 }

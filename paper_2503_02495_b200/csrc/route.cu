@@ -25,7 +25,7 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
                               int* __restrict__ expert_idx,
                               int* __restrict__ patch_idx, float* __restrict__ gate, float* __restrict__ p_samp,
                               float* __restrict__ p_patch, int* __restrict__ offsets, int* __restrict__ load,
-                              int* __restrict__ ticket) {
+                              int* __restrict__ ticket, const PlanPtrs plan) {
     __shared__ float ps[32];               // sample gate
     __shared__ int sel[32];                // chosen experts, ascending
     __shared__ int cnts[32];               // Eq. 16: patches each expert receives in the first routing stage
@@ -116,6 +116,7 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
             expert_idx[(size_t)b * k + s] = lane;
             atomicAdd(&load[lane], 1);
         }
+        if (lane == 0 && plan.sample_mask) plan.sample_mask[b] = mask;
     }
     __syncthreads();
     int take = min(c, n_elig);
@@ -142,14 +143,24 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
                 }
             const bool pick = valid && rank < take;
             const unsigned mask = __ballot_sync(0xffffffffu, pick);
+            const int pos = before + __popc(mask & ((1u << lane) - 1u));
+            const float g = use_gate ? ps[i] * v : 1.0f;
             if (pick) {
-                const int pos = before + __popc(mask & ((1u << lane) - 1u));
                 out_idx[pos] = j;
-                out_gate[pos] = use_gate ? ps[i] * v : 1.0f;
+                out_gate[pos] = g;
+            }
+            if (plan.inv_row && valid) {        // the inverse of Eq. 18, relative to the pair's first routed row
+                plan.inv_row[((size_t)b * m + j) * k + s] = pick ? pos * l_p : -1;
+                plan.inv_gate[((size_t)b * m + j) * k + s] = pick ? g : 0.f;
             }
             before += __popc(mask);
         }
         for (int pos = before + lane; pos < c; pos += 32) { out_idx[pos] = -1; out_gate[pos] = 0.f; }
+        if (plan.inv_row)
+            for (int j = n_elig + lane; j < m; j += 32) {       // patches of pad tokens only
+                plan.inv_row[((size_t)b * m + j) * k + s] = -1;
+                plan.inv_gate[((size_t)b * m + j) * k + s] = 0.f;
+            }
     }
     // Eq. 23 as row offsets: the CTA that completes the last sample turns the loads into a prefix sum
     __syncthreads();
@@ -158,6 +169,7 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
         s_last = (atomicAdd(ticket, 1) == B - 1);
     }
     __syncthreads();
+    __shared__ int s_offs[34];
     if (s_last && warp == 0) {
         __threadfence();
         const int rows_per_pair = c * l_p;
@@ -173,8 +185,39 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
             const int v = __shfl_up_sync(0xffffffffu, incl, o);
             if (lane >= o) incl += v;
         }
-        if (lane < n) offsets[lane] = incl - rows;
-        if (lane == n - 1) offsets[n] = incl;
+        if (lane < n) { offsets[lane] = incl - rows; s_offs[lane] = incl - rows; }
+        if (lane == n - 1) { offsets[n] = incl; s_offs[n] = incl; }
+    }
+    // The part of the routing plan that needs every sample's choice, by the same CTA: where every pair's rows start
+    // and which pair owns every slot of every expert's region.  One pass over the samples' expert sets per expert
+    // (a warp per expert, 32 samples per step), so rows inside a region ascend with the sample.
+    if (plan.pair_row && s_last) {
+        unsigned* s_mask = (unsigned*)pp;           // [B] (pp is free now)
+        __syncthreads();
+        for (int b2 = tid; b2 < B; b2 += NT) s_mask[b2] = __ldcg(plan.sample_mask + b2);
+        __syncthreads();
+        const int l_a = c * l_p;
+        for (int i = warp; i < n; i += NT / 32) {
+            int running = 0;
+            for (int b0 = 0; b0 < B; b0 += 32) {
+                const int b2 = b0 + lane;
+                const unsigned mk = b2 < B ? s_mask[b2] : 0u;
+                const bool mine = (mk >> i) & 1u;
+                const unsigned ball = __ballot_sync(0xffffffffu, mine);
+                if (mine) {        // the chosen experts of a sample ascend: expert i sits in slot #(chosen experts below i)
+                    const int s = __popc(mk & ((1u << i) - 1u));
+                    const int q = running + __popc(ball & ((1u << lane) - 1u));
+                    plan.pair_row[(size_t)b2 * k + s] = s_offs[i] + q * l_a;
+                    plan.slot_pair[(size_t)i * B + q] = b2 * k + s;
+                }
+                running += __popc(ball);
+            }
+            if (lane == 0) plan.expert_end[i] = s_offs[i] + running * l_a;
+        }
+        if (plan.tail) {
+            const long long r0 = s_offs[n], r1 = min(plan.rows_max, r0 + 128);
+            for (long long q = tid; q < (r1 - r0) * plan.tail_row_vecs; q += NT) plan.tail[r0 * plan.tail_row_vecs + q] = make_uint4(0, 0, 0, 0);
+        }
     }
 }
 
@@ -198,7 +241,7 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
              int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
              float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
              int* __restrict__ ctl /* word 1: ticket, words 8..: expert loads */, int* __restrict__ sample_ticket /* [B] */,
-             int* __restrict__ patch_ticket /* [B*m] */) {
+             int* __restrict__ patch_ticket /* [B*m] */, const PlanPtrs plan /* all null: no plan is written */) {
     pdl_trigger();
     pdl_wait();
     constexpr int V = Vec16<T>::N;
@@ -356,7 +399,7 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
         __threadfence();
         // ---- 3. this CTA completed sample b ----
         select_sample<NT>((float*)s_dyn4, scores, 1, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
-                      p_patch, offsets, ctl + 8, ctl + 1);
+                      p_patch, offsets, ctl + 8, ctl + 1, plan);
     }
 }
 
@@ -370,7 +413,7 @@ route_patch_scores_kernel(const T* __restrict__ W_r, const float* __restrict__ p
                           int B, int Lv, int d, int n, int k, int m, int c, int l_p, int rsplit, int use_gate,
                           int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
                           float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
-                          int* __restrict__ ctl, int* __restrict__ sample_ticket) {
+                          int* __restrict__ ctl, int* __restrict__ sample_ticket, const PlanPtrs plan) {
     pdl_trigger();
     pdl_wait();
     constexpr int NT = kScoreThreads;
@@ -453,7 +496,7 @@ route_patch_scores_kernel(const T* __restrict__ W_r, const float* __restrict__ p
     if (!s_mine) return;
     __threadfence();
     select_sample<kScoreThreads>(s_sel, scores, 1, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch,
-                  offsets, ctl + 8, ctl + 1);
+                  offsets, ctl + 8, ctl + 1, plan);
 }
 
 struct RouteWs { size_t tickets, ptickets, scores, pool, total; int nchunks, CT, rsplit, rows_per_cta, wblk_bytes; size_t smem; bool two_kernels, small_ctas; };
@@ -503,7 +546,10 @@ RouteWs route_ws(const Dims& D) {
 // scores, pooled sums); its control block must have been zero when first used.
 uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void* W_r, int32_t* expert_idx,
                         int32_t* patch_idx, float* gate, float* p_samp, float* p_patch, int32_t* expert_offsets,
-                        char* base, const RouteWs& W, cudaStream_t stream, bool profile) {
+                        char* base, const RouteWs& W, cudaStream_t stream, bool profile, const PlanPtrs& plan = PlanPtrs()) {
+    // with a plan the CTA that completes the last sample keeps one word per sample in dynamic shared memory
+    const size_t plan_smem = plan.pair_row ? (size_t)D.B * sizeof(unsigned) : 0;
+    const size_t smem0 = W.smem > plan_smem ? W.smem : plan_smem;
     int* ctl = (int*)base;             // word 0 status (unused here), word 1 ticket, words 8.. expert loads
     int* tickets = (int*)(base + W.tickets);
     int* ptickets = (int*)(base + W.ptickets);
@@ -513,16 +559,16 @@ uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void
     dim3 grid((unsigned)(D.B * D.m * W.nchunks * W.rsplit)), grid2((unsigned)(D.B * D.m));
 #define UOE_ROUTE_ARGS(T) (const T*)x, (const T*)W_r, pool, scores, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, \
         W.nchunks, W.rsplit, W.rows_per_cta, W.wblk_bytes, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, \
-        tickets, ptickets
+        tickets, ptickets, plan
     cudaError_t e;
     if (!W.two_kernels) {
         ProfScope ps(profile ? "route" : nullptr, stream);
         if (W.small_ctas) {
-            if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0, 64>, grid, dim3(64), W.smem, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
-            else e = launch_k(route_kernel<float, 0, 64>, grid, dim3(64), W.smem, stream, UOE_ROUTE_ARGS(float));
+            if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0, 64>, grid, dim3(64), smem0, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
+            else e = launch_k(route_kernel<float, 0, 64>, grid, dim3(64), smem0, stream, UOE_ROUTE_ARGS(float));
         } else {
-            if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0, kScoreThreads>, grid, dim3(kScoreThreads), W.smem, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
-            else e = launch_k(route_kernel<float, 0, kScoreThreads>, grid, dim3(kScoreThreads), W.smem, stream, UOE_ROUTE_ARGS(float));
+            if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0, kScoreThreads>, grid, dim3(kScoreThreads), smem0, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
+            else e = launch_k(route_kernel<float, 0, kScoreThreads>, grid, dim3(kScoreThreads), smem0, stream, UOE_ROUTE_ARGS(float));
         }
         if (e != cudaSuccess) return UOE_ERR_CUDA;
         UOE_LAUNCHED();
@@ -537,9 +583,10 @@ uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void
     UOE_LAUNCHED();
     {
         ProfScope ps(profile ? "route_select" : nullptr, stream);
-        const size_t sel = (size_t)D.n * D.m * sizeof(float);
+        size_t sel = (size_t)D.n * D.m * sizeof(float);
+        if (sel < plan_smem) sel = plan_smem;
 #define UOE_SCORE_ARGS(T) (const T*)W_r, pool, scores, D.B, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.rsplit, use_gate, expert_idx, \
-        patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, tickets
+        patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, tickets, plan
 #define UOE_SCORE_LAUNCH(T, NMAX) launch_k(route_patch_scores_kernel<T, NMAX>, grid2, dim3(kScoreThreads), sel, stream, UOE_SCORE_ARGS(T))
         if (D.bf16) {
             if (D.n <= 8) e = UOE_SCORE_LAUNCH(__nv_bfloat16, 8);
@@ -577,6 +624,19 @@ uoe_status route_check(const uoe_problem* prob, Dims& D, RouteWs& W, const void*
 }  // namespace
 
 size_t route_workspace_bytes(const Dims& D) { return route_ws(D).total; }
+
+bool route_can_plan(const Dims& D) { return (size_t)D.B * sizeof(unsigned) <= 32 * 1024; }
+
+uoe_status route_run(const uoe_problem* prob, const void* x, const void* W_r, const RoutingPtrs& r, char* scratch,
+                     cudaStream_t stream, const PlanPtrs* plan) {
+    Dims D;
+    RouteWs W;
+    uoe_status st = route_check(prob, D, W, x, W_r, r.expert_idx, r.patch_idx, r.gate, r.p_samp, r.p_patch, r.expert_offsets);
+    if (st != UOE_OK) return st;
+    if (plan && !route_can_plan(D)) return UOE_ERR_UNSUPPORTED;
+    return route_launch(D, prob->flags, x, W_r, r.expert_idx, r.patch_idx, r.gate, r.p_samp, r.p_patch, r.expert_offsets, scratch,
+                        W, stream, true, plan ? *plan : PlanPtrs());
+}
 
 }  // namespace uoe
 

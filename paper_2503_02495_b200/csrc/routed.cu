@@ -160,7 +160,8 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __restrict__ inv_row,
                const float* __restrict__ inv_gate, T* __restrict__ y, int L, int Lv, int d, int m, int k,
-               int l_p, int residual, int use_gate, int rows_per_cta, const float* __restrict__ rvec) {
+               int l_p, int residual, int use_gate, int rows_per_cta, const float* __restrict__ rvec,
+               const int* __restrict__ pair_row /* not null: inv_row holds offsets from the pair's first row */) {
     pdl_trigger();
     pdl_wait();
     constexpr int V = Vec16<T>::N;
@@ -169,7 +170,9 @@ combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __re
     const int bj = blockIdx.x, b = bj / m, j = bj % m;
     const int r0 = blockIdx.y * rows_per_cta, r1 = min(l_p, r0 + rows_per_cta);
     if (threadIdx.x < k) {
-        srow[threadIdx.x] = inv_row[(size_t)bj * k + threadIdx.x];
+        const int rel = inv_row[(size_t)bj * k + threadIdx.x];
+        const int base = pair_row ? pair_row[(size_t)b * k + threadIdx.x] : 0;
+        srow[threadIdx.x] = rel >= 0 ? rel + base : -1;
         sg[threadIdx.x] = use_gate ? inv_gate[(size_t)bj * k + threadIdx.x] : 1.0f;
     }
     __syncthreads();
@@ -328,11 +331,13 @@ uoe_status launch_combine(const Dims& D, const void* x, const void* z, const Pla
     if (D.bf16)
         launch_k(combine_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, s, 
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)z, P.inv_row, P.inv_gate, (__nv_bfloat16*)y, D.L, D.Lv,
-            D.d, D.m, D.k, D.l_p, residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec);
+            D.d, D.m, D.k, D.l_p, residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec,
+            P.inv_relative ? (const int*)P.pair_row : (const int*)nullptr);
     else
         launch_k(combine_kernel<float>, grid, dim3(kThreads), 0, s, (const float*)x, (const float*)z, P.inv_row, P.inv_gate,
                                                        (float*)y, D.L, D.Lv, D.d, D.m, D.k, D.l_p,
-                                                       residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec);
+                                                       residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec,
+                                                       P.inv_relative ? (const int*)P.pair_row : (const int*)nullptr);
     UOE_LAUNCHED();
     return UOE_OK;
 }
