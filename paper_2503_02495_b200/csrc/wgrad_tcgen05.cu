@@ -8,9 +8,12 @@
 // TMEM accumulator are the same as in the forward grouped GEMM.  The output is float32 and overwritten
 // (each epilogue warp stages [32 rows x 32 columns] in swizzled shared memory and issues one TMA tensor
 // store); an expert with no rows gets zeros.
-// A tile's cost is its expert's row count, so the tile list is ordered by descending row count and dealt to the
-// CTAs in a snake (wave w goes 0..G-1 if w is even, G-1..0 if odd): every CTA gets nearly the same number of K
-// steps whatever the load skew, with a fixed assignment (no atomics, deterministic).
+// A tile's cost is its expert's row count, so the tile list is ordered by descending row count and handed out
+// longest first: a CTA's first tile is its own index, every further one comes from a counter in the workspace's
+// control block that the producer warp advances when it is ready for more work (greedy list scheduling: the CTAs
+// finish within one cheap tile of each other whatever the load skew).  Which CTA computes a tile varies from run to
+// run; the result does not, because every output tile is computed whole, in a fixed K order, by one CTA.  The last
+// CTA to finish leaves the counters at zero for the next launch.
 #include "kernels.cuh"
 #include "tc.cuh"
 #include "tmap.cuh"
@@ -22,6 +25,8 @@ using namespace tc;
 
 constexpr int BM = 128, BK = 64;
 constexpr int A_BLOCK_BYTES = BM * BK * 2;
+constexpr int kSchedSlots = 4;       // tiles the producer may run ahead of the slowest consumer
+constexpr int kSchedWord = 64;       // words [64, 66) of the workspace's control block: next tile, CTAs finished
 
 // MT = 2: 256 x BN output tiles (two 128-row accumulators fed by the same Q stage), one accumulator set
 // drained by eight epilogue warps; MT = 1: 128 x BN tiles with two accumulator sets.
@@ -44,13 +49,16 @@ struct WCtl {
     int abort_flag;
     int offs[34];
     int perm[32];                  // experts by descending row count
+    uint64_t sfull[kSchedSlots], sempty[kSchedSlots];
+    int sched_tile[kSchedSlots];   // tiles handed from the producer warp to the MMA thread and the epilogue warps
 };
 
 template <int BN, int MT>
 __global__ void __launch_bounds__(WCfg<BN, MT>::THREADS, 1)
 wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CUtensorMap tmQ,
              const __grid_constant__ CUtensorMap tmW, const int* __restrict__ offsets, int n, int M, int N,
-             int ksplit, int* status, int gather_p, int gather_q, const int* __restrict__ src_patch, int l_p, int Bm) {
+             int ksplit, int* status, int gather_p, int gather_q, const int* __restrict__ src_patch, int l_p, int Bm,
+             int* __restrict__ sched /* [2], zero between launches */) {
     pdl_trigger();
     using Cf = WCfg<BN, MT>;
     extern __shared__ uint8_t smem_raw[];
@@ -62,6 +70,7 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
     if (threadIdx.x == 0) {
         for (int s = 0; s < Cf::STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 32 * Cf::EPI_WARPS); }
+        for (int q = 0; q < kSchedSlots; ++q) { mbar_init(&ctl->sfull[q], 1); mbar_init(&ctl->sempty[q], 1 + Cf::EPI_WARPS); }
         ctl->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmP);
@@ -104,9 +113,16 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         kb_cnt = max(0, min(num_kb, kb_lo + per) - kb_lo);
     };
 
-    // the tile this CTA works in wave `wave` of the snake
-    auto snake_tile = [&](int wave) {
-        return wave * (int)gridDim.x + ((wave & 1) ? (int)gridDim.x - 1 - (int)blockIdx.x : (int)blockIdx.x);
+    // Consumer side of the tile hand-off (one thread per consumer warp calls it): the next tile of this CTA, or a value
+    // >= total_tiles when there is none (also after a wait ran out).
+    auto next_tile = [&](int& slot, uint32_t& sphase) {
+        int tile = total_tiles;
+        if (mbar_wait(&ctl->sfull[slot], sphase, abort_flag, status) && !*abort_flag) {
+            tile = ctl->sched_tile[slot];
+            mbar_arrive(&ctl->sempty[slot]);
+        }
+        if (++slot == kSchedSlots) { slot = 0; sphase ^= 1; }
+        return tile;
     };
 
     if (warp == 0) {
@@ -115,9 +131,21 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         uint32_t phase = 0, issued = 0, issued_parity = 0;
         bool stop = false;
         const int sub_rows = (gather_p || gather_q) ? min(l_p, BK) : BK, nsub = BK / sub_rows;
-        for (int wave = 0; wave * (int)gridDim.x < total_tiles && !stop; ++wave) {
-            const int tile = snake_tile(wave);
-            if (tile >= total_tiles) continue;
+        int slot = 0;
+        uint32_t sphase = 0;
+        for (bool first = true; !stop; first = false) {
+            int tile = total_tiles;
+            if (lane == 0) {       // hand the next tile (or the end marker) to the consumers
+                if (mbar_wait(&ctl->sempty[slot], sphase ^ 1, abort_flag, status) && !*abort_flag) {
+                    tile = first ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(sched, 1);
+                    if (tile > total_tiles) tile = total_tiles;
+                }
+                ctl->sched_tile[slot] = tile;
+                mbar_arrive(&ctl->sfull[slot]);
+            }
+            tile = __shfl_sync(0xffffffffu, tile, 0);
+            if (++slot == kSchedSlots) { slot = 0; sphase ^= 1; }
+            if (tile >= total_tiles) break;
             int e, m0, n0, ks, kb_lo, num_kb;
             decode(tile, e, m0, n0, ks, kb_lo, num_kb);
             const int r0 = ctl->offs[e] + kb_lo * BK;
@@ -174,9 +202,11 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool stop = false;
-            for (int wave = 0; wave * (int)gridDim.x < total_tiles && !stop; ++wave) {
-                const int tile = snake_tile(wave);
-                if (tile >= total_tiles) continue;
+            int slot = 0;
+            uint32_t sphase = 0;
+            while (!stop) {
+                const int tile = next_tile(slot, sphase);
+                if (tile >= total_tiles) break;
                 int e, m0, n0, ks, kb_lo, num_kb;
                 decode(tile, e, m0, n0, ks, kb_lo, num_kb);
                 if (!mbar_wait(&ctl->tempty[acc], acc_phase ^ 1, abort_flag, status) || *abort_flag) break;
@@ -208,9 +238,13 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         const int half = (warp - 2) >> 2;
         int acc = 0;
         uint32_t acc_phase = 0;
-        for (int wave = 0; wave * (int)gridDim.x < total_tiles; ++wave) {
-            const int tile = snake_tile(wave);
-            if (tile >= total_tiles) continue;
+        int slot = 0;
+        uint32_t sphase = 0;
+        for (;;) {
+            int tile = 0;
+            if (lane == 0) tile = next_tile(slot, sphase);
+            tile = __shfl_sync(0xffffffffu, tile, 0);
+            if (tile >= total_tiles) break;
             int e, m0, n0, ks, kb_lo, num_kb;
             decode(tile, e, m0, n0, ks, kb_lo, num_kb);
             const bool ready = mbar_wait(&ctl->tfull[acc], acc_phase, abort_flag, status) && !*abort_flag;
@@ -219,21 +253,23 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
             const int wrow0 = (ks * n + e) * M + m0 + half * BM + quarter * 32;   // first row of this warp's piece in [ksplit*n*M, N]
             const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (MT == 2 ? half * BN : acc * BN);
             uint8_t* stg = smem + Cf::STAGES * Cf::STAGE + 1024 + (warp - 2) * Cf::STG_BYTES;
+            // the TMEM read of the next piece is in flight while this one is staged and stored
+            uint32_t v[32];
+            if (num_kb > 0) {
+                tmem_ld32(taddr, v);
+            } else {
+#pragma unroll
+                for (int q = 0; q < 32; ++q) v[q] = 0u;
+            }
 #pragma unroll 1
             for (int ch = 0; ch < BN / 32; ++ch) {
-                uint32_t v[32];
-                if (num_kb > 0) {
-                    tmem_ld32(taddr + ch * 32, v);
-                    tmem_ld_wait();
-                } else {
-#pragma unroll
-                    for (int q = 0; q < 32; ++q) v[q] = 0u;
-                }
+                if (num_kb > 0) tmem_ld_wait();
                 if (lane == 0) bulk_wait_read();      // the previous store has finished reading the piece
                 __syncwarp();
 #pragma unroll
                 for (int q = 0; q < 8; ++q)
                     *(uint4*)(stg + lane * 128 + ((q ^ (lane & 7)) << 4)) = make_uint4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+                if (num_kb > 0 && ch + 1 < BN / 32) tmem_ld32(taddr + (ch + 1) * 32, v);
                 fence_async_smem();
                 __syncwarp();
                 if (lane == 0) { tma_store_2d(&tmW, stg, n0 + ch * 32, wrow0); bulk_commit(); }
@@ -249,6 +285,14 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
     if (warp == 1) {
         __syncwarp();
         tmem_dealloc(tmem_base, Cf::TMEM_COLS);
+    }
+    if (threadIdx.x == 0) {         // this CTA's last fetch lies before the barrier above: the last CTA to get here resets
+        __threadfence();
+        if (atomicAdd(sched + 1, 1) == (int)gridDim.x - 1) {
+            sched[0] = 0;
+            sched[1] = 0;
+            __threadfence();
+        }
     }
 }
 
@@ -310,7 +354,7 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
     int grid = (int)(tiles < sm_count() ? tiles : sm_count());
     ProfScope ps(label, s);
     launch_k(kern, grid, dim3(Cf::THREADS), Cf::SMEM, s, tmP, tmQ, tmW, offsets, n, M, N, ksplit, status, g.gather_p ? 1 : 0,
-             g.gather_q ? 1 : 0, g.src_patch, g.l_p, g.Bm);
+             g.gather_q ? 1 : 0, g.src_patch, g.l_p, g.Bm, status + kSchedWord);
     UOE_LAUNCHED();
     if (ksplit > 1) {
         const long long vecs = (long long)n * M * N / 4;
@@ -345,6 +389,7 @@ size_t wgrad_scratch_bytes(int n, int M, int N, long long rows_max) {
 uoe_status launch_wgrad_bf16(const void* P, const void* Q, float* dW, const int* offsets, int n, int M, int N,
                              long long rows_max, const char* label, int* status, cudaStream_t s, float* part,
                              const WgradGather& g) {
+    if (!status) return UOE_ERR_INVALID_ARG;       // the tile counters live in the control block behind the status word
     if (M % BM != 0 || N % 64 != 0 || n > 32) return UOE_ERR_UNSUPPORTED;
     if ((g.gather_p || g.gather_q) && (!g.src_patch || !wgrad_can_gather(g.l_p))) return UOE_ERR_INVALID_ARG;
     const int bn = gemm_bf16_bn(N);
