@@ -270,7 +270,7 @@ uoe_status uoe_block_forward(const uoe_problem* att, const uoe_problem* mlp, con
  * synchronise the device or touch the allocator (a latency-critical serving loop, a plugin hosted by
  * a framework that owns all device memory and offers no way to request scratch, start-up code that
  * runs before the host application's memory pool exists).  Such a caller can pass its inputs and
- * outputs but has nowhere to get the extra buffer that uoe_route needs for its pooled sums, scores and tickets.
+ * outputs but has nowhere to get the extra buffer that uoe_route needs for its partial scores and tickets.
  *
  * Here that buffer is a fixed array of UOE_ROUTE_STATIC_SCRATCH_BYTES compiled into the library's
  * device image, so every GPU on which the library is loaded holds that many bytes until the process
@@ -288,7 +288,7 @@ uoe_status uoe_block_forward(const uoe_problem* att, const uoe_problem* mlp, con
  *     give wrong routing: order them, or use uoe_route with separate workspaces.
  *   - No device status word is kept for this variant (uoe_read_device_status does not apply).
  */
-#define UOE_ROUTE_STATIC_SCRATCH_BYTES (8 << 20)
+#define UOE_ROUTE_STATIC_SCRATCH_BYTES (2 << 20)
 uoe_status uoe_route_static(const uoe_problem* prob, const void* x, const void* W_r,
                             int32_t* expert_idx /* [B,k] */, int32_t* patch_idx /* [B,k,c] */,
                             float* gate /* [B,k,c] */, float* p_samp /* [B,n] */, float* p_patch /* [B,n,m] */,

@@ -234,7 +234,7 @@ def uoe_route(prob: Problem, x, W_r, out: Routing | None = None, ws=None, check:
     return r
 
 
-UOE_ROUTE_STATIC_SCRATCH_BYTES = 8 << 20
+UOE_ROUTE_STATIC_SCRATCH_BYTES = 2 << 20
 
 
 def uoe_route_static(prob: Problem, x, W_r, out: Routing | None = None) -> Routing:

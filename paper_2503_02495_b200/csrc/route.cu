@@ -1,12 +1,11 @@
 // uoe_route: router scoring (Eq. 13-14, 21) and fused top-k expert / top-c patch selection (Eq. 17, 22-23).
-//   Every CTA streams one (patch, column chunk, row slice) of x with 16-byte loads and sums its rows per column.
-//   The CTA that completes a patch (a ticket per patch; none when the patch is one CTA's work) multiplies the
-//   pooled columns by W_r; the CTA that completes a sample (a ticket per sample) runs that sample's selection:
-//   both softmaxes, rank-based selection with warp ballots, gates; the CTA that completes the last sample turns
-//   the per-expert loads into row offsets.  One kernel for small inputs (64-thread CTAs when the patches are
-//   many and tiny); for large inputs a first kernel that only streams and a second with one CTA per patch.
-//   Tickets and loads are reset by their last user, so a scratch area whose control block was zeroed once
-//   (uoe_workspace_init, or the static array of uoe_route_static) serves any number of calls of any shapes.
+//   Every CTA streams one (patch, column chunk, row slice) of x with 16-byte loads, sums its rows per column and
+//   multiplies the sums by W_r, so that only scores leave the CTA.  The CTA that completes a sample (a ticket per
+//   sample) runs that sample's selection: both softmaxes, rank-based selection with warp ballots, gates; the CTA that
+//   completes the last sample turns the per-expert loads into row offsets.  One kernel for small inputs (64-thread
+//   CTAs when the patches are many and tiny); for large inputs a first kernel that only streams and a second with one
+//   CTA per sample.  Tickets and loads are reset by their last user, so a scratch area whose control block was
+//   zeroed once (uoe_workspace_init, or the static array of uoe_route_static) serves any number of calls of any shapes.
 // Also here: uoe_route_balance (Eq. 15-16, 42-44) and uoe_route_static.
 #include "kernels.cuh"
 
@@ -221,27 +220,26 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
     }
 }
 
-// Three steps, in one kernel (MODE 0) or two (MODE 1, then route_patch_scores_kernel):
-//   1. grid B*m * nchunks * rsplit, column chunk fastest: a CTA takes one column chunk of one row slice of a
-//      patch, sums its rows per column and stores the sums, pool_part[patch, row slice, column].  CTAs that run
-//      at the same time cover neighbouring chunks of the same rows, so together they read x linearly.  CT
-//      threads span the columns of the chunk (16 bytes each), 256/CT span rows.
-//   2. one CTA per patch (MODE 0: the CTA that completes the patch; else the second kernel) adds the row slices in
-//      fixed order and multiplies by W_r:  scores[patch, i] = sum over the patch's real tokens of x[t,:] . W_r[:,i]
-//   3. the CTA that completes a sample runs its selection (select_sample).
-// MODE 0 serves small inputs, where a second launch costs more than the work; two kernels serve large ones,
-// where step 1 should be nothing but streaming.
-// Dynamic shared memory: max(n*m floats for step 3, the blocks of W_r rows for step 2).
+// Scoring (Eq. 13, 21) and selection, in one kernel or two.  Grid B*m * nchunks * rsplit, column chunk fastest: a CTA
+// takes one column chunk of one row slice of a patch (CT threads span the columns of the chunk, 16 bytes each, NT/CT
+// span rows).  CTAs that run at the same time cover neighbouring chunks of the same rows, so together they read x
+// linearly.  The CTA first asks for the rows of W_r that belong to its columns (cp.async into shared memory, landing
+// behind the x loads), sums its rows of x per column, and multiplies the column sums by those rows: n partial scores,
+// score_part[patch, part, i], are all that leaves the CTA -- pooled activations never reach global memory.
+//   TICKET   the CTA that completes a sample (a ticket per sample, m * parts arrivals) runs its selection, which adds
+//            the parts in ascending order.  One launch: for small inputs.
+//   !TICKET  the kernel does nothing but stream and dot, and route_select_kernel (one CTA per sample) follows.  For
+//            large inputs, where a second launch costs less than CTAs that carry the selection code and its registers.
+// Dynamic shared memory: max(n*m floats for the selection, the CTA's block of W_r rows).
 
-template <typename T, int MODE, int NT>
-__global__ void __launch_bounds__(NT, NT == 64 ? 16 : (MODE == 1 ? 6 : 5))
-route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ pool_part,
-             float* __restrict__ scores, int B, int L, int Lv, int d, int n, int k, int m, int c, int l_p, int CT,
-             int nchunks, int rsplit, int rows_per_cta, int wblk_bytes, int use_gate,
+template <typename T, bool TICKET, int NT>
+__global__ void __launch_bounds__(NT, NT == 64 ? 16 : (TICKET ? 5 : 6))
+route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ scores, int B, int L, int Lv, int d,
+             int n, int k, int m, int c, int l_p, int CT, int nchunks, int rsplit, int rows_per_cta, int use_gate,
              int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
              float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
              int* __restrict__ ctl /* word 1: ticket, words 8..: expert loads */, int* __restrict__ sample_ticket /* [B] */,
-             int* __restrict__ patch_ticket /* [B*m] */, const PlanPtrs plan /* all null: no plan is written */) {
+             const PlanPtrs plan /* all null: no plan is written */) {
     pdl_trigger();
     pdl_wait();
     constexpr int V = Vec16<T>::N;
@@ -252,38 +250,25 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
     const int nparts = nchunks * rsplit;
     const int bj = blockIdx.x / nparts;
     const int b = bj / m, j = bj % m;
+    const int part = blockIdx.x % nparts;
+    const int chunk = part % nchunks, rs = part / nchunks;
+    const int c0 = chunk * CT * V, cw = min(CT * V, d - c0);          // this CTA's columns: [c0, c0 + cw)
 
-    // step 2 set-up (used by the CTA that completes a patch)
-    const int groups = NT / n;                    // thread (group g, expert i) strides over the columns
-    const int i = tid % n, g = tid / n;
-    int cb = (wblk_bytes / (n * (int)sizeof(T))) / V * V;
-    cb = min(cb, NT * V);
-    const int col_lo = 0, col_hi = d;
-    const int nblk = col_hi > col_lo ? (col_hi - col_lo + cb - 1) / cb : 0;
-    const float* pp_bj = pool_part + (size_t)bj * rsplit * d;
-    auto stage_w = [&](int blk) {
-        const int c0 = col_lo + blk * cb, cw = min(cb, col_hi - c0);
-        const uint4* src = (const uint4*)(W_r + (size_t)c0 * n);
-        uint4* dst = s_dyn4 + (blk & 1) * (wblk_bytes / 16);
+    {   // the W_r rows of these columns: cw * n consecutive elements (cw and the rows' start are multiples of V elements)
         const int nvec = cw * n * (int)sizeof(T) / 16;
+        const uint4* src = (const uint4*)(W_r + (size_t)c0 * n);
         for (int q = tid; q < nvec; q += NT)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(dst + q)), "l"(src + q) : "memory");
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(s_dyn4 + q)), "l"(src + q) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
-    };
-    // a patch that is one CTA's work (one part, all columns in one block) never leaves the CTA: its pooled sums
-    // stay in shared memory, no ticket is taken, and the W_r rows are fetched behind the x loads
-    const bool direct = MODE == 0 && nparts == 1 && d <= cb;
-    if (direct) stage_w(0);
+    }
 
+    // ---- column sums of this CTA's rows ----
+    const int ct = tid % CT, rt = tid / CT, RT = NT / CT;
+    const int col = c0 + ct * V;
+    float cs[V];
     {
-        // ---- 1. column sums of this CTA's rows ----
-        const int part = blockIdx.x % nparts;
-        const int chunk = part % nchunks, rs = part / nchunks;
-        const int ct = tid % CT, rt = tid / CT, RT = NT / CT;
-        const int col = (chunk * CT + ct) * V;
         const int row_lo = rs * rows_per_cta;
         const int rows = min(max(0, min(l_p, Lv - j * l_p)), row_lo + rows_per_cta);      // this slice: [row_lo, rows)
-        float cs[V];
 #pragma unroll
         for (int v = 0; v < V; ++v) cs[v] = 0.f;
         if (col < d) {
@@ -317,233 +302,113 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
 #pragma unroll
                     for (int v = 0; v < V; ++v) cs[v] += s_cs[(q * CT + ct) * V + v];
         }
-        if (direct) {
-            if (rt == 0 && col < d) {
-#pragma unroll
-                for (int v = 0; v < V; ++v) s_cs[col + v] = cs[v];      // slot 0 of this thread's own column group
-            }
-        } else {
-            if (rt == 0 && col < d) {
-                float4* dst = (float4*)(pool_part + ((size_t)bj * rsplit + rs) * d + col);
-#pragma unroll
-                for (int v = 0; v < V; v += 4) dst[v / 4] = make_float4(cs[v], cs[v + 1], cs[v + 2], cs[v + 3]);
-            }
-            if constexpr (MODE == 1) return;
-            __threadfence();
-            __syncthreads();
-            if (tid == 0) {
-                __threadfence();
-                s_mine = (atomicAdd(&patch_ticket[bj], 1) == nparts - 1);
-                if (s_mine) patch_ticket[bj] = 0;         // left at zero for the next call
-            }
-            __syncthreads();
-            if (!s_mine) return;
-            __threadfence();
-        }
     }
 
-    if constexpr (MODE != 1) {
-        // ---- 2. scores[bj, :] = pooled columns . W_r, W_r rows staged block
-        //         by block in shared memory (double-buffered when the range takes more than one block) ----
+    // ---- score_part[bj, part, :] = column sums . W_r rows, out of shared memory; thread (group g, expert i) strides
+    //      over the CTA's columns ----
+    if (rt == 0 && col < d) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) s_cs[ct * V + v] = cs[v];       // the slot this thread itself wrote above: no one else reads it
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    {
+        const int groups = NT / n;
+        const int i = tid % n, g = tid / n;
+        const T* s_w = (const T*)s_dyn4;
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        if (!direct && nblk > 0) stage_w(0);
-        for (int blk = 0; blk < nblk; ++blk) {
-            const int c0 = col_lo + blk * cb, cw = min(cb, col_hi - c0);
-            if (blk + 1 < nblk) stage_w(blk + 1);
-            for (int q4 = direct ? cw : tid; q4 < cw / 4; q4 += NT) {        // add the row slices, fixed order, loads batched by four
-                const float4* p0 = (const float4*)(pp_bj + c0) + q4;
-                float4 acc = __ldcg(p0);
-                for (int r0 = 1; r0 < rsplit; r0 += 4) {
-                    float4 t[4];
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (r0 + u < rsplit) t[u] = __ldcg((const float4*)((const float*)p0 + (size_t)(r0 + u) * d));
-#pragma unroll
-                    for (int u = 0; u < 4; ++u)
-                        if (r0 + u < rsplit) { acc.x += t[u].x; acc.y += t[u].y; acc.z += t[u].z; acc.w += t[u].w; }
-                }
-                *(float4*)(s_cs + 4 * q4) = acc;
+        if (g < groups) {           // four independent chains, then the tail: a fixed summation order
+            int cc = g;
+            for (; cc + 3 * groups < cw; cc += 4 * groups) {
+                a0 = fmaf(s_cs[cc], to_f32(s_w[cc * n + i]), a0);
+                a1 = fmaf(s_cs[cc + groups], to_f32(s_w[(cc + groups) * n + i]), a1);
+                a2 = fmaf(s_cs[cc + 2 * groups], to_f32(s_w[(cc + 2 * groups) * n + i]), a2);
+                a3 = fmaf(s_cs[cc + 3 * groups], to_f32(s_w[(cc + 3 * groups) * n + i]), a3);
             }
-            if (blk + 1 < nblk) asm volatile("cp.async.wait_group 1;" ::: "memory");
-            else asm volatile("cp.async.wait_group 0;" ::: "memory");
-            __syncthreads();
-            const T* s_w = (const T*)(s_dyn4 + (blk & 1) * (wblk_bytes / 16));
-            if (g < groups) {           // four independent chains, then the tail: a fixed summation order
-                int cc = g;
-                for (; cc + 3 * groups < cw; cc += 4 * groups) {
-                    a0 = fmaf(s_cs[cc], to_f32(s_w[cc * n + i]), a0);
-                    a1 = fmaf(s_cs[cc + groups], to_f32(s_w[(cc + groups) * n + i]), a1);
-                    a2 = fmaf(s_cs[cc + 2 * groups], to_f32(s_w[(cc + 2 * groups) * n + i]), a2);
-                    a3 = fmaf(s_cs[cc + 3 * groups], to_f32(s_w[(cc + 3 * groups) * n + i]), a3);
-                }
-                for (; cc < cw; cc += groups) a0 = fmaf(s_cs[cc], to_f32(s_w[cc * n + i]), a0);
-            }
-            __syncthreads();
+            for (; cc < cw; cc += groups) a0 = fmaf(s_cs[cc], to_f32(s_w[cc * n + i]), a0);
         }
+        __syncthreads();
         s_cs[tid] = (a0 + a1) + (a2 + a3);
         __syncthreads();
         if (tid < n) {
             float sum = 0.f;
             for (int q = 0; q < groups; ++q) sum += s_cs[q * n + tid];
-            scores[(size_t)bj * n + tid] = sum;
+            scores[((size_t)bj * nparts + part) * n + tid] = sum;
             __threadfence();
         }
+    }
+    if constexpr (TICKET) {
         __syncthreads();
         if (tid == 0) {
             __threadfence();
-            s_mine = (atomicAdd(&sample_ticket[b], 1) == m - 1);
-            if (s_mine) sample_ticket[b] = 0;
+            s_mine = (atomicAdd(&sample_ticket[b], 1) == m * nparts - 1);
+            if (s_mine) sample_ticket[b] = 0;         // left at zero for the next call
         }
         __syncthreads();
         if (!s_mine) return;
         __threadfence();
-        // ---- 3. this CTA completed sample b ----
-        select_sample<NT>((float*)s_dyn4, scores, 1, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
-                      p_patch, offsets, ctl + 8, ctl + 1, plan);
+        // ---- this CTA completed sample b ----
+        select_sample<NT>((float*)s_dyn4, scores, nparts, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
+                          p_patch, offsets, ctl + 8, ctl + 1, plan);
     }
 }
 
-// Steps 2 and 3 as a kernel of their own (after a MODE 1 launch): grid B*m, one CTA per patch.  Thread t owns
-// columns t, t + 256, ...: it adds the row slices of pool_part for its column (fixed order), reads that column's
-// row of W_r (n consecutive elements) and accumulates one partial score per expert in registers; the CTA then
-// reduces the partials in a fixed order.  NMAX >= n bounds the register tile.
-template <typename T, int NMAX>
+// Selection as a kernel of its own (after a route_kernel launch without tickets): grid B, one CTA per sample.
 __global__ void __launch_bounds__(kScoreThreads)
-route_patch_scores_kernel(const T* __restrict__ W_r, const float* __restrict__ pool_part, float* __restrict__ scores,
-                          int B, int Lv, int d, int n, int k, int m, int c, int l_p, int rsplit, int use_gate,
-                          int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
-                          float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
-                          int* __restrict__ ctl, int* __restrict__ sample_ticket, const PlanPtrs plan) {
+route_select_kernel(const float* __restrict__ scores, int nparts, int B, int Lv, int n, int k, int m, int c, int l_p,
+                    int use_gate, int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
+                    float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
+                    int* __restrict__ ctl, const PlanPtrs plan) {
     pdl_trigger();
     pdl_wait();
-    constexpr int NT = kScoreThreads;
-    constexpr int V = Vec16<T>::N;
     extern __shared__ float s_sel[];
-    __shared__ float s_red[NT / 32][NMAX];
-    __shared__ int s_mine;
-    const int bj = blockIdx.x, b = bj / m, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const float* pp_bj = pool_part + (size_t)bj * rsplit * d;
-    const bool vec_rows = (n % V) == 0;           // a row of W_r is a whole number of 16-byte pieces
-    float acc[NMAX];
-#pragma unroll
-    for (int i = 0; i < NMAX; ++i) acc[i] = 0.f;
-    // four columns per round: every load of a round (row slices in batches of four, W_r rows) is issued before
-    // the first use, so a round costs one trip to L2 / HBM
-    for (int c0 = tid; c0 < d; c0 += 4 * NT) {
-        float p[4] = {0.f, 0.f, 0.f, 0.f};
-        uint4 wv[4][NMAX / V];
-        if (vec_rows) {
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-                for (int q = 0; q < NMAX / V; ++q)
-                    if (c0 + u * NT < d && q * V < n) wv[u][q] = *(const uint4*)(W_r + (size_t)(c0 + u * NT) * n + q * V);
-        }
-        for (int r0 = 0; r0 < rsplit; r0 += 4) {
-            float t[4][4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-                for (int r = 0; r < 4; ++r)
-                    t[u][r] = (c0 + u * NT < d && r0 + r < rsplit) ? __ldcg(pp_bj + (size_t)(r0 + r) * d + c0 + u * NT) : 0.f;
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-#pragma unroll
-                for (int r = 0; r < 4; ++r) p[u] += t[u][r];       // ascending slice order
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (c0 + u * NT >= d) continue;
-            if (vec_rows) {
-#pragma unroll
-                for (int q = 0; q < NMAX / V; ++q) {
-                    if (q * V < n) {
-                        float f[V];
-                        unpack16<T>(wv[u][q], f);
-#pragma unroll
-                        for (int v = 0; v < V; ++v) acc[q * V + v] = fmaf(p[u], f[v], acc[q * V + v]);
-                    }
-                }
-            } else {
-                const T* wrow = W_r + (size_t)(c0 + u * NT) * n;
-#pragma unroll
-                for (int i = 0; i < NMAX; ++i)
-                    if (i < n) acc[i] = fmaf(p[u], to_f32(wrow[i]), acc[i]);
-            }
-        }
-    }
-#pragma unroll
-    for (int i = 0; i < NMAX; ++i) {
-        float v = acc[i];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-        if (lane == 0) s_red[warp][i] = v;
-    }
-    __syncthreads();
-    if (tid < n) {
-        float sum = 0.f;
-        for (int q = 0; q < NT / 32; ++q) sum += s_red[q][tid];
-        scores[(size_t)bj * n + tid] = sum;
-        __threadfence();
-    }
-    __syncthreads();
-    if (tid == 0) {
-        __threadfence();
-        s_mine = (atomicAdd(&sample_ticket[b], 1) == m - 1);
-        if (s_mine) sample_ticket[b] = 0;
-    }
-    __syncthreads();
-    if (!s_mine) return;
-    __threadfence();
-    select_sample<kScoreThreads>(s_sel, scores, 1, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch,
-                  offsets, ctl + 8, ctl + 1, plan);
+    select_sample<kScoreThreads>(s_sel, scores, nparts, blockIdx.x, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate,
+                                 p_samp, p_patch, offsets, ctl + 8, ctl + 1, plan);
 }
 
-struct RouteWs { size_t tickets, ptickets, scores, pool, total; int nchunks, CT, rsplit, rows_per_cta, wblk_bytes; size_t smem; bool two_kernels, small_ctas; };
+struct RouteWs { size_t tickets, scores, total; int nchunks, CT, rsplit, rows_per_cta; size_t smem, wb; bool two_kernels, small_ctas; };
+
+constexpr int kWblkBytes = 16384;       // shared memory for a CTA's rows of W_r
 
 RouteWs route_ws(const Dims& D) {
     const int V = 16 / D.esize;
     int CT = kScoreThreads;
-    while (CT > 1 && (CT / 2) * V >= D.d) CT /= 2;
+    // the fewest column threads that still cover d, and few enough that their rows of W_r fit the staging block
+    while (CT > 1 && ((CT / 2) * V >= D.d || (size_t)CT * V * D.n * D.esize > (size_t)kWblkBytes)) CT /= 2;
     const int nchunks = (D.d + CT * V - 1) / (CT * V);
     const int rows_per_cta = 32 * (kScoreThreads / CT);       // at most four 8-deep load batches per thread
     const int rsplit = (D.l_p + rows_per_cta - 1) / rows_per_cta;
-    // The control block has a fixed size whatever the problem: status block, then the sample and patch tickets.
-    // Data starts behind it, so no problem shape ever writes data where another shape keeps its tickets, and a
-    // scratch area zeroed once serves calls of any shapes in any order.
+    // The control block has a fixed size whatever the problem: status block, then the sample tickets.  Data starts
+    // behind it, so no problem shape ever writes data where another shape keeps its tickets, and a scratch area
+    // zeroed once serves calls of any shapes in any order.
     RouteWs r;
     r.tickets = kStatusBytes;
-    r.ptickets = r.tickets + (size_t)D.B * sizeof(int);
     WsCarver w;
     w.take(kControlBytes);
-    // a second launch pays off once step 1 moves enough bytes that it should do nothing but stream; its step-2
-    // CTAs each take a column range whose W_r rows fit one block
+    // a second launch pays off once the first moves enough bytes that it should do nothing but stream
     r.two_kernels = nchunks * rsplit > 1 && (size_t)D.B * D.L * D.d * D.esize >= ((size_t)64 << 20);
-    r.wblk_bytes = 16384;
-    r.scores = w.take((size_t)D.B * D.m * D.n * sizeof(float));
-    r.pool = w.take((size_t)D.B * D.m * rsplit * D.d * sizeof(float));
+    r.scores = w.take((size_t)D.B * D.m * nchunks * rsplit * D.n * sizeof(float));
     r.rsplit = rsplit;
     r.rows_per_cta = rows_per_cta;
     r.total = w.off;
     r.nchunks = nchunks;
     r.CT = CT;
     const size_t sel = (size_t)D.n * D.m * sizeof(float);
-    size_t wb = (r.two_kernels ? 1 : 2) * (size_t)r.wblk_bytes;
+    r.wb = (size_t)(CT * V < D.d ? CT * V : D.d) * D.n * D.esize;
     // Many small patches (a patch is one CTA's work and a few KB): 64-thread CTAs with exactly the shared memory they
     // need, so that all of them are resident at once and the per-CTA chain (loads, dots, ticket) is paid once.
-    r.small_ctas = !r.two_kernels && nchunks == 1 && rsplit == 1 && D.d <= 64 * V && D.l_p <= 32 &&
-                   (size_t)D.d * D.n * D.esize <= (size_t)r.wblk_bytes && (long long)D.B * D.m >= 1024;
+    r.small_ctas = nchunks * rsplit == 1 && D.d <= 64 * V && D.l_p <= 32 && (size_t)D.d * D.n * D.esize <= (size_t)kWblkBytes &&
+                   (long long)D.B * D.m >= 1024;
     if (r.small_ctas) {
         r.CT = 64;
         r.rows_per_cta = D.l_p;
-        wb = ((size_t)D.d * D.n * D.esize + 15) / 16 * 16;
     }
-    r.smem = sel > wb ? sel : wb;
+    r.smem = r.two_kernels ? r.wb : (sel > r.wb ? sel : r.wb);
     return r;
 }
 
-// The launch shared by uoe_route and uoe_route_static.  `base` is the scratch (control block with the tickets,
-// scores, pooled sums); its control block must have been zero when first used.
+// The launch shared by uoe_route and uoe_route_static.  `base` is the scratch (control block with the tickets, then
+// the scores); its control block must have been zero when first used.
 uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void* W_r, int32_t* expert_idx,
                         int32_t* patch_idx, float* gate, float* p_samp, float* p_patch, int32_t* expert_offsets,
                         char* base, const RouteWs& W, cudaStream_t stream, bool profile, const PlanPtrs& plan = PlanPtrs()) {
@@ -552,55 +417,34 @@ uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void
     const size_t smem0 = W.smem > plan_smem ? W.smem : plan_smem;
     int* ctl = (int*)base;             // word 0 status (unused here), word 1 ticket, words 8.. expert loads
     int* tickets = (int*)(base + W.tickets);
-    int* ptickets = (int*)(base + W.ptickets);
     float* scores = (float*)(base + W.scores);
-    float* pool = (float*)(base + W.pool);
     const int use_gate = ((flags & UOE_FLAG_GATE) ? 1 : 0) | ((flags & UOE_FLAG_DYNAMIC_C) ? 2 : 0);     // selection flags
-    dim3 grid((unsigned)(D.B * D.m * W.nchunks * W.rsplit)), grid2((unsigned)(D.B * D.m));
-#define UOE_ROUTE_ARGS(T) (const T*)x, (const T*)W_r, pool, scores, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, \
-        W.nchunks, W.rsplit, W.rows_per_cta, W.wblk_bytes, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, \
-        tickets, ptickets, plan
+    dim3 grid((unsigned)(D.B * D.m * W.nchunks * W.rsplit));
+#define UOE_ROUTE_ARGS(T) (const T*)x, (const T*)W_r, scores, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, \
+        W.nchunks, W.rsplit, W.rows_per_cta, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, \
+        tickets, plan
+#define UOE_ROUTE_LAUNCH(T, TICKET, NT, SMEM) \
+        launch_k(route_kernel<T, TICKET, NT>, grid, dim3(NT), SMEM, stream, UOE_ROUTE_ARGS(T))
     cudaError_t e;
-    if (!W.two_kernels) {
-        ProfScope ps(profile ? "route" : nullptr, stream);
-        if (W.small_ctas) {
-            if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0, 64>, grid, dim3(64), smem0, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
-            else e = launch_k(route_kernel<float, 0, 64>, grid, dim3(64), smem0, stream, UOE_ROUTE_ARGS(float));
-        } else {
-            if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 0, kScoreThreads>, grid, dim3(kScoreThreads), smem0, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
-            else e = launch_k(route_kernel<float, 0, kScoreThreads>, grid, dim3(kScoreThreads), smem0, stream, UOE_ROUTE_ARGS(float));
-        }
-        if (e != cudaSuccess) return UOE_ERR_CUDA;
-        UOE_LAUNCHED();
-        return UOE_OK;
-    }
     {
         ProfScope ps(profile ? "route" : nullptr, stream);
-        if (D.bf16) e = launch_k(route_kernel<__nv_bfloat16, 1, kScoreThreads>, grid, dim3(kScoreThreads), 0, stream, UOE_ROUTE_ARGS(__nv_bfloat16));
-        else e = launch_k(route_kernel<float, 1, kScoreThreads>, grid, dim3(kScoreThreads), 0, stream, UOE_ROUTE_ARGS(float));
+        if (W.two_kernels) e = D.bf16 ? UOE_ROUTE_LAUNCH(__nv_bfloat16, false, kScoreThreads, W.smem) : UOE_ROUTE_LAUNCH(float, false, kScoreThreads, W.smem);
+        else if (W.small_ctas) e = D.bf16 ? UOE_ROUTE_LAUNCH(__nv_bfloat16, true, 64, smem0) : UOE_ROUTE_LAUNCH(float, true, 64, smem0);
+        else e = D.bf16 ? UOE_ROUTE_LAUNCH(__nv_bfloat16, true, kScoreThreads, smem0) : UOE_ROUTE_LAUNCH(float, true, kScoreThreads, smem0);
     }
+#undef UOE_ROUTE_LAUNCH
+#undef UOE_ROUTE_ARGS
     if (e != cudaSuccess) return UOE_ERR_CUDA;
     UOE_LAUNCHED();
+    if (!W.two_kernels) return UOE_OK;
     {
         ProfScope ps(profile ? "route_select" : nullptr, stream);
         size_t sel = (size_t)D.n * D.m * sizeof(float);
         if (sel < plan_smem) sel = plan_smem;
-#define UOE_SCORE_ARGS(T) (const T*)W_r, pool, scores, D.B, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.rsplit, use_gate, expert_idx, \
-        patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, tickets, plan
-#define UOE_SCORE_LAUNCH(T, NMAX) launch_k(route_patch_scores_kernel<T, NMAX>, grid2, dim3(kScoreThreads), sel, stream, UOE_SCORE_ARGS(T))
-        if (D.bf16) {
-            if (D.n <= 8) e = UOE_SCORE_LAUNCH(__nv_bfloat16, 8);
-            else if (D.n <= 16) e = UOE_SCORE_LAUNCH(__nv_bfloat16, 16);
-            else e = UOE_SCORE_LAUNCH(__nv_bfloat16, 32);
-        } else {
-            if (D.n <= 8) e = UOE_SCORE_LAUNCH(float, 8);
-            else if (D.n <= 16) e = UOE_SCORE_LAUNCH(float, 16);
-            else e = UOE_SCORE_LAUNCH(float, 32);
-        }
-#undef UOE_SCORE_LAUNCH
-#undef UOE_SCORE_ARGS
+        e = launch_k(route_select_kernel, dim3(D.B), dim3(kScoreThreads), sel, stream, (const float*)scores, W.nchunks * W.rsplit,
+                     D.B, D.Lv, D.n, D.k, D.m, D.c, D.l_p, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch,
+                     expert_offsets, ctl, plan);
     }
-#undef UOE_ROUTE_ARGS
     if (e != cudaSuccess) return UOE_ERR_CUDA;
     UOE_LAUNCHED();
     return UOE_OK;
@@ -617,7 +461,7 @@ uoe_status route_check(const uoe_problem* prob, Dims& D, RouteWs& W, const void*
     if ((size_t)D.n * D.m * sizeof(float) > 36 * 1024) return UOE_ERR_UNSUPPORTED;   // gate values of a sample in shared memory
     W = route_ws(D);
     if ((long long)D.B * D.m * W.nchunks * W.rsplit > 0x7fffffffll) return UOE_ERR_UNSUPPORTED;
-    if (W.ptickets + (size_t)D.B * D.m * sizeof(int) > kControlBytes) return UOE_ERR_UNSUPPORTED;   // tickets must fit the control block
+    if (W.tickets + (size_t)D.B * sizeof(int) > kControlBytes) return UOE_ERR_UNSUPPORTED;   // tickets must fit the control block
     return UOE_OK;
 }
 

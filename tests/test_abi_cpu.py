@@ -85,8 +85,8 @@ def test_every_entry_point_validates_on_the_host(uoe):
     ok_rope = uoe.Problem(B=2, L=256, L_valid=256, d=256, n=4, k=2, m=8, c=4, H=4, d_h=64, d_rope=32)
     assert uoe.uoe_workspace_bytes(ok_rope, uoe.UOE_OP_SMHA_FWD) > 0
     assert uoe.uoe_workspace_bytes(ok_rope, uoe.UOE_OP_SMHA_BWD) > uoe.uoe_workspace_bytes(ok_rope, uoe.UOE_OP_SMHA_FWD)
-    # the router's tickets live in a fixed control block: more patches than it holds is "unsupported", not a fault
-    huge = uoe.Problem(B=70000, L=64, L_valid=64, d=64, n=4, k=2, m=8, c=4, d_e=64).c_struct()
+    # the router's tickets live in a fixed control block: more samples than it holds is "unsupported", not a fault
+    huge = uoe.Problem(B=300000, L=64, L_valid=64, d=64, n=4, k=2, m=8, c=4, d_e=64).c_struct()
     dummy = ctypes.c_void_p(4096)        # non-null, 16-byte aligned, never dereferenced: validation fails first
     lib.uoe_route.restype = ctypes.c_int
     st = lib.uoe_route(ctypes.byref(huge), dummy, dummy, dummy, dummy, dummy, dummy, dummy, dummy, dummy,
