@@ -24,7 +24,6 @@ struct PlanPtrs {
     int* src_patch = nullptr;    // [Rmax/l_p] source patch (b*m + j) of every l_p-row block of the routed buffers, -1 = zero rows
     int* slot_pair = nullptr;    // [n,B]    plan written by the router kernel: pair (b*k + s) of the q-th sample in expert i's
                                  //          region (it replaces src_patch, which that plan does not fill)
-    unsigned* sample_mask = nullptr;   // [B]  plan written by the router kernel: chosen experts of every sample as a bit set
     bool inv_relative = false;   // inv_row holds offsets from pair_row (plan written by the router kernel)
     // plan written by the router kernel only: a routed buffer whose first rows past the last expert region are
     // zero-filled (up to 128 of them, as many as a 128-row tile that starts inside the last region can reach)
@@ -56,7 +55,7 @@ inline bool can_fuse_gather(const Dims& D) {
 inline size_t plan_bytes(const Dims& D, bool with_rows = false) {
     return align_up((size_t)D.B * D.k * 4, 1024) + 2 * align_up((size_t)D.B * D.m * D.k * 4, 1024) + 1024 +
            (with_rows ? 2 * align_up((size_t)D.Rmax * 4, 1024) : 0) + align_up((size_t)(D.Rmax / D.l_p + 1) * 4, 1024) +
-           align_up((size_t)D.n * D.B * 4, 1024) + align_up((size_t)D.B * 4, 1024);
+           align_up((size_t)D.n * D.B * 4, 1024);
 }
 inline PlanPtrs plan_ptrs(const Dims& D, char* base, bool with_rows = false) {
     PlanPtrs p;
@@ -75,8 +74,6 @@ inline PlanPtrs plan_ptrs(const Dims& D, char* base, bool with_rows = false) {
     p.src_patch = (int*)base;
     base += align_up((size_t)(D.Rmax / D.l_p + 1) * 4, 1024);
     p.slot_pair = (int*)base;
-    base += align_up((size_t)D.n * D.B * 4, 1024);
-    p.sample_mask = (unsigned*)base;
     return p;
 }
 

@@ -18,80 +18,85 @@ namespace {
 constexpr int kScoreThreads = 256;
 
 // Selection for sample b by one CTA of NT threads (all threads call).  pp: n*m floats of shared memory.
+// Written for a short dependent chain (the router is latency-bound on all but the largest inputs): three phases
+// separated by CTA barriers, then the ticket.
+//   A  a warp works 32/np2 patches at a time (np2 = n rounded up to a power of two), one lane per (patch, expert):
+//      adds the parts of the score in ascending order, softmax over the experts of the patch through segment
+//      shuffles (Eq. 14), first-stage counts of Eq. 15 when the capacity is dynamic; the raw scores are summed per
+//      expert on the side for the sample gate
+//   B  warp 0: sample gate (Eq. 21), top-k experts (Eq. 22); the other warps write p_patch
+//   C  a warp per chosen expert: top-c patches by rank counting (Eq. 17), gates, the inverse map of the plan
+// The CTA that completes the last sample (a ticket) turns every sample's expert set (one bit mask per sample, masks[B]
+// in the scratch area) into per-expert row offsets (Eq. 23) and, for the plan, each pair's first row.
 template <int NT>
 __device__ void select_sample(float* pp, const float* __restrict__ partial, int nparts, int b, int B, int Lv, int n, int k,
                               int m, int c, int l_p, int sel_flags /* bit 0: gate weights, bit 1: dynamic capacity */,
                               int* __restrict__ expert_idx,
                               int* __restrict__ patch_idx, float* __restrict__ gate, float* __restrict__ p_samp,
-                              float* __restrict__ p_patch, int* __restrict__ offsets, int* __restrict__ load,
+                              float* __restrict__ p_patch, int* __restrict__ offsets, unsigned* __restrict__ masks,
                               int* __restrict__ ticket, const PlanPtrs plan) {
+    constexpr int NW = NT / 32;
+    constexpr int kMaskCache = 1024;       // samples whose masks the last CTA keeps in shared memory
     __shared__ float ps[32];               // sample gate
+    __shared__ float s_raw[NW][32];        // per warp: sum over its patches of the raw scores, per expert
     __shared__ int sel[32];                // chosen experts, ascending
-    __shared__ int cnts[32];               // Eq. 16: patches each expert receives in the first routing stage
+    __shared__ int cnts[32];               // Eq. 16: patches each expert receives in the first routing stage; later: samples per expert
     __shared__ int s_last;
+    __shared__ unsigned s_masks[kMaskCache];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int use_gate = sel_flags & 1, dynamic_c = (sel_flags >> 1) & 1;
     if (tid < 32) cnts[tid] = 0;
     const int n_elig = (Lv + l_p - 1) / l_p;       // patches holding at least one real token (a prefix)
+    int np2 = 1;
+    while (np2 < n) np2 <<= 1;
+    const int G = 32 / np2;                         // patches a warp works at a time
+    if (dynamic_c) __syncthreads();                 // cnts is zero before the first count
 
-    for (int idx = tid; idx < n * m; idx += NT) {
-        const int i = idx / m, j = idx % m;
-        const float* p = partial + ((size_t)(b * m + j) * nparts) * n + i;
-        float s = 0.f;
-        for (int ch = 0; ch < nparts; ++ch) s += __ldcg(p + (size_t)ch * n);     // written by other CTAs: read from L2
-        pp[idx] = s;
-    }
-    __syncthreads();
-    if (tid < n) {                          // Eq. 21: mean over the real tokens, then W_r
-        float s = 0.f;
-        for (int j = 0; j < m; ++j) s += pp[tid * m + j];
-        ps[tid] = s / (float)Lv;
-    }
-    __syncthreads();
-    // Eq. 14: softmax over the experts of every patch.  The exponentials and divisions run one element per thread; the
-    // per-patch maximum and sum (ascending expert order) one patch per thread.
-    __shared__ float colstat[1024];         // per patch: maximum, then sum
-    for (int idx = tid; idx < n * m; idx += NT) {
-        const int j = idx % m;
-        const int cnt = max(0, min(l_p, Lv - j * l_p));
-        pp[idx] = cnt > 0 ? pp[idx] / (float)cnt : 0.f;
-    }
-    __syncthreads();
-    for (int j = tid; j < m; j += NT) {
-        float mx = -INFINITY;
-        for (int i = 0; i < n; ++i) mx = fmaxf(mx, pp[i * m + j]);
-        colstat[j] = mx;
-    }
-    __syncthreads();
-    for (int idx = tid; idx < n * m; idx += NT) pp[idx] = expf(pp[idx] - colstat[idx % m]);
-    __syncthreads();
-    for (int j = tid; j < m; j += NT) {
-        float sum = 0.f;
-        for (int i = 0; i < n; ++i) sum += pp[i * m + j];
-        colstat[j] = sum;
-    }
-    __syncthreads();
-    for (int idx = tid; idx < n * m; idx += NT) {
-        const float pr = pp[idx] / colstat[idx % m];
-        pp[idx] = pr;
-        p_patch[(size_t)b * n * m + idx] = pr;
-    }
-    __syncthreads();
-    if (dynamic_c) {                        // Eq. 15: every real patch goes to its k best experts (ties: lower index)
-        for (int j = tid; j < n_elig; j += NT) {
-            for (int i = 0; i < n; ++i) {
-                const float v = pp[i * m + j];
+    // ---- A ----
+    {
+        const int seg = lane / np2, i = lane % np2, seg_base = lane - i;
+        float raw_acc = 0.f;
+        for (int j0 = warp * G; j0 < m; j0 += NW * G) {
+            const int j = j0 + seg;
+            const bool valid = j < m && i < n;
+            float s = 0.f;
+            if (valid) {
+                const float* p = partial + ((size_t)(b * m + j) * nparts) * n + i;
+                for (int ch = 0; ch < nparts; ++ch) s += __ldcg(p + (size_t)ch * n);     // written by other CTAs: read from L2
+            }
+            raw_acc += s;
+            const int cnt = valid ? max(0, min(l_p, Lv - j * l_p)) : 0;
+            const float g = valid ? (cnt > 0 ? s / (float)cnt : 0.f) : -INFINITY;       // Eq. 13: mean over the patch's real tokens
+            float mx = g;
+            for (int o = np2 >> 1; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            const float e = valid ? expf(g - mx) : 0.f;
+            float sum = e;
+            for (int o = np2 >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            const float pr = e / sum;                    // (lanes outside the problem: 0/0, never used)
+            if (valid) pp[i * m + j] = pr;
+            if (dynamic_c) {                        // Eq. 15: every real patch goes to its k best experts (ties: lower index)
                 int rank = 0;
                 for (int q = 0; q < n; ++q) {
-                    const float w = pp[q * m + j];
-                    rank += (w > v) || (w == v && q < i);
+                    const float w = __shfl_sync(0xffffffffu, pr, seg_base + q);
+                    rank += (w > pr) || (w == pr && q < i);
                 }
-                if (rank < k) atomicAdd(&cnts[i], 1);
+                if (valid && j < n_elig && rank < k) atomicAdd(&cnts[i], 1);
             }
         }
+        for (int o = np2; o < 32; o <<= 1) raw_acc += __shfl_xor_sync(0xffffffffu, raw_acc, o);     // over the warp's segments
+        if (lane < n) s_raw[warp][lane] = raw_acc;
     }
+    __syncthreads();
+
+    // ---- B ----
     if (warp == 0) {
-        const float v = lane < n ? ps[lane] : -INFINITY;
+        float v = -INFINITY;
+        if (lane < n) {                         // Eq. 21: mean over the real tokens, then W_r
+            float s = 0.f;
+#pragma unroll
+            for (int q = 0; q < NW; ++q) s += s_raw[q][lane];
+            v = s / (float)Lv;
+        }
         float mx = v;
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -113,18 +118,23 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
             const int s = __popc(mask & ((1u << lane) - 1u));
             sel[s] = lane;
             expert_idx[(size_t)b * k + s] = lane;
-            atomicAdd(&load[lane], 1);
         }
-        if (lane == 0 && plan.sample_mask) plan.sample_mask[b] = mask;
+        if (lane == 0) masks[b] = mask;
+    }
+    if (NW == 1 || warp > 0) {
+        const int t0 = NW == 1 ? tid : tid - 32, nt = NW == 1 ? NT : NT - 32;
+        for (int idx = t0; idx < n * m; idx += nt) p_patch[(size_t)b * n * m + idx] = pp[idx];
     }
     __syncthreads();
+
+    // ---- C ----
     int take = min(c, n_elig);
     if (dynamic_c) {                        // Eq. 16: c = the largest first-stage count, capped by the slots available
         int c_dyn = 0;
         for (int i = 0; i < n; ++i) c_dyn = max(c_dyn, cnts[i]);
         take = min(take, c_dyn);
     }
-    for (int s = warp; s < k; s += NT / 32) {       // Eq. 17 for the s-th chosen expert
+    for (int s = warp; s < k; s += NW) {            // Eq. 17 for the s-th chosen expert
         const int i = sel[s];
         const float* v_i = pp + i * m;
         int* out_idx = patch_idx + ((size_t)b * k + s) * c;
@@ -135,11 +145,13 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
             const bool valid = j < n_elig;
             const float v = valid ? v_i[j] : 0.f;
             int rank = 0;
-            if (valid)
-                for (int jj = 0; jj < n_elig; ++jj) {
-                    const float w = v_i[jj];
-                    rank += (w > v) || (w == v && jj < j);
-                }
+            for (int jj0 = 0; jj0 < n_elig; jj0 += 8) {      // eight broadcast reads at a time
+                float w[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) w[u] = jj0 + u < n_elig ? v_i[jj0 + u] : -INFINITY;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) rank += (w[u] > v) || (w[u] == v && jj0 + u < j);
+            }
             const bool pick = valid && rank < take;
             const unsigned mask = __ballot_sync(0xffffffffu, pick);
             const int pos = before + __popc(mask & ((1u << lane) - 1u));
@@ -161,60 +173,64 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
                 plan.inv_gate[((size_t)b * m + j) * k + s] = 0.f;
             }
     }
-    // Eq. 23 as row offsets: the CTA that completes the last sample turns the loads into a prefix sum
+
+    // ---- the CTA that completes the last sample: Eq. 23 as row offsets, and the part of the routing plan that needs
+    //      every sample's choice (where every pair's rows start, which pair owns every slot of every expert's region) ----
     __syncthreads();
     if (tid == 0) {
         __threadfence();
         s_last = (atomicAdd(ticket, 1) == B - 1);
     }
     __syncthreads();
-    __shared__ int s_offs[34];
-    if (s_last && warp == 0) {
-        __threadfence();
-        const int rows_per_pair = c * l_p;
-        int rows = 0;
-        if (lane < n) {
-            rows = (__ldcg(load + lane) * rows_per_pair + UOE_ROW_ALIGN - 1) / UOE_ROW_ALIGN * UOE_ROW_ALIGN;
-            load[lane] = 0;                 // left at zero for the next call
+    if (!s_last) return;
+    __threadfence();
+    if (tid == 0) *ticket = 0;              // left at zero for the next call
+    if (tid < 32) cnts[tid] = 0;
+    __syncthreads();
+    for (int b2 = tid; b2 < B; b2 += NT) {           // samples per expert
+        unsigned mk = __ldcg(masks + b2);
+        if (b2 < kMaskCache) s_masks[b2] = mk;
+        while (mk) {
+            const int i = __ffs(mk) - 1;
+            mk &= mk - 1;
+            atomicAdd(&cnts[i], 1);
         }
-        if (lane == 0) *ticket = 0;
-        int incl = rows;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const int v = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += v;
-        }
-        if (lane < n) { offsets[lane] = incl - rows; s_offs[lane] = incl - rows; }
-        if (lane == n - 1) { offsets[n] = incl; s_offs[n] = incl; }
     }
-    // The part of the routing plan that needs every sample's choice, by the same CTA: where every pair's rows start
-    // and which pair owns every slot of every expert's region.  One pass over the samples' expert sets per expert
-    // (a warp per expert, 32 samples per step), so rows inside a region ascend with the sample.
-    if (plan.pair_row && s_last) {
-        unsigned* s_mask = (unsigned*)pp;           // [B] (pp is free now)
-        __syncthreads();
-        for (int b2 = tid; b2 < B; b2 += NT) s_mask[b2] = __ldcg(plan.sample_mask + b2);
-        __syncthreads();
-        const int l_a = c * l_p;
-        for (int i = warp; i < n; i += NT / 32) {
+    __syncthreads();
+    const int l_a = c * l_p;
+    const int rows = lane < n ? (cnts[lane] * l_a + UOE_ROW_ALIGN - 1) / UOE_ROW_ALIGN * UOE_ROW_ALIGN : 0;
+    int incl = rows;                        // every warp scans for itself
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    const int total_rows = __shfl_sync(0xffffffffu, incl, n - 1);
+    if (warp == 0) {
+        if (lane < n) offsets[lane] = incl - rows;
+        if (lane == 0) offsets[n] = total_rows;
+    }
+    if (plan.pair_row) {                    // a warp per expert, 32 samples per step: rows inside a region ascend with the sample
+        for (int i = warp; i < n; i += NW) {
+            const int off_i = __shfl_sync(0xffffffffu, incl - rows, i);
             int running = 0;
             for (int b0 = 0; b0 < B; b0 += 32) {
                 const int b2 = b0 + lane;
-                const unsigned mk = b2 < B ? s_mask[b2] : 0u;
+                const unsigned mk = b2 < B ? (b2 < kMaskCache ? s_masks[b2] : __ldcg(masks + b2)) : 0u;
                 const bool mine = (mk >> i) & 1u;
                 const unsigned ball = __ballot_sync(0xffffffffu, mine);
                 if (mine) {        // the chosen experts of a sample ascend: expert i sits in slot #(chosen experts below i)
                     const int s = __popc(mk & ((1u << i) - 1u));
                     const int q = running + __popc(ball & ((1u << lane) - 1u));
-                    plan.pair_row[(size_t)b2 * k + s] = s_offs[i] + q * l_a;
+                    plan.pair_row[(size_t)b2 * k + s] = off_i + q * l_a;
                     plan.slot_pair[(size_t)i * B + q] = b2 * k + s;
                 }
                 running += __popc(ball);
             }
-            if (lane == 0) plan.expert_end[i] = s_offs[i] + running * l_a;
+            if (lane == 0) plan.expert_end[i] = off_i + running * l_a;
         }
         if (plan.tail) {
-            const long long r0 = s_offs[n], r1 = min(plan.rows_max, r0 + 128);
+            const long long r0 = total_rows, r1 = min(plan.rows_max, r0 + 128);
             for (long long q = tid; q < (r1 - r0) * plan.tail_row_vecs; q += NT) plan.tail[r0 * plan.tail_row_vecs + q] = make_uint4(0, 0, 0, 0);
         }
     }
@@ -233,12 +249,12 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
 // Dynamic shared memory: max(n*m floats for the selection, the CTA's block of W_r rows).
 
 template <typename T, bool TICKET, int NT>
-__global__ void __launch_bounds__(NT, NT == 64 ? 16 : (TICKET ? 5 : 6))
+__global__ void __launch_bounds__(NT, NT == 64 ? (TICKET ? 16 : 32) : (TICKET ? 5 : 6))
 route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restrict__ scores, int B, int L, int Lv, int d,
              int n, int k, int m, int c, int l_p, int CT, int nchunks, int rsplit, int rows_per_cta, int use_gate,
              int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
              float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
-             int* __restrict__ ctl /* word 1: ticket, words 8..: expert loads */, int* __restrict__ sample_ticket /* [B] */,
+             int* __restrict__ ctl /* word 1: ticket */, int* __restrict__ sample_ticket /* [B] */, unsigned* __restrict__ masks /* [B] */,
              const PlanPtrs plan /* all null: no plan is written */) {
     pdl_trigger();
     pdl_wait();
@@ -258,7 +274,7 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
         const int nvec = cw * n * (int)sizeof(T) / 16;
         const uint4* src = (const uint4*)(W_r + (size_t)c0 * n);
         for (int q = tid; q < nvec; q += NT)
-            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(s_dyn4 + q)), "l"(src + q) : "memory");
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(s_dyn4 + q)), "l"(src + q) : "memory");
         asm volatile("cp.async.commit_group;" ::: "memory");
     }
 
@@ -349,7 +365,7 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
         __threadfence();
         // ---- this CTA completed sample b ----
         select_sample<NT>((float*)s_dyn4, scores, nparts, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp,
-                          p_patch, offsets, ctl + 8, ctl + 1, plan);
+                          p_patch, offsets, masks, ctl + 1, plan);
     }
 }
 
@@ -358,17 +374,18 @@ __global__ void __launch_bounds__(kScoreThreads)
 route_select_kernel(const float* __restrict__ scores, int nparts, int B, int Lv, int n, int k, int m, int c, int l_p,
                     int use_gate, int* __restrict__ expert_idx, int* __restrict__ patch_idx, float* __restrict__ gate,
                     float* __restrict__ p_samp, float* __restrict__ p_patch, int* __restrict__ offsets,
-                    int* __restrict__ ctl, const PlanPtrs plan) {
+                    int* __restrict__ ctl, unsigned* __restrict__ masks, const PlanPtrs plan) {
     pdl_trigger();
     pdl_wait();
     extern __shared__ float s_sel[];
     select_sample<kScoreThreads>(s_sel, scores, nparts, blockIdx.x, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate,
-                                 p_samp, p_patch, offsets, ctl + 8, ctl + 1, plan);
+                                 p_samp, p_patch, offsets, masks, ctl + 1, plan);
 }
 
 struct RouteWs { size_t tickets, scores, total; int nchunks, CT, rsplit, rows_per_cta; size_t smem, wb; bool two_kernels, small_ctas; };
 
 constexpr int kWblkBytes = 16384;       // shared memory for a CTA's rows of W_r
+constexpr size_t kMaskOffset = kControlBytes / 2;      // control block: status block, sample tickets [B]; second half: expert masks [B]
 
 RouteWs route_ws(const Dims& D) {
     const int V = 16 / D.esize;
@@ -403,6 +420,8 @@ RouteWs route_ws(const Dims& D) {
         r.CT = 64;
         r.rows_per_cta = D.l_p;
     }
+    // they also hand the selection to a second launch: thousands of CTAs would otherwise each pay a fence and a ticket
+    if (r.small_ctas) r.two_kernels = true;
     r.smem = r.two_kernels ? r.wb : (sel > r.wb ? sel : r.wb);
     return r;
 }
@@ -412,24 +431,23 @@ RouteWs route_ws(const Dims& D) {
 uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void* W_r, int32_t* expert_idx,
                         int32_t* patch_idx, float* gate, float* p_samp, float* p_patch, int32_t* expert_offsets,
                         char* base, const RouteWs& W, cudaStream_t stream, bool profile, const PlanPtrs& plan = PlanPtrs()) {
-    // with a plan the CTA that completes the last sample keeps one word per sample in dynamic shared memory
-    const size_t plan_smem = plan.pair_row ? (size_t)D.B * sizeof(unsigned) : 0;
-    const size_t smem0 = W.smem > plan_smem ? W.smem : plan_smem;
-    int* ctl = (int*)base;             // word 0 status (unused here), word 1 ticket, words 8.. expert loads
+    const size_t smem0 = W.smem;
+    int* ctl = (int*)base;             // word 0 status (unused here), word 1 ticket
     int* tickets = (int*)(base + W.tickets);
+    unsigned* masks = (unsigned*)(base + kMaskOffset);      // every sample's expert set; data, at a place no ticket ever uses
     float* scores = (float*)(base + W.scores);
     const int use_gate = ((flags & UOE_FLAG_GATE) ? 1 : 0) | ((flags & UOE_FLAG_DYNAMIC_C) ? 2 : 0);     // selection flags
     dim3 grid((unsigned)(D.B * D.m * W.nchunks * W.rsplit));
 #define UOE_ROUTE_ARGS(T) (const T*)x, (const T*)W_r, scores, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, \
         W.nchunks, W.rsplit, W.rows_per_cta, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, \
-        tickets, plan
+        tickets, masks, plan
 #define UOE_ROUTE_LAUNCH(T, TICKET, NT, SMEM) \
         launch_k(route_kernel<T, TICKET, NT>, grid, dim3(NT), SMEM, stream, UOE_ROUTE_ARGS(T))
     cudaError_t e;
     {
         ProfScope ps(profile ? "route" : nullptr, stream);
-        if (W.two_kernels) e = D.bf16 ? UOE_ROUTE_LAUNCH(__nv_bfloat16, false, kScoreThreads, W.smem) : UOE_ROUTE_LAUNCH(float, false, kScoreThreads, W.smem);
-        else if (W.small_ctas) e = D.bf16 ? UOE_ROUTE_LAUNCH(__nv_bfloat16, true, 64, smem0) : UOE_ROUTE_LAUNCH(float, true, 64, smem0);
+        if (W.small_ctas) e = D.bf16 ? UOE_ROUTE_LAUNCH(__nv_bfloat16, false, 64, W.smem) : UOE_ROUTE_LAUNCH(float, false, 64, W.smem);
+        else if (W.two_kernels) e = D.bf16 ? UOE_ROUTE_LAUNCH(__nv_bfloat16, false, kScoreThreads, W.smem) : UOE_ROUTE_LAUNCH(float, false, kScoreThreads, W.smem);
         else e = D.bf16 ? UOE_ROUTE_LAUNCH(__nv_bfloat16, true, kScoreThreads, smem0) : UOE_ROUTE_LAUNCH(float, true, kScoreThreads, smem0);
     }
 #undef UOE_ROUTE_LAUNCH
@@ -439,11 +457,10 @@ uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void
     if (!W.two_kernels) return UOE_OK;
     {
         ProfScope ps(profile ? "route_select" : nullptr, stream);
-        size_t sel = (size_t)D.n * D.m * sizeof(float);
-        if (sel < plan_smem) sel = plan_smem;
+        const size_t sel = (size_t)D.n * D.m * sizeof(float);
         e = launch_k(route_select_kernel, dim3(D.B), dim3(kScoreThreads), sel, stream, (const float*)scores, W.nchunks * W.rsplit,
                      D.B, D.Lv, D.n, D.k, D.m, D.c, D.l_p, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch,
-                     expert_offsets, ctl, plan);
+                     expert_offsets, ctl, masks, plan);
     }
     if (e != cudaSuccess) return UOE_ERR_CUDA;
     UOE_LAUNCHED();
@@ -461,7 +478,7 @@ uoe_status route_check(const uoe_problem* prob, Dims& D, RouteWs& W, const void*
     if ((size_t)D.n * D.m * sizeof(float) > 36 * 1024) return UOE_ERR_UNSUPPORTED;   // gate values of a sample in shared memory
     W = route_ws(D);
     if ((long long)D.B * D.m * W.nchunks * W.rsplit > 0x7fffffffll) return UOE_ERR_UNSUPPORTED;
-    if (W.tickets + (size_t)D.B * sizeof(int) > kControlBytes) return UOE_ERR_UNSUPPORTED;   // tickets must fit the control block
+    if (W.tickets + (size_t)D.B * sizeof(int) > kMaskOffset) return UOE_ERR_UNSUPPORTED;   // tickets and expert masks must fit the control block
     return UOE_OK;
 }
 
@@ -469,7 +486,7 @@ uoe_status route_check(const uoe_problem* prob, Dims& D, RouteWs& W, const void*
 
 size_t route_workspace_bytes(const Dims& D) { return route_ws(D).total; }
 
-bool route_can_plan(const Dims& D) { return (size_t)D.B * sizeof(unsigned) <= 32 * 1024; }
+bool route_can_plan(const Dims&) { return true; }
 
 uoe_status route_run(const uoe_problem* prob, const void* x, const void* W_r, const RoutingPtrs& r, char* scratch,
                      cudaStream_t stream, const PlanPtrs* plan) {
