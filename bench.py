@@ -602,6 +602,55 @@ def measure_gpu(args, w: gen.Workload, dev, world: int, steps: int, warmup: int,
     return res
 
 
+def single_mode_of(dev, steps: int):
+    """The two selection modes the paper uses on their own (end of Section III-B), on the language-model and image
+    shapes: pure data selection (k = n, Eq. 12-20) and pure expert selection (c = m, Eq. 21-26), each timed through
+    its shortcut and through the general routed path (UOE_FLAG_GENERAL_PATH), whole block forward, same protocol
+    as the small workloads (L2 flushed before every step, one CUDA event pair per step)."""
+    import torch
+
+    import paper_2503_02495_b200 as uoe
+    from paper_2503_02495_b200.workload import problem_of, to_dev
+
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream()
+    out = {}
+    for name in ("cfg2_lm", "cfg4_vit"):
+        w0 = gen.WORKLOADS[name]
+        for mode, w in (("data_selection_k=n", w0.replace(k=w0.n)), ("expert_selection_c=m", w0.replace(c=w0.m))):
+            h = host_inputs(w)
+            wd = {k: to_dev(v, dev) for k, v in h.items() if k not in ("x", "dy")}
+            x_dev = to_dev(h["x"], dev)
+            rec = {"k": w.k, "n": w.n, "c": w.c, "m": w.m, "routed_rows": w.R}
+            ys = []
+            for label, general in (("shortcut_ms", False), ("general_path_ms", True)):
+                pa, pm = problem_of(w, "att", general_path=general), problem_of(w, "mlp", general_path=general)
+                ws = uoe.alloc_block_workspace(pa, pm, dev)
+                u, y = torch.empty_like(x_dev), torch.empty_like(x_dev)
+                run = lambda: uoe.uoe_block_forward(pa, pm, x_dev, wd, u=u, y=y, ws=ws, check=False)
+                for _ in range(3):
+                    run()
+                torch.cuda.synchronize()
+                ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+                for e0, e1 in ev:
+                    flush.zero_()
+                    e0.record(stream)
+                    run()
+                    e1.record(stream)
+                torch.cuda.synchronize()
+                st = uoe.uoe_read_device_status(ws)
+                if st != 0:
+                    raise RuntimeError("device status in the single-mode run: " + uoe.status_string(st))
+                rec[label] = sum(e0.elapsed_time(e1) for e0, e1 in ev) / steps
+                ys.append(y.clone())
+            rec["saved_us"] = (rec["general_path_ms"] - rec["shortcut_ms"]) * 1e3
+            rec["same_bits"] = bool(torch.equal(ys[0], ys[1]))
+            out[name + ":" + mode] = rec
+    del flush
+    torch.cuda.empty_cache()
+    return out
+
+
 TENSOR_KERNELS = ("gemm1_act", "gemm2", "mlp_fused", "qkv_proj", "out_proj", "attention", "bwd_da_dh", "bwd_dx", "wgrad_W1", "wgrad_W2",
                   "attn_bwd_dkdv", "attn_bwd_dq", "bwd_do", "bwd_dx_att", "wgrad_Wo", "wgrad_Wqkv")
 HBM_KERNELS = ("route", "gather", "combine", "pool")
@@ -740,6 +789,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
             del mo
             others[name] = bo
         line["workloads"] = others
+        line["single_mode"] = single_mode_of(dev, min(args.steps, 50))
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -71,10 +71,24 @@ enum {
     UOE_FLAG_RESIDUAL = 1,     /* y = x + sum(...) (the selective residual of Eq. 20); else y = sum(...) */
     UOE_FLAG_GATE = 2,         /* combine weight = P_samp[b,i] * P_patch[b,i,j]; else 1 (Eq. 20 literal) */
     UOE_FLAG_CAUSAL = 4,       /* SMHA: shared lower-triangular mask over the gathered tokens (Fig. 4) */
-    UOE_FLAG_DYNAMIC_C = 8     /* uoe_route: two-stage routing (Eq. 15-16): every chosen expert of a sample takes
+    UOE_FLAG_DYNAMIC_C = 8,    /* uoe_route: two-stage routing (Eq. 15-16): every chosen expert of a sample takes
                                   min(c, c_b) patches, c_b = the largest number of patches any expert receives when
                                   each patch goes to its k best experts; the remaining slots are unused (-1) */
+    UOE_FLAG_GENERAL_PATH = 16 /* take the general routed path even for the two single-mode cases below (same results;
+                                  for verification and for measuring what the special cases save) */
 };
+
+/*
+ * The two selection modes the paper uses on their own (end of Section III-B) are recognised from the problem and
+ * take shorter paths with the same results:
+ *   k == n  pure data selection (Eq. 12-20): every sample uses all n experts.  No expert ranking; every expert's
+ *           region holds exactly B pairs, so expert_offsets and each pair's rows follow from (b, i) alone and no
+ *           step of the router waits for the other samples.
+ *   c >= number of patches that hold a real token, without UOE_FLAG_DYNAMIC_C  pure expert selection (Eq. 21-26): a
+ *           chosen expert takes the whole sample.  No patch ranking; slot u of a pair is patch u, so neither the
+ *           router nor the consumers inside uoe_block_forward build or read a patch plan or an inverse map: the
+ *           combine finds the at most k rows of a token from the pair's first row and the token's position.
+ */
 
 typedef enum { UOE_OP_ROUTE = 0, UOE_OP_MLP_FWD = 1, UOE_OP_MLP_BWD = 2, UOE_OP_SMHA_FWD = 3, UOE_OP_SMHA_BWD = 4,
                UOE_OP_BALANCE_BWD = 5 } uoe_op;

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libuoe.so")
 UOE_ROW_ALIGN = 128
 UOE_F32, UOE_BF16 = 0, 1
 ACTS = {"gelu_erf": 0, "gelu_tanh": 1, "silu": 2, "identity": 3}
-UOE_FLAG_RESIDUAL, UOE_FLAG_GATE, UOE_FLAG_CAUSAL, UOE_FLAG_DYNAMIC_C = 1, 2, 4, 8
+UOE_FLAG_RESIDUAL, UOE_FLAG_GATE, UOE_FLAG_CAUSAL, UOE_FLAG_DYNAMIC_C, UOE_FLAG_GENERAL_PATH = 1, 2, 4, 8, 16
 UOE_OP_ROUTE, UOE_OP_MLP_FWD, UOE_OP_MLP_BWD, UOE_OP_SMHA_FWD, UOE_OP_SMHA_BWD = 0, 1, 2, 3, 4
 UOE_OP_BALANCE_BWD = 5
 
@@ -61,10 +61,12 @@ class Problem:
     causal: bool = False
     dynamic_c: bool = False
     d_rope: int = 0
+    general_path: bool = False      # UOE_FLAG_GENERAL_PATH: no single-mode shortcuts (same results)
 
     def c_struct(self) -> _Problem:
         flags = (UOE_FLAG_RESIDUAL if self.residual else 0) | (UOE_FLAG_GATE if self.gate else 0) | \
-                (UOE_FLAG_CAUSAL if self.causal else 0) | (UOE_FLAG_DYNAMIC_C if self.dynamic_c else 0)
+                (UOE_FLAG_CAUSAL if self.causal else 0) | (UOE_FLAG_DYNAMIC_C if self.dynamic_c else 0) | \
+                (UOE_FLAG_GENERAL_PATH if self.general_path else 0)
         return _Problem(self.B, self.L, self.L_valid, self.d, self.n, self.k, self.m, self.c, self.d_e, self.H,
                         self.d_h, UOE_BF16 if self.dtype == "bf16" else UOE_F32, ACTS[self.act], flags, self.d_rope)
 

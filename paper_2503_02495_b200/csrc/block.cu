@@ -116,6 +116,8 @@ extern "C" uoe_status uoe_block_forward(const uoe_problem* att, const uoe_proble
         const SmhaFwdBufs B{bufs + W.so.xg, bufs + W.so.q, bufs + W.so.k, bufs + W.so.v, bufs + W.so.o, bufs + W.so.z};
         if (route_can_plan(Da)) {
             P.inv_relative = true;
+            P.identity_patches = route_whole_samples(Da, att->flags);
+            P.gate = R.gate;
             P.tail = (uint4*)B.v; P.tail_row_vecs = (long long)Da.d_g * Da.esize / 16; P.rows_max = Da.Rmax;
             st = route_run(att, cur, Wr_att, R, scratch, stream, &P);
             if (st != UOE_OK) return st;
@@ -137,6 +139,8 @@ extern "C" uoe_status uoe_block_forward(const uoe_problem* att, const uoe_proble
         PlanPtrs P = plan_ptrs(Dm, base + W.plan_mlp);
         if (route_can_plan(Dm)) {
             P.inv_relative = true;
+            P.identity_patches = route_whole_samples(Dm, mlp->flags);
+            P.gate = R.gate;
             st = route_run(mlp, cur, Wr_mlp, R, scratch, stream, &P);
             if (st != UOE_OK) return st;
         } else {

@@ -25,6 +25,11 @@ struct PlanPtrs {
     int* slot_pair = nullptr;    // [n,B]    plan written by the router kernel: pair (b*k + s) of the q-th sample in expert i's
                                  //          region (it replaces src_patch, which that plan does not fill)
     bool inv_relative = false;   // inv_row holds offsets from pair_row (plan written by the router kernel)
+    // plan written by the router kernel, whole samples per expert (every chosen expert takes every patch that holds a
+    // real token, Eq. 21-26): slot u of a pair is patch u, so inv_row, inv_gate and patch_idx are neither written nor
+    // read; the combine takes its weights from the router's gate array [B,k,c]
+    bool identity_patches = false;
+    const float* gate = nullptr;
     // plan written by the router kernel only: a routed buffer whose first rows past the last expert region are
     // zero-filled (up to 128 of them, as many as a 128-row tile that starts inside the last region can reach)
     uint4* tail = nullptr;
@@ -45,6 +50,11 @@ struct RoutingPtrs {
 // `plan` the routing plan is written by the same kernels (inv_row relative to pair_row), so no plan kernel is needed;
 // route_can_plan says whether the problem allows that.
 bool route_can_plan(const Dims& D);
+// Whether the router treats the problem as pure expert selection (whole samples per expert, Eq. 21-26): then a plan it
+// writes has identity_patches set and holds no inverse map.
+inline bool route_whole_samples(const Dims& D, uint32_t flags) {
+    return !(flags & (UOE_FLAG_DYNAMIC_C | UOE_FLAG_GENERAL_PATH)) && D.c >= (D.Lv + D.l_p - 1) / D.l_p;
+}
 uoe_status route_run(const uoe_problem* prob, const void* x, const void* W_r, const RoutingPtrs& r, char* scratch,
                      cudaStream_t stream, const PlanPtrs* plan);
 // Gathering through the GEMM's own TMA loads needs whole patches inside a 128-row tile, 8-row swizzle groups
@@ -86,12 +96,14 @@ struct SrcMap {
     const int* patch_idx = nullptr;    // [B,k,c]
     const int* expert_end = nullptr;   // [n]
     int B = 0, k = 0, c = 0, m = 0, l_p = 0;
+    int n_elig = -1;                   // >= 0: slot u of a pair is patch u for u < n_elig (whole samples per expert), patch_idx is not read
     __host__ __device__ bool on() const { return src_patch != nullptr || slot_pair != nullptr; }
 };
 inline SrcMap src_map_of(const Dims& D, const PlanPtrs& P, const int* patch_idx) {
     SrcMap g;
     if (P.inv_relative) { g.slot_pair = P.slot_pair; g.patch_idx = patch_idx; g.expert_end = P.expert_end; }
     else g.src_patch = P.src_patch;
+    if (P.inv_relative && P.identity_patches) g.n_elig = (D.Lv + D.l_p - 1) / D.l_p;
     g.B = D.B; g.k = D.k; g.c = D.c; g.m = D.m; g.l_p = D.l_p;
     return g;
 }
@@ -108,7 +120,8 @@ __device__ __forceinline__ int src_of(const SrcMap& g, int r, int e, int off_e, 
         if (r < g.expert_end[e]) {
             const int rel = r - off_e, l_a = g.c * g.l_p;
             const int pair = g.slot_pair[(size_t)e * g.B + rel / l_a];
-            const int pj = g.patch_idx[(size_t)pair * g.c + (rel % l_a) / g.l_p];
+            const int u = (rel % l_a) / g.l_p;
+            const int pj = g.n_elig >= 0 ? (u < g.n_elig ? u : -1) : g.patch_idx[(size_t)pair * g.c + u];
             if (pj >= 0 && pj < g.m) src = (pair / g.k) * g.m + pj;
         }
     }

@@ -30,7 +30,8 @@ constexpr int kScoreThreads = 256;
 // in the scratch area) into per-expert row offsets (Eq. 23) and, for the plan, each pair's first row.
 template <int NT>
 __device__ void select_sample(float* pp, const float* __restrict__ partial, int nparts, int b, int B, int Lv, int n, int k,
-                              int m, int c, int l_p, int sel_flags /* bit 0: gate weights, bit 1: dynamic capacity */,
+                              int m, int c, int l_p,
+                              int sel_flags /* bit 0: gate weights, bit 1: dynamic capacity, bit 2: general path only */,
                               int* __restrict__ expert_idx,
                               int* __restrict__ patch_idx, float* __restrict__ gate, float* __restrict__ p_samp,
                               float* __restrict__ p_patch, int* __restrict__ offsets, unsigned* __restrict__ masks,
@@ -47,6 +48,9 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
     const int use_gate = sel_flags & 1, dynamic_c = (sel_flags >> 1) & 1;
     if (tid < 32) cnts[tid] = 0;
     const int n_elig = (Lv + l_p - 1) / l_p;       // patches holding at least one real token (a prefix)
+    // the single-mode cases: every sample uses all experts (Eq. 12-20) / a chosen expert takes the whole sample (Eq. 21-26)
+    const bool all_experts = !(sel_flags & 4) && k == n;
+    const bool all_patches = !(sel_flags & 4) && !dynamic_c && c >= n_elig;
     int np2 = 1;
     while (np2 < n) np2 <<= 1;
     const int G = 32 / np2;                         // patches a warp works at a time
@@ -108,10 +112,11 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
         if (lane < n) { ps[lane] = pr; p_samp[(size_t)b * n + lane] = pr; }
         // Eq. 22: rank = number of experts that beat this one (larger value, or equal with lower index)
         int rank = 0;
-        for (int i = 0; i < n; ++i) {
-            const float w = __shfl_sync(0xffffffffu, pr, i);
-            rank += (w > pr) || (w == pr && i < lane);
-        }
+        if (!all_experts)
+            for (int i = 0; i < n; ++i) {
+                const float w = __shfl_sync(0xffffffffu, pr, i);
+                rank += (w > pr) || (w == pr && i < lane);
+            }
         const bool pick = lane < n && rank < k;
         const unsigned mask = __ballot_sync(0xffffffffu, pick);
         if (pick) {
@@ -145,6 +150,7 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
             const bool valid = j < n_elig;
             const float v = valid ? v_i[j] : 0.f;
             int rank = 0;
+            if (!all_patches)
             for (int jj0 = 0; jj0 < n_elig; jj0 += 8) {      // eight broadcast reads at a time
                 float w[8];
 #pragma unroll
@@ -160,14 +166,14 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
                 out_idx[pos] = j;
                 out_gate[pos] = g;
             }
-            if (plan.inv_row && valid) {        // the inverse of Eq. 18, relative to the pair's first routed row
+            if (plan.inv_row && valid && !all_patches) {        // the inverse of Eq. 18, relative to the pair's first routed row
                 plan.inv_row[((size_t)b * m + j) * k + s] = pick ? pos * l_p : -1;
                 plan.inv_gate[((size_t)b * m + j) * k + s] = pick ? g : 0.f;
             }
             before += __popc(mask);
         }
         for (int pos = before + lane; pos < c; pos += 32) { out_idx[pos] = -1; out_gate[pos] = 0.f; }
-        if (plan.inv_row)
+        if (plan.inv_row && !all_patches)
             for (int j = n_elig + lane; j < m; j += 32) {       // patches of pad tokens only
                 plan.inv_row[((size_t)b * m + j) * k + s] = -1;
                 plan.inv_gate[((size_t)b * m + j) * k + s] = 0.f;
@@ -176,6 +182,24 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
 
     // ---- the CTA that completes the last sample: Eq. 23 as row offsets, and the part of the routing plan that needs
     //      every sample's choice (where every pair's rows start, which pair owns every slot of every expert's region) ----
+    if (all_experts) {
+        // every expert's region holds the B samples in order: nothing here depends on another sample, no ticket
+        const int l_a = c * l_p;
+        const int region = (B * l_a + UOE_ROW_ALIGN - 1) / UOE_ROW_ALIGN * UOE_ROW_ALIGN;
+        if (plan.pair_row && tid < n) {
+            plan.pair_row[(size_t)b * k + tid] = tid * region + b * l_a;
+            plan.slot_pair[(size_t)tid * B + b] = b * k + tid;
+        }
+        if (b == 0) {
+            if (tid <= n) offsets[tid] = tid * region;
+            if (plan.pair_row && tid < n) plan.expert_end[tid] = tid * region + B * l_a;
+            if (plan.pair_row && plan.tail) {
+                const long long r0 = (long long)n * region, r1 = min(plan.rows_max, r0 + 128);
+                for (long long q = tid; q < (r1 - r0) * plan.tail_row_vecs; q += NT) plan.tail[r0 * plan.tail_row_vecs + q] = make_uint4(0, 0, 0, 0);
+            }
+        }
+        return;
+    }
     __syncthreads();
     if (tid == 0) {
         __threadfence();
@@ -436,7 +460,8 @@ uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void
     int* tickets = (int*)(base + W.tickets);
     unsigned* masks = (unsigned*)(base + kMaskOffset);      // every sample's expert set; data, at a place no ticket ever uses
     float* scores = (float*)(base + W.scores);
-    const int use_gate = ((flags & UOE_FLAG_GATE) ? 1 : 0) | ((flags & UOE_FLAG_DYNAMIC_C) ? 2 : 0);     // selection flags
+    const int use_gate = ((flags & UOE_FLAG_GATE) ? 1 : 0) | ((flags & UOE_FLAG_DYNAMIC_C) ? 2 : 0) |
+                         ((flags & UOE_FLAG_GENERAL_PATH) ? 4 : 0);                                       // selection flags
     dim3 grid((unsigned)(D.B * D.m * W.nchunks * W.rsplit));
 #define UOE_ROUTE_ARGS(T) (const T*)x, (const T*)W_r, scores, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, \
         W.nchunks, W.rsplit, W.rows_per_cta, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, expert_offsets, ctl, \

@@ -161,7 +161,9 @@ __global__ void __launch_bounds__(kThreads)
 combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __restrict__ inv_row,
                const float* __restrict__ inv_gate, T* __restrict__ y, int L, int Lv, int d, int m, int k,
                int l_p, int residual, int use_gate, int rows_per_cta, const float* __restrict__ rvec,
-               const int* __restrict__ pair_row /* not null: inv_row holds offsets from the pair's first row */) {
+               const int* __restrict__ pair_row /* not null: inv_row holds offsets from the pair's first row */,
+               const float* __restrict__ gate_bkc /* not null: whole samples per expert (slot u is patch u): no inverse map,
+                                                     weights from the router's gate array [B,k,c] */, int c) {
     pdl_trigger();
     pdl_wait();
     constexpr int V = Vec16<T>::N;
@@ -170,10 +172,15 @@ combine_kernel(const T* __restrict__ x, const T* __restrict__ z, const int* __re
     const int bj = blockIdx.x, b = bj / m, j = bj % m;
     const int r0 = blockIdx.y * rows_per_cta, r1 = min(l_p, r0 + rows_per_cta);
     if (threadIdx.x < k) {
-        const int rel = inv_row[(size_t)bj * k + threadIdx.x];
-        const int base = pair_row ? pair_row[(size_t)b * k + threadIdx.x] : 0;
-        srow[threadIdx.x] = rel >= 0 ? rel + base : -1;
-        sg[threadIdx.x] = use_gate ? inv_gate[(size_t)bj * k + threadIdx.x] : 1.0f;
+        if (gate_bkc) {          // Eq. 26: the token's row in every chosen expert follows from its position alone
+            srow[threadIdx.x] = j * l_p < Lv ? pair_row[(size_t)b * k + threadIdx.x] + j * l_p : -1;
+            sg[threadIdx.x] = use_gate ? gate_bkc[((size_t)b * k + threadIdx.x) * c + j] : 1.0f;
+        } else {
+            const int rel = inv_row[(size_t)bj * k + threadIdx.x];
+            const int base = pair_row ? pair_row[(size_t)b * k + threadIdx.x] : 0;
+            srow[threadIdx.x] = rel >= 0 ? rel + base : -1;
+            sg[threadIdx.x] = use_gate ? inv_gate[(size_t)bj * k + threadIdx.x] : 1.0f;
+        }
     }
     __syncthreads();
     const int vpr = d / V;
@@ -327,17 +334,19 @@ uoe_status launch_combine(const Dims& D, const void* x, const void* z, const Pla
     if (rows_per_cta < 1) rows_per_cta = 1;
     if (rows_per_cta > D.l_p) rows_per_cta = D.l_p;
     dim3 grid(D.B * D.m, (D.l_p + rows_per_cta - 1) / rows_per_cta);
+    const bool ident = P.inv_relative && P.identity_patches && P.gate != nullptr;
     ProfScope ps("combine", s);
     if (D.bf16)
         launch_k(combine_kernel<__nv_bfloat16>, grid, dim3(kThreads), 0, s, 
             (const __nv_bfloat16*)x, (const __nv_bfloat16*)z, P.inv_row, P.inv_gate, (__nv_bfloat16*)y, D.L, D.Lv,
             D.d, D.m, D.k, D.l_p, residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec,
-            P.inv_relative ? (const int*)P.pair_row : (const int*)nullptr);
+            P.inv_relative ? (const int*)P.pair_row : (const int*)nullptr, ident ? P.gate : (const float*)nullptr, D.c);
     else
         launch_k(combine_kernel<float>, grid, dim3(kThreads), 0, s, (const float*)x, (const float*)z, P.inv_row, P.inv_gate,
                                                        (float*)y, D.L, D.Lv, D.d, D.m, D.k, D.l_p,
                                                        residual ? 1 : 0, use_gate ? 1 : 0, rows_per_cta, rvec,
-                                                       P.inv_relative ? (const int*)P.pair_row : (const int*)nullptr);
+                                                       P.inv_relative ? (const int*)P.pair_row : (const int*)nullptr,
+                                                       ident ? P.gate : (const float*)nullptr, D.c);
     UOE_LAUNCHED();
     return UOE_OK;
 }
