@@ -750,7 +750,7 @@ def run_ours(args, w: gen.Workload, rank: int, local_rank: int, world: int):
 
     solo = world == 1 and args.part == "all"
     m = measure_gpu(args, w, dev, world, args.steps, args.warmup, True, with_parity=solo and not args.skip_cpu_baseline,
-                    sustain_s=1.2 if solo else 0.0)
+                    sustain_s=1.2 if solo and not args.no_sustained else 0.0)
     ms_step, e2e_ms = max_over_ranks([m["ms_step"], m["e2e_ms"]], world, dev)
     if rank != 0:
         if world > 1:
@@ -806,6 +806,7 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="omit the oracle timing and the parity block (profiling runs)")
     ap.add_argument("--backward", action="store_true", help="add the backward of every half of the block to the step")
     ap.add_argument("--part", default="all", choices=["all", "route"], help="time only a part of the step (profiling runs)")
+    ap.add_argument("--no-sustained", action="store_true", help="omit the second-long sustained run (profiling runs)")
     ap.add_argument("--no-others", "--no-scale", dest="no_others", action="store_true",
                     help="only the selected workload: do not add the other workloads' blocks to the line")
     args = ap.parse_args()

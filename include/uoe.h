@@ -324,6 +324,10 @@ uoe_status uoe_read_device_status(void* ws, void* cuda_stream);
 /* Number of this library's kernel launches enqueued by this process so far (for benchmarks). */
 int64_t uoe_launch_count(void);
 
+/* Number of TMA tensor maps this process has encoded so far.  Encoded maps are kept in a table keyed by buffer
+ * address and shape, so repeated calls on the same buffers encode nothing new (for benchmarks and tests). */
+int64_t uoe_tensor_map_encodings(void);
+
 /*
  * Per-kernel timing for benchmarks (instrumentation; the paper times whole passes with a profiler,
  * Section IV).  uoe_profile_enable(1) clears the record list and starts recording: from then on every

@@ -124,6 +124,8 @@ def _load():
     lib.uoe_read_device_status.argtypes = [vp, vp]
     lib.uoe_launch_count.restype = ctypes.c_int64
     lib.uoe_launch_count.argtypes = []
+    lib.uoe_tensor_map_encodings.restype = ctypes.c_int64
+    lib.uoe_tensor_map_encodings.argtypes = []
     lib.uoe_profile_enable.restype = None
     lib.uoe_profile_enable.argtypes = [ctypes.c_int]
     lib.uoe_profile_count.restype = ctypes.c_int
@@ -172,6 +174,10 @@ def uoe_workspace_bytes(prob: Problem, op: int) -> int:
 
 def uoe_launch_count() -> int:
     return int(_lib.uoe_launch_count())
+
+
+def uoe_tensor_map_encodings() -> int:
+    return int(_lib.uoe_tensor_map_encodings())
 
 
 def uoe_profile_enable(on: bool) -> None:

@@ -1,5 +1,6 @@
 // Entry points that launch nothing: sizes, status text, status read-back, launch counter.
 #include "kernels.cuh"
+#include "tmap.cuh"
 
 #include <vector>
 
@@ -98,3 +99,5 @@ extern "C" uoe_status uoe_read_device_status(void* ws, void* cuda_stream) {
 }
 
 extern "C" int64_t uoe_launch_count(void) { return g_launch_count; }
+
+extern "C" int64_t uoe_tensor_map_encodings(void) { return tmap_encode_count(); }

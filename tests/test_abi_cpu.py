@@ -22,7 +22,7 @@ def test_library_exports_every_declared_symbol(uoe):
     header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
     names = set(re.findall(r"\b(uoe_[a-z_0-9]+)\s*\(", header))
     assert {"uoe_route", "uoe_mlp_forward", "uoe_mlp_backward", "uoe_smha_forward", "uoe_workspace_bytes",
-            "uoe_max_routed_rows", "uoe_status_string", "uoe_read_device_status", "uoe_workspace_init", "uoe_launch_count",
+            "uoe_max_routed_rows", "uoe_status_string", "uoe_read_device_status", "uoe_workspace_init", "uoe_launch_count", "uoe_tensor_map_encodings",
             "uoe_profile_enable", "uoe_profile_count", "uoe_profile_get"} <= names
     lib = ctypes.CDLL(uoe.LIB_PATH)
     for nm in names:

@@ -163,3 +163,21 @@ def test_block_forward_rejects_bad_arguments_before_launching():
         uoe.uoe_block_forward(pa, pm2, x, wd, ws=uoe.alloc_block_workspace(pa, pm2))
     assert uoe.uoe_launch_count() == n0
     assert uoe.uoe_block_workspace_bytes(None, None) == 0
+
+
+def test_repeated_calls_on_the_same_buffers_encode_no_new_tensor_maps():
+    import paper_2503_02495_b200 as uoe
+    w = gen.WORKLOADS["cfg2_lm"].replace(B=2)
+    pa, pm = problem_of(w, "att"), problem_of(w, "mlp")
+    x = to_dev(gen.make_x(w))
+    wd = {k: to_dev(v) for k, v in _weights(w).items()}
+    ws = uoe.alloc_block_workspace(pa, pm)
+    u, y = torch.empty_like(x), torch.empty_like(x)
+    uoe.uoe_block_forward(pa, pm, x, wd, u=u, y=y, ws=ws)
+    n1 = uoe.uoe_tensor_map_encodings()
+    assert n1 > 0
+    y1 = y.clone()
+    for _ in range(3):
+        uoe.uoe_block_forward(pa, pm, x, wd, u=u, y=y, ws=ws)
+    assert uoe.uoe_tensor_map_encodings() == n1
+    assert torch.equal(y, y1)

@@ -35,6 +35,10 @@ CASES = {
     "fused_fwd_d512": _w(B=4, L=256, L_valid=256, m=8, c=4, d=512, n=4, k=2, d_ff=1024, act="gelu_tanh"),
     # long K and many row tiles: 256-row GEMM tiles with half tiles at the region ends
     "tall_tiles": _w(B=40, L=1152, L_valid=1152, m=9, c=3, d=1024, n=4, k=2, d_ff=4096, w_std=0.02),
+    # imbalanced loads on shapes large enough for the 256-row GEMM tiles and for the weight-gradient kernel's
+    # 256 x 256 tiles handed out longest-first (320 of them, the experts' row counts far apart)
+    "tall_tiles_skewed": _w(B=40, L=1152, L_valid=1152, m=9, c=3, d=1024, n=4, k=2, d_ff=4096, w_std=0.02),
+    "wgrad_256_skewed": _w(B=12, L=1152, L_valid=1152, m=9, c=3, d=1024, n=5, k=2, d_ff=5 * 4096, w_std=0.02),
 }
 
 
@@ -60,15 +64,15 @@ def _run(w, residual, use_gate, skew=0.0):
 @pytest.mark.parametrize("residual", [False, True])
 def test_backward_matches_oracle(name, residual):
     w = CASES[name]
-    if name == "tall_tiles" and residual:
+    if w.B * w.L > 10000 and residual:
         pytest.skip("large case: run once")
-    got, ref, ro = _run(w, residual, True, skew=3.0 if name == "skewed" else 0.0)
+    got, ref, ro = _run(w, residual, True, skew=(3.0 if name == "skewed" else 12.0) if "skewed" in name else 0.0)
     for nm, g, r in zip(("dx", "dW1", "dW2", "dW_r"), got, ref[:4]):
         err = rel_inf(g, r)
         print(f"{name} residual={residual} {nm}: {err:.3e}  (|ref|max {np.abs(r).max():.3e})")
         assert err <= TOL, nm
-    if name == "skewed":
-        assert ro.load.min() == 0 or ro.load.max() >= 2 * ro.load.mean()      # the load really is uneven
+    if "skewed" in name:
+        assert ro.load.min() == 0 or ro.load.max() >= 1.5 * ro.load.mean()      # the load really is uneven
 
 
 def test_backward_without_gates_has_zero_router_gradient():

@@ -35,12 +35,15 @@ CASES = {
     "lm_shape": gen.WORKLOADS["cfg2_lm"].replace(B=4),
     "long_shape": gen.WORKLOADS["cfg3_long"].replace(B=2),
     "vit_shape": gen.WORKLOADS["cfg4_vit"].replace(B=12),
+    # imbalanced expert loads (every sample pushed toward one expert drawn with Zipf weights) on the language-model shape
+    "lm_shape_skewed": gen.WORKLOADS["cfg2_lm"].replace(B=6),
 }
 
 
-def _run(w, residual, use_gate=True, d_rope=0):
+def _run(w, residual, use_gate=True, d_rope=0, skew=0.0):
     import paper_2503_02495_b200 as uoe
-    x, Wr = gen.make_x(w), gen.make_router(w, "att")
+    Wr = gen.make_router(w, "att")
+    x = gen.make_x(w, skew_beta=skew, W_r=Wr.f64) if skew else gen.make_x(w)
     if not w.name.startswith("cfg"):
         Wr = gen.store(Wr.f64 * 20, w.dtype)
     Wq, Wk, Wv, Wo = gen.make_attn_weights(w)
@@ -60,9 +63,9 @@ def _run(w, residual, use_gate=True, d_rope=0):
 @pytest.mark.parametrize("residual", [False, True])
 def test_smha_backward_matches_oracle(name, residual):
     w = CASES[name]
-    if residual and name.endswith("_shape"):
+    if residual and "_shape" in name:
         pytest.skip("larger case: run once")
-    got, ref = _run(w, residual)
+    got, ref = _run(w, residual, skew=4.0 if "skewed" in name else 0.0)
     for nm, g, r in zip(NAMES, got, ref[:6]):
         assert np.isfinite(g).all(), nm
         err = rel_inf(g, r)
