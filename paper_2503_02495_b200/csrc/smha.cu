@@ -92,7 +92,6 @@ uoe_status uoe::smha_forward_check(const uoe_problem* prob, Dims& D, const void*
     if (!aligned16(x) || !aligned16(Wq) || !aligned16(Wk) || !aligned16(Wv) || !aligned16(Wo) || !aligned16(y))
         return UOE_ERR_INVALID_ARG;
     if (!D.bf16 || D.d_h != 64) return UOE_ERR_UNSUPPORTED;     // tensor-core path: bf16, 64-wide heads
-    if ((long long)D.B * D.k > 65535) return UOE_ERR_UNSUPPORTED;  // the attention grid carries the pairs on its z axis
     return UOE_OK;
 }
 
