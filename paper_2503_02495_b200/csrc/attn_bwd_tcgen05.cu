@@ -170,6 +170,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             }
         }
         const int kv0 = k_tile * T;
+        const int keep_cols = (qrow < l_a ? min(kv_end, causal ? qrow + 1 : kv_end) : 0) - kv0;     // kept columns of this key tile
         const int sw = trow & 7;
 #pragma unroll 1
         for (int ch = 2 * hsel; ch < 2 * hsel + 2; ++ch) {
@@ -177,11 +178,12 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
             tmem_ld32(t_lane + ch * 32, (uint32_t*)s_v);
             tmem_ld32(t_lane + 128 + ch * 32, (uint32_t*)dp_v);
             tmem_ld_wait();
+            // (one limit per row covers the three masks -- rows past the pair, keys past the real ones, the causal
+            // triangle --: tested clause by clause per element the test becomes branches per element)
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-                const int col = kv0 + ch * 32 + j;
-                const bool keep = qrow < l_a && col < kv_end && (!causal || col <= qrow);
-                const float p = keep ? exp2f(s_v[j] * scale_log2 - my_lse2) : 0.f;
+                const bool keep = ch * 32 + j < keep_cols;
+                const float p = keep ? ex2_approx(fmaf(s_v[j], scale_log2, -my_lse2)) : 0.f;
                 s_v[j] = p;
                 dp_v[j] = keep ? p * (dp_v[j] - my_delta) * inv_sqrt_dh : 0.f;
             }

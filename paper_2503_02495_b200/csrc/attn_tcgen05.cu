@@ -75,11 +75,6 @@ struct AttnArgs {
     int* status;
 };
 
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 
 template <bool FUSE_O>
 __global__ void __launch_bounds__(kAttnThreads, 1)

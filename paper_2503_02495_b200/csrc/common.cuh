@@ -243,6 +243,13 @@ __device__ __forceinline__ float act_apply(float h, int act) {
     }
 }
 
+// 2^x on the special-function unit (relative error about 2^-22; the results here are rounded to bfloat16)
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ float tanh_fast(float x) {
     float y;
     asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
