@@ -137,11 +137,7 @@ attn_stream_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     auto wait = [&](uint64_t* bar, uint32_t parity) { return mbar_wait(bar, parity, abort_flag, status) && !*abort_flag; };
     // the same for the one-thread roles (TMA, MMA), which sit on the critical path between the softmax warps' steps:
     // they poll without letting the hardware suspend them first
-    auto wait1 = [&](uint64_t* bar, uint32_t parity) {
-        for (int it = 0; it < 20000; ++it)
-            if (mbar_test_wait(bar, parity)) return !*abort_flag;
-        return mbar_wait(bar, parity, abort_flag, status) && !*abort_flag;
-    };
+    auto wait1 = [&](uint64_t* bar, uint32_t parity) { return mbar_wait_spin(bar, parity, abort_flag, status) && !*abort_flag; };
 
     if (role == 1) {
         // =========================== TMA warp ===========================

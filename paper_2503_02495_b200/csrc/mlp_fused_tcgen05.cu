@@ -122,13 +122,20 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
             if (++stage == STAGES) { stage = 0; phase ^= 1; }
         };
+        const bool gathered = smap.on();
+        const int nbox_a = gathered ? BM / l_p : 1;                         // <= 16
+        // where a tile's rows come from (two dependent look-ups in global memory when A is gathered): found for the
+        // next tile while this tile's first W2 blocks are in flight and the ring is full anyway
+        int e_next = 0, row0_next = 0, src_next = 0;
+        auto look_up = [&](int tile) {
+            if (tile >= total_tiles) return;
+            locate(tile, e_next, row0_next);
+            if (gathered && lane < nbox_a) src_next = src_of(smap, row0_next + lane * l_p, e_next, ctl->offs[e_next], Bm);   // Bm: zero-filled box
+        };
+        look_up(blockIdx.x);
         for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
-            int e, row0;
-            locate(tile, e, row0);
-            const bool gathered = smap.on();
-            const int nbox_a = gathered ? BM / l_p : 1;                         // <= 16
-            int my_src = 0;
-            if (gathered && lane < nbox_a) my_src = src_of(smap, row0 + lane * l_p, e, ctl->offs[e], Bm);   // Bm: zero-filled box
+            const int e = e_next, row0 = row0_next, my_src = src_next;
+            bool looked = false;
             for (int kb = 0; kb < kb1 && !stop; ++kb) {
                 if (!acquire(STAGE)) { stop = true; break; }
                 uint8_t* sa = smem + stage * STAGE;
@@ -148,8 +155,10 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     uint8_t* sb = smem + stage * STAGE + A_BYTES;
                     if (lane < nbox) tma_load_3d(sb + lane * 8192, &tmW2, j * 256 + lane * 64, kb * BK, e, &ctl->full[stage]);
                     advance();
+                    if (!looked && j * kb2 + kb + 1 == STAGES) { look_up(tile + gridDim.x); looked = true; }
                 }
             }
+            if (!looked) look_up(tile + gridDim.x);
         }
         if (lane == 0 && *abort_flag) {      // let this CTA's own copies land before it exits
             for (int s = 0; s < STAGES; ++s)

@@ -62,6 +62,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return false;
 }
 
+// The same for a role that is one thread (a TMA producer, an MMA issuer) and sits between other warps' steps: it
+// polls without letting the hardware suspend it first (a suspended try_wait answers a few hundred ns late), then
+// falls back to the bounded wait above.
+__device__ __forceinline__ bool mbar_wait_spin(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* status) {
+    for (int it = 0; it < 20000; ++it)
+        if (mbar_test_wait(bar, parity)) return true;
+    return mbar_wait(bar, parity, abort_flag, status);
+}
+
 // ---- TMA --------------------------------------------------------------------------------------
 __device__ __forceinline__ void prefetch_tmap(const CUtensorMap* m) {
     asm volatile("prefetch.tensormap [%0];" :: "l"(m) : "memory");
