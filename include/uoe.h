@@ -175,8 +175,9 @@ uoe_status uoe_route_balance_backward(const uoe_problem* prob, const void* x, co
  *   y[b,t,:] = x[b,t,:] + sum over (expert i, patch j) that selected token t of
  *              gate[b,i,j] * ( phi( x[b,t,:] W1[i] + b1[i] ) W2[i] + b2[i] )
  * W1 [n,d,d_e] holds the column slices of the first layer, W2 [n,d_e,d] the row slices of the
- * second (Eq. 1-7); no activation follows the second layer.  b1 [n,d_e], b2 [n,d] may be NULL
- * (biases are supported for float32 only).  The routing arrays are the outputs of uoe_route or any
+ * second (Eq. 1-7); no activation follows the second layer.  b1 [n,d_e], b2 [n,d] (in prob->dtype) may be NULL;
+ * they are the in-place bias of the batched product (Section III-D.2): b1[i] enters before phi, b2[i] is added to
+ * expert i's output before the combine weight (the backward entry point does not return their gradients).  The routing arrays are the outputs of uoe_route or any
  * arrays of the same form supplied by the caller (sorted, in range, offsets consistent with
  * expert_idx).  With UOE_FLAG_GATE the combine weight is gate[b,s,u], otherwise 1.  saved_h, if
  * not NULL, receives the pre-activation x W1[i] of every routed row,

@@ -234,7 +234,7 @@ uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s);
 bool mlp_can_fuse(const Dims& D);
 uoe_status launch_mlp_fused(const Dims& D, const void* A, const void* W1, const void* W2, void* z, void* pre,
                             const int* offsets, int act, const void* gather_x, const SrcMap& map, int* status,
-                            cudaStream_t s);
+                            cudaStream_t s, const void* b1 = nullptr, const void* b2 = nullptr);
 
 // ---- forward halves behind the routing plan (shared by the per-half entry points and the block entry) ----
 struct MlpFwdBufs { void* xg; void* a; void* z; };

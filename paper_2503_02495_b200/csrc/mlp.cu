@@ -51,9 +51,9 @@ uoe_status uoe::mlp_forward_run(const Dims& D, const uoe_problem* prob, const vo
     GemmArgs g2{a, W2, b2, z, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
     g1.label = "gemm1_act";
     g2.label = "gemm2";
-    if (mlp_can_fuse(D)) {                    // (bf16: no biases)      narrow experts: both GEMMs in one kernel, the hidden tile stays on chip
+    if (mlp_can_fuse(D)) {                    // narrow experts: both GEMMs in one kernel, the hidden tile stays on chip
         st = launch_mlp_fused(D, xg, W1, W2, z, saved_h, expert_offsets, prob->act, fused ? x : nullptr, map, status,
-                              stream);
+                              stream, b1, b2);
         if (st != UOE_OK) return st;
     } else if (D.bf16) {
         st = launch_gemm_bf16(g1, status, stream);
@@ -79,7 +79,8 @@ uoe_status uoe::mlp_forward_check(const uoe_problem* prob, Dims& D, const void* 
     if (!aligned16(x) || !aligned16(W1) || !aligned16(W2) || !aligned16(y) || (saved_h && !aligned16(saved_h)))
         return UOE_ERR_INVALID_ARG;
     if ((D.d_e * D.esize) % 16 != 0) return UOE_ERR_UNSUPPORTED;
-    if (D.bf16 && (b1 || b2)) return UOE_ERR_UNSUPPORTED;
+    if ((b1 && !aligned16(b1)) || (b2 && !aligned16(b2))) return UOE_ERR_INVALID_ARG;
+    if (D.bf16 && (b1 || b2) && D.d_e % 64 != 0) return UOE_ERR_UNSUPPORTED;
     return UOE_OK;
 }
 

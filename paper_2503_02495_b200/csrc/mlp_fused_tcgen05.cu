@@ -48,7 +48,8 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  const __grid_constant__ CUtensorMap tmW1, const __grid_constant__ CUtensorMap tmW2,
                  const __grid_constant__ CUtensorMap tmZ, __nv_bfloat16* __restrict__ pre,
                  const int* __restrict__ offsets, int n, int d, int act, int* status,
-                 const SrcMap smap, int l_p, int Bm) {
+                 const SrcMap smap, int l_p, int Bm,
+                 const __nv_bfloat16* __restrict__ b1 /* [n, 256] or null */, const __nv_bfloat16* __restrict__ b2 /* [n, d] or null */) {
     pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -246,6 +247,16 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 float f[64];
 #pragma unroll
                 for (int q = 0; q < 64; ++q) f[q] = __uint_as_float(v[q]);
+                if (b1) {                                    // the expert's bias row of the first layer
+                    const uint4* bp = (const uint4*)(b1 + (size_t)e * DE + g * 64);
+#pragma unroll
+                    for (int q8 = 0; q8 < 8; ++q8) {
+                        float bv[8];
+                        unpack16<__nv_bfloat16>(bp[q8], bv);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) f[8 * q8 + q] += bv[q];
+                    }
+                }
                 if (pre) {
                     uint4* dst = (uint4*)(pre + (size_t)(row0 + trow) * DE + g * 64);
 #pragma unroll
@@ -279,6 +290,12 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     float f[8];
 #pragma unroll
                     for (int q = 0; q < 8; ++q) f[q] = __uint_as_float(v[8 * c + q]);
+                    if (b2) {                                // the expert's bias row of the second layer
+                        float bv[8];
+                        unpack16<__nv_bfloat16>(*(const uint4*)(b2 + (size_t)e * d + g * 64 + 8 * c), bv);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) f[q] += bv[q];
+                    }
                     *(uint4*)(stg + lane * 128 + ((c ^ (lane & 7)) << 4)) = pack8(f);
                 }
                 fence_async_smem();
@@ -305,10 +322,10 @@ mlp_fused_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 bool mlp_can_fuse(const Dims& D) { return D.bf16 && D.d_e == DE && D.d % 64 == 0 && D.d <= 512 && D.n <= 31; }
 
 // A: routed rows [rows_max, d] (or gathered from gather_x through src_patch), W1 [n, d, 256], W2 [n, 256, d],
-// z [rows_max, d]; pre (optional) [rows_max, 256] receives the pre-activation.
+// z [rows_max, d]; pre (optional) [rows_max, 256] receives the pre-activation; b1 [n, 256], b2 [n, d] optional biases.
 uoe_status launch_mlp_fused(const Dims& D, const void* A, const void* W1, const void* W2, void* z, void* pre,
                             const int* offsets, int act, const void* gather_x, const SrcMap& map, int* status,
-                            cudaStream_t s) {
+                            cudaStream_t s, const void* b1, const void* b2) {
     if (!mlp_can_fuse(D) || D.Rmax % BM != 0) return UOE_ERR_UNSUPPORTED;
     if (gather_x && (!map.on() || D.l_p < 8 || D.l_p % 8 != 0 || BM % D.l_p != 0)) return UOE_ERR_INVALID_ARG;
     static DeviceOnce once;
@@ -350,7 +367,8 @@ uoe_status launch_mlp_fused(const Dims& D, const void* A, const void* W1, const 
     if (grid < 1) grid = 1;
     ProfScope ps("mlp_fused", s);
     launch_k(mlp_fused_kernel, dim3(grid), dim3(THREADS), (size_t)SMEM, s, tmA, tmX, tmW1, tmW2, tmZ, (__nv_bfloat16*)pre, offsets,
-             D.n, D.d, act, status, gather_x ? map : SrcMap(), D.l_p, (int)(D.B * D.m));
+             D.n, D.d, act, status, gather_x ? map : SrcMap(), D.l_p, (int)(D.B * D.m), (const __nv_bfloat16*)b1,
+             (const __nv_bfloat16*)b2);
     UOE_LAUNCHED();
     return UOE_OK;
 }

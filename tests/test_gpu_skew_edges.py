@@ -85,3 +85,37 @@ def test_float32_path_with_bias():
     ro = orc.with_selection(x.f64, Wr.f64, r.expert_idx.cpu().numpy(), r.patch_idx.cpu().numpy(), w.m, w.L_valid)
     ref = orc.mlp_forward(x.f64, W1.f64, W2.f64, ro, w.act, residual=False, b1=b1.f64, b2=b2.f64)
     assert rel_inf(to_f64(y), ref) <= 1e-4
+
+
+@pytest.mark.parametrize("kw", [dict(d=384, d_ff=768, n=3),                 # narrow experts: the one-kernel MLP
+                                dict(d=256, d_ff=2048, n=4),                # 512-wide experts: two grouped GEMMs
+                                dict(d=128, d_ff=4 * 192, n=4)])            # 64-column GEMM tiles
+def test_bfloat16_path_with_bias(kw):
+    """The in-place bias of the batched product (Section III-D.2) on the tensor-core path: b1 before phi, b2 on every
+    expert's output before the combine weight."""
+    import paper_2503_02495_b200 as uoe
+    base = dict(B=5, L=224, L_valid=197, m=14, c=7, k=2, H=0, d_h=0, dtype="bf16", w_std=0.05, act="silu")
+    base.update(kw)
+    w = gen.tiny(**base)
+    x, Wr = gen.make_x(w), gen.store(gen.make_router(w).f64 * 20, "bf16")
+    W1, W2 = gen.make_mlp_weights(w)
+    b1 = gen.store(gen.normal(7, 20, (w.n, w.d_e), 0.2), "bf16")
+    b2 = gen.store(gen.normal(7, 21, (w.n, w.d), 0.2), "bf16")
+    prob = problem_of(w, "mlp", residual=False)
+    xd = to_dev(x)
+    r = uoe.uoe_route(prob, xd, to_dev(Wr))
+    saved_h = uoe.alloc_saved_h(prob)
+    y = uoe.uoe_mlp_forward(prob, xd, to_dev(W1), to_dev(W2), r, b1=to_dev(b1), b2=to_dev(b2), saved_h=saved_h)
+    ro = orc.with_selection(x.f64, Wr.f64, r.expert_idx.cpu().numpy(), r.patch_idx.cpu().numpy(), w.m, w.L_valid)
+    ref = orc.mlp_forward(x.f64, W1.f64, W2.f64, ro, w.act, residual=False, b1=b1.f64, b2=b2.f64)
+    ref0 = orc.mlp_forward(x.f64, W1.f64, W2.f64, ro, w.act, residual=False)
+    assert np.abs(ref - ref0).max() > 0.05 * np.abs(ref).max()          # the biases matter in this case
+    assert rel_inf(to_f64(y), ref) <= TOL
+    # the saved pre-activation includes b1: first real row of the first pair of expert e
+    offs = r.expert_offsets.cpu().numpy()
+    e_idx, p_idx = r.expert_idx.cpu().numpy(), r.patch_idx.cpu().numpy()
+    b, s = 0, 0
+    e, j = int(e_idx[b, s]), int(p_idx[b, s, 0])
+    row = int(offs[e]) + int((e_idx[:b] == e).sum()) * w.c * (w.L // w.m)
+    h_ref = x.f64[b, j * (w.L // w.m)] @ W1.f64[e] + b1.f64[e]
+    assert np.abs(to_f64(saved_h[row]) - h_ref).max() <= TOL * np.abs(h_ref).max()
