@@ -32,6 +32,11 @@ CASES = {
     "three_tiles_ragged": _w(B=2, L=512, L_valid=512, m=8, c=5, d=128, n=4, k=2, H=4),
     "three_tiles_causal_pad": _w(B=2, L=512, L_valid=470, m=8, c=5, d=128, n=4, k=3, H=8, causal=True),
     "full_selection": _w(k=2, c=6, causal=True),
+    # many (sample, expert) pairs: at least two units per SM, the launches that take the persistent two-pipeline kernel
+    # (the cases above and cfg2 / cfg3 have fewer and take the one-unit-per-CTA kernel; cfg4 takes the persistent one)
+    "many_pairs_causal_pad": _w(B=80, L=256, L_valid=250, m=8, c=6, d=64, n=2, k=2, H=2, causal=True),
+    "many_pairs_two_heads": _w(B=80, L=256, L_valid=256, m=8, c=6, d=128, n=2, k=2, H=4),
+    "many_pairs_three_tiles": _w(B=52, L=512, L_valid=470, m=8, c=5, d=128, n=4, k=3, H=4, causal=True),
     "cfg2": gen.WORKLOADS["cfg2_lm"],
     "cfg3": gen.WORKLOADS["cfg3_long"],
     "cfg4": gen.WORKLOADS["cfg4_vit"],
@@ -67,7 +72,7 @@ def test_attention_term_matches_oracle(name):
     assert np.all(y[:, w.L_valid:] == 0)
 
 
-@pytest.mark.parametrize("name", ["one_tile", "pad_causal", "cfg2", "cfg4"])
+@pytest.mark.parametrize("name", ["one_tile", "pad_causal", "many_pairs_causal_pad", "cfg2", "cfg4"])
 def test_residual_output_matches_oracle(name):
     w = CASES[name]
     y, ref, x, r, ro, _ = _run(w, residual=True)
@@ -76,7 +81,8 @@ def test_residual_output_matches_oracle(name):
 
 
 @pytest.mark.parametrize("name,d_rope", [("one_tile_causal", 64), ("pad", 32), ("three_tiles_causal_pad", 16),
-                                         ("two_heads_per_expert", 32), ("cfg3", 32), ("cfg4", 64)])
+                                         ("two_heads_per_expert", 32), ("many_pairs_three_tiles", 32), ("cfg3", 32),
+                                         ("cfg4", 64)])
 def test_attention_with_rotary_embedding_matches_oracle(name, d_rope):
     """Eq. 32: the last d_rope channels of every head of q and k rotated by the token's position in its sample."""
     w = CASES[name]
@@ -118,9 +124,10 @@ def test_full_selection_equals_multihead_attention():
         assert rel_inf(y[b], acc) <= TOL
 
 
-def test_lse_output():
+@pytest.mark.parametrize("name", ["three_tiles_causal_pad", "many_pairs_two_heads", "many_pairs_causal_pad"])
+def test_lse_output(name):
     import paper_2503_02495_b200 as uoe
-    w = CASES["three_tiles_causal_pad"]
+    w = CASES[name]
     y, (ref, lse_ref), x, r, ro, lse = _run(w, residual=False, want_lse=True)
     assert rel_inf(y, ref) <= TOL
     lse = lse.cpu().numpy()
