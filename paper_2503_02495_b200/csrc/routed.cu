@@ -8,6 +8,38 @@ namespace {
 constexpr int kThreads = 256;
 
 // ---------------------------------------------------------------------------------------------
+// pair rows for many samples: one CTA passes over expert_idx [B,k] once, a warp per expert, 32 samples per step,
+// and writes where every (sample, slot) pair's rows start (samples ascending inside an expert's region).  O(B k)
+// work in all, where plan_kernel's own scan of the earlier samples is O(B k) per sample.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPlanScanMaxB = 512;        // up to here every sample's CTA scans the earlier samples itself
+
+__global__ void __launch_bounds__(1024)
+plan_rows_kernel(const int* __restrict__ expert_idx, const int* __restrict__ offsets, int B, int n, int k, int l_a,
+                 int* __restrict__ pair_row, int* status) {
+    pdl_trigger();
+    pdl_wait();
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int i = warp; i < n; i += 32) {
+        const int off_i = offsets[i];
+        int running = 0;
+        for (int b0 = 0; b0 < B; b0 += 32) {
+            const int b = b0 + lane;
+            int slot = -1;
+            if (b < B)
+                for (int s = 0; s < k; ++s) {
+                    const int e = expert_idx[(size_t)b * k + s];
+                    if (e < 0 || e >= n) set_status(status, UOE_ERR_DEVICE_INDEX);
+                    if (e == i) slot = s;
+                }
+            const unsigned ball = __ballot_sync(0xffffffffu, slot >= 0);
+            if (slot >= 0) pair_row[(size_t)b * k + slot] = off_i + (running + __popc(ball & ((1u << lane) - 1u))) * l_a;
+            running += __popc(ball);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // plan: grid B, 128 threads, dynamic shared memory 8*k*c bytes.  Everything a sample needs from global memory
 // (its routing arrays, the offsets, the expert choices of the samples before it) is fetched in one round of
 // independent loads; the rest runs out of shared memory.
@@ -18,7 +50,7 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
             int* __restrict__ pair_row, int* __restrict__ inv_row, float* __restrict__ inv_gate,
             int* __restrict__ expert_end, int* status, float* __restrict__ row_gate, float* __restrict__ row_valid,
             int Lv, int use_gate, int* __restrict__ src_patch, uint4* __restrict__ tail, long long tail_row_vecs,
-            long long rows_max) {
+            long long rows_max, int rows_given /* pair_row already holds every pair's first row (plan_rows_kernel) */) {
     pdl_trigger();
     pdl_wait();
     extern __shared__ int s_dyn[];
@@ -42,7 +74,7 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
         s_pi[idx] = pj;
         s_g[idx] = gate[(size_t)b * k * c + idx];
     }
-    {   // choices of the samples before b, per expert: lane i of each warp counts expert i through ballots
+    if (!rows_given) {   // choices of the samples before b, per expert: lane i of each warp counts expert i through ballots
         int acc = 0;
         const int lane = tid & 31;
         for (int i0 = 0; i0 < b * k; i0 += 128) {
@@ -57,9 +89,9 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
     }
     __syncthreads();
     if (tid < k) {
-        const int row = offs[my_e[tid]] + hist[my_e[tid]] * l_a;
+        const int row = rows_given ? pair_row[b * k + tid] : offs[my_e[tid]] + hist[my_e[tid]] * l_a;
         prow[tid] = row;
-        pair_row[b * k + tid] = row;
+        if (!rows_given) pair_row[b * k + tid] = row;
     }
     __syncthreads();
     for (int idx = tid; idx < m * k; idx += 128) {          // inverse map: which routed rows feed patch j
@@ -79,9 +111,20 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
     }
     if (b == B - 1) {          // the last sample has seen every choice: ends of the expert regions, padding blocks
         __shared__ int s_end[32];
-        if (tid < k) atomicAdd(&hist[my_e[tid]], 1);
-        __syncthreads();
-        if (tid < n) s_end[tid] = expert_end[tid] = offs[tid] + hist[tid] * l_a;
+        if (rows_given) {      // the last pair of a region starts l_a rows before its end: the largest first row per expert
+            if (tid < n) s_end[tid] = offs[tid];
+            __syncthreads();
+            for (int idx = tid; idx < B * k; idx += 128) {
+                const int e = expert_idx[idx];
+                if (e >= 0 && e < n) atomicMax(&s_end[e], pair_row[idx] + l_a);
+            }
+            __syncthreads();
+            if (tid < n) expert_end[tid] = s_end[tid];
+        } else {
+            if (tid < k) atomicAdd(&hist[my_e[tid]], 1);
+            __syncthreads();
+            if (tid < n) s_end[tid] = expert_end[tid] = offs[tid] + hist[tid] * l_a;
+        }
         __syncthreads();
         for (int i = 0; i < n; ++i)
             for (int rb = s_end[i] / l_p + tid; rb < offs[i + 1] / l_p; rb += 128) src_patch[rb] = -1;
@@ -302,10 +345,16 @@ uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_id
                        long long tail_row_bytes) {
     const size_t smem = (size_t)D.k * D.c * 8;
     if (smem > 32 * 1024) return UOE_ERR_UNSUPPORTED;      // a sample's routing arrays live in shared memory
+    const bool many = D.B > kPlanScanMaxB;
+    if (many) {
+        ProfScope ps("plan_rows", s);
+        launch_k(plan_rows_kernel, dim3(1), dim3(1024), 0, s, expert_idx, offsets, D.B, D.n, D.k, D.l_a, P.pair_row, status);
+        UOE_LAUNCHED();
+    }
     ProfScope ps("plan", s);
     launch_k(plan_kernel, dim3(D.B), dim3(128), smem, s, expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
                                     P.pair_row, P.inv_row, P.inv_gate, P.expert_end, status, P.row_gate, P.row_valid,
-                                    D.Lv, use_gate ? 1 : 0, P.src_patch, (uint4*)tail, tail_row_bytes / 16, D.Rmax);
+                                    D.Lv, use_gate ? 1 : 0, P.src_patch, (uint4*)tail, tail_row_bytes / 16, D.Rmax, many ? 1 : 0);
     UOE_LAUNCHED();
     return UOE_OK;
 }

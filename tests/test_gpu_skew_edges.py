@@ -119,3 +119,29 @@ def test_bfloat16_path_with_bias(kw):
     row = int(offs[e]) + int((e_idx[:b] == e).sum()) * w.c * (w.L // w.m)
     h_ref = x.f64[b, j * (w.L // w.m)] @ W1.f64[e] + b1.f64[e]
     assert np.abs(to_f64(saved_h[row]) - h_ref).max() <= TOL * np.abs(h_ref).max()
+
+
+def test_many_samples_take_the_one_pass_pair_rows():
+    """More than 512 samples: the plan's pair rows come from one pass over expert_idx instead of every sample scanning
+    the samples before it; forward (MLP and attention) and MLP backward against the oracle, skewed loads."""
+    import paper_2503_02495_b200 as uoe
+    w = gen.tiny(B=700, L=32, L_valid=29, m=4, c=2, d=64, n=5, k=2, d_ff=5 * 64, H=5, d_h=64, dtype="bf16", w_std=0.05)
+    res = _block(w, skew=2.0)
+    for block, (err, load) in res.items():
+        assert err <= TOL, (block, err)
+        assert load.sum() == w.B * w.k
+    w = gen.tiny(B=600, L=32, L_valid=29, m=4, c=2, d=128, n=5, k=2, d_ff=5 * 128, H=0, d_h=0, dtype="bf16", w_std=0.05)
+    Wr = gen.store(gen.make_router(w).f64 * 10, w.dtype)
+    x = gen.make_x(w, skew_beta=2.0, W_r=Wr.f64)
+    W1, W2 = gen.make_mlp_weights(w)
+    dy = gen.make_dy(w)
+    prob = problem_of(w, "mlp", residual=False)
+    xd, W1d, W2d, Wrd = to_dev(x), to_dev(W1), to_dev(W2), to_dev(Wr)
+    r = uoe.uoe_route(prob, xd, Wrd)
+    saved_h = uoe.alloc_saved_h(prob)
+    uoe.uoe_mlp_forward(prob, xd, W1d, W2d, r, saved_h=saved_h)
+    got = uoe.uoe_mlp_backward(prob, xd, W1d, W2d, Wrd, r, saved_h, to_dev(dy))
+    ro = orc.with_selection(x.f64, Wr.f64, r.expert_idx.cpu().numpy(), r.patch_idx.cpu().numpy(), w.m, w.L_valid)
+    ref = orc.mlp_backward(x.f64, W1.f64, W2.f64, Wr.f64, ro, dy.f64, w.act, False, True)
+    for nm, g, rr in zip(("dx", "dW1", "dW2", "dW_r"), got, ref[:4]):
+        assert rel_inf(to_f64(g), rr) <= TOL, nm
