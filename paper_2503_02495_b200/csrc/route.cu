@@ -35,7 +35,8 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
                               int* __restrict__ expert_idx,
                               int* __restrict__ patch_idx, float* __restrict__ gate, float* __restrict__ p_samp,
                               float* __restrict__ p_patch, int* __restrict__ offsets, unsigned* __restrict__ masks,
-                              int* __restrict__ ticket, const PlanPtrs plan) {
+                              int* __restrict__ ticket, const PlanPtrs plan,
+                              const float* local_scores = nullptr /* [m,n] in shared memory: used instead of `partial` */) {
     constexpr int NW = NT / 32;
     constexpr int kMaskCache = 1024;       // samples whose masks the last CTA keeps in shared memory
     __shared__ float ps[32];               // sample gate
@@ -65,8 +66,12 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
             const bool valid = j < m && i < n;
             float s = 0.f;
             if (valid) {
-                const float* p = partial + ((size_t)(b * m + j) * nparts) * n + i;
-                for (int ch = 0; ch < nparts; ++ch) s += __ldcg(p + (size_t)ch * n);     // written by other CTAs: read from L2
+                if (local_scores) {
+                    s = local_scores[j * n + i];
+                } else {
+                    const float* p = partial + ((size_t)(b * m + j) * nparts) * n + i;
+                    for (int ch = 0; ch < nparts; ++ch) s += __ldcg(p + (size_t)ch * n);     // written by other CTAs: read from L2
+                }
             }
             raw_acc += s;
             const int cnt = valid ? max(0, min(l_p, Lv - j * l_p)) : 0;
@@ -393,6 +398,91 @@ route_kernel(const T* __restrict__ x, const T* __restrict__ W_r, float* __restri
     }
 }
 
+// One CTA per sample, for many samples of few small patches (image-sized inputs: a sample is a few hundred KB and
+// there are at least as many samples as SMs).  The CTA's thread groups (CT column threads each) take the sample's
+// patches in turn, a thread summing all rows of its 16-byte column piece, so no partial result crosses a thread; the
+// pooled patches meet W_r (staged once per CTA) in shared memory and the selection follows in the same CTA: no scores
+// in global memory, no ticket per sample, one launch.
+constexpr int kSampleThreads = 512;
+
+template <typename T>
+__global__ void __launch_bounds__(kSampleThreads, 2)
+route_sample_kernel(const T* __restrict__ x, const T* __restrict__ W_r, int B, int L, int Lv, int d, int n, int k, int m, int c,
+                    int l_p, int CT, int use_gate, int* __restrict__ expert_idx, int* __restrict__ patch_idx,
+                    float* __restrict__ gate, float* __restrict__ p_samp, float* __restrict__ p_patch,
+                    int* __restrict__ offsets, int* __restrict__ ctl, unsigned* __restrict__ masks, const PlanPtrs plan) {
+    pdl_trigger();
+    pdl_wait();
+    constexpr int V = Vec16<T>::N;
+    constexpr int NT = kSampleThreads;
+    extern __shared__ uint4 s_dyn4[];
+    const int wbytes = (d * n * (int)sizeof(T) + 15) / 16 * 16;
+    const T* s_w = (const T*)s_dyn4;                                          // W_r [d, n]
+    float* s_pool = (float*)((char*)s_dyn4 + wbytes);                         // [m, d] column sums of every patch
+    float* s_sc = s_pool + (size_t)m * d;                                     // [m, n] scores
+    float* s_pp = s_sc + (size_t)m * n;                                       // [n, m] gate values (selection)
+    const int tid = threadIdx.x, b = blockIdx.x;
+    {
+        const int nvec = d * n * (int)sizeof(T) / 16;
+        const uint4* src = (const uint4*)W_r;
+        for (int q = tid; q < nvec; q += NT)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 16;" :: "r"((uint32_t)__cvta_generic_to_shared(s_dyn4 + q)), "l"(src + q) : "memory");
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    }
+    // ---- column sums: group g takes patches g, g + G, ... ----
+    const int G = NT / CT, g = tid / CT, col = (tid % CT) * V;
+    for (int j = g; j < m; j += G) {
+        const int rows = max(0, min(l_p, Lv - j * l_p));
+        float cs[V];
+#pragma unroll
+        for (int v = 0; v < V; ++v) cs[v] = 0.f;
+        if (col < d) {
+            const T* base = x + ((size_t)b * L + (size_t)j * l_p) * d + col;
+            int r = 0;
+            for (; r + 7 < rows; r += 8) {
+                uint4 q[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) q[u] = ld_stream16(base + (size_t)(r + u) * d);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    float f[V];
+                    unpack16<T>(q[u], f);
+#pragma unroll
+                    for (int v = 0; v < V; ++v) cs[v] += f[v];
+                }
+            }
+            for (; r < rows; ++r) {
+                float f[V];
+                unpack16<T>(ld_stream16(base + (size_t)r * d), f);
+#pragma unroll
+                for (int v = 0; v < V; ++v) cs[v] += f[v];
+            }
+#pragma unroll
+            for (int v = 0; v < V; ++v) s_pool[(size_t)j * d + col + v] = cs[v];
+        }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncthreads();
+    // ---- scores[j, i] = pooled patch j . W_r[:, i]: `parts` threads per score, columns dealt round robin, summed by a
+    //      fixed shuffle tree ----
+    int parts = 1;
+    while (parts < 32 && 2 * parts * m * n <= NT) parts <<= 1;
+    for (int p0 = 0; p0 < m * n; p0 += NT / parts) {
+        const int p = p0 + tid / parts, sub = tid % parts;
+        float acc = 0.f;
+        if (p < m * n) {
+            const int j = p / n, i = p % n;
+            const float* pj = s_pool + (size_t)j * d;
+            for (int cc = sub; cc < d; cc += parts) acc = fmaf(pj[cc], to_f32(s_w[cc * n + i]), acc);
+        }
+        for (int o = parts >> 1; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (p < m * n && sub == 0) s_sc[p] = acc;
+    }
+    __syncthreads();
+    select_sample<NT>(s_pp, nullptr, 1, b, B, Lv, n, k, m, c, l_p, use_gate, expert_idx, patch_idx, gate, p_samp, p_patch, offsets,
+                      masks, ctl + 1, plan, s_sc);
+}
+
 // Selection as a kernel of its own (after a route_kernel launch without tickets): grid B, one CTA per sample.
 __global__ void __launch_bounds__(kScoreThreads)
 route_select_kernel(const float* __restrict__ scores, int nparts, int B, int Lv, int n, int k, int m, int c, int l_p,
@@ -406,7 +496,7 @@ route_select_kernel(const float* __restrict__ scores, int nparts, int B, int Lv,
                                  p_samp, p_patch, offsets, masks, ctl + 1, plan);
 }
 
-struct RouteWs { size_t tickets, scores, total; int nchunks, CT, rsplit, rows_per_cta; size_t smem, wb; bool two_kernels, small_ctas; };
+struct RouteWs { size_t tickets, scores, total; int nchunks, CT, rsplit, rows_per_cta; size_t smem, wb; bool two_kernels, small_ctas, per_sample; size_t sample_smem; };
 
 constexpr int kWblkBytes = 16384;       // shared memory for a CTA's rows of W_r
 constexpr size_t kMaskOffset = kControlBytes / 2;      // control block: status block, sample tickets [B]; second half: expert masks [B]
@@ -446,6 +536,17 @@ RouteWs route_ws(const Dims& D) {
     }
     // they also hand the selection to a second launch: thousands of CTAs would otherwise each pay a fence and a ticket
     if (r.small_ctas) r.two_kernels = true;
+    // ... unless a whole sample is one CTA's work (route_sample_kernel): at least one CTA per SM, patches of one column
+    // chunk, at most 64 rows per thread, everything of a sample in half an SM's shared memory
+    {
+        int CTs = 1;
+        while (CTs * V < D.d) CTs <<= 1;
+        const int Gs = CTs <= kSampleThreads ? kSampleThreads / CTs : 0;
+        r.sample_smem = ((size_t)D.d * D.n * D.esize + 15) / 16 * 16 + ((size_t)D.m * D.d + 2 * (size_t)D.m * D.n) * sizeof(float);
+        r.per_sample = Gs >= 1 && D.B >= 128 && D.l_p <= 32 && ((D.m + Gs - 1) / Gs) * D.l_p <= 64 && r.sample_smem <= 100 * 1024 &&
+                       (size_t)D.B * D.L * D.d * D.esize < ((size_t)64 << 20);
+        if (r.per_sample) r.CT = CTs;
+    }
     r.smem = r.two_kernels ? r.wb : (sel > r.wb ? sel : r.wb);
     return r;
 }
@@ -469,6 +570,24 @@ uoe_status route_launch(const Dims& D, uint32_t flags, const void* x, const void
 #define UOE_ROUTE_LAUNCH(T, TICKET, NT, SMEM) \
         launch_k(route_kernel<T, TICKET, NT>, grid, dim3(NT), SMEM, stream, UOE_ROUTE_ARGS(T))
     cudaError_t e;
+    if (W.per_sample) {
+        static DeviceOnce once_bf16, once_f32;
+        const uoe_status so = D.bf16 ? smem_opt_in(once_bf16, route_sample_kernel<__nv_bfloat16>, 100 * 1024)
+                                     : smem_opt_in(once_f32, route_sample_kernel<float>, 100 * 1024);
+        if (so != UOE_OK) return so;
+        ProfScope ps(profile ? "route" : nullptr, stream);
+        if (D.bf16)
+            e = launch_k(route_sample_kernel<__nv_bfloat16>, dim3(D.B), dim3(kSampleThreads), W.sample_smem, stream, (const __nv_bfloat16*)x,
+                         (const __nv_bfloat16*)W_r, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, use_gate, expert_idx, patch_idx,
+                         gate, p_samp, p_patch, expert_offsets, ctl, masks, plan);
+        else
+            e = launch_k(route_sample_kernel<float>, dim3(D.B), dim3(kSampleThreads), W.sample_smem, stream, (const float*)x,
+                         (const float*)W_r, D.B, D.L, D.Lv, D.d, D.n, D.k, D.m, D.c, D.l_p, W.CT, use_gate, expert_idx, patch_idx,
+                         gate, p_samp, p_patch, expert_offsets, ctl, masks, plan);
+        if (e != cudaSuccess) return UOE_ERR_CUDA;
+        UOE_LAUNCHED();
+        return UOE_OK;
+    }
     {
         ProfScope ps(profile ? "route" : nullptr, stream);
         if (W.small_ctas) e = D.bf16 ? UOE_ROUTE_LAUNCH(__nv_bfloat16, false, 64, W.smem) : UOE_ROUTE_LAUNCH(float, false, 64, W.smem);
