@@ -144,9 +144,21 @@ rvec_kernel(const T* __restrict__ W_r, const float* __restrict__ G, float* __res
     const int bj = blockIdx.x;
     if (threadIdx.x < n) sG[threadIdx.x] = G[(size_t)bj * n + threadIdx.x];
     __syncthreads();
+    constexpr int V = Vec16<T>::N;
+    const bool vec_rows = (n % V) == 0;               // a row of W_r is a whole number of 16-byte pieces
     for (int dd = threadIdx.x; dd < d; dd += kThreads) {
         float a = 0.f;
-        for (int i = 0; i < n; ++i) a = fmaf(to_f32(W_r[(size_t)dd * n + i]), sG[i], a);
+        if (vec_rows) {
+            const uint4* wr = (const uint4*)(W_r + (size_t)dd * n);
+            for (int q = 0; q < n / V; ++q) {
+                float f[V];
+                unpack16<T>(wr[q], f);
+#pragma unroll
+                for (int v = 0; v < V; ++v) a = fmaf(f[v], sG[q * V + v], a);
+            }
+        } else {
+            for (int i = 0; i < n; ++i) a = fmaf(to_f32(W_r[(size_t)dd * n + i]), sG[i], a);
+        }
         rvec[(size_t)bj * d + dd] = a;
     }
 }
