@@ -69,8 +69,17 @@ __device__ void select_sample(float* pp, const float* __restrict__ partial, int 
                 if (local_scores) {
                     s = local_scores[j * n + i];
                 } else {
+                    // written by other CTAs: read from L2, eight loads in flight, added in ascending order
                     const float* p = partial + ((size_t)(b * m + j) * nparts) * n + i;
-                    for (int ch = 0; ch < nparts; ++ch) s += __ldcg(p + (size_t)ch * n);     // written by other CTAs: read from L2
+                    int ch = 0;
+                    for (; ch + 7 < nparts; ch += 8) {
+                        float t[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) t[u] = __ldcg(p + (size_t)(ch + u) * n);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) s += t[u];
+                    }
+                    for (; ch < nparts; ++ch) s += __ldcg(p + (size_t)ch * n);
                 }
             }
             raw_acc += s;
