@@ -131,6 +131,13 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
         uint32_t phase = 0, issued = 0, issued_parity = 0;
         bool stop = false;
         const int sub_rows = (gather_p || gather_q) ? min(l_p, BK) : BK, nsub = BK / sub_rows;
+        // Source patches of a gathered operand: l_p is a power of two that divides 128, so the slab `sub` of K block kb
+        // of a region that starts at routed row r0 lies in routed patch r0 / l_p + (64 kb + sub_rows sub) / l_p.  The
+        // warp keeps a window of 32 consecutive entries of src_patch in its lanes and reads them with a shuffle: a
+        // look-up in global memory in front of every copy would set the pace of the whole ring.
+        const int lp_shift = __ffs(l_p) - 1;
+        const int my_sub = nsub == 1 ? 0 : (lane & 15) % nsub;
+        const bool gathers = gather_p || gather_q;
         int slot = 0;
         uint32_t sphase = 0;
         for (bool first = true; !stop; first = false) {
@@ -149,7 +156,21 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
             int e, m0, n0, ks, kb_lo, num_kb;
             decode(tile, e, m0, n0, ks, kb_lo, num_kb);
             const int r0 = ctl->offs[e] + kb_lo * BK;
+            const int patch_end = gathers ? (r0 + num_kb * BK + l_p - 1) >> lp_shift : 0;     // routed patches of this tile's rows
+            int win0 = r0 >> lp_shift;
+            int win = (gathers && win0 + lane < patch_end) ? src_patch[win0 + lane] : 0;
             for (int kb = 0; kb < num_kb; ++kb) {
+                int src = 0, prow = 0;
+                if (gathers) {
+                    const int row = r0 + kb * BK;
+                    if (((row + BK - 1) >> lp_shift) >= win0 + 32) {      // (uniform) the block's last slab is past the window
+                        win0 = row >> lp_shift;
+                        win = win0 + lane < patch_end ? src_patch[win0 + lane] : 0;
+                    }
+                    src = __shfl_sync(0xffffffffu, win, (((row + my_sub * sub_rows) >> lp_shift) - win0) & 31);
+                    if (src < 0) src = Bm;                                // no patch: the zero-filled box past the end
+                    prow = (row + my_sub * sub_rows) & (l_p - 1);
+                }
                 int ok = 1;
                 if (lane == 0) ok = (mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) && !*abort_flag) ? 1 : 0;
                 ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -158,33 +179,27 @@ wgrad_kernel(const __grid_constant__ CUtensorMap tmP, const __grid_constant__ CU
                 uint8_t* sb = sa + Cf::A_BYTES;
                 if (lane == 0) mbar_arrive_expect_tx(&ctl->full[stage], Cf::STAGE);
                 __syncwarp();
-                // a gathered operand (Eq. 18 inside the contraction) comes from the source tensor [Bm patches, l_p, cols]:
-                // the 64 routed rows of a K block are 64 / sub_rows slabs of sub_rows rows, each inside one patch
+                // An operand is a tensor of [column blocks of 64][rows][64 columns], so one copy brings all the column
+                // blocks of a stage (the pace of this loop is set by the number of copies it issues, not by their bytes).
+                // A gathered operand (Eq. 18 inside the contraction) comes from the source tensor
+                // [Bm patches][column blocks][l_p rows][64]: the 64 routed rows of a K block are 64 / sub_rows slabs of
+                // sub_rows rows, each inside one patch; with one slab it is one copy as well, with more the boxes are one
+                // column block wide and lane (block, slab) issues its own.
                 const int row = r0 + kb * BK;
                 if (lane < 16) {
-                    const int cnt = (TM / 64) * (gather_p ? nsub : 1);
-                    if (lane < cnt) {
-                        if (gather_p) {
-                            const int cb = lane / nsub, sub = lane % nsub, rr = row + sub * sub_rows;
-                            int src = src_patch[rr / l_p];
-                            if (src < 0) src = Bm;                    // out of range: zero-filled box
-                            tma_load_3d(sa + cb * 8192 + sub * sub_rows * 128, &tmP, m0 + cb * 64, rr % l_p, src, &ctl->full[stage]);
-                        } else {
-                            tma_load_2d(sa + lane * 8192, &tmP, m0 + lane * 64, row, &ctl->full[stage]);
-                        }
+                    if (!gather_p) {
+                        if (lane == 0) tma_load_3d(sa, &tmP, 0, row, m0 / 64, &ctl->full[stage]);
+                    } else if (lane < (nsub == 1 ? 1 : (TM / 64) * nsub)) {
+                        const int cb = nsub == 1 ? 0 : lane / nsub;
+                        tma_load_4d(sa + cb * 8192 + my_sub * sub_rows * 128, &tmP, 0, prow, m0 / 64 + cb, src, &ctl->full[stage]);
                     }
                 } else {
                     const int l2 = lane - 16;
-                    const int cnt = (BN / 64) * (gather_q ? nsub : 1);
-                    if (l2 < cnt) {
-                        if (gather_q) {
-                            const int cb = l2 / nsub, sub = l2 % nsub, rr = row + sub * sub_rows;
-                            int src = src_patch[rr / l_p];
-                            if (src < 0) src = Bm;
-                            tma_load_3d(sb + cb * 8192 + sub * sub_rows * 128, &tmQ, n0 + cb * 64, rr % l_p, src, &ctl->full[stage]);
-                        } else {
-                            tma_load_2d(sb + l2 * 8192, &tmQ, n0 + l2 * 64, row, &ctl->full[stage]);
-                        }
+                    if (!gather_q) {
+                        if (l2 == 0) tma_load_3d(sb, &tmQ, 0, row, n0 / 64, &ctl->full[stage]);
+                    } else if (l2 < (nsub == 1 ? 1 : (BN / 64) * nsub)) {
+                        const int cb = nsub == 1 ? 0 : l2 / nsub;
+                        tma_load_4d(sb + cb * 8192 + my_sub * sub_rows * 128, &tmQ, 0, prow, n0 / 64 + cb, src, &ctl->full[stage]);
                     }
                 }
                 issued |= 1u << stage;
@@ -322,27 +337,22 @@ uoe_status launch_w(const void* P, const void* Q, float* dW, const int* offsets,
         const uoe_status st = smem_opt_in(once, kern, Cf::SMEM);
         if (st != UOE_OK) return st;
     }
+    // operands as [column blocks of 64][rows][64 columns]; a gathered one as [Bm patches][column blocks][l_p rows][64]
     CUtensorMap tmP, tmQ;
-    const uint32_t box[2] = {64, BK};
-    const uint32_t gbox[3] = {64, (uint32_t)(g.l_p < BK ? g.l_p : BK), 1};
-    if (g.gather_p) {      // P rows come from the source tensor [Bm patches, l_p, M]
-        const uint64_t dims[3] = {(uint64_t)M, (uint64_t)g.l_p, (uint64_t)g.Bm};
-        const uint64_t str[2] = {(uint64_t)M * 2, (uint64_t)M * 2 * g.l_p};
-        if (!make_tmap(&tmP, P, 3, dims, str, gbox)) return UOE_ERR_CUDA;
-    } else {
-        const uint64_t dims[2] = {(uint64_t)M, (uint64_t)rows_max};
-        const uint64_t str[1] = {(uint64_t)M * 2};
-        if (!make_tmap(&tmP, P, 2, dims, str, box)) return UOE_ERR_CUDA;
-    }
-    if (g.gather_q) {
-        const uint64_t dims[3] = {(uint64_t)N, (uint64_t)g.l_p, (uint64_t)g.Bm};
-        const uint64_t str[2] = {(uint64_t)N * 2, (uint64_t)N * 2 * g.l_p};
-        if (!make_tmap(&tmQ, Q, 3, dims, str, gbox)) return UOE_ERR_CUDA;
-    } else {
-        const uint64_t dims[2] = {(uint64_t)N, (uint64_t)rows_max};
-        const uint64_t str[1] = {(uint64_t)N * 2};
-        if (!make_tmap(&tmQ, Q, 2, dims, str, box)) return UOE_ERR_CUDA;
-    }
+    const int sub_rows = g.l_p < BK ? g.l_p : BK;
+    auto operand_map = [&](CUtensorMap* tm, const void* base, int cols, int tile_cols, bool gathered) {
+        if (gathered) {
+            const uint64_t dims[4] = {64, (uint64_t)g.l_p, (uint64_t)cols / 64, (uint64_t)g.Bm};
+            const uint64_t str[3] = {(uint64_t)cols * 2, 128, (uint64_t)cols * 2 * g.l_p};
+            const uint32_t box[4] = {64, (uint32_t)sub_rows, (uint32_t)(sub_rows == BK ? tile_cols / 64 : 1), 1};
+            return make_tmap(tm, base, 4, dims, str, box);
+        }
+        const uint64_t dims[3] = {64, (uint64_t)rows_max, (uint64_t)cols / 64};
+        const uint64_t str[2] = {(uint64_t)cols * 2, 128};
+        const uint32_t box[3] = {64, BK, (uint32_t)tile_cols / 64};
+        return make_tmap(tm, base, 3, dims, str, box);
+    };
+    if (!operand_map(&tmP, P, M, MT * BM, g.gather_p) || !operand_map(&tmQ, Q, N, BN, g.gather_q)) return UOE_ERR_CUDA;
     CUtensorMap tmW;      // the output (or the per-split partial outputs) as [ksplit*n*M, N] float32, [32 x 32] pieces
     {
         const uint64_t dims[2] = {(uint64_t)N, (uint64_t)ksplit * n * M};

@@ -39,6 +39,9 @@ CASES = {
     # 256 x 256 tiles handed out longest-first (320 of them, the experts' row counts far apart)
     "tall_tiles_skewed": _w(B=40, L=1152, L_valid=1152, m=9, c=3, d=1024, n=4, k=2, d_ff=4096, w_std=0.02),
     "wgrad_256_skewed": _w(B=12, L=1152, L_valid=1152, m=9, c=3, d=1024, n=5, k=2, d_ff=5 * 4096, w_std=0.02),
+    # the same tiles with patches shorter than a 64-row contraction block (two gathered boxes per block), pad tokens,
+    # and an expert that may get no rows at all
+    "wgrad_256_short_patches_skewed": _w(B=10, L=288, L_valid=270, m=9, c=4, d=1024, n=5, k=2, d_ff=5 * 4096, w_std=0.02),
 }
 
 
