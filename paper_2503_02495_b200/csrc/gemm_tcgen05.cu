@@ -137,9 +137,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     const int num_kb = K / (BK * Cf::KSUB);
     const int total_tiles = ctl->tstart[n] * n_tiles;
 
-    // row tile -> expert, first row, number of 128-row blocks it holds
+    // row tile -> expert, first row, number of 128-row blocks it holds.  A CTA's tiles come in ascending order, so the
+    // search starts at the expert of its previous tile (e is carried by the caller, 0 before the first tile).
     auto locate = [&](int row_tile, int& e, int& row0, int& blocks) {
-        e = 0;
         while (e + 1 < n && row_tile >= ctl->tstart[e + 1]) ++e;
         const int i = row_tile - ctl->tstart[e];
         row0 = ctl->offs[e] + i * (Cf::UNIT * BM);
@@ -153,10 +153,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         uint32_t issued = 0, issued_parity = 0;      // per stage: a load is in flight with this parity
         bool stop = false;
         constexpr int BN_CTA = PAIR ? BN / 2 : BN;              // B columns this CTA loads
-        constexpr int nbox_b = B_KMAJOR ? 1 : BN_CTA / 64;
+        // one copy per operand and stage wherever the rows of a stage are consecutive in memory: the pace of this loop is
+        // set by the number of copies it issues.  W [n, K, N] is mapped as [n][N/64 column blocks][K][64], so a box holds
+        // all the column blocks of a tile; the three side-by-side matrices take one copy each.
+        constexpr int nbox_b = SIDE3 ? 3 : 1;
         const CUtensorMap* tmB_lane = lane == 0 ? &tmB0 : (lane == 1 ? &tmB1 : &tmB2);
+        int e = 0;
         for (int tile = worker; tile < total_tiles && !stop; tile += workers) {
-            int e, row0, blocks;
+            int row0, blocks;
             locate(tile / n_tiles, e, row0, blocks);
             const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
             const CUtensorMap* tmB = mat == 0 ? &tmB0 : (mat == 1 ? &tmB1 : &tmB2);
@@ -164,10 +168,14 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const int my_blocks = PAIR ? (rank < blocks ? 1 : 0) : blocks;
             const int arow0 = row0 + rank * BM;
             const bool gathered = smap.on();
-            const int nbox_a = gathered ? my_blocks * (BM / l_p) : my_blocks;   // <= 32
+            const int nbox_a = gathered ? my_blocks * (BM / l_p) : (my_blocks > 0 ? 1 : 0);   // <= 32; a routed buffer: one box
             int my_src = 0;                                                     // source patch of this lane's box
-            if (gathered && lane < nbox_a) my_src = src_of(smap, arow0 + lane * l_p, e, ctl->offs[e], Bm);
-            const uint32_t stage_bytes = Cf::KSUB * (blocks * A_BLOCK_BYTES + (PAIR ? 2 : 1) * Cf::B_BYTES);   // both CTAs' bytes
+            {
+                const int bx = PAIR ? lane % 16 : lane;       // (pairs: lanes 16.. copy the round's second sub-block)
+                if (gathered && bx < nbox_a) my_src = src_of(smap, arow0 + bx * l_p, e, ctl->offs[e], Bm);
+            }
+            // (pairs: both CTAs' bytes; a routed buffer's box is always MT blocks high, rows past the tile included)
+            const uint32_t stage_bytes = Cf::KSUB * ((gathered || PAIR ? blocks : MT) * A_BLOCK_BYTES + (PAIR ? 2 : 1) * Cf::B_BYTES);
             for (int kb = 0; kb < num_kb; ++kb) {
                 int ok = 1;
                 if (lane == 0) ok = (mbar_wait(&ctl->empty[stage], phase ^ 1, abort_flag, status) && !*abort_flag) ? 1 : 0;
@@ -180,29 +188,30 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if constexpr (PAIR) {
                     const uint32_t full0 = map_to_cta(&ctl->full[stage], 0);    // rank 0's barrier counts both CTAs' bytes
                     const int bcol0 = col0 + rank * BN_CTA;
-#pragma unroll
-                    for (int j = 0; j < Cf::KSUB; ++j) {
+                    // lane (j, box): sub-block j of the round; the sub-blocks' copies leave in the same instruction
+                    {
+                        const int j = lane / 16, bx = lane % 16;              // KSUB = 2
                         const int k0 = (kb * Cf::KSUB + j) * BK;
                         uint8_t* sa_j = sa + j * Cf::SUB;
                         uint8_t* sb_j = sa_j + Cf::A_BYTES;
-                        if (lane < nbox_a) {
-                            if (gathered) tma_load_3d_pair(sa_j + lane * l_p * 128, &tmX, k0, 0, my_src, full0);
+                        if (bx < nbox_a) {
+                            if (gathered) tma_load_3d_pair(sa_j + bx * l_p * 128, &tmX, k0, 0, my_src, full0);
                             else tma_load_2d_pair(sa_j, &tmA, k0, arow0, full0);
                         }
-                        if (lane < nbox_b) {
+                        if (bx == 0) {
                             if (B_KMAJOR) tma_load_3d_pair(sb_j, tmB, k0, bcol0, e, full0);
-                            else tma_load_3d_pair(sb_j + lane * 8192, tmB, bcol0 + lane * 64, k0, e, full0);
+                            else tma_load_4d_pair(sb_j, tmB, 0, k0, bcol0 / 64, e, full0);
                         }
                     }
                 } else {
                     if (lane < nbox_a) {
                         if (gathered) tma_load_3d(sa + lane * l_p * 128, &tmX, kb * BK, 0, my_src, &ctl->full[stage]);
-                        else tma_load_2d(sa + lane * A_BLOCK_BYTES, &tmA, kb * BK, row0 + lane * BM, &ctl->full[stage]);
+                        else tma_load_2d(sa, &tmA, kb * BK, row0, &ctl->full[stage]);
                     }
                     if (lane < nbox_b) {
-                        if (SIDE3) tma_load_3d(sb + lane * 8192, tmB_lane, 0, kb * BK, e, &ctl->full[stage]);
+                        if (SIDE3) tma_load_4d(sb + lane * 8192, tmB_lane, 0, kb * BK, 0, e, &ctl->full[stage]);
                         else if (B_KMAJOR) tma_load_3d(sb, tmB, kb * BK, col0, e, &ctl->full[stage]);
-                        else tma_load_3d(sb + lane * 8192, tmB, col0 + lane * 64, kb * BK, e, &ctl->full[stage]);
+                        else tma_load_4d(sb, tmB, 0, kb * BK, col0 / 64, e, &ctl->full[stage]);
                     }
                 }
                 issued |= 1u << stage;
@@ -221,8 +230,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool stop = false;
+            int e = 0;
             for (int tile = worker; tile < total_tiles && !stop; tile += workers) {
-                int e, row0, blocks;
+                int row0, blocks;
                 locate(tile / n_tiles, e, row0, blocks);
                 if (!mbar_wait(&ctl->tempty[acc], acc_phase ^ 1, abort_flag, status) || *abort_flag) break;
                 tc_fence_after();
@@ -286,8 +296,9 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             __syncwarp();
             if (lane == 0) { tma_store_2d(tm, stg, c0, r0); bulk_commit(); }
         };
+        int e = 0;
         for (int tile = worker; tile < total_tiles; tile += workers) {
-            int e, row0, blocks;
+            int row0, blocks;
             locate(tile / n_tiles, e, row0, blocks);
             const int mat = (tile % n_tiles) / n_tiles_mat, col0 = ((tile % n_tiles) % n_tiles_mat) * BN;
             const CUtensorMap* tmC = mat == 0 ? &tmC0 : (mat == 1 ? &tmC1 : &tmC2);
@@ -403,7 +414,7 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     } else {
         const uint64_t dims[2] = {(uint64_t)g.K, (uint64_t)g.rows_max};
         const uint64_t str[1] = {(uint64_t)g.K * 2};
-        const uint32_t box[2] = {BK, BM};
+        const uint32_t box[2] = {BK, (uint32_t)(MT * BM)};      // all the 128-row blocks of a tile in one box
         if (!make_tmap(&tmA, g.A, 2, dims, str, box)) return UOE_ERR_CUDA;
         tmX = tmA;
     }
@@ -415,11 +426,11 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
             const uint64_t str[2] = {(uint64_t)g.K * 2, (uint64_t)g.K * g.N * 2};
             const uint32_t box[3] = {BK, PAIR ? BN / 2 : BN, 1};
             if (!make_tmap(&tmB[q], Ws[q], 3, dims, str, box)) return UOE_ERR_CUDA;
-        } else {              // W [n, K, N]
-            const uint64_t dims[3] = {(uint64_t)g.N, (uint64_t)g.K, (uint64_t)g.n};
-            const uint64_t str[2] = {(uint64_t)g.N * 2, (uint64_t)g.K * g.N * 2};
-            const uint32_t box[3] = {64, BK, 1};
-            if (!make_tmap(&tmB[q], Ws[q], 3, dims, str, box)) return UOE_ERR_CUDA;
+        } else {              // W [n, K, N] as [n][N/64 column blocks][K][64]
+            const uint64_t dims[4] = {64, (uint64_t)g.K, (uint64_t)g.N / 64, (uint64_t)g.n};
+            const uint64_t str[3] = {(uint64_t)g.N * 2, 128, (uint64_t)g.K * g.N * 2};
+            const uint32_t box[4] = {64, BK, (uint32_t)(BN == 192 ? 1 : (PAIR ? BN / 2 : BN) / 64), 1};
+            if (!make_tmap(&tmB[q], Ws[q], 4, dims, str, box)) return UOE_ERR_CUDA;
         }
     }
     // outputs as [rows_max, N], written in [32 rows x 64 columns] pieces
@@ -469,6 +480,7 @@ uoe_status dispatch(const GemmArgs& g, int* status, cudaStream_t s) {
         if (bn == 256 && g.K % 128 == 0 && tiles256 >= 2 * sm_count()) return launch_one<256, B_KMAJOR, BWD, 1, true>(g, status, s);
     }
     if constexpr (!BWD) {
+        if (bn == 256 && g.K % 128 == 0 && tiles256 >= 2 * sm_count()) return launch_one<256, B_KMAJOR, BWD, 1, true>(g, status, s);
         if (bn == 256 && g.K >= 1024 && tiles256 >= 2 * sm_count()) return launch_one<256, B_KMAJOR, BWD, 2>(g, status, s);
     }
     if (bn == 256) return launch_one<256, B_KMAJOR, BWD, 1>(g, status, s);
