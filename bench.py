@@ -661,29 +661,29 @@ HBM_KERNELS = ("route", "gather", "combine", "pool")
 # changed since, the line reports null instead of a stale figure.  (workload, kernel label) ->
 # (bytes per launch at the benchmark's size, source file, sha1 prefix, profiles/ summary)
 NCU_TRAFFIC = {
-    ("cfg5_scale", "wgrad_W2"): (948.3e6, "wgrad_tcgen05.cu", "b87f76756f15", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg5_scale", "wgrad_W1"): (854.0e6, "wgrad_tcgen05.cu", "b87f76756f15", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg5_scale", "gemm1_act"): (906.5e6, "gemm_tcgen05.cu", "f8c89f063c38", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg5_scale", "gemm2"): (736.5e6, "gemm_tcgen05.cu", "f8c89f063c38", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg5_scale", "bwd_da_dh"): (1105.2e6, "gemm_tcgen05.cu", "f8c89f063c38", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg5_scale", "bwd_dx"): (736.8e6, "gemm_tcgen05.cu", "f8c89f063c38", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg5_scale", "combine"): (1052.4e6, "routed.cu", "3796fde38da4", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg5_scale", "route"): (271.1e6, "route.cu", "9bbafba6931c", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg2_lm", "route"): (8.47e6, "route.cu", "9bbafba6931c", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg2_lm", "mlp_fused"): (12.34e6, "mlp_fused_tcgen05.cu", "4d093230b636", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg2_lm", "attention"): (6.87e6, "attn_tcgen05.cu", "9739abc79f14", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg2_lm", "combine"): (25.18e6, "routed.cu", "3796fde38da4", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg2_lm", "qkv_proj"): (9.73e6, "gemm_tcgen05.cu", "f8c89f063c38", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg3_long", "route"): (16.85e6, "route.cu", "9bbafba6931c", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg3_long", "mlp_fused"): (8.97e6, "mlp_fused_tcgen05.cu", "4d093230b636", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg3_long", "attention"): (6.48e6, "attn_tcgen05.cu", "9739abc79f14", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg3_long", "combine"): (25.18e6, "routed.cu", "3796fde38da4", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg3_long", "qkv_proj"): (8.29e6, "gemm_tcgen05.cu", "f8c89f063c38", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg4_vit", "route"): (39.91e6, "route.cu", "9bbafba6931c", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg4_vit", "mlp_fused"): (57.27e6, "mlp_fused_tcgen05.cu", "4d093230b636", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg4_vit", "attention"): (39.34e6, "attn_tcgen05.cu", "9739abc79f14", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg4_vit", "combine"): (124.34e6, "routed.cu", "3796fde38da4", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg4_vit", "qkv_proj"): (40.13e6, "gemm_tcgen05.cu", "f8c89f063c38", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg5_scale", "wgrad_W2"): (944.6e6, "wgrad_tcgen05.cu", "60af6e835bc7", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg5_scale", "wgrad_W1"): (859.8e6, "wgrad_tcgen05.cu", "60af6e835bc7", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg5_scale", "gemm1_act"): (941.6e6, "gemm_tcgen05.cu", "f7363c30cfda", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg5_scale", "gemm2"): (739.9e6, "gemm_tcgen05.cu", "f7363c30cfda", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg5_scale", "bwd_da_dh"): (1106.7e6, "gemm_tcgen05.cu", "f7363c30cfda", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg5_scale", "bwd_dx"): (740.0e6, "gemm_tcgen05.cu", "f7363c30cfda", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg5_scale", "combine"): (1049.8e6, "routed.cu", "af00419374c5", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg5_scale", "route"): (270.5e6, "route.cu", "b4b9b9429eca", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg2_lm", "route"): (8.5e6, "route.cu", "b4b9b9429eca", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg2_lm", "mlp_fused"): (12.4e6, "mlp_fused_tcgen05.cu", "dbfbf455fb44", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg2_lm", "attention"): (6.9e6, "attn_tcgen05.cu", "4e097eabc901", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg2_lm", "combine"): (25.2e6, "routed.cu", "af00419374c5", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg2_lm", "qkv_proj"): (9.7e6, "gemm_tcgen05.cu", "f7363c30cfda", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg3_long", "route"): (16.85e6, "route.cu", "b4b9b9429eca", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg3_long", "mlp_fused"): (9.0e6, "mlp_fused_tcgen05.cu", "dbfbf455fb44", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg3_long", "attention"): (6.5e6, "attn_tcgen05.cu", "4e097eabc901", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg3_long", "combine"): (25.2e6, "routed.cu", "af00419374c5", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg3_long", "qkv_proj"): (8.3e6, "gemm_tcgen05.cu", "f7363c30cfda", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg4_vit", "route"): (38.8e6, "route.cu", "b4b9b9429eca", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg4_vit", "mlp_fused"): (55.0e6, "mlp_fused_tcgen05.cu", "dbfbf455fb44", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg4_vit", "attention"): (39.5e6, "attn_tcgen05.cu", "4e097eabc901", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg4_vit", "combine"): (123.7e6, "routed.cu", "af00419374c5", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg4_vit", "qkv_proj"): (40.0e6, "gemm_tcgen05.cu", "f7363c30cfda", "profiles/dram_traffic_per_kernel.md"),
 }
 
 

@@ -5,23 +5,25 @@
 //
 // One persistent CTA per SM walks the (row tile, BN-column tile) list; expert regions are padded to 128
 // rows, so a 128-row block never straddles two experts.  Warp roles:
-//   warp 0      TMA producer (lane 0 runs the pipeline; the boxes of a stage are issued one per lane):
-//               A tile [MT*128 x 64] and B tile [64 x BN] per K step into a 128B-swizzled ring
+//   warp 0      TMA producer (lane 0 runs the pipeline; boxes of a stage that need separate copies are issued one per
+//               lane): A tile [MT*128 x 64] and B tile [64 x BN] per K step into a 128B-swizzled ring
 //   warp 1      MMA issuer: tcgen05.mma 128 x BN x 16 into TMEM accumulators
 //   warps 2..   epilogue: tcgen05.ld the accumulator (one row per thread), activation, bf16, then a
 //               [32 rows x 64 columns] piece per warp staged in swizzled shared memory and written with one
 //               TMA tensor store (full 128-byte lines instead of 16-byte scattered stores)
-// Two tile heights:
+// Three tile shapes:
 //   MT = 1  128-row tiles, two TMEM accumulators: the epilogue of tile t overlaps the main loop of tile t+1
-//   MT = 2  256-row tiles (two 128-row accumulators fed by the same B stage): a third fewer operand bytes
-//           per flop, which is what bounds the ring at large K (the ring holds ~1 us of MMA work against an
-//           L2/HBM latency of the same order); one accumulator set, drained by eight epilogue warps.
-//           A 256-row unit at the end of an expert region may hold a single 128-row block ("half tile").
 //   PAIR    256-row tiles worked by a cluster of two CTAs (tcgen05 cta_group::2): CTA r of the pair loads row block r
 //           of A and half r of the B tile's columns, the even CTA issues 256 x BN x 16 MMAs that read both CTAs'
-//           shared memory and write 128 rows into each CTA's TMEM.  Operand bytes per flop as with MT = 2, but each
-//           CTA keeps two accumulator sets, so the epilogue runs under the next main loop; one barrier round covers
-//           128 columns of K.  Used for the backward epilogue, which is too long to leave exposed.
+//           shared memory and write 128 rows into each CTA's TMEM.  A third fewer operand bytes per flop than MT = 1,
+//           and each CTA still keeps two accumulator sets, so the epilogue runs under the next main loop; one barrier
+//           round covers 128 columns of K.  Taken, forward and backward, whenever there are at least two such tiles
+//           per SM and K is a multiple of 128.
+//   MT = 2  256-row tiles in one CTA (two 128-row accumulators fed by the same B stage): the same operand bytes per
+//           flop, but one accumulator set, so the drain of a tile is exposed; left for K that is not a multiple of
+//           128.  A 256-row unit at the end of an expert region may hold a single 128-row block ("half tile").
+// Every stage is filled by as few copies as its layout allows (one box for a routed A tile, one for a B tile: the
+// weights [n, K, N] are mapped as [n][N/64 column blocks][K][64]); only a gathered A needs a box per source patch.
 // The A operand is either a routed buffer (2-D tensor map) or gathered on the fly from x, one TMA box per
 // source patch (Eq. 18 inside the GEMM).
 #include "kernels.cuh"
