@@ -32,6 +32,9 @@ CASES = {
     # ... and with a width that is not a multiple of 128 (17 K blocks): GEMM1 takes the 256-row tiles of one CTA
     "tall_tiles_k1088": gen.tiny(B=40, L=1152, L_valid=1152, m=9, c=3, d=1088, n=4, k=2, d_ff=4096, dtype="bf16",
                                  w_std=0.02),
+    # CTA-pair tiles with x gathered in 16-token patches (eight boxes per 128-row block and K step, two K steps per round)
+    "pair_tiles_short_patches": gen.tiny(B=80, L=256, L_valid=250, m=16, c=8, d=512, n=4, k=2, d_ff=4096, dtype="bf16",
+                                         w_std=0.03),
     # narrow experts (d_e = 256): both GEMMs in one kernel; 64 output columns, a ragged second output half, pad
     # tokens, and a patch length the GEMM cannot gather by itself (routed copy of x as the A operand)
     "fused_d64": gen.tiny(B=3, L=96, L_valid=96, m=6, c=3, d=64, n=2, k=1, d_ff=512, dtype="bf16", w_std=0.05),

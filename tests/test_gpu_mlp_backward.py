@@ -41,6 +41,8 @@ CASES = {
     "wgrad_256_skewed": _w(B=12, L=1152, L_valid=1152, m=9, c=3, d=1024, n=5, k=2, d_ff=5 * 4096, w_std=0.02),
     # the same tiles with patches shorter than a 64-row contraction block (two gathered boxes per block), pad tokens,
     # and an expert that may get no rows at all
+    # CTA-pair GEMMs with 16-token patches: dy gathered in eight boxes per block in the dA/dh step, x in GEMM1
+    "pair_tiles_short_patches": _w(B=80, L=256, L_valid=250, m=16, c=8, d=512, n=4, k=2, d_ff=4096, w_std=0.03),
     "wgrad_256_short_patches_skewed": _w(B=10, L=288, L_valid=270, m=9, c=4, d=1024, n=5, k=2, d_ff=5 * 4096, w_std=0.02),
 }
 
