@@ -89,7 +89,8 @@ def test_float32_path_with_bias():
 
 @pytest.mark.parametrize("kw", [dict(d=384, d_ff=768, n=3),                 # narrow experts: the one-kernel MLP
                                 dict(d=256, d_ff=2048, n=4),                # 512-wide experts: two grouped GEMMs
-                                dict(d=128, d_ff=4 * 192, n=4)])            # 64-column GEMM tiles
+                                dict(d=128, d_ff=4 * 192, n=4),             # 64-column GEMM tiles
+                                dict(d=512, d_ff=4096, n=4, B=80, L=256, L_valid=250, m=16, c=8)])   # 256-row tiles on CTA pairs
 def test_bfloat16_path_with_bias(kw):
     """The in-place bias of the batched product (Section III-D.2) on the tensor-core path: b1 before phi, b2 on every
     expert's output before the combine weight."""
