@@ -75,6 +75,7 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                  int n, int K, int N, int nmat, int act, int* status, const __nv_bfloat16* __restrict__ bwd_h,
                  const float* __restrict__ row_gate, const float* __restrict__ row_valid, float* __restrict__ dg_part,
                  const __nv_bfloat16* __restrict__ bias /* [n, N] or null: added before the activation (forward epilogue) */,
+                 const float* __restrict__ blk_scale /* [rows / 128] or null: factor on the activated output (forward epilogue) */,
                  const __grid_constant__ CUtensorMap tmX, const SrcMap smap, int l_p, int Bm,
                  const __grid_constant__ CUtensorMap tmC0, const __grid_constant__ CUtensorMap tmC1,
                  const __grid_constant__ CUtensorMap tmC2, const __grid_constant__ CUtensorMap tmPre) {
@@ -361,6 +362,11 @@ gemm_bf16_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                         }
                         if (pre) stage_store(f, &tmPre, col0 + g * 64, wrow0);
                         act_apply_n<64>(f, act);
+                        if (blk_scale) {
+                            const float sc = blk_scale[(row0 + half * BM) >> 7];
+#pragma unroll
+                            for (int q = 0; q < 64; ++q) f[q] *= sc;
+                        }
                         if (SIDE3) stage_store(f, g == 0 ? &tmC0 : (g == 1 ? &tmC1 : &tmC2), 0, wrow0);
                         else stage_store(f, tmC, col0 + g * 64, wrow0);
                     }
@@ -464,7 +470,7 @@ uoe_status launch_one(const GemmArgs& g, int* status, cudaStream_t s) {
     launch(kern, dim3(grid), dim3(Cf::THREADS), (size_t)Cf::SMEM, s, tmA, tmB[0], tmB[1], tmB[2], (__nv_bfloat16*)g.C, (__nv_bfloat16*)g.C1,
                                              (__nv_bfloat16*)g.C2, (__nv_bfloat16*)g.pre, g.offsets, g.n, g.K, g.N,
                                              nmat, g.act, status, (const __nv_bfloat16*)g.bwd_h, g.row_gate, g.row_valid,
-                                             g.dg_part, (const __nv_bfloat16*)g.bias, tmX, smap, g.l_p, g.Bm, tmC[0],
+                                             g.dg_part, (const __nv_bfloat16*)g.bias, g.blk_scale, tmX, smap, g.l_p, g.Bm, tmC[0],
                                              tmC[1], tmC[2], tmPre);
     UOE_LAUNCHED();
     return UOE_OK;
@@ -494,7 +500,7 @@ uoe_status dispatch(const GemmArgs& g, int* status, cudaStream_t s) {
 
 uoe_status launch_gemm_bf16(const GemmArgs& g, int* status, cudaStream_t s) {
     if (g.K % BK != 0 || g.N % 64 != 0 || g.nmat > 3) return UOE_ERR_UNSUPPORTED;
-    if (g.bias && (g.bwd || g.nmat > 1)) return UOE_ERR_UNSUPPORTED;      // a bias row per expert: plain forward GEMMs only
+    if ((g.bias || g.blk_scale) && (g.bwd || g.nmat > 1)) return UOE_ERR_UNSUPPORTED;      // a bias row per expert, a factor per block: plain forward GEMMs only
     if (g.nmat > 1 && g.pre) return UOE_ERR_UNSUPPORTED;
     if (g.gather_x && ((!g.src_patch && !g.map.on()) || g.l_p < 8 || g.l_p % 8 != 0 || BM % g.l_p != 0)) return UOE_ERR_INVALID_ARG;
     if (g.rows_max % BM != 0 || g.n > 31) return UOE_ERR_UNSUPPORTED;

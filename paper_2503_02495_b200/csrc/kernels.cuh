@@ -181,6 +181,9 @@ struct GemmArgs {
     const int* src_patch = nullptr;
     int l_p = 0, Bm = 0;
     SrcMap map;             // if map.on(): used instead of src_patch (the router-written plan has no src_patch table)
+    // bf16 path, forward epilogue: C[r,:] is multiplied, after the activation, by blk_scale[r / 128] (one combine weight
+    // per 128-row block, Eq. 40 applied ahead of the second layer; `pre` keeps the unscaled pre-activation)
+    const float* blk_scale = nullptr;
     bool bwd = false;
     const void* bwd_h = nullptr;
     const float* row_gate = nullptr;
@@ -238,6 +241,12 @@ uoe_status launch_mlp_fused(const Dims& D, const void* A, const void* W1, const 
 
 // ---- forward halves behind the routing plan (shared by the per-half entry points and the block entry) ----
 struct MlpFwdBufs { void* xg; void* a; void* z; };
+// Second layer + combine walked by output patch (patches of 128 tokens): whether the problem and plan allow it, the
+// per-block combine weights it needs the first layer to apply, and the launch itself.
+bool gemm2_patch_can(const Dims& D, const PlanPtrs& P, const void* b2);
+uoe_status launch_block_gate(const Dims& D, const PlanPtrs& P, bool use_gate, float* blk, cudaStream_t s);
+uoe_status launch_gemm2_patch(const Dims& D, const void* a, const void* W2, const void* x, void* y, const int* offsets,
+                              const PlanPtrs& P, bool residual, int* status, cudaStream_t s);
 struct SmhaFwdBufs { void *xg, *q, *k, *v, *o, *z; };
 struct SmhaFwdOffsets { size_t xg, q, k, v, o, z; };
 // bytes of the routed buffers of a forward half and their offsets (0 for a buffer the path does not need)

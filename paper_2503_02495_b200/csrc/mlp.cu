@@ -51,6 +51,17 @@ uoe_status uoe::mlp_forward_run(const Dims& D, const uoe_problem* prob, const vo
     GemmArgs g2{a, W2, b2, z, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, false, D.Rmax};
     g1.label = "gemm1_act";
     g2.label = "gemm2";
+    if (!mlp_can_fuse(D) && gemm2_patch_can(D, P, b2)) {
+        // patches of 128 tokens: the first layer applies the combine weights (one per 128-row block, kept where z would
+        // be), the second layer is walked by output patch and writes y itself
+        float* blk = (float*)z;
+        st = launch_block_gate(D, P, (prob->flags & UOE_FLAG_GATE) != 0, blk, stream);
+        if (st != UOE_OK) return st;
+        g1.blk_scale = blk;
+        st = launch_gemm_bf16(g1, status, stream);
+        if (st != UOE_OK) return st;
+        return launch_gemm2_patch(D, a, W2, x, y, expert_offsets, P, (prob->flags & UOE_FLAG_RESIDUAL) != 0, status, stream);
+    }
     if (mlp_can_fuse(D)) {                    // narrow experts: both GEMMs in one kernel, the hidden tile stays on chip
         st = launch_mlp_fused(D, xg, W1, W2, z, saved_h, expert_offsets, prob->act, fused ? x : nullptr, map, status,
                               stream, b1, b2);
