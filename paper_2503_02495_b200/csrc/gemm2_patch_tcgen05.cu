@@ -8,6 +8,10 @@
 // runs the K loops of all selecting experts into one TMEM accumulator, in ascending slot order, adds x in the epilogue
 // and stores y: the per-expert outputs z never reach memory and the sum over experts stays in float32.  Pad tokens and
 // patches nobody selected get y = x (or 0 without the residual).
+// A tile costs as many K loops as its patch has experts (none to k), so the tiles are handed out as the CTAs get to
+// them: a CTA's first tile is its own index, every further one comes from a counter in the workspace's control block
+// that the producer warp advances (which CTA computes a tile varies from run to run; the result does not, every tile
+// being computed whole, in a fixed order, by one CTA).  The last CTA to finish leaves the counters at zero.
 //   warp 0      TMA producer: per 64-wide K step an A block [128 x 64] of a' and a W2 block [64 x 256] (one box each)
 //   warp 1      MMA issuer: tcgen05.mma 128 x 256 x 16, two accumulator sets (the epilogue of a tile runs under the
 //               next tile's main loop)
@@ -28,12 +32,16 @@ constexpr int STAGES = 4;
 constexpr int EPI_WARPS = 8, THREADS = 64 + 32 * EPI_WARPS, STG_BYTES = 32 * 128;
 constexpr int SMEM = STAGES * STAGE + 1024 + 1024 + EPI_WARPS * STG_BYTES;
 constexpr int KMAX = 8;            // experts per sample this kernel handles
+constexpr int kSchedSlots = 4;     // tiles the producer may run ahead of the slowest consumer
+constexpr int kSchedWord = 64;     // words [64, 66) of the workspace's control block: next tile, CTAs finished (zero between launches)
 
 struct PCtl {
     uint64_t full[STAGES], empty[STAGES], tfull[2], tempty[2];
     uint32_t tmem_base;
     int abort_flag;
     int offs[34];
+    uint64_t sfull[kSchedSlots], sempty[kSchedSlots];
+    int sched_tile[kSchedSlots];   // tiles handed from the producer warp to the MMA thread and the epilogue warps
 };
 
 __global__ void __launch_bounds__(THREADS, 1)
@@ -41,7 +49,7 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                    const __grid_constant__ CUtensorMap tmY, const __nv_bfloat16* __restrict__ x,
                    const int* __restrict__ inv_row, const int* __restrict__ pair_row, int inv_relative,
                    const int* __restrict__ offsets, int n, int Bm, int m, int k, int K, int N, int Lv, int residual,
-                   int* status) {
+                   int* status, int* __restrict__ sched /* [2], zero between launches */) {
     pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -52,6 +60,7 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(&ctl->tfull[a], 1); mbar_init(&ctl->tempty[a], 32 * EPI_WARPS); }
+        for (int q = 0; q < kSchedSlots; ++q) { mbar_init(&ctl->sfull[q], 1); mbar_init(&ctl->sempty[q], 1 + EPI_WARPS); }
         ctl->abort_flag = 0;
         fence_barrier_init();
         prefetch_tmap(&tmA);
@@ -75,12 +84,37 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         return r;
     };
 
+    // consumer side of the tile hand-off (one thread per consumer warp): this CTA's next tile, or >= total_tiles at the end
+    auto next_tile = [&](int& slot, uint32_t& sphase) {
+        int tile = total_tiles;
+        if (mbar_wait(&ctl->sfull[slot], sphase, abort_flag, status) && !*abort_flag) {
+            tile = ctl->sched_tile[slot];
+            mbar_arrive(&ctl->sempty[slot]);
+        }
+        if (++slot == kSchedSlots) { slot = 0; sphase ^= 1; }
+        return tile;
+    };
+
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         int stage = 0;
         uint32_t phase = 0, issued = 0, issued_parity = 0;
         bool stop = false;
-        for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+        int slot = 0;
+        uint32_t sphase = 0;
+        for (bool first = true; !stop; first = false) {
+            int tile = total_tiles;
+            if (lane == 0) {       // hand the next tile (or the end marker) to the consumers
+                if (mbar_wait(&ctl->sempty[slot], sphase ^ 1, abort_flag, status) && !*abort_flag) {
+                    tile = first ? (int)blockIdx.x : (int)gridDim.x + atomicAdd(sched, 1);
+                    if (tile > total_tiles) tile = total_tiles;
+                }
+                ctl->sched_tile[slot] = tile;
+                mbar_arrive(&ctl->sfull[slot]);
+            }
+            tile = __shfl_sync(0xffffffffu, tile, 0);
+            if (++slot == kSchedSlots) { slot = 0; sphase ^= 1; }
+            if (tile >= total_tiles) break;
             const int p = tile / n_tiles, n0 = (tile % n_tiles) * BN;
             int rows[KMAX];
 #pragma unroll
@@ -118,7 +152,11 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool stop = false;
-            for (int tile = blockIdx.x; tile < total_tiles && !stop; tile += gridDim.x) {
+            int slot = 0;
+            uint32_t sphase = 0;
+            while (!stop) {
+                const int tile = next_tile(slot, sphase);
+                if (tile >= total_tiles) break;
                 const int p = tile / n_tiles;
                 int cnt = 0;
                 for (int s = 0; s < k; ++s) cnt += inv_row[(size_t)p * k + s] >= 0 ? 1 : 0;
@@ -147,7 +185,13 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         int acc = 0;
         uint32_t acc_phase = 0;
         uint8_t* stg = smem + STAGES * STAGE + 1024 + (warp - 2) * STG_BYTES;
-        for (int tile = blockIdx.x; tile < total_tiles; tile += gridDim.x) {
+        int slot = 0;
+        uint32_t sphase = 0;
+        for (;;) {
+            int tile = 0;
+            if (lane == 0) tile = next_tile(slot, sphase);
+            tile = __shfl_sync(0xffffffffu, tile, 0);
+            if (tile >= total_tiles) break;
             const int p = tile / n_tiles, n0 = (tile % n_tiles) * BN;
             int cnt = 0;
             for (int s = 0; s < k; ++s) cnt += inv_row[(size_t)p * k + s] >= 0 ? 1 : 0;
@@ -207,6 +251,14 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
         __syncwarp();
         tmem_dealloc(tmem_base, 2 * BN);
     }
+    if (threadIdx.x == 0) {         // this CTA's last fetch lies before the barrier above: the last CTA to get here resets
+        __threadfence();
+        if (atomicAdd(sched + 1, 1) == (int)gridDim.x - 1) {
+            sched[0] = 0;
+            sched[1] = 0;
+            __threadfence();
+        }
+    }
 }
 
 // blk[r / 128] = combine weight of the 128-row block that starts at routed row r, for every selected (patch, slot)
@@ -241,6 +293,7 @@ uoe_status launch_block_gate(const Dims& D, const PlanPtrs& P, bool use_gate, fl
 
 uoe_status launch_gemm2_patch(const Dims& D, const void* a, const void* W2, const void* x, void* y, const int* offsets,
                               const PlanPtrs& P, bool residual, int* status, cudaStream_t s) {
+    if (!status) return UOE_ERR_INVALID_ARG;       // the tile counters live in the control block behind the status word
     static DeviceOnce once;
     {
         const uoe_status st = smem_opt_in(once, gemm2_patch_kernel, SMEM);
@@ -270,7 +323,7 @@ uoe_status launch_gemm2_patch(const Dims& D, const void* a, const void* W2, cons
     ProfScope ps("gemm2", s);
     launch_k(gemm2_patch_kernel, dim3(grid), dim3(THREADS), (size_t)SMEM, s, tmA, tmB, tmY, (const __nv_bfloat16*)x,
              (const int*)P.inv_row, (const int*)P.pair_row, P.inv_relative ? 1 : 0, offsets, D.n, D.B * D.m, D.m, D.k, D.d_e,
-             D.d, D.Lv, residual ? 1 : 0, status);
+             D.d, D.Lv, residual ? 1 : 0, status, status + kSchedWord);
     UOE_LAUNCHED();
     return UOE_OK;
 }
