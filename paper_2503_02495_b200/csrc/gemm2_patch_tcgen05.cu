@@ -8,6 +8,8 @@
 // runs the K loops of all selecting experts into one TMEM accumulator, in ascending slot order, adds x in the epilogue
 // and stores y: the per-expert outputs z never reach memory and the sum over experts stays in float32.  Pad tokens and
 // patches nobody selected get y = x (or 0 without the residual).
+// The backward uses the same kernel for dx (derivative of Eq. 38 and 40): a' is dh (the gate is inside it), the weights
+// are W1 read K-major ([n, d, d_e]: dx_g = dh W1^T), x is dy, and the router's per-patch vector is added on real tokens.
 // A tile costs as many K loops as its patch has experts (none to k), so the tiles are handed out as the CTAs get to
 // them: a CTA's first tile is its own index, every further one comes from a counter in the workspace's control block
 // that the producer warp advances (which CTA computes a tile varies from run to run; the result does not, every tile
@@ -44,12 +46,14 @@ struct PCtl {
     int sched_tile[kSchedSlots];   // tiles handed from the producer warp to the MMA thread and the epilogue warps
 };
 
+template <bool B_KMAJOR>
 __global__ void __launch_bounds__(THREADS, 1)
 gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                    const __grid_constant__ CUtensorMap tmY, const __nv_bfloat16* __restrict__ x,
                    const int* __restrict__ inv_row, const int* __restrict__ pair_row, int inv_relative,
                    const int* __restrict__ offsets, int n, int Bm, int m, int k, int K, int N, int Lv, int residual,
-                   int* status, int* __restrict__ sched /* [2], zero between launches */) {
+                   int* status, int* __restrict__ sched /* [2], zero between launches */,
+                   const float* __restrict__ rvec /* [patches, N] added on real tokens, or null */) {
     pdl_trigger();
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -133,7 +137,8 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                     if (lane == 0) {
                         mbar_arrive_expect_tx(&ctl->full[stage], STAGE);
                         tma_load_2d(sa, &tmA, kb * BK, rows[s], &ctl->full[stage]);
-                        tma_load_4d(sa + A_BYTES, &tmB, 0, kb * BK, n0 / 64, e, &ctl->full[stage]);
+                        if (B_KMAJOR) tma_load_3d(sa + A_BYTES, &tmB, kb * BK, n0, e, &ctl->full[stage]);
+                        else tma_load_4d(sa + A_BYTES, &tmB, 0, kb * BK, n0 / 64, e, &ctl->full[stage]);
                     }
                     issued |= 1u << stage;
                     issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
@@ -148,7 +153,7 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------- MMA issuer ----------------
-            constexpr uint32_t idesc = instr_desc_bf16(BM, BN, false, true);
+            constexpr uint32_t idesc = instr_desc_bf16(BM, BN, false, !B_KMAJOR);
             int stage = 0, acc = 0;
             uint32_t phase = 0, acc_phase = 0;
             bool stop = false;
@@ -170,7 +175,8 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                     const uint32_t sa = smem_u32(smem + stage * STAGE), sb = sa + A_BYTES;
 #pragma unroll
                     for (int ks = 0; ks < BK / 16; ++ks)
-                        mma_bf16(d_tmem, smem_desc(sa + ks * 32, 16, 1024), smem_desc(sb + ks * 2048, 8192, 1024), idesc, (i | ks) != 0);
+                        mma_bf16(d_tmem, smem_desc(sa + ks * 32, 16, 1024),
+                                 B_KMAJOR ? smem_desc(sb + ks * 32, 16, 1024) : smem_desc(sb + ks * 2048, 8192, 1024), idesc, (i | ks) != 0);
                     mma_commit(&ctl->empty[stage]);
                     if (++stage == STAGES) { stage = 0; phase ^= 1; }
                 }
@@ -215,6 +221,14 @@ gemm2_patch_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constan
                 } else {
 #pragma unroll
                     for (int q = 0; q < 64; ++q) f[q] = 0.f;
+                }
+                if (rvec && real) {
+                    const float4* rp = (const float4*)(rvec + (size_t)p * N + n0 + g * 64);
+#pragma unroll
+                    for (int q4 = 0; q4 < 16; ++q4) {
+                        const float4 rq = rp[q4];
+                        f[4 * q4] += rq.x; f[4 * q4 + 1] += rq.y; f[4 * q4 + 2] += rq.z; f[4 * q4 + 3] += rq.w;
+                    }
                 }
                 if (residual) {
                     const uint4* xp = (const uint4*)(x + grow * N + n0 + g * 64);
@@ -292,11 +306,13 @@ uoe_status launch_block_gate(const Dims& D, const PlanPtrs& P, bool use_gate, fl
 }
 
 uoe_status launch_gemm2_patch(const Dims& D, const void* a, const void* W2, const void* x, void* y, const int* offsets,
-                              const PlanPtrs& P, bool residual, int* status, cudaStream_t s) {
+                              const PlanPtrs& P, bool residual, int* status, cudaStream_t s, bool w_kmajor,
+                              const float* rvec, const char* label) {
     if (!status) return UOE_ERR_INVALID_ARG;       // the tile counters live in the control block behind the status word
-    static DeviceOnce once;
+    static DeviceOnce once[2];
     {
-        const uoe_status st = smem_opt_in(once, gemm2_patch_kernel, SMEM);
+        const uoe_status st = w_kmajor ? smem_opt_in(once[1], gemm2_patch_kernel<true>, SMEM)
+                                       : smem_opt_in(once[0], gemm2_patch_kernel<false>, SMEM);
         if (st != UOE_OK) return st;
     }
     CUtensorMap tmA, tmB, tmY;
@@ -306,7 +322,12 @@ uoe_status launch_gemm2_patch(const Dims& D, const void* a, const void* W2, cons
         const uint32_t box[2] = {BK, BM};
         if (!make_tmap(&tmA, a, 2, dims, str, box)) return UOE_ERR_CUDA;
     }
-    {                     // W2 [n, d_e, d] as [n][d/64 column blocks][d_e][64]
+    if (w_kmajor) {       // W [n, d, d_e]: rows of the output dimension, the contraction contiguous
+        const uint64_t dims[3] = {(uint64_t)D.d_e, (uint64_t)D.d, (uint64_t)D.n};
+        const uint64_t str[2] = {(uint64_t)D.d_e * 2, (uint64_t)D.d_e * D.d * 2};
+        const uint32_t box[3] = {BK, BN, 1};
+        if (!make_tmap(&tmB, W2, 3, dims, str, box)) return UOE_ERR_CUDA;
+    } else {              // W2 [n, d_e, d] as [n][d/64 column blocks][d_e][64]
         const uint64_t dims[4] = {64, (uint64_t)D.d_e, (uint64_t)D.d / 64, (uint64_t)D.n};
         const uint64_t str[3] = {(uint64_t)D.d * 2, 128, (uint64_t)D.d_e * D.d * 2};
         const uint32_t box[4] = {64, BK, BN / 64, 1};
@@ -320,10 +341,14 @@ uoe_status launch_gemm2_patch(const Dims& D, const void* a, const void* W2, cons
     }
     const long long tiles = (long long)D.B * D.m * (D.d / BN);
     const int grid = (int)(tiles < sm_count() ? tiles : sm_count());
-    ProfScope ps("gemm2", s);
-    launch_k(gemm2_patch_kernel, dim3(grid), dim3(THREADS), (size_t)SMEM, s, tmA, tmB, tmY, (const __nv_bfloat16*)x,
-             (const int*)P.inv_row, (const int*)P.pair_row, P.inv_relative ? 1 : 0, offsets, D.n, D.B * D.m, D.m, D.k, D.d_e,
-             D.d, D.Lv, residual ? 1 : 0, status, status + kSchedWord);
+    ProfScope ps(label, s);
+    auto go = [&](auto kern) {
+        launch_k(kern, dim3(grid), dim3(THREADS), (size_t)SMEM, s, tmA, tmB, tmY, (const __nv_bfloat16*)x,
+                 (const int*)P.inv_row, (const int*)P.pair_row, P.inv_relative ? 1 : 0, offsets, D.n, D.B * D.m, D.m, D.k, D.d_e,
+                 D.d, D.Lv, residual ? 1 : 0, status, status + kSchedWord, rvec);
+    };
+    if (w_kmajor) go(gemm2_patch_kernel<true>);
+    else go(gemm2_patch_kernel<false>);
     UOE_LAUNCHED();
     return UOE_OK;
 }

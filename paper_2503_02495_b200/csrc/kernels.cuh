@@ -245,8 +245,10 @@ struct MlpFwdBufs { void* xg; void* a; void* z; };
 // per-block combine weights it needs the first layer to apply, and the launch itself.
 bool gemm2_patch_can(const Dims& D, const PlanPtrs& P, const void* b2);
 uoe_status launch_block_gate(const Dims& D, const PlanPtrs& P, bool use_gate, float* blk, cudaStream_t s);
+// (w_kmajor: the weights are [n, d, d_e] and the product is a' W^T, the backward's dx; rvec [B*m, d]: added on real tokens)
 uoe_status launch_gemm2_patch(const Dims& D, const void* a, const void* W2, const void* x, void* y, const int* offsets,
-                              const PlanPtrs& P, bool residual, int* status, cudaStream_t s);
+                              const PlanPtrs& P, bool residual, int* status, cudaStream_t s, bool w_kmajor = false,
+                              const float* rvec = nullptr, const char* label = "gemm2");
 struct SmhaFwdBufs { void *xg, *q, *k, *v, *o, *z; };
 struct SmhaFwdOffsets { size_t xg, q, k, v, o, z; };
 // bytes of the routed buffers of a forward half and their offsets (0 for a buffer the path does not need)

@@ -440,10 +440,14 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
     st = launch_wgrad_bf16(ag, fused ? dy : dyg, dW2, expert_offsets, D.n, D.d_e, D.d, D.Rmax, "wgrad_W2", status, stream,
                            wgrad_scratch_bytes(D.n, D.d_e, D.d, D.Rmax) ? (float*)(base + W.wgpart) : nullptr, gq);
     if (st != UOE_OK) return st;
-    GemmArgs gx{dh, W1, nullptr, dxg, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, true, D.Rmax};
-    gx.label = "bwd_dx";
-    st = launch_gemm_bf16(gx, status, stream);
-    if (st != UOE_OK) return st;
+    // patches of 128 tokens: dx_g and the combine are one kernel walked by output patch, after the router's term is known
+    const bool patch_major = gemm2_patch_can(D, P, nullptr);
+    if (!patch_major) {
+        GemmArgs gx{dh, W1, nullptr, dxg, nullptr, expert_offsets, D.n, D.d_e, D.d, UOE_ACT_IDENTITY, true, D.Rmax};
+        gx.label = "bwd_dx";
+        st = launch_gemm_bf16(gx, status, stream);
+        if (st != UOE_OK) return st;
+    }
     st = launch_wgrad_bf16(fused ? x : xg, dh, dW1, expert_offsets, D.n, D.d, D.d_e, D.Rmax, "wgrad_W1", status, stream,
                            wgrad_scratch_bytes(D.n, D.d, D.d_e, D.Rmax) ? (float*)(base + W.wgpart) : nullptr, gp);
     if (st != UOE_OK) return st;
@@ -456,6 +460,9 @@ extern "C" uoe_status uoe_mlp_backward(const uoe_problem* prob, const void* x, c
         UOE_CUDA_OK(cudaMemsetAsync(dW_r, 0, (size_t)D.d * D.n * sizeof(float), stream));
     }
     // dx = dy (selective residual) + the routed input gradients (the gate is already inside dh) + router term
+    if (patch_major)
+        return launch_gemm2_patch(D, dh, W1, dy, dx, expert_offsets, P, residual, status, stream, true,
+                                  use_gate ? rvec : nullptr, "bwd_dx");
     return launch_combine(D, dy, dxg, P, residual, false, dx, stream, use_gate ? rvec : nullptr);
 }
 
