@@ -40,11 +40,11 @@ plan_rows_kernel(const int* __restrict__ expert_idx, const int* __restrict__ off
 }
 
 // ---------------------------------------------------------------------------------------------
-// plan: grid B, 128 threads, dynamic shared memory 8*k*c bytes.  Everything a sample needs from global memory
+// plan: grid B, 128 threads (512 when the backward asks for long per-row arrays), dynamic shared memory 8*k*c bytes.  Everything a sample needs from global memory
 // (its routing arrays, the offsets, the expert choices of the samples before it) is fetched in one round of
 // independent loads; the rest runs out of shared memory.
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(512)
 plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_idx, const float* __restrict__ gate,
             const int* __restrict__ offsets, int B, int n, int k, int m, int c, int l_p,
             int* __restrict__ pair_row, int* __restrict__ inv_row, float* __restrict__ inv_gate,
@@ -57,7 +57,7 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
     int* s_pi = s_dyn;                         // [k*c] patch indices of this sample
     float* s_g = (float*)(s_dyn + k * c);      // [k*c] gates
     __shared__ int my_e[32], prow[32], hist[33], offs[34];
-    const int b = blockIdx.x, tid = threadIdx.x;
+    const int b = blockIdx.x, tid = threadIdx.x, NT = blockDim.x;      // NT: 128 or 512 (long per-row arrays)
     const int l_a = c * l_p;
     if (tid < 33) hist[tid] = 0;
     __syncthreads();
@@ -68,7 +68,7 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
         my_e[tid] = e;
     }
     if (tid <= n) offs[tid] = offsets[tid];
-    for (int idx = tid; idx < k * c; idx += 128) {
+    for (int idx = tid; idx < k * c; idx += NT) {
         const int pj = patch_idx[(size_t)b * k * c + idx];
         if (pj < -1 || pj >= m) set_status(status, UOE_ERR_DEVICE_INDEX);
         s_pi[idx] = pj;
@@ -77,7 +77,7 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
     if (!rows_given) {   // choices of the samples before b, per expert: lane i of each warp counts expert i through ballots
         int acc = 0;
         const int lane = tid & 31;
-        for (int i0 = 0; i0 < b * k; i0 += 128) {
+        for (int i0 = 0; i0 < b * k; i0 += NT) {
             const int idx = i0 + tid;
             const int e = idx < b * k ? expert_idx[idx] : -1;
             for (int i = 0; i < n; ++i) {
@@ -94,7 +94,7 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
         if (!rows_given) pair_row[b * k + tid] = row;
     }
     __syncthreads();
-    for (int idx = tid; idx < m * k; idx += 128) {          // inverse map: which routed rows feed patch j
+    for (int idx = tid; idx < m * k; idx += NT) {          // inverse map: which routed rows feed patch j
         const int j = idx / k, s = idx % k;
         int row = -1;
         float g = 0.f;
@@ -104,7 +104,7 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
         inv_gate[((size_t)b * m + j) * k + s] = g;
     }
     // source patch of every l_p-row block (used when the GEMM gathers its own A operand)
-    for (int idx = tid; idx < k * c; idx += 128) {
+    for (int idx = tid; idx < k * c; idx += NT) {
         const int s = idx / c, u = idx % c;
         const int pj = s_pi[idx];
         src_patch[prow[s] / l_p + u] = (pj >= 0 && pj < m) ? b * m + pj : -1;
@@ -114,7 +114,7 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
         if (rows_given) {      // the last pair of a region starts l_a rows before its end: the largest first row per expert
             if (tid < n) s_end[tid] = offs[tid];
             __syncthreads();
-            for (int idx = tid; idx < B * k; idx += 128) {
+            for (int idx = tid; idx < B * k; idx += NT) {
                 const int e = expert_idx[idx];
                 if (e >= 0 && e < n) atomicMax(&s_end[e], pair_row[idx] + l_a);
             }
@@ -127,16 +127,16 @@ plan_kernel(const int* __restrict__ expert_idx, const int* __restrict__ patch_id
         }
         __syncthreads();
         for (int i = 0; i < n; ++i)
-            for (int rb = s_end[i] / l_p + tid; rb < offs[i + 1] / l_p; rb += 128) src_patch[rb] = -1;
+            for (int rb = s_end[i] / l_p + tid; rb < offs[i + 1] / l_p; rb += NT) src_patch[rb] = -1;
     }
     if (tail) {
         const long long r0 = offs[n];
         const long long total = (rows_max - r0) * tail_row_vecs;
-        for (long long q = (long long)b * 128 + tid; q < total; q += (long long)B * 128)
+        for (long long q = (long long)b * NT + tid; q < total; q += (long long)B * NT)
             tail[r0 * tail_row_vecs + q] = make_uint4(0, 0, 0, 0);
     }
     if (row_gate) {                          // per-row weights for the backward
-        for (int idx = tid; idx < k * l_a; idx += 128) {
+        for (int idx = tid; idx < k * l_a; idx += NT) {
             const int s = idx / l_a, r = idx % l_a, u = r / l_p;
             const int pj = s_pi[s * c + u];
             const bool real = pj >= 0 && pj < m && pj * l_p + (r % l_p) < Lv;
@@ -352,7 +352,8 @@ uoe_status launch_plan(const Dims& D, const int* expert_idx, const int* patch_id
         UOE_LAUNCHED();
     }
     ProfScope ps("plan", s);
-    launch_k(plan_kernel, dim3(D.B), dim3(128), smem, s, expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
+    const int threads = (P.row_gate && (long long)D.k * D.l_a >= 4096) ? 512 : 128;      // the backward's per-row weights: k*l_a rows per sample
+    launch_k(plan_kernel, dim3(D.B), dim3(threads), smem, s, expert_idx, patch_idx, gate, offsets, D.B, D.n, D.k, D.m, D.c, D.l_p,
                                     P.pair_row, P.inv_row, P.inv_gate, P.expert_end, status, P.row_gate, P.row_valid,
                                     D.Lv, use_gate ? 1 : 0, P.src_patch, (uint4*)tail, tail_row_bytes / 16, D.Rmax, many ? 1 : 0);
     UOE_LAUNCHED();
