@@ -682,17 +682,17 @@ NCU_TRAFFIC = {
     ("cfg2_lm", "route"): (8.5e6, "route.cu", "b4b9b9429eca", "profiles/dram_traffic_per_kernel.md"),
     ("cfg2_lm", "mlp_fused"): (12.3e6, "mlp_fused_tcgen05.cu", "dbfbf455fb44", "profiles/dram_traffic_per_kernel.md"),
     ("cfg2_lm", "attention"): (6.9e6, "attn_tcgen05.cu", "4e097eabc901", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg2_lm", "combine"): (25.2e6, "routed.cu", "af00419374c5", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg2_lm", "combine"): (25.2e6, "routed.cu", "a26f173c1050", "profiles/dram_traffic_per_kernel.md"),
     ("cfg2_lm", "qkv_proj"): (9.7e6, "gemm_tcgen05.cu", "e9e4cad6259f", "profiles/dram_traffic_per_kernel.md"),
     ("cfg3_long", "route"): (16.9e6, "route.cu", "b4b9b9429eca", "profiles/dram_traffic_per_kernel.md"),
     ("cfg3_long", "mlp_fused"): (9.0e6, "mlp_fused_tcgen05.cu", "dbfbf455fb44", "profiles/dram_traffic_per_kernel.md"),
     ("cfg3_long", "attention"): (6.5e6, "attn_tcgen05.cu", "4e097eabc901", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg3_long", "combine"): (25.2e6, "routed.cu", "af00419374c5", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg3_long", "combine"): (25.2e6, "routed.cu", "a26f173c1050", "profiles/dram_traffic_per_kernel.md"),
     ("cfg3_long", "qkv_proj"): (8.3e6, "gemm_tcgen05.cu", "e9e4cad6259f", "profiles/dram_traffic_per_kernel.md"),
     ("cfg4_vit", "route"): (38.8e6, "route.cu", "b4b9b9429eca", "profiles/dram_traffic_per_kernel.md"),
     ("cfg4_vit", "mlp_fused"): (55.7e6, "mlp_fused_tcgen05.cu", "dbfbf455fb44", "profiles/dram_traffic_per_kernel.md"),
     ("cfg4_vit", "attention"): (39.5e6, "attn_tcgen05.cu", "4e097eabc901", "profiles/dram_traffic_per_kernel.md"),
-    ("cfg4_vit", "combine"): (123.7e6, "routed.cu", "af00419374c5", "profiles/dram_traffic_per_kernel.md"),
+    ("cfg4_vit", "combine"): (123.7e6, "routed.cu", "a26f173c1050", "profiles/dram_traffic_per_kernel.md"),
     ("cfg4_vit", "qkv_proj"): (39.9e6, "gemm_tcgen05.cu", "e9e4cad6259f", "profiles/dram_traffic_per_kernel.md"),
 }
 
